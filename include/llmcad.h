@@ -1,0 +1,221 @@
+/*
+ * llmcad.h -- C ABI of the B200 (sm_100a) token-tree verification library.
+ *
+ * One call of llmcad_verify_tree() is the target model's single-pass verification
+ * of a draft token tree (LLMCad, arXiv 2309.04255, Sec. 3.2 "Token tree
+ * verification and rectification"): a LLaMA-style decoder forward over all N tree
+ * nodes at once, each node at position prefix_len + depth and attending to the
+ * prefix KV cache plus its own ancestors (the mask table of Sec. 3.2 "Tree
+ * decoder"), then the depth-first search for the longest verified root-to-node
+ * path, then the rollback of the cache to that path.
+ *
+ * Conventions
+ *   - Every pointer marked DEVICE is memory of the current CUDA device, owned by
+ *     the caller and only borrowed for the duration of the enqueued work. Every
+ *     pointer marked HOST is ordinary host memory.
+ *   - `stream` arguments are a cudaStream_t passed as void*. Calls enqueue work on
+ *     that stream and return without synchronising unless stated otherwise.
+ *   - A context is not thread-safe and serves one stream at a time.
+ *   - Return value: LLMCAD_OK or a negative host-detected error. Errors found on
+ *     the device (malformed tree, token id out of range, a wait that ran out) are
+ *     written to scalars[LLMCAD_S_STATUS]; all later phases of that pass then do
+ *     nothing: the cache below prefix_len is untouched and new_prefix_len equals
+ *     prefix_len. Kernels never trap and never wait without a limit.
+ *   - There is no CPU fallback: every step below runs in CUDA kernels of this
+ *     library, and every entry point fails with LLMCAD_ERR_CUDA when no device is
+ *     usable.
+ *
+ * Model (the LLaMA shape): pre-norm residual blocks, RMSNorm, no biases, n_kv_heads
+ * = n_heads, rotary position embedding on interleaved pairs (x[2t], x[2t+1]) with
+ * angle pos * rope_base^(-2t/head_dim), softmax scale 1/sqrt(head_dim), SwiGLU
+ * FFN, separate embedding and lm_head. Weights are row-major [out][in].
+ * dtype bf16: weights, cached K/V and GEMM input activations are bf16; residual
+ * stream, accumulators, softmax, norms and logits are fp32. dtype fp32: all fp32.
+ *
+ * KV cache layout: [n_layers][2 (K,V)][n_heads][max_seq][head_dim] in the model
+ * dtype. Slots 0..prefix_len-1 hold the prefix; during a pass the tree nodes'
+ * rows sit at slots prefix_len..prefix_len+N-1; after the pass slots
+ * 0..new_prefix_len-1 hold prefix + verified path, the rest is unspecified.
+ */
+#ifndef LLMCAD_H
+#define LLMCAD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LLMCAD_MAX_TREE 128
+
+enum {
+    LLMCAD_OK = 0,
+    LLMCAD_ERR_INVALID_ARG = -1, /* NULL pointer, non-positive size, N < 1 */
+    LLMCAD_ERR_UNSUPPORTED = -2, /* N > max_tree or > 128, head_dim not 64/128, unknown dtype, odd sizes */
+    LLMCAD_ERR_CAPACITY = -3,    /* prefix_len + N > max_seq */
+    LLMCAD_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (see llmcad_last_cuda_error) */
+    /* device-detected, reported in scalars[LLMCAD_S_STATUS] */
+    LLMCAD_ERR_BAD_TREE = 1,  /* parent_idx[0] != -1, or parent_idx[i] not in [0, i) */
+    LLMCAD_ERR_BAD_TOKEN = 2, /* token id outside [0, vocab) */
+    LLMCAD_ERR_TIMEOUT = 3,   /* a bounded device-side wait ran out */
+    LLMCAD_ERR_NAN = 4        /* a logit was NaN */
+};
+
+enum { LLMCAD_F32 = 0, LLMCAD_BF16 = 1 };
+
+/* flags of llmcad_config */
+enum {
+    LLMCAD_FLAG_SIMT_GEMM = 1, /* use the plain-ALU GEMM even for bf16 (debugging aid) */
+    LLMCAD_FLAG_SIMT_ATTN = 2  /* use the plain-ALU attention even for bf16 (debugging aid) */
+};
+
+/* indices into the scalars[8] output */
+enum {
+    LLMCAD_S_ACCEPTED_LEN = 0,   /* nodes on the verified path, root included (>= 1) */
+    LLMCAD_S_NEXT_TOKEN = 1,     /* target's output at the last verified node */
+    LLMCAD_S_NEW_PREFIX_LEN = 2, /* prefix_len + accepted_len */
+    LLMCAD_S_N_CORRECT = 3,      /* verified draft tokens = accepted_len - 1 */
+    LLMCAD_S_N_ALL = 4,          /* draft tokens on the longest branch through the last verified node */
+    LLMCAD_S_RECTIFIED = 5,      /* 1 if the last verified node had draft children (all wrong) */
+    LLMCAD_S_STATUS = 6,         /* 0 or a device-detected error */
+    LLMCAD_S_RESERVED = 7
+};
+
+typedef struct llmcad_ctx llmcad_ctx;
+
+typedef struct {
+    int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+    int32_t max_seq;  /* cache capacity in slots */
+    int32_t max_tree; /* largest N this context will see, <= LLMCAD_MAX_TREE */
+    float rms_eps, rope_base;
+    int32_t dtype; /* LLMCAD_F32 or LLMCAD_BF16 */
+    int32_t flags;
+} llmcad_config;
+
+/* Unpacked weights of one layer, DEVICE pointers, row-major [out][in]. */
+typedef struct {
+    const void *attn_norm; /* [d] */
+    const void *wq, *wk, *wv, *wo; /* [d][d] */
+    const void *ffn_norm;  /* [d] */
+    const void *w_gate, *w_up; /* [f][d] */
+    const void *w_down;    /* [d][f] */
+} llmcad_layer_weights;
+
+typedef struct {
+    const void *tok_embed;  /* [V][d] */
+    const void *final_norm; /* [d] */
+    const void *lm_head;    /* [V][d] */
+} llmcad_global_weights;
+
+/* Outputs of a pass: DEVICE pointers, caller-owned. */
+typedef struct {
+    float *logits;          /* [N][vocab] fp32, or NULL when not wanted */
+    int32_t *argmax;        /* [N]: lowest index of each node's maximum logit */
+    int32_t *accepted_path; /* [max_tree]: node indices of the verified path, root first */
+    int32_t *scalars;       /* [8], see LLMCAD_S_* */
+} llmcad_result;
+
+/* The same outputs in HOST memory, for llmcad_verify_tree_host. */
+typedef struct {
+    float *logits;          /* [N][vocab] or NULL */
+    int32_t *argmax;        /* [N] */
+    int32_t *accepted_path; /* [max_tree] */
+    int32_t *scalars;       /* [8] */
+} llmcad_host_result;
+
+int llmcad_version(void);
+const char *llmcad_strerror(int code);
+/* Text of the last CUDA error this library saw on the calling thread's context. */
+const char *llmcad_last_cuda_error(void);
+
+/* Create a context for one model shape on the current device. Allocates the
+ * context's own workspaces (activations of max_tree nodes, partial tiles, attention
+ * partials: a few tens of MB). Fails with LLMCAD_ERR_CUDA without a usable GPU. */
+int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out);
+void llmcad_destroy(llmcad_ctx *ctx);
+
+/* Bytes of the KV cache / of the packed weight buffer for this configuration.
+ * The caller allocates both as DEVICE memory (256-byte aligned). */
+size_t llmcad_kv_cache_bytes(const llmcad_config *cfg);
+size_t llmcad_packed_weight_bytes(const llmcad_config *cfg);
+
+/* One-time packing into the layout the kernels stream: per layer attn_norm,
+ * [wq;wk;wv] as one [3d][d] matrix, wo, ffn_norm, [w_gate;w_up] as one [2f][d]
+ * matrix, w_down; then tok_embed, final_norm, lm_head. Device-to-device copies on
+ * `stream`; the sources may be freed once the stream has run them.
+ * llmcad_pack_layer packs layer `layer`; llmcad_pack_globals the three shared
+ * tensors. All of them must have been called before the first pass. */
+int llmcad_pack_layer(llmcad_ctx *ctx, int32_t layer, const llmcad_layer_weights *src /*HOST struct of DEVICE ptrs*/,
+                      void *packed /*DEVICE*/, void *stream);
+int llmcad_pack_globals(llmcad_ctx *ctx, const llmcad_global_weights *src, void *packed /*DEVICE*/, void *stream);
+
+/* Sec. 3.2: one verification pass.
+ *   packed       DEVICE, from the pack calls
+ *   kv_cache     DEVICE, layout above; slots < prefix_len are read, slots
+ *                prefix_len .. prefix_len+N-1 are written, then the verified path is
+ *                moved to slots prefix_len .. new_prefix_len-1
+ *   tree_tokens  DEVICE int32[N]; node 0 is the root: the last committed token whose
+ *                K/V is not in the cache yet; it is always verified
+ *   parent_idx   DEVICE int32[N], parent_idx[0] = -1, 0 <= parent_idx[i] < i
+ *   out          HOST struct of DEVICE pointers
+ * Asynchronous on `stream`. */
+int llmcad_verify_tree(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t prefix_len,
+                       const int32_t *tree_tokens, const int32_t *parent_idx, int32_t n,
+                       const llmcad_result *out, void *stream);
+
+/* The same pass for callers holding HOST buffers: copies tokens and parents to the
+ * device, runs the pass, copies argmax, path, scalars (and logits when out->logits
+ * is not NULL) back, and synchronises `stream` before returning. The host buffers
+ * should be pinned for the copies to be asynchronous; pageable memory works too. */
+int llmcad_verify_tree_host(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t prefix_len,
+                            const int32_t *tree_tokens /*HOST*/, const int32_t *parent_idx /*HOST*/, int32_t n,
+                            const llmcad_host_result *out, void *stream);
+
+/* Fill cache slots prefix_len .. prefix_len+n-1 from n tokens (a chain-shaped tree
+ * whose nodes are all committed): the "examine them sequentially" case of Sec. 3.2
+ * run in one shot. Any n >= 1; processed in chunks of max_tree. last_logits, when
+ * not NULL, receives the fp32 logits [vocab] at the last token (DEVICE). */
+int llmcad_prefill(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t prefix_len,
+                   const int32_t *tokens /*DEVICE*/, int32_t n, float *last_logits /*DEVICE or NULL*/, void *stream);
+
+/* ---- single steps of the pass, exported for parity tests and kernel benchmarks ---- */
+
+/* Mask table of Sec. 3.2 "Tree decoder": depth[i], pos[i] = prefix_len + depth[i] and
+ * the ancestor-or-self bitmask anc[i][4] (bit j of the 128-bit row i set iff node j is
+ * i or an ancestor of i). status receives 0 or LLMCAD_ERR_BAD_TREE. All DEVICE. */
+int llmcad_tree_prep(const int32_t *parent_idx, int32_t n, int32_t prefix_len, int32_t *depth, int32_t *pos,
+                     uint32_t *anc /*[n][4]*/, int32_t *status, void *stream);
+
+/* Depth-first verified-sequence search and rollback of Sec. 3.2 on a given argmax
+ * array: writes accepted_path and scalars, and moves the verified nodes' K/V rows
+ * of every layer from slot prefix_len+path[j] to slot prefix_len+j.
+ * kv_cache may be NULL (search only). All DEVICE. */
+int llmcad_accept_compact(llmcad_ctx *ctx, void *kv_cache, int32_t prefix_len, const int32_t *tree_tokens,
+                          const int32_t *parent_idx, const int32_t *argmax, int32_t n,
+                          int32_t *accepted_path, int32_t *scalars, void *stream);
+
+/* Tree-masked attention alone (one layer): q [n][H][hd]; k, v [H][kv_stride][hd] with
+ * the prefix at slots 0..prefix_len-1 and the tree nodes at prefix_len..prefix_len+n-1;
+ * o [n][H][hd]. dtype as in llmcad_config. All DEVICE. */
+int llmcad_tree_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, int32_t kv_stride,
+                          int32_t prefix_len, const int32_t *parent_idx, int32_t n, void *o, void *stream);
+
+/* Skinny GEMM alone: y[n][n_out] (fp32) = x[n][n_in] W[n_out][n_in]^T with W and x in
+ * the context's dtype; the weight-streaming step of Sec. 3.2's one-shot verification
+ * (parameters visited once for all n tokens). n <= max_tree. All DEVICE. */
+int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, int32_t n_out, int32_t n_in,
+                       int32_t n, void *stream);
+
+/* For the entry points that have no scalars output (prefill, tree_attention, skinny_gemm):
+ * synchronises `stream` and returns the context's own device status word of the last such
+ * call: 0, a device-detected LLMCAD_ERR_* (> 0), or LLMCAD_ERR_CUDA. */
+int llmcad_last_status(llmcad_ctx *ctx, void *stream);
+
+/* Number of kernels this library has launched through this context so far. */
+int64_t llmcad_launch_count(const llmcad_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LLMCAD_H */

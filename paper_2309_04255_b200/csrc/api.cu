@@ -1,0 +1,567 @@
+// C ABI of the library (see include/llmcad.h): contexts, weight packing, and the host-side
+// sequencing of one verification pass. All arithmetic of the pass runs in the kernels of the
+// other translation units; this file only validates arguments and enqueues them in order.
+#include <cuda.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "attention_tc.cuh"
+#include "common.cuh"
+#include "gemm_tc.cuh"
+
+using namespace llmcad;
+
+namespace {
+
+thread_local char g_cuda_err[256] = "";
+
+bool cuda_ok(cudaError_t e, const char *what)
+{
+    if (e == cudaSuccess) return true;
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+    return false;
+}
+
+#define CUDA_TRY(expr)                                             \
+    do {                                                           \
+        if (!cuda_ok((expr), #expr)) return LLMCAD_ERR_CUDA;       \
+    } while (0)
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct PackedLayout {
+    size_t attn_norm, wqkv, wo, ffn_norm, wgu, wdown, layer_bytes;  // offsets inside one layer
+    size_t tok_embed, final_norm, lm_head, total;                   // offsets from the start of the buffer
+};
+
+PackedLayout packed_layout(const llmcad_config &c)
+{
+    const size_t e = c.dtype == LLMCAD_F32 ? 4 : 2;
+    const size_t d = c.d_model, f = c.d_ffn, v = c.vocab;
+    PackedLayout L{};
+    size_t o = 0;
+    L.attn_norm = o; o = align_up(o + d * e, 256);
+    L.wqkv = o;      o = align_up(o + 3 * d * d * e, 256);
+    L.wo = o;        o = align_up(o + d * d * e, 256);
+    L.ffn_norm = o;  o = align_up(o + d * e, 256);
+    L.wgu = o;       o = align_up(o + 2 * f * d * e, 256);
+    L.wdown = o;     o = align_up(o + d * f * e, 256);
+    L.layer_bytes = o;
+    o = L.layer_bytes * (size_t)c.n_layers;
+    L.tok_embed = o;  o = align_up(o + v * d * e, 256);
+    L.final_norm = o; o = align_up(o + d * e, 256);
+    L.lm_head = o;    o = align_up(o + v * d * e, 256);
+    L.total = o;
+    return L;
+}
+
+int check_config(const llmcad_config *c)
+{
+    if (c == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    if (c->n_layers < 0 || c->d_model <= 0 || c->n_heads <= 0 || c->head_dim <= 0 || c->d_ffn <= 0 || c->vocab <= 0 ||
+        c->max_seq <= 0 || c->max_tree <= 0)
+        return LLMCAD_ERR_INVALID_ARG;
+    if (c->dtype != LLMCAD_F32 && c->dtype != LLMCAD_BF16) return LLMCAD_ERR_UNSUPPORTED;
+    if (c->max_tree > LLMCAD_MAX_TREE) return LLMCAD_ERR_UNSUPPORTED;
+    if (c->head_dim != 64 && c->head_dim != 128) return LLMCAD_ERR_UNSUPPORTED;
+    if (c->n_heads * c->head_dim != c->d_model) return LLMCAD_ERR_UNSUPPORTED;
+    if (c->d_model % 8 || c->d_ffn % 8) return LLMCAD_ERR_UNSUPPORTED;
+    return LLMCAD_OK;
+}
+
+}  // namespace
+
+struct llmcad_ctx {
+    llmcad_config cfg;
+    PackedLayout lay;
+    int n_sms = 0;
+    size_t elem = 2;
+    bool tc_gemm = false, tc_attn = false;
+    // activations of up to 128 nodes
+    float *x = nullptr;       // residual stream [128][d] fp32
+    void *xn = nullptr;       // normalised GEMM input [128][d]
+    void *q = nullptr;        // rotated queries [128][d]
+    void *att = nullptr;      // attention output [128][d]
+    void *h = nullptr;        // SwiGLU output [128][f]
+    float *logits = nullptr;  // [128][V], used when the caller does not want logits
+    TreeBuffers tb{};
+    int32_t *ibuf = nullptr;  // tokens[128], parent[128], argmax[128], path[128], scalars[8], chain[128]
+    float *partials = nullptr;
+    uint32_t *flags = nullptr;
+    float *attn_ws = nullptr;
+    uint32_t *attn_counters = nullptr;
+    uint32_t epoch = 0;
+    int64_t launches = 0;
+    // tensor maps
+    const void *maps_for = nullptr;
+    std::vector<CUtensorMap> w_maps;   // [L][4] (qkv, o, gate/up, down) + lm_head
+    CUtensorMap act_maps[9][3];        // [n_pad/16][xn, att, h]
+    bool act_ready[9] = {false, false, false, false, false, false, false, false, false};
+
+    int32_t *tokens_dev() const { return ibuf; }
+    int32_t *parent_dev() const { return ibuf + 128; }
+    int32_t *argmax_dev() const { return ibuf + 256; }
+    int32_t *path_dev() const { return ibuf + 384; }
+    int32_t *scalars_dev() const { return ibuf + 512; }
+    int32_t *chain_dev() const { return ibuf + 520; }
+};
+
+namespace {
+
+int ensure_weight_maps(llmcad_ctx *ctx, const void *packed)
+{
+    if (!ctx->tc_gemm || ctx->maps_for == packed) return LLMCAD_OK;
+    const llmcad_config &c = ctx->cfg;
+    const uint64_t d = c.d_model, f = c.d_ffn;
+    ctx->w_maps.assign((size_t)c.n_layers * 4 + 1, CUtensorMap{});
+    const char *base = static_cast<const char *>(packed);
+    bool ok = true;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
+        ok &= make_tensor_map_bf16(&ctx->w_maps[l * 4 + 0], lb + ctx->lay.wqkv, 3 * d, d, 128);
+        ok &= make_tensor_map_bf16(&ctx->w_maps[l * 4 + 1], lb + ctx->lay.wo, d, d, 128);
+        ok &= make_tensor_map_bf16(&ctx->w_maps[l * 4 + 2], lb + ctx->lay.wgu, 2 * f, d, 128);
+        ok &= make_tensor_map_bf16(&ctx->w_maps[l * 4 + 3], lb + ctx->lay.wdown, d, f, 128);
+    }
+    ok &= make_tensor_map_bf16(&ctx->w_maps[(size_t)c.n_layers * 4], base + ctx->lay.lm_head, c.vocab, d, 128);
+    if (!ok) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed for a weight matrix");
+        return LLMCAD_ERR_CUDA;
+    }
+    ctx->maps_for = packed;
+    return LLMCAD_OK;
+}
+
+int ensure_act_maps(llmcad_ctx *ctx, int n_pad)
+{
+    const int slot = n_pad / 16;
+    if (!ctx->tc_gemm || ctx->act_ready[slot]) return LLMCAD_OK;
+    const llmcad_config &c = ctx->cfg;
+    bool ok = true;
+    ok &= make_tensor_map_bf16(&ctx->act_maps[slot][0], ctx->xn, 128, c.d_model, n_pad);
+    ok &= make_tensor_map_bf16(&ctx->act_maps[slot][1], ctx->att, 128, c.d_model, n_pad);
+    ok &= make_tensor_map_bf16(&ctx->act_maps[slot][2], ctx->h, 128, c.d_ffn, n_pad);
+    if (!ok) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed for an activation buffer");
+        return LLMCAD_ERR_CUDA;
+    }
+    ctx->act_ready[slot] = true;
+    return LLMCAD_OK;
+}
+
+// One GEMM of the pass: W is `which` of layer l (or the lm_head when l < 0).
+int run_gemm(llmcad_ctx *ctx, const void *packed, int l, int which, int act, int n_in, const EpiParams &ep, int n_pad,
+             int32_t *status, cudaStream_t st)
+{
+    const char *base = static_cast<const char *>(packed);
+    const void *xin = act == 0 ? ctx->xn : act == 1 ? ctx->att : ctx->h;
+    ctx->launches++;
+    if (ctx->tc_gemm) {
+        const size_t mi = l < 0 ? (size_t)ctx->cfg.n_layers * 4 : (size_t)l * 4 + which;
+        ctx->epoch++;
+        CUDA_TRY(launch_gemm_tc(ctx->w_maps[mi], ctx->act_maps[n_pad / 16][act], n_in, n_pad, ctx->n_sms, ctx->partials,
+                                ctx->flags, ctx->epoch, status, ep, st));
+        return LLMCAD_OK;
+    }
+    const void *W;
+    if (l < 0) W = base + ctx->lay.lm_head;
+    else {
+        const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
+        W = lb + (which == 0 ? ctx->lay.wqkv : which == 1 ? ctx->lay.wo : which == 2 ? ctx->lay.wgu : ctx->lay.wdown);
+    }
+    CUDA_TRY(launch_gemm_simt(W, xin, ctx->cfg.dtype, n_in, ep, status, st));
+    return LLMCAD_OK;
+}
+
+int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, int kv_stride, int P, int n, void *o,
+                  int32_t *status, cudaStream_t st)
+{
+    const llmcad_config &c = ctx->cfg;
+    if (ctx->tc_attn) {
+        int launched = 0;
+        CUDA_TRY(launch_attention_tc(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->attn_ws,
+                                     ctx->attn_counters, ctx->n_sms, status, st, &launched));
+        ctx->launches += launched;
+        return LLMCAD_OK;
+    }
+    if (sizeof(float) * (size_t)(c.head_dim + P + n) > 200 * 1024) return LLMCAD_ERR_UNSUPPORTED;
+    ctx->launches++;
+    CUDA_TRY(launch_attention_simt(q, k, v, c.dtype, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, status, st));
+    return LLMCAD_OK;
+}
+
+// Decoder forward over n nodes: tree prep, embedding, all layers; K/V of node i go to cache slot
+// P+i. When logits != nullptr the final norm and lm_head run too.
+int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, const int32_t *tokens,
+                const int32_t *parent, int n, float *logits, int32_t *status, cudaStream_t st)
+{
+    const llmcad_config &c = ctx->cfg;
+    const int d = c.d_model, f = c.d_ffn, hd = c.head_dim, H = c.n_heads, S = c.max_seq;
+    const int n_pad = (n + 15) / 16 * 16;
+    const char *base = static_cast<const char *>(packed);
+    int rc;
+    if ((rc = ensure_weight_maps(ctx, packed)) != LLMCAD_OK) return rc;
+    if ((rc = ensure_act_maps(ctx, n_pad)) != LLMCAD_OK) return rc;
+
+    CUDA_TRY(launch_tree_prep(parent, tokens, n, P, c.vocab, hd, c.rope_base, ctx->tb, status, st));
+    CUDA_TRY(launch_embed(base + ctx->lay.tok_embed, c.dtype, tokens, n, d, ctx->x, status, st));
+    ctx->launches += 2;
+
+    const size_t kv_layer = (size_t)2 * H * S * hd * ctx->elem;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
+        char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)l;
+        char *vl = kl + kv_layer / 2;
+        EpiParams ep{};
+        ep.n = n;
+
+        CUDA_TRY(launch_rmsnorm(ctx->x, lb + ctx->lay.attn_norm, c.dtype, n, d, c.rms_eps, ctx->xn, status, st));
+        ctx->launches++;
+        ep.mode = EPI_QKV; ep.n_out = 3 * d; ep.q_out = ctx->q; ep.k_cache = kl; ep.v_cache = vl;
+        ep.rope_cs = ctx->tb.rope_cs; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P;
+        if ((rc = run_gemm(ctx, packed, l, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+
+        if ((rc = run_attention(ctx, ctx->q, kl, vl, S, P, n, ctx->att, status, st)) != LLMCAD_OK) return rc;
+
+        ep = EpiParams{}; ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
+        if ((rc = run_gemm(ctx, packed, l, 1, 1, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+
+        CUDA_TRY(launch_rmsnorm(ctx->x, lb + ctx->lay.ffn_norm, c.dtype, n, d, c.rms_eps, ctx->xn, status, st));
+        ctx->launches++;
+        ep = EpiParams{}; ep.n = n; ep.mode = EPI_SWIGLU; ep.n_out = f; ep.h = ctx->h;
+        if ((rc = run_gemm(ctx, packed, l, 2, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+
+        ep = EpiParams{}; ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
+        if ((rc = run_gemm(ctx, packed, l, 3, 2, f, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+    }
+    if (logits != nullptr) {
+        CUDA_TRY(launch_rmsnorm(ctx->x, base + ctx->lay.final_norm, c.dtype, n, d, c.rms_eps, ctx->xn, status, st));
+        ctx->launches++;
+        EpiParams ep{};
+        ep.n = n; ep.mode = EPI_PLAIN; ep.n_out = c.vocab; ep.y = logits; ep.ldy = c.vocab;
+        if ((rc = run_gemm(ctx, packed, -1, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+    }
+    return LLMCAD_OK;
+}
+
+int check_pass_args(const llmcad_ctx *ctx, const void *packed, const void *kv, int P, const void *tok, const void *par, int n)
+{
+    if (ctx == nullptr || packed == nullptr || kv == nullptr || tok == nullptr || par == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    if (n < 1 || P < 0) return LLMCAD_ERR_INVALID_ARG;
+    if (n > ctx->cfg.max_tree) return LLMCAD_ERR_UNSUPPORTED;
+    if ((long long)P + n > ctx->cfg.max_seq) return LLMCAD_ERR_CAPACITY;
+    return LLMCAD_OK;
+}
+
+}  // namespace
+
+// =============================================================================================
+extern "C" {
+
+int llmcad_version(void) { return 100; }
+
+const char *llmcad_strerror(int code)
+{
+    switch (code) {
+    case LLMCAD_OK: return "ok";
+    case LLMCAD_ERR_INVALID_ARG: return "invalid argument";
+    case LLMCAD_ERR_UNSUPPORTED: return "unsupported size, shape or dtype";
+    case LLMCAD_ERR_CAPACITY: return "prefix_len + n exceeds the cache capacity";
+    case LLMCAD_ERR_CUDA: return "CUDA call failed";
+    case LLMCAD_ERR_BAD_TREE: return "malformed tree (parent_idx)";
+    case LLMCAD_ERR_BAD_TOKEN: return "token id out of range";
+    case LLMCAD_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case LLMCAD_ERR_NAN: return "NaN logit";
+    default: return "unknown error";
+    }
+}
+
+const char *llmcad_last_cuda_error(void) { return g_cuda_err; }
+
+size_t llmcad_kv_cache_bytes(const llmcad_config *cfg)
+{
+    if (check_config(cfg) != LLMCAD_OK) return 0;
+    const size_t e = cfg->dtype == LLMCAD_F32 ? 4 : 2;
+    return (size_t)cfg->n_layers * 2 * cfg->n_heads * cfg->max_seq * cfg->head_dim * e;
+}
+
+size_t llmcad_packed_weight_bytes(const llmcad_config *cfg)
+{
+    if (check_config(cfg) != LLMCAD_OK) return 0;
+    return packed_layout(*cfg).total;
+}
+
+int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
+{
+    if (out == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    *out = nullptr;
+    int rc = check_config(cfg);
+    if (rc != LLMCAD_OK) return rc;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    cudaDeviceProp prop;
+    CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+    llmcad_ctx *ctx = new (std::nothrow) llmcad_ctx();
+    if (ctx == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    ctx->cfg = *cfg;
+    ctx->lay = packed_layout(*cfg);
+    ctx->n_sms = prop.multiProcessorCount;
+    ctx->elem = cfg->dtype == LLMCAD_F32 ? 4 : 2;
+    const bool sm100 = prop.major == 10;
+    ctx->tc_gemm = sm100 && cfg->dtype == LLMCAD_BF16 && !(cfg->flags & LLMCAD_FLAG_SIMT_GEMM);
+    ctx->tc_attn = cfg->dtype == LLMCAD_BF16 && cfg->head_dim == 128 && !(cfg->flags & LLMCAD_FLAG_SIMT_ATTN);
+
+    const size_t d = cfg->d_model, f = cfg->d_ffn, hd = cfg->head_dim;
+    auto alloc = [&](void **p, size_t bytes) {
+        if (!cuda_ok(cudaMalloc(p, bytes), "cudaMalloc")) return false;
+        return cuda_ok(cudaMemset(*p, 0, bytes), "cudaMemset");
+    };
+    bool ok = true;
+    ok = ok && alloc((void **)&ctx->x, 128 * d * 4);
+    ok = ok && alloc(&ctx->xn, 128 * d * ctx->elem);
+    ok = ok && alloc(&ctx->q, 128 * d * ctx->elem);
+    ok = ok && alloc(&ctx->att, 128 * d * ctx->elem);
+    ok = ok && alloc(&ctx->h, 128 * f * ctx->elem);
+    ok = ok && alloc((void **)&ctx->logits, (size_t)128 * cfg->vocab * 4);
+    ok = ok && alloc((void **)&ctx->tb.depth, 128 * 4);
+    ok = ok && alloc((void **)&ctx->tb.pos, 128 * 4);
+    ok = ok && alloc((void **)&ctx->tb.anc, 128 * 16);
+    ok = ok && alloc((void **)&ctx->tb.rope_cs, 128 * (hd / 2) * sizeof(float2));
+    ok = ok && alloc((void **)&ctx->ibuf, (520 + 128) * 4);
+    ok = ok && alloc((void **)&ctx->partials, gemm_tc_partial_floats(ctx->n_sms, 128) * 4);
+    ok = ok && alloc((void **)&ctx->flags, (size_t)ctx->n_sms * 4);
+    ok = ok && alloc((void **)&ctx->attn_ws, attention_tc_workspace_bytes(cfg->n_heads, ctx->n_sms));
+    ok = ok && alloc((void **)&ctx->attn_counters, (size_t)cfg->n_heads * 8 * 4);
+    if (ok) {
+        std::vector<int32_t> chain(128);
+        for (int i = 0; i < 128; ++i) chain[i] = i - 1;
+        ok = cuda_ok(cudaMemcpy(ctx->chain_dev(), chain.data(), 128 * 4, cudaMemcpyHostToDevice), "cudaMemcpy");
+    }
+    if (!ok) {
+        llmcad_destroy(ctx);
+        return LLMCAD_ERR_CUDA;
+    }
+    *out = ctx;
+    return LLMCAD_OK;
+}
+
+void llmcad_destroy(llmcad_ctx *ctx)
+{
+    if (ctx == nullptr) return;
+    void *ptrs[] = {ctx->x, ctx->xn, ctx->q, ctx->att, ctx->h, ctx->logits, ctx->tb.depth, ctx->tb.pos, ctx->tb.anc,
+                    ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->flags, ctx->attn_ws, ctx->attn_counters};
+    for (void *p : ptrs)
+        if (p != nullptr) cudaFree(p);
+    delete ctx;
+}
+
+int llmcad_pack_layer(llmcad_ctx *ctx, int32_t layer, const llmcad_layer_weights *src, void *packed, void *stream)
+{
+    if (ctx == nullptr || src == nullptr || packed == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return LLMCAD_ERR_INVALID_ARG;
+    if (!src->attn_norm || !src->wq || !src->wk || !src->wv || !src->wo || !src->ffn_norm || !src->w_gate || !src->w_up ||
+        !src->w_down)
+        return LLMCAD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t e = ctx->elem, d = ctx->cfg.d_model, f = ctx->cfg.d_ffn;
+    char *lb = static_cast<char *>(packed) + ctx->lay.layer_bytes * (size_t)layer;
+    auto cp = [&](size_t off, const void *s, size_t bytes) {
+        return cudaMemcpyAsync(lb + off, s, bytes, cudaMemcpyDeviceToDevice, st);
+    };
+    CUDA_TRY(cp(ctx->lay.attn_norm, src->attn_norm, d * e));
+    CUDA_TRY(cp(ctx->lay.wqkv, src->wq, d * d * e));
+    CUDA_TRY(cp(ctx->lay.wqkv + d * d * e, src->wk, d * d * e));
+    CUDA_TRY(cp(ctx->lay.wqkv + 2 * d * d * e, src->wv, d * d * e));
+    CUDA_TRY(cp(ctx->lay.wo, src->wo, d * d * e));
+    CUDA_TRY(cp(ctx->lay.ffn_norm, src->ffn_norm, d * e));
+    CUDA_TRY(cp(ctx->lay.wgu, src->w_gate, f * d * e));
+    CUDA_TRY(cp(ctx->lay.wgu + f * d * e, src->w_up, f * d * e));
+    CUDA_TRY(cp(ctx->lay.wdown, src->w_down, d * f * e));
+    return LLMCAD_OK;
+}
+
+int llmcad_pack_globals(llmcad_ctx *ctx, const llmcad_global_weights *src, void *packed, void *stream)
+{
+    if (ctx == nullptr || src == nullptr || packed == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    if (!src->tok_embed || !src->final_norm || !src->lm_head) return LLMCAD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t e = ctx->elem, d = ctx->cfg.d_model, v = ctx->cfg.vocab;
+    char *b = static_cast<char *>(packed);
+    CUDA_TRY(cudaMemcpyAsync(b + ctx->lay.tok_embed, src->tok_embed, v * d * e, cudaMemcpyDeviceToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(b + ctx->lay.final_norm, src->final_norm, d * e, cudaMemcpyDeviceToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(b + ctx->lay.lm_head, src->lm_head, v * d * e, cudaMemcpyDeviceToDevice, st));
+    return LLMCAD_OK;
+}
+
+int llmcad_verify_tree(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t prefix_len,
+                       const int32_t *tree_tokens, const int32_t *parent_idx, int32_t n, const llmcad_result *out,
+                       void *stream)
+{
+    int rc = check_pass_args(ctx, packed, kv_cache, prefix_len, tree_tokens, parent_idx, n);
+    if (rc != LLMCAD_OK) return rc;
+    if (out == nullptr || out->argmax == nullptr || out->accepted_path == nullptr || out->scalars == nullptr)
+        return LLMCAD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const llmcad_config &c = ctx->cfg;
+    int32_t *status = out->scalars + LLMCAD_S_STATUS;
+    float *logits = out->logits != nullptr ? out->logits : ctx->logits;
+    CUDA_TRY(cudaMemsetAsync(out->scalars, 0, 8 * sizeof(int32_t), st));
+    if ((rc = run_forward(ctx, packed, kv_cache, prefix_len, tree_tokens, parent_idx, n, logits, status, st)) != LLMCAD_OK)
+        return rc;
+    CUDA_TRY(launch_argmax(logits, n, c.vocab, out->argmax, status, st));
+    CUDA_TRY(launch_accept(parent_idx, tree_tokens, out->argmax, n, prefix_len, out->accepted_path, out->scalars, st));
+    CUDA_TRY(launch_compact(kv_cache, c.dtype, c.n_layers, c.n_heads, c.max_seq, c.head_dim, prefix_len,
+                            out->accepted_path, out->scalars, st));
+    ctx->launches += 3;
+    return LLMCAD_OK;
+}
+
+int llmcad_verify_tree_host(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t prefix_len,
+                            const int32_t *tree_tokens, const int32_t *parent_idx, int32_t n,
+                            const llmcad_host_result *out, void *stream)
+{
+    int rc = check_pass_args(ctx, packed, kv_cache, prefix_len, tree_tokens, parent_idx, n);
+    if (rc != LLMCAD_OK) return rc;
+    if (out == nullptr || out->argmax == nullptr || out->accepted_path == nullptr || out->scalars == nullptr)
+        return LLMCAD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CUDA_TRY(cudaMemcpyAsync(ctx->tokens_dev(), tree_tokens, n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(ctx->parent_dev(), parent_idx, n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    llmcad_result dev{};
+    dev.logits = out->logits != nullptr ? ctx->logits : nullptr;
+    dev.argmax = ctx->argmax_dev();
+    dev.accepted_path = ctx->path_dev();
+    dev.scalars = ctx->scalars_dev();
+    rc = llmcad_verify_tree(ctx, packed, kv_cache, prefix_len, ctx->tokens_dev(), ctx->parent_dev(), n, &dev, stream);
+    if (rc != LLMCAD_OK) return rc;
+    // argmax[128], path[128] and scalars[8] are contiguous in the context's integer buffer
+    CUDA_TRY(cudaMemcpyAsync(out->argmax, ctx->argmax_dev(), n * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaMemcpyAsync(out->accepted_path, ctx->path_dev(), n * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaMemcpyAsync(out->scalars, ctx->scalars_dev(), 8 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    if (out->logits != nullptr)
+        CUDA_TRY(cudaMemcpyAsync(out->logits, ctx->logits, (size_t)n * ctx->cfg.vocab * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return LLMCAD_OK;
+}
+
+int llmcad_prefill(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t prefix_len, const int32_t *tokens,
+                   int32_t n, float *last_logits, void *stream)
+{
+    if (ctx == nullptr || packed == nullptr || kv_cache == nullptr || tokens == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    if (n < 1 || prefix_len < 0) return LLMCAD_ERR_INVALID_ARG;
+    if ((long long)prefix_len + n > ctx->cfg.max_seq) return LLMCAD_ERR_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
+    CUDA_TRY(cudaMemsetAsync(ctx->scalars_dev(), 0, 8 * sizeof(int32_t), st));
+    const int chunk = ctx->cfg.max_tree;
+    for (int done = 0; done < n; done += chunk) {
+        const int m = n - done < chunk ? n - done : chunk;
+        const bool last = done + m == n;
+        // a chain whose "prefix" is everything before it; every node is committed, nothing to roll back
+        int rc = run_forward(ctx, packed, kv_cache, prefix_len + done, tokens + done, ctx->chain_dev(), m,
+                             (last && last_logits != nullptr) ? ctx->logits : nullptr, status, st);
+        if (rc != LLMCAD_OK) return rc;
+        if (last && last_logits != nullptr)
+            CUDA_TRY(cudaMemcpyAsync(last_logits, ctx->logits + (size_t)(m - 1) * ctx->cfg.vocab,
+                                     (size_t)ctx->cfg.vocab * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    }
+    return LLMCAD_OK;
+}
+
+int llmcad_tree_prep(const int32_t *parent_idx, int32_t n, int32_t prefix_len, int32_t *depth, int32_t *pos,
+                     uint32_t *anc, int32_t *status, void *stream)
+{
+    if (!parent_idx || !depth || !pos || !anc || !status) return LLMCAD_ERR_INVALID_ARG;
+    if (n < 1 || prefix_len < 0) return LLMCAD_ERR_INVALID_ARG;
+    if (n > LLMCAD_MAX_TREE) return LLMCAD_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    TreeBuffers tb{depth, pos, anc, nullptr};
+    CUDA_TRY(launch_tree_prep(parent_idx, nullptr, n, prefix_len, 0, 0, 0.f, tb, status, st));
+    return LLMCAD_OK;
+}
+
+int llmcad_accept_compact(llmcad_ctx *ctx, void *kv_cache, int32_t prefix_len, const int32_t *tree_tokens,
+                          const int32_t *parent_idx, const int32_t *argmax, int32_t n, int32_t *accepted_path,
+                          int32_t *scalars, void *stream)
+{
+    if (!ctx || !tree_tokens || !parent_idx || !argmax || !accepted_path || !scalars) return LLMCAD_ERR_INVALID_ARG;
+    if (n < 1 || prefix_len < 0) return LLMCAD_ERR_INVALID_ARG;
+    if (n > ctx->cfg.max_tree) return LLMCAD_ERR_UNSUPPORTED;
+    if ((long long)prefix_len + n > ctx->cfg.max_seq) return LLMCAD_ERR_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const llmcad_config &c = ctx->cfg;
+    CUDA_TRY(cudaMemsetAsync(scalars, 0, 8 * sizeof(int32_t), st));
+    // the search trusts the tree: validate it first (a malformed tree lands in scalars[status])
+    CUDA_TRY(launch_tree_prep(parent_idx, tree_tokens, n, prefix_len, c.vocab, c.head_dim, c.rope_base, ctx->tb,
+                              scalars + LLMCAD_S_STATUS, st));
+    CUDA_TRY(launch_accept(parent_idx, tree_tokens, argmax, n, prefix_len, accepted_path, scalars, st));
+    ctx->launches += 2;
+    if (kv_cache != nullptr) {
+        CUDA_TRY(launch_compact(kv_cache, c.dtype, c.n_layers, c.n_heads, c.max_seq, c.head_dim, prefix_len, accepted_path,
+                                scalars, st));
+        ctx->launches++;
+    }
+    return LLMCAD_OK;
+}
+
+int llmcad_tree_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, int32_t kv_stride,
+                          int32_t prefix_len, const int32_t *parent_idx, int32_t n, void *o, void *stream)
+{
+    if (!ctx || !q || !k || !v || !parent_idx || !o) return LLMCAD_ERR_INVALID_ARG;
+    if (n < 1 || prefix_len < 0 || kv_stride < prefix_len + n) return LLMCAD_ERR_INVALID_ARG;
+    if (n > ctx->cfg.max_tree) return LLMCAD_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
+    CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    TreeBuffers tb = ctx->tb;
+    tb.rope_cs = nullptr;
+    CUDA_TRY(launch_tree_prep(parent_idx, nullptr, n, prefix_len, 0, 0, 0.f, tb, status, st));
+    ctx->launches++;
+    return run_attention(ctx, q, k, v, kv_stride, prefix_len, n, o, status, st);
+}
+
+int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, int32_t n_out, int32_t n_in, int32_t n,
+                       void *stream)
+{
+    if (!ctx || !w || !x || !y) return LLMCAD_ERR_INVALID_ARG;
+    if (n_out < 1 || n_in < 1 || n < 1) return LLMCAD_ERR_INVALID_ARG;
+    if (n > ctx->cfg.max_tree || n_in % 8) return LLMCAD_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
+    CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    EpiParams ep{};
+    ep.mode = EPI_PLAIN; ep.n = n; ep.n_out = n_out; ep.y = y; ep.ldy = n_out;
+    ctx->launches++;
+    if (ctx->tc_gemm) {
+        const int n_pad = (n + 15) / 16 * 16;
+        CUtensorMap mw, mx;
+        // rows of x beyond n are outside the tensor: the copy engine fills them with zeros
+        if (!make_tensor_map_bf16(&mw, w, n_out, n_in, 128) || !make_tensor_map_bf16(&mx, x, n, n_in, n_pad)) {
+            snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
+            return LLMCAD_ERR_CUDA;
+        }
+        ctx->epoch++;
+        CUDA_TRY(launch_gemm_tc(mw, mx, n_in, n_pad, ctx->n_sms, ctx->partials, ctx->flags, ctx->epoch, status, ep, st));
+        return LLMCAD_OK;
+    }
+    CUDA_TRY(launch_gemm_simt(w, x, ctx->cfg.dtype, n_in, ep, status, st));
+    return LLMCAD_OK;
+}
+
+int llmcad_last_status(llmcad_ctx *ctx, void *stream)
+{
+    if (ctx == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t v = 0;
+    CUDA_TRY(cudaMemcpyAsync(&v, ctx->scalars_dev() + LLMCAD_S_STATUS, sizeof(v), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return v;
+}
+
+int64_t llmcad_launch_count(const llmcad_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

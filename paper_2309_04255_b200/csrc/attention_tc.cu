@@ -1,0 +1,311 @@
+// Tree-masked attention on tensor cores (bf16, head_dim 128).
+//
+// Per head the keys are the prefix slots 0..P-1 (visible to every node) followed by the tree
+// nodes at slots P..P+n-1, of which node i sees the ones whose bit is set in its ancestor-or-self
+// row (the mask table of Sec. 3.2 "Tree decoder"). The prefix K/V bytes dominate, and a layer has
+// few heads, so the key range of each head is split over several CTAs (grid = splits x heads,
+// sized to about two CTAs per SM): each CTA streams its key range once through a cp.async
+// double buffer in shared memory, keeps an online softmax per query row, and writes an
+// unnormalised partial (max, sum, output); the CTA that finishes a head last (an atomic ticket,
+// nobody waits) merges the partials and writes the bf16 output.
+//
+// Inside a CTA warp w owns query rows 16w..16w+15 (n <= 128 nodes -> at most 8 warps busy);
+// QK^T and PV are mma.sync m16n8k16 bf16 with fp32 accumulation, scores never leave registers.
+#include "attention_tc.cuh"
+
+namespace llmcad {
+
+namespace {
+
+constexpr int kHd = 128;
+constexpr int kKeyTile = 64;
+constexpr int kAtThreads = 256;
+constexpr int kRowBytes = kHd * 2;            // 256-byte rows = 16 chunks of 16 bytes
+constexpr int kWsRow = kHd + 2;               // partial row: 128 outputs, max, sum
+constexpr int kMaxSplits = 16;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// 16-byte chunk c of row r lives at chunk c ^ (r & 7): ldmatrix reads of 8 consecutive rows at one
+// logical chunk then touch 8 different bank groups.
+__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4)); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid)
+{
+    const int sz = valid ? 16 : 0;  // size 0: the 16 destination bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm4_t(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kAtThreads)
+attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
+                    const __nv_bfloat16 *__restrict__ v, int n_heads, int kv_stride, int P, int n, int n_pad,
+                    const uint32_t *__restrict__ anc, __nv_bfloat16 *o, float *ws, uint32_t *counters, int splits,
+                    int tiles_per_split, const int32_t *status)
+{
+    if (*status) return;
+    extern __shared__ __align__(128) uint8_t sm[];
+    uint8_t *s_q = sm;                                      // [n_pad][256 B]
+    uint8_t *s_k = s_q + (size_t)n_pad * kRowBytes;         // [2][64][256 B]
+    uint8_t *s_v = s_k + 2 * kKeyTile * kRowBytes;          // [2][64][256 B]
+    __shared__ int s_last;
+
+    const int split = blockIdx.x, head = blockIdx.y;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_keys = P + n;
+    const int n_tiles = (n_keys + kKeyTile - 1) / kKeyTile;
+    const int t_begin = split * tiles_per_split;
+    const int t_end = min(n_tiles, t_begin + tiles_per_split);
+    const __nv_bfloat16 *kh = k + (size_t)head * kv_stride * kHd;
+    const __nv_bfloat16 *vh = v + (size_t)head * kv_stride * kHd;
+
+    auto load_tile = [&](int t, int buf) {
+        const int key0 = t * kKeyTile;
+        uint8_t *dk = s_k + (size_t)buf * kKeyTile * kRowBytes, *dv = s_v + (size_t)buf * kKeyTile * kRowBytes;
+        for (int c = tid; c < kKeyTile * 16; c += kAtThreads) {
+            const int r = c >> 4, ch = c & 15;
+            const int key = key0 + r;
+            const bool ok = key < n_keys;
+            const size_t off = (size_t)(ok ? key : 0) * kHd + ch * 8;
+            cp_async16(smem_u32(dk) + swz(r, ch), kh + off, ok);
+            cp_async16(smem_u32(dv) + swz(r, ch), vh + off, ok);
+        }
+    };
+
+    // queries of this head (rows >= n are zero) and the first key tile
+    for (int c = tid; c < n_pad * 16; c += kAtThreads) {
+        const int r = c >> 4, ch = c & 15;
+        const bool ok = r < n;
+        cp_async16(smem_u32(s_q) + swz(r, ch), q + ((size_t)(ok ? r : 0) * n_heads + head) * kHd + ch * 8, ok);
+    }
+    if (t_begin < t_end) load_tile(t_begin, 0);
+    cp_commit();
+
+    const int q_tiles = n_pad >> 4;
+    const bool active = warp < q_tiles;
+    const int row0 = warp * 16 + (lane >> 2), row1 = row0 + 8;   // the two query rows this thread holds
+    uint32_t anc0[4] = {0, 0, 0, 0}, anc1[4] = {0, 0, 0, 0};
+    if (active) {
+        for (int w = 0; w < 4; ++w) {
+            if (row0 < n) anc0[w] = anc[row0 * 4 + w];
+            if (row1 < n) anc1[w] = anc[row1 * 4 + w];
+        }
+    }
+
+    const float scale_log2 = 1.4426950408889634f * rsqrtf((float)kHd);
+    uint32_t qf[8][4];
+    float oacc[16][4];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f;
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+    for (int t = t_begin; t < t_end; ++t) {
+        const int buf = (t - t_begin) & 1;
+        cp_wait<0>();
+        __syncthreads();                       // tile t (and Q) visible; everyone is done with the other buffer
+        if (t + 1 < t_end) load_tile(t + 1, buf ^ 1);
+        cp_commit();
+        if (t == t_begin && active) {
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                ldsm4(smem_u32(s_q) + swz(warp * 16 + (lane & 15), ks * 2 + (lane >> 4)), qf[ks]);
+        }
+        if (!active) continue;
+        const uint32_t kb = smem_u32(s_k) + buf * kKeyTile * kRowBytes;
+        const uint32_t vb = smem_u32(s_v) + buf * kKeyTile * kRowBytes;
+
+        // ---- S = Q K^T for 64 keys: 8 n-tiles of 8 keys
+        float s[8][4];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t b[4];
+                const int key = np * 16 + (lane & 7) + ((lane >> 4) << 3);
+                ldsm4(kb + swz(key, ks * 2 + ((lane >> 3) & 1)), b);
+                mma_bf16(s[2 * np], qf[ks], b[0], b[1]);
+                mma_bf16(s[2 * np + 1], qf[ks], b[2], b[3]);
+            }
+        }
+        // ---- scale, mask (tree region and the ragged end only), online softmax
+        const int key_base = t * kKeyTile;
+        const bool needs_mask = key_base + kKeyTile > P;
+        float tmax0 = -INFINITY, tmax1 = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float val = s[j][e] * scale_log2;
+                if (needs_mask) {
+                    const int key = key_base + j * 8 + ((lane & 3) << 1) + (e & 1);
+                    if (key >= P) {
+                        const int node = key - P;
+                        const uint32_t *a = (e < 2) ? anc0 : anc1;
+                        const bool vis = node < n && ((a[node >> 5] >> (node & 31)) & 1u);
+                        if (!vis) val = -INFINITY;
+                    }
+                }
+                s[j][e] = val;
+                if (e < 2) tmax0 = fmaxf(tmax0, val); else tmax1 = fmaxf(tmax1, val);
+            }
+        }
+        tmax0 = fmaxf(tmax0, __shfl_xor_sync(0xffffffffu, tmax0, 1));
+        tmax0 = fmaxf(tmax0, __shfl_xor_sync(0xffffffffu, tmax0, 2));
+        tmax1 = fmaxf(tmax1, __shfl_xor_sync(0xffffffffu, tmax1, 1));
+        tmax1 = fmaxf(tmax1, __shfl_xor_sync(0xffffffffu, tmax1, 2));
+        const float mn0 = fmaxf(m0, tmax0), mn1 = fmaxf(m1, tmax1);
+        // a row that has seen no visible key yet keeps max = -inf: use 0 as the reference to avoid inf - inf
+        const float ref0 = (mn0 == -INFINITY) ? 0.f : mn0, ref1 = (mn1 == -INFINITY) ? 0.f : mn1;
+        const float alpha0 = exp2f(m0 - ref0), alpha1 = exp2f(m1 - ref1);
+        m0 = mn0; m1 = mn1;
+        float rs0 = 0.f, rs1 = 0.f;
+        uint32_t pa[4][4];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float p0 = exp2f(s[j][0] - ref0), p1 = exp2f(s[j][1] - ref0);
+            const float p2 = exp2f(s[j][2] - ref1), p3 = exp2f(s[j][3] - ref1);
+            rs0 += p0 + p1; rs1 += p2 + p3;
+            pa[j >> 1][(j & 1) * 2 + 0] = pack_bf16(p0, p1);
+            pa[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
+        }
+        l0 = l0 * alpha0 + rs0; l1 = l1 * alpha1 + rs1;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) { oacc[j][0] *= alpha0; oacc[j][1] *= alpha0; oacc[j][2] *= alpha1; oacc[j][3] *= alpha1; }
+        // ---- O += P V: k = 64 keys (4 steps of 16), n = 128 dims (8 pairs of n-tiles)
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+            for (int dp = 0; dp < 8; ++dp) {
+                uint32_t b[4];
+                const int key = kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                ldsm4_t(vb + swz(key, dp * 2 + (lane >> 4)), b);
+                mma_bf16(oacc[2 * dp], pa[kk], b[0], b[1]);
+                mma_bf16(oacc[2 * dp + 1], pa[kk], b[2], b[3]);
+            }
+        }
+    }
+    cp_wait<0>();
+
+    // ---- row sums over the four threads of a row
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+
+    if (splits == 1) {
+        if (active) {
+            const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int dim = j * 8 + ((lane & 3) << 1);
+                if (row0 < n) *reinterpret_cast<uint32_t *>(o + ((size_t)row0 * n_heads + head) * kHd + dim) = pack_bf16(oacc[j][0] * i0, oacc[j][1] * i0);
+                if (row1 < n) *reinterpret_cast<uint32_t *>(o + ((size_t)row1 * n_heads + head) * kHd + dim) = pack_bf16(oacc[j][2] * i1, oacc[j][3] * i1);
+            }
+        }
+        return;
+    }
+
+    // ---- partial result of this split
+    float *wsp = ws + ((size_t)head * splits + split) * n_pad * kWsRow;
+    if (active) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int dim = j * 8 + ((lane & 3) << 1);
+            *reinterpret_cast<float2 *>(wsp + (size_t)row0 * kWsRow + dim) = make_float2(oacc[j][0], oacc[j][1]);
+            *reinterpret_cast<float2 *>(wsp + (size_t)row1 * kWsRow + dim) = make_float2(oacc[j][2], oacc[j][3]);
+        }
+        if ((lane & 3) == 0) {
+            *reinterpret_cast<float2 *>(wsp + (size_t)row0 * kWsRow + kHd) = make_float2(m0, l0);
+            *reinterpret_cast<float2 *>(wsp + (size_t)row1 * kWsRow + kHd) = make_float2(m1, l1);
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const uint32_t ticket = atomicAdd(counters + head, 1u);
+        s_last = (ticket == (uint32_t)splits - 1);
+        if (s_last) counters[head] = 0;   // ready for the next launch (stream order separates them)
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    // ---- merge: out[row] = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M)
+    const float *wh = ws + (size_t)head * splits * n_pad * kWsRow;
+    for (int idx = tid; idx < n * (kHd / 2); idx += kAtThreads) {
+        const int row = idx / (kHd / 2), dim = (idx % (kHd / 2)) * 2;
+        float M = -INFINITY;
+        for (int sp = 0; sp < splits; ++sp) M = fmaxf(M, __ldcg(wh + ((size_t)sp * n_pad + row) * kWsRow + kHd));
+        float L = 0.f, a0 = 0.f, a1 = 0.f;
+        for (int sp = 0; sp < splits; ++sp) {
+            const float *r = wh + ((size_t)sp * n_pad + row) * kWsRow;
+            const float2 ml = __ldcg(reinterpret_cast<const float2 *>(r + kHd));
+            if (ml.x == -INFINITY) continue;
+            const float w = exp2f(ml.x - M);
+            const float2 ov = __ldcg(reinterpret_cast<const float2 *>(r + dim));
+            L += ml.y * w; a0 += ov.x * w; a1 += ov.y * w;
+        }
+        const float inv = L > 0.f ? 1.f / L : 0.f;
+        *reinterpret_cast<uint32_t *>(o + ((size_t)row * n_heads + head) * kHd + dim) = pack_bf16(a0 * inv, a1 * inv);
+    }
+}
+
+size_t attention_tc_workspace_bytes(int n_heads, int n_sms)
+{
+    (void)n_sms;
+    return (size_t)n_heads * kMaxSplits * LLMCAD_MAX_TREE * kWsRow * sizeof(float);
+}
+
+cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
+                                int n, const uint32_t *anc, void *o, float *ws, uint32_t *counters, int n_sms,
+                                int32_t *status, cudaStream_t st, int *launched)
+{
+    if (hd != kHd) return cudaErrorInvalidValue;
+    const int n_pad = (n + 15) / 16 * 16;
+    const int n_tiles = (P + n + kKeyTile - 1) / kKeyTile;
+    int splits = (2 * n_sms + n_heads - 1) / n_heads;
+    if (splits > kMaxSplits) splits = kMaxSplits;
+    if (splits > n_tiles) splits = n_tiles;
+    if (splits < 1) splits = 1;
+    const int tiles_per_split = (n_tiles + splits - 1) / splits;
+    splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
+    const size_t smem = (size_t)n_pad * kRowBytes + 4 * kKeyTile * kRowBytes;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * kRowBytes + 4 * kKeyTile * kRowBytes);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    dim3 grid(splits, n_heads);
+    attention_tc_kernel<<<grid, kAtThreads, smem, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
+                                                       (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc,
+                                                       (__nv_bfloat16 *)o, ws, counters, splits, tiles_per_split, status);
+    if (launched) *launched = 1;
+    return cudaGetLastError();
+}
+
+}  // namespace llmcad

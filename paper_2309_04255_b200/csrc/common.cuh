@@ -1,0 +1,120 @@
+// Shared declarations of the token-tree verification library (device + host side).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/llmcad.h"
+
+namespace llmcad {
+
+// ---------------------------------------------------------------- element access
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// ---------------------------------------------------------------- GEMM epilogues
+// What a GEMM does with a finished pair of output values of one tree node.
+enum EpiMode : int {
+    EPI_PLAIN = 0,   // y[i][r] = acc                                   (fp32)
+    EPI_QKV = 1,     // rotate q,k pairs at pos[i]; q -> q buffer, k,v -> cache slot P+i
+    EPI_RESID = 2,   // x[i][r] += acc                                   (fp32 residual stream)
+    EPI_SWIGLU = 3,  // h[i][r] = silu(gate) * up                        (pair = gate row r, up row r)
+};
+
+struct EpiParams {
+    int mode;
+    int n;         // tree nodes
+    int n_out;     // output features (rows of W); for EPI_SWIGLU the FFN width f
+    // EPI_PLAIN
+    float *y;
+    int ldy;
+    // EPI_RESID
+    float *x;      // [n][n_out]
+    // EPI_SWIGLU
+    void *h;       // [n][f] activation dtype
+    // EPI_QKV
+    void *q_out;   // [n][d] activation dtype
+    void *k_cache; // this layer's K: [H][S][hd]
+    void *v_cache;
+    const float2 *rope_cs;  // [n][hd/2] (cos, sin) of pos[i] * base^(-2t/hd)
+    int d, hd, S, P;
+};
+
+// (v0, v1) are the accumulators of output rows (r0, r0+1), r0 even, of node i; for
+// EPI_SWIGLU they are (gate, up) of output feature r0. has1 says whether row r0+1 exists.
+template <typename T>
+__device__ __forceinline__ void epilogue_pair(const EpiParams &ep, int r0, int i, float v0, float v1, bool has1)
+{
+    switch (ep.mode) {
+    case EPI_PLAIN:
+        ep.y[(size_t)i * ep.ldy + r0] = v0;
+        if (has1) ep.y[(size_t)i * ep.ldy + r0 + 1] = v1;
+        break;
+    case EPI_RESID:
+        ep.x[(size_t)i * ep.n_out + r0] += v0;
+        if (has1) ep.x[(size_t)i * ep.n_out + r0 + 1] += v1;
+        break;
+    case EPI_SWIGLU: {
+        float s = v0 / (1.0f + __expf(-v0));
+        reinterpret_cast<T *>(ep.h)[(size_t)i * ep.n_out + r0] = from_f32<T>(s * v1);
+        break;
+    }
+    case EPI_QKV: {
+        const int sec = r0 / ep.d, c = r0 - sec * ep.d;
+        const int head = c / ep.hd, e = c - head * ep.hd;
+        float o0 = v0, o1 = v1;
+        if (sec < 2) {
+            const float2 cs = ep.rope_cs[(size_t)i * (ep.hd >> 1) + (e >> 1)];
+            o0 = v0 * cs.x - v1 * cs.y;
+            o1 = v0 * cs.y + v1 * cs.x;
+        }
+        T *dst;
+        if (sec == 0) dst = reinterpret_cast<T *>(ep.q_out) + (size_t)i * ep.d + c;
+        else dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P + i) * ep.hd + e;
+        dst[0] = from_f32<T>(o0);
+        dst[1] = from_f32<T>(o1);
+        break;
+    }
+    }
+}
+
+// ---------------------------------------------------------------- bounded waits
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every device-side wait gives up after 2 s
+
+// ---------------------------------------------------------------- launchers (host)
+struct TreeBuffers {
+    int32_t *depth, *pos;
+    uint32_t *anc;      // [n][4]
+    float2 *rope_cs;    // [n][hd/2]
+};
+
+cudaError_t launch_tree_prep(const int32_t *parent, const int32_t *tokens, int n, int P, int vocab, int hd,
+                             float rope_base, TreeBuffers tb, int32_t *status, cudaStream_t st);
+cudaError_t launch_embed(const void *E, int dtype, const int32_t *tokens, int n, int d, float *x, const int32_t *status,
+                         cudaStream_t st);
+cudaError_t launch_rmsnorm(const float *x, const void *g, int dtype, int n, int d, float eps, void *out,
+                           const int32_t *status, cudaStream_t st);
+cudaError_t launch_argmax(const float *logits, int n, int vocab, int32_t *argmax, int32_t *status, cudaStream_t st);
+cudaError_t launch_accept(const int32_t *parent, const int32_t *tokens, const int32_t *argmax, int n, int P,
+                          int32_t *path, int32_t *scalars, cudaStream_t st);
+cudaError_t launch_compact(void *kv, int dtype, int n_layers, int n_heads, int S, int hd, int P, const int32_t *path,
+                           const int32_t *scalars, cudaStream_t st);
+cudaError_t launch_gemm_simt(const void *W, const void *x, int dtype, int n_in, const EpiParams &ep,
+                             const int32_t *status, cudaStream_t st);
+cudaError_t launch_attention_simt(const void *q, const void *k, const void *v, int dtype, int n_heads, int hd,
+                                  int kv_stride, int P, int n, const uint32_t *anc, void *o, const int32_t *status,
+                                  cudaStream_t st);
+
+}  // namespace llmcad

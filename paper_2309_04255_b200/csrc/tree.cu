@@ -1,0 +1,279 @@
+// Integer side of the pass: mask table, embedding gather, argmax, verified-path search,
+// cache rollback. Everything here is bit-exact by construction.
+#include "common.cuh"
+
+namespace llmcad {
+
+// ------------------------------------------------------------------------------------------
+// Mask table (Sec. 3.2 "Tree decoder"): block i handles node i. Thread 0 walks from the node to
+// the root, checking every link it uses (0 <= parent < child, root has -1), which yields the
+// node's depth and its ancestor-or-self bit row. All threads then fill the node's rotary table
+// row at position prefix_len + depth in fp64.
+__global__ void tree_prep_kernel(const int32_t *__restrict__ parent, const int32_t *__restrict__ tokens, int n, int P,
+                                 int vocab, int hd, double rope_base, int32_t *depth, int32_t *pos, uint32_t *anc,
+                                 float2 *rope_cs, int32_t *status)
+{
+    __shared__ int s_depth;
+    const int i = blockIdx.x;
+    if (threadIdx.x == 0) {
+        uint32_t bits[4] = {0, 0, 0, 0};
+        int d = 0, cur = i, err = 0;
+        if (tokens != nullptr && (tokens[i] < 0 || tokens[i] >= vocab)) err = LLMCAD_ERR_BAD_TOKEN;
+        // cur strictly decreases, so the walk ends within n steps whatever the array holds
+        while (true) {
+            bits[cur >> 5] |= 1u << (cur & 31);
+            const int p = parent[cur];
+            if (cur == 0) {
+                if (p != -1) err = LLMCAD_ERR_BAD_TREE;
+                break;
+            }
+            if (p < 0 || p >= cur) { err = LLMCAD_ERR_BAD_TREE; break; }
+            cur = p;
+            ++d;
+        }
+        if (err) atomicCAS(status, 0, err);
+        depth[i] = d;
+        pos[i] = P + d;
+        for (int w = 0; w < 4; ++w) anc[i * 4 + w] = bits[w];
+        s_depth = d;
+    }
+    __syncthreads();
+    if (rope_cs != nullptr) {
+        const double p = (double)(P + s_depth);
+        for (int t = threadIdx.x; t < hd / 2; t += blockDim.x) {
+            const double ang = p * pow(rope_base, -2.0 * t / hd);
+            double sn, cs;
+            sincos(ang, &sn, &cs);
+            rope_cs[(size_t)i * (hd / 2) + t] = make_float2((float)cs, (float)sn);
+        }
+    }
+}
+
+cudaError_t launch_tree_prep(const int32_t *parent, const int32_t *tokens, int n, int P, int vocab, int hd,
+                             float rope_base, TreeBuffers tb, int32_t *status, cudaStream_t st)
+{
+    tree_prep_kernel<<<n, 64, 0, st>>>(parent, tokens, n, P, vocab, hd, (double)rope_base, tb.depth, tb.pos, tb.anc,
+                                       tb.rope_cs, status);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_kernel(const T *__restrict__ E, const int32_t *__restrict__ tokens, int d, float *x,
+                             const int32_t *status)
+{
+    if (*status) return;
+    const int i = blockIdx.x;
+    const T *row = E + (size_t)tokens[i] * d;
+    for (int k = threadIdx.x; k < d; k += blockDim.x) x[(size_t)i * d + k] = to_f32<T>(row[k]);
+}
+
+cudaError_t launch_embed(const void *E, int dtype, const int32_t *tokens, int n, int d, float *x, const int32_t *status,
+                         cudaStream_t st)
+{
+    if (dtype == LLMCAD_F32) embed_kernel<float><<<n, 256, 0, st>>>((const float *)E, tokens, d, x, status);
+    else embed_kernel<__nv_bfloat16><<<n, 256, 0, st>>>((const __nv_bfloat16 *)E, tokens, d, x, status);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// RMSNorm of the fp32 residual stream into the GEMM input dtype.
+template <typename T>
+__global__ void rmsnorm_kernel(const float *__restrict__ x, const T *__restrict__ g, int d, float eps, T *out,
+                               const int32_t *status)
+{
+    if (*status) return;
+    __shared__ float red[32];
+    const int i = blockIdx.x;
+    const float *xi = x + (size_t)i * d;
+    float ss = 0.f;
+    for (int k = threadIdx.x; k < d; k += blockDim.x) ss += xi[k] * xi[k];
+    for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (threadIdx.x == 0) red[0] = v;
+    }
+    __syncthreads();
+    const float r = rsqrtf(red[0] / d + eps);
+    for (int k = threadIdx.x; k < d; k += blockDim.x) out[(size_t)i * d + k] = from_f32<T>(xi[k] * r * to_f32<T>(g[k]));
+}
+
+cudaError_t launch_rmsnorm(const float *x, const void *g, int dtype, int n, int d, float eps, void *out,
+                           const int32_t *status, cudaStream_t st)
+{
+    if (dtype == LLMCAD_F32) rmsnorm_kernel<float><<<n, 256, 0, st>>>(x, (const float *)g, d, eps, (float *)out, status);
+    else rmsnorm_kernel<__nv_bfloat16><<<n, 256, 0, st>>>(x, (const __nv_bfloat16 *)g, d, eps, (__nv_bfloat16 *)out, status);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Greedy choice of the target at every node: lowest index of the maximum; a NaN sets status.
+__global__ void argmax_kernel(const float *__restrict__ logits, int vocab, int32_t *argmax, int32_t *status)
+{
+    if (*status) return;
+    __shared__ float s_v[32];
+    __shared__ int s_i[32];
+    const int i = blockIdx.x;
+    const float *row = logits + (size_t)i * vocab;
+    float best = -INFINITY;
+    int bi = 0x7fffffff;
+    bool nan = false;
+    for (int t = threadIdx.x; t < vocab; t += blockDim.x) {
+        const float v = row[t];
+        nan |= (v != v);
+        if (v > best || (v == best && t < bi)) { best = v; bi = t; }
+    }
+    if (nan) atomicCAS(status, 0, LLMCAD_ERR_NAN);
+    for (int o = 16; o; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { s_v[threadIdx.x >> 5] = best; s_i[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const int nw = blockDim.x >> 5;
+        best = threadIdx.x < nw ? s_v[threadIdx.x] : -INFINITY;
+        bi = threadIdx.x < nw ? s_i[threadIdx.x] : 0x7fffffff;
+        for (int o = 16; o; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+        }
+        if (threadIdx.x == 0) argmax[i] = (bi == 0x7fffffff) ? 0 : bi;
+    }
+}
+
+cudaError_t launch_argmax(const float *logits, int n, int vocab, int32_t *argmax, int32_t *status, cudaStream_t st)
+{
+    argmax_kernel<<<n, 256, 0, st>>>(logits, vocab, argmax, status);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Verified-sequence search (Sec. 3.2 "Depth-first verified sequence searching"), data-parallel
+// form: node c is verified iff every link on its root path is correct (the child's draft token
+// equals the target's output at the parent). The verified sequence ends at the deepest verified
+// node, ties to the lowest index. One block of 128 threads, thread c = node c.
+__global__ void accept_kernel(const int32_t *__restrict__ parent, const int32_t *__restrict__ tokens,
+                              const int32_t *__restrict__ argmax, int n, int P, int32_t *path, int32_t *scalars)
+{
+    __shared__ int s_par[LLMCAD_MAX_TREE];
+    __shared__ unsigned char s_link[LLMCAD_MAX_TREE];
+    __shared__ int s_key[4];
+    __shared__ int s_best, s_haschild;
+    const int c = threadIdx.x;
+    const int status = scalars[LLMCAD_S_STATUS];
+    if (status) {  // an earlier phase failed: report an empty result, leave the cache as it was
+        if (c == 0) {
+            scalars[LLMCAD_S_ACCEPTED_LEN] = 0;
+            scalars[LLMCAD_S_NEXT_TOKEN] = -1;
+            scalars[LLMCAD_S_NEW_PREFIX_LEN] = P;
+            scalars[LLMCAD_S_N_CORRECT] = 0;
+            scalars[LLMCAD_S_N_ALL] = 0;
+            scalars[LLMCAD_S_RECTIFIED] = 0;
+            scalars[LLMCAD_S_RESERVED] = 0;
+        }
+        return;
+    }
+    if (c < n) {
+        const int p = parent[c];
+        s_par[c] = p;
+        s_link[c] = (c == 0) ? 1 : (tokens[c] == argmax[p]);
+    }
+    if (c == 0) s_haschild = 0;
+    __syncthreads();
+    int key = -1, d = 0;
+    if (c < n) {
+        bool ok = true;
+        for (int cur = c; cur > 0; cur = s_par[cur]) { ok &= (s_link[cur] != 0); ++d; }
+        if (ok) key = (d << 8) | (LLMCAD_MAX_TREE - 1 - c);
+    }
+    int m = key;
+    for (int o = 16; o; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((c & 31) == 0) s_key[c >> 5] = m;
+    __syncthreads();
+    if (c == 0) {
+        const int mm = max(max(s_key[0], s_key[1]), max(s_key[2], s_key[3]));
+        s_best = LLMCAD_MAX_TREE - 1 - (mm & 0xff);
+    }
+    __syncthreads();
+    const int best = s_best;
+    // longest draft branch through the verified end node: deepest node that has it on its root path
+    int below = -1;
+    if (c < n) {
+        for (int cur = c;; cur = s_par[cur]) {
+            if (cur == best) { below = d; break; }
+            if (cur <= 0 || cur < best) break;
+        }
+        if (c > 0 && s_par[c] == best) s_haschild = 1;
+    }
+    for (int o = 16; o; o >>= 1) below = max(below, __shfl_xor_sync(0xffffffffu, below, o));
+    __syncthreads();
+    if ((c & 31) == 0) s_key[c >> 5] = below;
+    __syncthreads();
+    if (c == 0) {
+        int len = 1;
+        for (int cur = best; cur > 0; cur = s_par[cur]) ++len;
+        int j = len - 1;
+        for (int cur = best; j >= 0; cur = s_par[cur], --j) path[j] = cur;
+        scalars[LLMCAD_S_ACCEPTED_LEN] = len;
+        scalars[LLMCAD_S_NEXT_TOKEN] = argmax[best];
+        scalars[LLMCAD_S_NEW_PREFIX_LEN] = P + len;
+        scalars[LLMCAD_S_N_CORRECT] = len - 1;
+        scalars[LLMCAD_S_N_ALL] = max(max(s_key[0], s_key[1]), max(s_key[2], s_key[3]));
+        scalars[LLMCAD_S_RECTIFIED] = s_haschild;
+        scalars[LLMCAD_S_RESERVED] = 0;
+    }
+}
+
+cudaError_t launch_accept(const int32_t *parent, const int32_t *tokens, const int32_t *argmax, int n, int P,
+                          int32_t *path, int32_t *scalars, cudaStream_t st)
+{
+    accept_kernel<<<1, LLMCAD_MAX_TREE, 0, st>>>(parent, tokens, argmax, n, P, path, scalars);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Rollback (Sec. 3.2): for every layer, K and V, head: move the row at slot P+path[j] to slot P+j.
+// path is strictly increasing with path[j] >= j, so for one fixed 16-byte column of one head an
+// ascending copy never reads a slot it has already overwritten; each thread owns one such column
+// and walks j upwards (eight rows are read before they are written to keep loads in flight).
+__global__ void compact_kernel(uint4 *kv, int n_lkh, int S, int chunks, int P, const int32_t *__restrict__ path,
+                               const int32_t *__restrict__ scalars)
+{
+    if (scalars[LLMCAD_S_STATUS]) return;
+    const int len = scalars[LLMCAD_S_ACCEPTED_LEN];
+    const long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (w >= (long long)n_lkh * chunks) return;
+    const int lkh = (int)(w / chunks), ch = (int)(w % chunks);
+    uint4 *base = kv + ((size_t)lkh * S + P) * chunks + ch;
+    int j0 = 0;
+    while (j0 < len && path[j0] == j0) ++j0;  // rows already in place
+    for (int j = j0; j < len; j += 8) {
+        uint4 tmp[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (j + u < len) tmp[u] = base[(size_t)path[j + u] * chunks];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (j + u < len) base[(size_t)(j + u) * chunks] = tmp[u];
+    }
+}
+
+cudaError_t launch_compact(void *kv, int dtype, int n_layers, int n_heads, int S, int hd, int P, const int32_t *path,
+                           const int32_t *scalars, cudaStream_t st)
+{
+    const int elem = dtype == LLMCAD_F32 ? 4 : 2;
+    const int chunks = hd * elem / 16;
+    const int n_lkh = n_layers * 2 * n_heads;
+    const long long total = (long long)n_lkh * chunks;
+    const int block = 128;
+    compact_kernel<<<(unsigned)((total + block - 1) / block), block, 0, st>>>((uint4 *)kv, n_lkh, S, chunks, P, path, scalars);
+    return cudaGetLastError();
+}
+
+}  // namespace llmcad
