@@ -212,6 +212,13 @@ int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, 
  * call: 0, a device-detected LLMCAD_ERR_* (> 0), or LLMCAD_ERR_CUDA. */
 int llmcad_last_status(llmcad_ctx *ctx, void *stream);
 
+/* Per-launch timing for roofline reports. While enabled, every skinny-GEMM launch (kind 0) and
+ * every tree-attention launch (kind 1) of this context is bracketed by CUDA events on the
+ * launching stream. llmcad_get_kernel_timing waits for the recorded launches of `kind`, returns
+ * their summed duration and count since the last query, and forgets them. */
+int llmcad_set_kernel_timing(llmcad_ctx *ctx, int32_t enable);
+int llmcad_get_kernel_timing(llmcad_ctx *ctx, int32_t kind, double *total_ms /*HOST*/, int64_t *n_launches /*HOST*/);
+
 /* Number of kernels this library has launched through this context so far. */
 int64_t llmcad_launch_count(const llmcad_ctx *ctx);
 

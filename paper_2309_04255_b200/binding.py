@@ -29,7 +29,7 @@ EXPORTS = [
     "llmcad_kv_cache_bytes", "llmcad_packed_weight_bytes", "llmcad_pack_layer", "llmcad_pack_globals",
     "llmcad_verify_tree", "llmcad_verify_tree_host", "llmcad_prefill", "llmcad_tree_prep",
     "llmcad_accept_compact", "llmcad_tree_attention", "llmcad_skinny_gemm", "llmcad_launch_count",
-    "llmcad_last_status",
+    "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing",
 ]
 
 
@@ -96,6 +96,8 @@ def lib():
         L.llmcad_launch_count.argtypes = [vp]
         L.llmcad_launch_count.restype = C.c_int64
         L.llmcad_last_status.argtypes = [vp, vp]
+        L.llmcad_set_kernel_timing.argtypes = [vp, i32]
+        L.llmcad_get_kernel_timing.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         _lib = L
     return _lib
 
@@ -232,6 +234,14 @@ class Verifier:
 
     def last_status(self) -> int:
         return lib().llmcad_last_status(self.ctx, _stream())
+
+    def set_kernel_timing(self, on: bool):
+        _check(lib().llmcad_set_kernel_timing(self.ctx, 1 if on else 0), "llmcad_set_kernel_timing")
+
+    def get_kernel_timing(self, kind: int):
+        ms, cnt = C.c_double(), C.c_int64()
+        _check(lib().llmcad_get_kernel_timing(self.ctx, kind, C.byref(ms), C.byref(cnt)), "llmcad_get_kernel_timing")
+        return ms.value, cnt.value
 
     def launch_count(self) -> int:
         return lib().llmcad_launch_count(self.ctx)

@@ -100,6 +100,11 @@ struct llmcad_ctx {
     std::vector<CUtensorMap> w_maps;   // [L][4] (qkv, o, gate/up, down) + lm_head
     CUtensorMap act_maps[9][3];        // [n_pad/16][xn, att, h]
     bool act_ready[9] = {false, false, false, false, false, false, false, false, false};
+    // optional per-launch timing (events around every GEMM / attention launch)
+    bool timing = false;
+    struct Timed { int kind; cudaEvent_t a, b; };
+    std::vector<Timed> timed;
+    std::vector<cudaEvent_t> event_pool;
 
     int32_t *tokens_dev() const { return ibuf; }
     int32_t *parent_dev() const { return ibuf + 128; }
@@ -110,6 +115,38 @@ struct llmcad_ctx {
 };
 
 namespace {
+
+// Brackets one launch with events when kernel timing is on.
+struct TimedLaunch {
+    llmcad_ctx *ctx;
+    cudaStream_t st;
+    cudaEvent_t a = nullptr, b = nullptr;
+    int kind;
+    TimedLaunch(llmcad_ctx *c, int k, cudaStream_t s) : ctx(c), st(s), kind(k)
+    {
+        if (!ctx->timing) return;
+        a = take();
+        b = take();
+        if (a && b) cudaEventRecord(a, st);
+    }
+    ~TimedLaunch()
+    {
+        if (!ctx->timing || !a || !b) return;
+        cudaEventRecord(b, st);
+        ctx->timed.push_back({kind, a, b});
+    }
+    cudaEvent_t take()
+    {
+        if (!ctx->event_pool.empty()) {
+            cudaEvent_t e = ctx->event_pool.back();
+            ctx->event_pool.pop_back();
+            return e;
+        }
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+        return e;
+    }
+};
 
 int ensure_weight_maps(llmcad_ctx *ctx, const void *packed)
 {
@@ -159,6 +196,7 @@ int run_gemm(llmcad_ctx *ctx, const void *packed, int l, int which, int act, int
     const char *base = static_cast<const char *>(packed);
     const void *xin = act == 0 ? ctx->xn : act == 1 ? ctx->att : ctx->h;
     ctx->launches++;
+    TimedLaunch tl(ctx, 0, st);
     if (ctx->tc_gemm) {
         const size_t mi = l < 0 ? (size_t)ctx->cfg.n_layers * 4 : (size_t)l * 4 + which;
         ctx->epoch++;
@@ -180,6 +218,7 @@ int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, 
                   int32_t *status, cudaStream_t st)
 {
     const llmcad_config &c = ctx->cfg;
+    TimedLaunch tl(ctx, 1, st);
     if (ctx->tc_attn) {
         int launched = 0;
         CUDA_TRY(launch_attention_tc(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->attn_ws,
@@ -355,6 +394,8 @@ void llmcad_destroy(llmcad_ctx *ctx)
                     ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->flags, ctx->attn_ws, ctx->attn_counters};
     for (void *p : ptrs)
         if (p != nullptr) cudaFree(p);
+    for (auto &t : ctx->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+    for (auto e : ctx->event_pool) cudaEventDestroy(e);
     delete ctx;
 }
 
@@ -549,6 +590,35 @@ int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, 
         return LLMCAD_OK;
     }
     CUDA_TRY(launch_gemm_simt(w, x, ctx->cfg.dtype, n_in, ep, status, st));
+    return LLMCAD_OK;
+}
+
+int llmcad_set_kernel_timing(llmcad_ctx *ctx, int32_t enable)
+{
+    if (ctx == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    ctx->timing = enable != 0;
+    return LLMCAD_OK;
+}
+
+int llmcad_get_kernel_timing(llmcad_ctx *ctx, int32_t kind, double *total_ms, int64_t *n_launches)
+{
+    if (ctx == nullptr || total_ms == nullptr || n_launches == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    double ms = 0.0;
+    int64_t cnt = 0;
+    std::vector<llmcad_ctx::Timed> rest;
+    for (auto &t : ctx->timed) {
+        if (t.kind != kind) { rest.push_back(t); continue; }
+        CUDA_TRY(cudaEventSynchronize(t.b));
+        float f = 0.f;
+        CUDA_TRY(cudaEventElapsedTime(&f, t.a, t.b));
+        ms += f;
+        ++cnt;
+        ctx->event_pool.push_back(t.a);
+        ctx->event_pool.push_back(t.b);
+    }
+    ctx->timed.swap(rest);
+    *total_ms = ms;
+    *n_launches = cnt;
     return LLMCAD_OK;
 }
 
