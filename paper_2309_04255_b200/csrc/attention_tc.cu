@@ -3,15 +3,21 @@
 // Per head the keys are the prefix slots 0..P-1 (visible to every node) followed by the tree
 // nodes at slots P..P+n-1, of which node i sees the ones whose bit is set in its ancestor-or-self
 // row (the mask table of Sec. 3.2 "Tree decoder"). The prefix K/V bytes dominate, and a layer has
-// few heads, so the key range of each head is split over several CTAs (grid = splits x heads,
-// sized to about two CTAs per SM): each CTA streams its key range once through a cp.async
-// double buffer in shared memory, keeps an online softmax per query row, and writes an
-// unnormalised partial (max, sum, output); the CTA that finishes a head last (an atomic ticket,
-// nobody waits) merges the partials and writes the bf16 output.
+// few heads, so the key range of each head is split over the CTAs of one thread-block cluster
+// (grid = splits x heads, cluster = the splits of a head, about one CTA per SM in total): each
+// CTA streams its key range once through a four-stage cp.async ring in shared memory, keeps an
+// online softmax per query row and leaves an unnormalised partial (max, sum, output) in its own
+// shared memory; after a cluster barrier every CTA merges a share of the query rows by reading
+// the partials of its peers through distributed shared memory and writes the bf16 output. No
+// global workspace, no atomics.
 //
 // Inside a CTA warp w owns query rows 16w..16w+15 (n <= 128 nodes -> at most 8 warps busy);
 // QK^T and PV are mma.sync m16n8k16 bf16 with fp32 accumulation, scores never leave registers.
+#include <cooperative_groups.h>
+
 #include "attention_tc.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace llmcad {
 
@@ -22,7 +28,8 @@ constexpr int kKeyTile = 64;
 constexpr int kAtThreads = 256;
 constexpr int kRowBytes = kHd * 2;            // 256-byte rows = 16 chunks of 16 bytes
 constexpr int kWsRow = kHd + 2;               // partial row: 128 outputs, max, sum
-constexpr int kMaxSplits = 16;
+constexpr int kMaxSplits = 8;                 // portable cluster size
+constexpr int kStages = 4;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -65,15 +72,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 __global__ void __launch_bounds__(kAtThreads)
 attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
                     const __nv_bfloat16 *__restrict__ v, int n_heads, int kv_stride, int P, int n, int n_pad,
-                    const uint32_t *__restrict__ anc, __nv_bfloat16 *o, float *ws, uint32_t *counters, int splits,
-                    int tiles_per_split, const int32_t *status)
+                    const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
+                    const int32_t *status)
 {
-    if (*status) return;
+    if (*status) return;   // uniform over the grid: set only by kernels that ran before this one
     extern __shared__ __align__(128) uint8_t sm[];
     uint8_t *s_q = sm;                                      // [n_pad][256 B]
-    uint8_t *s_k = s_q + (size_t)n_pad * kRowBytes;         // [2][64][256 B]
-    uint8_t *s_v = s_k + 2 * kKeyTile * kRowBytes;          // [2][64][256 B]
-    __shared__ int s_last;
+    uint8_t *s_k = s_q + (size_t)n_pad * kRowBytes;         // [kStages][64][256 B]
+    uint8_t *s_v = s_k + kStages * kKeyTile * kRowBytes;    // [kStages][64][256 B]
 
     const int split = blockIdx.x, head = blockIdx.y;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -103,8 +109,10 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         const bool ok = r < n;
         cp_async16(smem_u32(s_q) + swz(r, ch), q + ((size_t)(ok ? r : 0) * n_heads + head) * kHd + ch * 8, ok);
     }
-    if (t_begin < t_end) load_tile(t_begin, 0);
-    cp_commit();
+    for (int st = 0; st < kStages - 1; ++st) {
+        if (t_begin + st < t_end) load_tile(t_begin + st, st);
+        cp_commit();                            // group 0 also carries the queries
+    }
 
     const int q_tiles = n_pad >> 4;
     const bool active = warp < q_tiles;
@@ -125,10 +133,10 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
     for (int t = t_begin; t < t_end; ++t) {
-        const int buf = (t - t_begin) & 1;
-        cp_wait<0>();
-        __syncthreads();                       // tile t (and Q) visible; everyone is done with the other buffer
-        if (t + 1 < t_end) load_tile(t + 1, buf ^ 1);
+        const int buf = (t - t_begin) % kStages;
+        cp_wait<kStages - 2>();
+        __syncthreads();                       // tile t (and Q) visible; everyone is done with tile t-1's buffer
+        if (t + kStages - 1 < t_end) load_tile(t + kStages - 1, (t + kStages - 1 - t_begin) % kStages);
         cp_commit();
         if (t == t_begin && active) {
 #pragma unroll
@@ -230,82 +238,103 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         return;
     }
 
-    // ---- partial result of this split
-    float *wsp = ws + ((size_t)head * splits + split) * n_pad * kWsRow;
+    // ---- partial result of this split, left in this CTA's shared memory (the K/V ring is done)
+    __syncthreads();
+    float *part = reinterpret_cast<float *>(sm);            // [n_pad][kWsRow]
     if (active) {
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
             const int dim = j * 8 + ((lane & 3) << 1);
-            *reinterpret_cast<float2 *>(wsp + (size_t)row0 * kWsRow + dim) = make_float2(oacc[j][0], oacc[j][1]);
-            *reinterpret_cast<float2 *>(wsp + (size_t)row1 * kWsRow + dim) = make_float2(oacc[j][2], oacc[j][3]);
+            *reinterpret_cast<float2 *>(part + (size_t)row0 * kWsRow + dim) = make_float2(oacc[j][0], oacc[j][1]);
+            *reinterpret_cast<float2 *>(part + (size_t)row1 * kWsRow + dim) = make_float2(oacc[j][2], oacc[j][3]);
         }
         if ((lane & 3) == 0) {
-            *reinterpret_cast<float2 *>(wsp + (size_t)row0 * kWsRow + kHd) = make_float2(m0, l0);
-            *reinterpret_cast<float2 *>(wsp + (size_t)row1 * kWsRow + kHd) = make_float2(m1, l1);
+            *reinterpret_cast<float2 *>(part + (size_t)row0 * kWsRow + kHd) = make_float2(m0, l0);
+            *reinterpret_cast<float2 *>(part + (size_t)row1 * kWsRow + kHd) = make_float2(m1, l1);
         }
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const uint32_t ticket = atomicAdd(counters + head, 1u);
-        s_last = (ticket == (uint32_t)splits - 1);
-        if (s_last) counters[head] = 0;   // ready for the next launch (stream order separates them)
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    // ---- merge: out[row] = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M)
-    const float *wh = ws + (size_t)head * splits * n_pad * kWsRow;
-    for (int idx = tid; idx < n * (kHd / 2); idx += kAtThreads) {
-        const int row = idx / (kHd / 2), dim = (idx % (kHd / 2)) * 2;
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.sync();                                          // all partials of this head are written
+    // ---- merge rows split, split + splits, ...: out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M)
+    const float *peer[kMaxSplits];
+#pragma unroll
+    for (int sp = 0; sp < kMaxSplits; ++sp) peer[sp] = sp < splits ? cluster.map_shared_rank(part, sp) : part;
+    const int my_rows = (n - split + splits - 1) / splits;   // rows split, split+splits, ... below n
+    for (int idx = tid; idx < my_rows * (kHd / 2); idx += kAtThreads) {
+        const int row = split + (idx / (kHd / 2)) * splits, dim = (idx % (kHd / 2)) * 2;
+        float2 ml[kMaxSplits], ov[kMaxSplits];
+#pragma unroll
+        for (int sp = 0; sp < kMaxSplits; ++sp) {
+            if (sp < splits) {
+                ml[sp] = *reinterpret_cast<const float2 *>(peer[sp] + (size_t)row * kWsRow + kHd);
+                ov[sp] = *reinterpret_cast<const float2 *>(peer[sp] + (size_t)row * kWsRow + dim);
+            } else {
+                ml[sp] = make_float2(-INFINITY, 0.f);
+                ov[sp] = make_float2(0.f, 0.f);
+            }
+        }
         float M = -INFINITY;
-        for (int sp = 0; sp < splits; ++sp) M = fmaxf(M, __ldcg(wh + ((size_t)sp * n_pad + row) * kWsRow + kHd));
+#pragma unroll
+        for (int sp = 0; sp < kMaxSplits; ++sp) M = fmaxf(M, ml[sp].x);
         float L = 0.f, a0 = 0.f, a1 = 0.f;
-        for (int sp = 0; sp < splits; ++sp) {
-            const float *r = wh + ((size_t)sp * n_pad + row) * kWsRow;
-            const float2 ml = __ldcg(reinterpret_cast<const float2 *>(r + kHd));
-            if (ml.x == -INFINITY) continue;
-            const float w = exp2f(ml.x - M);
-            const float2 ov = __ldcg(reinterpret_cast<const float2 *>(r + dim));
-            L += ml.y * w; a0 += ov.x * w; a1 += ov.y * w;
+#pragma unroll
+        for (int sp = 0; sp < kMaxSplits; ++sp) {
+            const float wgt = (ml[sp].x == -INFINITY) ? 0.f : exp2f(ml[sp].x - M);
+            L += ml[sp].y * wgt; a0 += ov[sp].x * wgt; a1 += ov[sp].y * wgt;
         }
         const float inv = L > 0.f ? 1.f / L : 0.f;
         *reinterpret_cast<uint32_t *>(o + ((size_t)row * n_heads + head) * kHd + dim) = pack_bf16(a0 * inv, a1 * inv);
     }
+    cluster.sync();                                          // peers may still be reading this CTA's partial
 }
 
 size_t attention_tc_workspace_bytes(int n_heads, int n_sms)
 {
-    (void)n_sms;
-    return (size_t)n_heads * kMaxSplits * LLMCAD_MAX_TREE * kWsRow * sizeof(float);
+    (void)n_heads; (void)n_sms;
+    return 256;   // the merge runs through distributed shared memory; no global workspace is needed
 }
 
 cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, float *ws, uint32_t *counters, int n_sms,
                                 int32_t *status, cudaStream_t st, int *launched)
 {
+    (void)ws; (void)counters;
     if (hd != kHd) return cudaErrorInvalidValue;
     const int n_pad = (n + 15) / 16 * 16;
     const int n_tiles = (P + n + kKeyTile - 1) / kKeyTile;
-    int splits = (2 * n_sms + n_heads - 1) / n_heads;
+    // one CTA per SM is resident (register file): aim for a single wave of heads x splits CTAs
+    int splits = n_sms / n_heads;
     if (splits > kMaxSplits) splits = kMaxSplits;
     if (splits > n_tiles) splits = n_tiles;
     if (splits < 1) splits = 1;
     const int tiles_per_split = (n_tiles + splits - 1) / splits;
     splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
-    const size_t smem = (size_t)n_pad * kRowBytes + 4 * kKeyTile * kRowBytes;
+    const size_t ring = (size_t)n_pad * kRowBytes + 2 * kStages * kKeyTile * kRowBytes;
+    const size_t part = (size_t)n_pad * kWsRow * sizeof(float);
+    const size_t smem = ring > part ? ring : part;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * kRowBytes + 4 * kKeyTile * kRowBytes);
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             128 * kRowBytes + 2 * kStages * kKeyTile * kRowBytes);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    dim3 grid(splits, n_heads);
-    attention_tc_kernel<<<grid, kAtThreads, smem, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
-                                                       (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc,
-                                                       (__nv_bfloat16 *)o, ws, counters, splits, tiles_per_split, status);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(splits, n_heads);
+    cfg.blockDim = dim3(kAtThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = splits;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (launched) *launched = 1;
-    return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, attention_tc_kernel, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
+                              (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc, (__nv_bfloat16 *)o, splits,
+                              tiles_per_split, status);
 }
 
 }  // namespace llmcad

@@ -61,7 +61,7 @@ __device__ __forceinline__ void epilogue_pair(const EpiParams &ep, int r0, int i
         if (has1) ep.x[(size_t)i * ep.n_out + r0 + 1] += v1;
         break;
     case EPI_SWIGLU: {
-        float s = v0 / (1.0f + __expf(-v0));
+        float s = v0 / (1.0f + expf(-v0));
         reinterpret_cast<T *>(ep.h)[(size_t)i * ep.n_out + r0] = from_f32<T>(s * v1);
         break;
     }

@@ -341,21 +341,49 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
                         for (int j = 0; j < 16; ++j) w[j] += __ldcg(src + (size_t)j * kTileM);
                     }
                 }
-                // fused epilogue on complete sums
+                // fused epilogue on complete sums; all loads of a 16-column chunk are issued before
+                // any dependent store so that they overlap instead of queueing behind each other
                 if (ep.mode == EPI_SWIGLU) {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (row_ok && c0 + j < ep.n) epilogue_pair<T>(ep, row, c0 + j, v[j], w[j], true);
-                } else if (ep.mode == EPI_QKV) {
+                    T *hrow = reinterpret_cast<T *>(ep.h) + row;
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
-                        if (!(lane & 1) && row_ok && c0 + j < ep.n) epilogue_pair<T>(ep, row, c0 + j, v[j], other, row + 1 < ep.n_out);
+                        if (row_ok && c0 + j < ep.n) {
+                            const float sg = v[j] / (1.0f + __expf(-v[j]));
+                            hrow[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(sg * w[j]);
+                        }
                     }
-                } else {
+                } else if (ep.mode == EPI_QKV) {
+                    const int sec = row / ep.d, cidx = row - sec * ep.d;
+                    const int head = cidx / ep.hd, e = cidx - head * ep.hd;
+                    float2 cs[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (row_ok && c0 + j < ep.n) epilogue_pair<T>(ep, row, c0 + j, v[j], 0.f, false);
+                        cs[j] = (sec < 2 && row_ok && c0 + j < ep.n) ? __ldg(ep.rope_cs + (size_t)(c0 + j) * (ep.hd >> 1) + (e >> 1))
+                                                                      : make_float2(1.f, 0.f);
+                    T *dst;
+                    size_t node_stride;
+                    if (sec == 0) { dst = reinterpret_cast<T *>(ep.q_out) + cidx; node_stride = ep.d; }
+                    else { dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P) * ep.hd + e; node_stride = ep.hd; }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        // the rotary partner (2t <-> 2t+1) lives in the neighbouring lane
+                        const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
+                        const float rot = (lane & 1) ? (other * cs[j].y + v[j] * cs[j].x) : (v[j] * cs[j].x - other * cs[j].y);
+                        if (row_ok && c0 + j < ep.n) dst[(size_t)(c0 + j) * node_stride] = from_f32<T>(rot);
+                    }
+                } else if (ep.mode == EPI_RESID) {
+                    float *xr = ep.x + row;
+                    float xo[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) xo[j] = (row_ok && c0 + j < ep.n) ? __ldcg(xr + (size_t)(c0 + j) * ep.n_out) : 0.f;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (row_ok && c0 + j < ep.n) xr[(size_t)(c0 + j) * ep.n_out] = xo[j] + v[j];
+                } else {
+                    float *yr = ep.y + row;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (row_ok && c0 + j < ep.n) yr[(size_t)(c0 + j) * ep.ldy] = v[j];
                 }
             }
             // accumulator buffer drained: hand it back to the MMA warp

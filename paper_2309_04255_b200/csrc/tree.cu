@@ -77,41 +77,93 @@ cudaError_t launch_embed(const void *E, int dtype, const int32_t *tokens, int n,
 }
 
 // ------------------------------------------------------------------------------------------
-// RMSNorm of the fp32 residual stream into the GEMM input dtype.
+// RMSNorm of the fp32 residual stream into the GEMM input dtype. One block per node; the row is
+// read once with 16-byte loads and kept in registers between the reduction and the scaling
+// (rows longer than 4 * kNormVec * blockDim fall back to re-reading).
+constexpr int kNormThreads = 512;
+constexpr int kNormVec = 4;   // float4 per thread held in registers -> d <= 8192
+
+template <typename T> __device__ __forceinline__ void store4(T *p, float a, float b, float c, float d);
+template <> __device__ __forceinline__ void store4<float>(float *p, float a, float b, float c, float d)
+{
+    *reinterpret_cast<float4 *>(p) = make_float4(a, b, c, d);
+}
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16 *p, float a, float b, float c, float d)
+{
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t *>(&lo);
+    u.y = *reinterpret_cast<uint32_t *>(&hi);
+    *reinterpret_cast<uint2 *>(p) = u;
+}
+
 template <typename T>
-__global__ void rmsnorm_kernel(const float *__restrict__ x, const T *__restrict__ g, int d, float eps, T *out,
-                               const int32_t *status)
+__global__ void __launch_bounds__(kNormThreads)
+rmsnorm_kernel(const float *__restrict__ x, const T *__restrict__ g, int d, float eps, T *__restrict__ out,
+               const int32_t *status)
 {
     if (*status) return;
-    __shared__ float red[32];
-    const int i = blockIdx.x;
-    const float *xi = x + (size_t)i * d;
+    __shared__ float red[kNormThreads / 32];
+    const int i = blockIdx.x, tid = threadIdx.x;
+    const float4 *xi = reinterpret_cast<const float4 *>(x + (size_t)i * d);
+    const int nv = d >> 2;                      // d is a multiple of 8
+    float4 r[kNormVec];
     float ss = 0.f;
-    for (int k = threadIdx.x; k < d; k += blockDim.x) ss += xi[k] * xi[k];
-    for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
-        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (threadIdx.x == 0) red[0] = v;
+#pragma unroll
+    for (int u = 0; u < kNormVec; ++u) {
+        const int k = tid + u * kNormThreads;
+        r[u] = k < nv ? __ldcg(xi + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+        ss += r[u].x * r[u].x + r[u].y * r[u].y + r[u].z * r[u].z + r[u].w * r[u].w;
     }
+    for (int k = tid + kNormVec * kNormThreads; k < nv; k += kNormThreads) {
+        const float4 t = __ldcg(xi + k);
+        ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+    }
+    for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((tid & 31) == 0) red[tid >> 5] = ss;
     __syncthreads();
-    const float r = rsqrtf(red[0] / d + eps);
-    for (int k = threadIdx.x; k < d; k += blockDim.x) out[(size_t)i * d + k] = from_f32<T>(xi[k] * r * to_f32<T>(g[k]));
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kNormThreads / 32; ++w) tot += red[w];
+    const float rs = rsqrtf(tot / d + eps);
+    T *oi = out + (size_t)i * d;
+#pragma unroll
+    for (int u = 0; u < kNormVec; ++u) {
+        const int k = tid + u * kNormThreads;
+        if (k < nv) {
+            const T *gk = g + 4 * k;
+            store4<T>(oi + 4 * k, r[u].x * rs * to_f32<T>(gk[0]), r[u].y * rs * to_f32<T>(gk[1]),
+                      r[u].z * rs * to_f32<T>(gk[2]), r[u].w * rs * to_f32<T>(gk[3]));
+        }
+    }
+    for (int k = tid + kNormVec * kNormThreads; k < nv; k += kNormThreads) {
+        const float4 t = __ldcg(xi + k);
+        const T *gk = g + 4 * k;
+        store4<T>(oi + 4 * k, t.x * rs * to_f32<T>(gk[0]), t.y * rs * to_f32<T>(gk[1]), t.z * rs * to_f32<T>(gk[2]),
+                  t.w * rs * to_f32<T>(gk[3]));
+    }
 }
 
 cudaError_t launch_rmsnorm(const float *x, const void *g, int dtype, int n, int d, float eps, void *out,
                            const int32_t *status, cudaStream_t st)
 {
-    if (dtype == LLMCAD_F32) rmsnorm_kernel<float><<<n, 256, 0, st>>>(x, (const float *)g, d, eps, (float *)out, status);
-    else rmsnorm_kernel<__nv_bfloat16><<<n, 256, 0, st>>>(x, (const __nv_bfloat16 *)g, d, eps, (__nv_bfloat16 *)out, status);
+    if (dtype == LLMCAD_F32) rmsnorm_kernel<float><<<n, kNormThreads, 0, st>>>(x, (const float *)g, d, eps, (float *)out, status);
+    else rmsnorm_kernel<__nv_bfloat16><<<n, kNormThreads, 0, st>>>(x, (const __nv_bfloat16 *)g, d, eps, (__nv_bfloat16 *)out, status);
     return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------
 // Greedy choice of the target at every node: lowest index of the maximum; a NaN sets status.
-__global__ void argmax_kernel(const float *__restrict__ logits, int vocab, int32_t *argmax, int32_t *status)
+constexpr int kArgmaxThreads = 1024;
+
+__device__ __forceinline__ void argmax_take(float v, int t, float &best, int &bi, bool &nan)
+{
+    nan |= (v != v);
+    if (v > best || (v == best && t < bi)) { best = v; bi = t; }
+}
+
+__global__ void __launch_bounds__(kArgmaxThreads)
+argmax_kernel(const float *__restrict__ logits, int vocab, int32_t *argmax, int32_t *status)
 {
     if (*status) return;
     __shared__ float s_v[32];
@@ -121,10 +173,17 @@ __global__ void argmax_kernel(const float *__restrict__ logits, int vocab, int32
     float best = -INFINITY;
     int bi = 0x7fffffff;
     bool nan = false;
-    for (int t = threadIdx.x; t < vocab; t += blockDim.x) {
-        const float v = row[t];
-        nan |= (v != v);
-        if (v > best || (v == best && t < bi)) { best = v; bi = t; }
+    if ((vocab & 3) == 0) {
+        const float4 *r4 = reinterpret_cast<const float4 *>(row);
+        for (int t = threadIdx.x; t < (vocab >> 2); t += kArgmaxThreads) {
+            const float4 q = __ldcg(r4 + t);
+            argmax_take(q.x, 4 * t, best, bi, nan);
+            argmax_take(q.y, 4 * t + 1, best, bi, nan);
+            argmax_take(q.z, 4 * t + 2, best, bi, nan);
+            argmax_take(q.w, 4 * t + 3, best, bi, nan);
+        }
+    } else {
+        for (int t = threadIdx.x; t < vocab; t += kArgmaxThreads) argmax_take(row[t], t, best, bi, nan);
     }
     if (nan) atomicCAS(status, 0, LLMCAD_ERR_NAN);
     for (int o = 16; o; o >>= 1) {
@@ -135,9 +194,8 @@ __global__ void argmax_kernel(const float *__restrict__ logits, int vocab, int32
     if ((threadIdx.x & 31) == 0) { s_v[threadIdx.x >> 5] = best; s_i[threadIdx.x >> 5] = bi; }
     __syncthreads();
     if (threadIdx.x < 32) {
-        const int nw = blockDim.x >> 5;
-        best = threadIdx.x < nw ? s_v[threadIdx.x] : -INFINITY;
-        bi = threadIdx.x < nw ? s_i[threadIdx.x] : 0x7fffffff;
+        best = s_v[threadIdx.x];
+        bi = s_i[threadIdx.x];
         for (int o = 16; o; o >>= 1) {
             const float ov = __shfl_xor_sync(0xffffffffu, best, o);
             const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
@@ -149,7 +207,7 @@ __global__ void argmax_kernel(const float *__restrict__ logits, int vocab, int32
 
 cudaError_t launch_argmax(const float *logits, int n, int vocab, int32_t *argmax, int32_t *status, cudaStream_t st)
 {
-    argmax_kernel<<<n, 256, 0, st>>>(logits, vocab, argmax, status);
+    argmax_kernel<<<n, kArgmaxThreads, 0, st>>>(logits, vocab, argmax, status);
     return cudaGetLastError();
 }
 
