@@ -219,6 +219,13 @@ int llmcad_last_status(llmcad_ctx *ctx, void *stream);
 int llmcad_set_kernel_timing(llmcad_ctx *ctx, int32_t enable);
 int llmcad_get_kernel_timing(llmcad_ctx *ctx, int32_t kind, double *total_ms /*HOST*/, int64_t *n_launches /*HOST*/);
 
+/* Tracing aid: while `trace` (DEVICE, [number of SMs][16] uint64, or NULL to stop) is set, every
+ * CTA of every tensor-core GEMM launch writes nanosecond timestamps of its phases there (entry,
+ * set-up done, weight prefetch issued, grid dependency resolved, last load issued, first tile
+ * landed, last MMA issued, accumulator ready, partial tiles ready, epilogue done, exit). The
+ * buffer holds the most recent launch. */
+int llmcad_set_gemm_trace(llmcad_ctx *ctx, uint64_t *trace);
+
 /* Number of kernels this library has launched through this context so far. */
 int64_t llmcad_launch_count(const llmcad_ctx *ctx);
 

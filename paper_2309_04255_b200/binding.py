@@ -29,7 +29,7 @@ EXPORTS = [
     "llmcad_kv_cache_bytes", "llmcad_packed_weight_bytes", "llmcad_pack_layer", "llmcad_pack_globals",
     "llmcad_verify_tree", "llmcad_verify_tree_host", "llmcad_prefill", "llmcad_tree_prep",
     "llmcad_accept_compact", "llmcad_tree_attention", "llmcad_skinny_gemm", "llmcad_launch_count",
-    "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing",
+    "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace",
 ]
 
 
@@ -96,6 +96,7 @@ def lib():
         L.llmcad_launch_count.argtypes = [vp]
         L.llmcad_launch_count.restype = C.c_int64
         L.llmcad_last_status.argtypes = [vp, vp]
+        L.llmcad_set_gemm_trace.argtypes = [vp, vp]
         L.llmcad_set_kernel_timing.argtypes = [vp, i32]
         L.llmcad_get_kernel_timing.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         _lib = L
@@ -234,6 +235,10 @@ class Verifier:
 
     def last_status(self) -> int:
         return lib().llmcad_last_status(self.ctx, _stream())
+
+    def set_gemm_trace(self, buf: Optional[torch.Tensor]):
+        """buf: int64 cuda tensor [n_sms][16] or None."""
+        _check(lib().llmcad_set_gemm_trace(self.ctx, _ptr(buf)), "llmcad_set_gemm_trace")
 
     def set_kernel_timing(self, on: bool):
         _check(lib().llmcad_set_kernel_timing(self.ctx, 1 if on else 0), "llmcad_set_kernel_timing")

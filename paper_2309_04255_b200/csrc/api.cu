@@ -91,10 +91,12 @@ struct llmcad_ctx {
     int32_t *ibuf = nullptr;  // tokens[128], parent[128], argmax[128], path[128], scalars[8], chain[128]
     float *partials = nullptr;
     uint32_t *flags = nullptr;
+    float *ssq[2] = {nullptr, nullptr};   // partial sums of squares for the folded attention / FFN norms
     float *attn_ws = nullptr;
     uint32_t *attn_counters = nullptr;
     uint32_t epoch = 0;
     int64_t launches = 0;
+    unsigned long long *trace = nullptr;   // optional GEMM timeline buffer (llmcad_set_gemm_trace)
     // tensor maps
     const void *maps_for = nullptr;
     std::vector<CUtensorMap> w_maps;   // [L][4] (qkv, o, gate/up, down) + lm_head
@@ -201,7 +203,7 @@ int run_gemm(llmcad_ctx *ctx, const void *packed, int l, int which, int act, int
         const size_t mi = l < 0 ? (size_t)ctx->cfg.n_layers * 4 : (size_t)l * 4 + which;
         ctx->epoch++;
         CUDA_TRY(launch_gemm_tc(ctx->w_maps[mi], ctx->act_maps[n_pad / 16][act], n_in, n_pad, ctx->n_sms, ctx->partials,
-                                ctx->flags, ctx->epoch, status, ep, st));
+                                ctx->flags, ctx->epoch, status, ep, st, ctx->trace));
         return LLMCAD_OK;
     }
     const void *W;
@@ -246,10 +248,56 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
     if ((rc = ensure_act_maps(ctx, n_pad)) != LLMCAD_OK) return rc;
 
     CUDA_TRY(launch_tree_prep(parent, tokens, n, P, c.vocab, hd, c.rope_base, ctx->tb, status, st));
-    CUDA_TRY(launch_embed(base + ctx->lay.tok_embed, c.dtype, tokens, n, d, ctx->x, status, st));
     ctx->launches += 2;
-
     const size_t kv_layer = (size_t)2 * H * S * hd * ctx->elem;
+
+    if (ctx->tc_gemm) {
+        // Tensor-core path: the RMSNorms are folded into the GEMMs. Whoever produces the residual
+        // stream (the embedding gather, the O and down GEMMs) also writes gain * x in bf16 and
+        // partial sums of squares; the consuming GEMM scales its accumulators by the per-node
+        // rsqrt(mean(x^2) + eps). Five kernels per layer.
+        const int tiles4 = 4 * ((d + 127) / 128);
+        CUDA_TRY(launch_embed_norm(base + ctx->lay.tok_embed, tokens, n, d,
+                                   c.n_layers > 0 ? base + ctx->lay.attn_norm : base + ctx->lay.final_norm, ctx->x, ctx->xn,
+                                   ctx->ssq[0], status, st));
+        int parts0 = 1;   // how many partials the next attention-norm consumer must add up
+        for (int l = 0; l < c.n_layers; ++l) {
+            const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
+            const char *next_attn_gain = (l + 1 < c.n_layers) ? lb + ctx->lay.layer_bytes + ctx->lay.attn_norm
+                                                              : base + ctx->lay.final_norm;
+            char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)l;
+            char *vl = kl + kv_layer / 2;
+            EpiParams ep{};
+            ep.n = n; ep.mode = EPI_QKV; ep.n_out = 3 * d; ep.q_out = ctx->q; ep.k_cache = kl; ep.v_cache = vl;
+            ep.rope_cs = ctx->tb.rope_cs; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P;
+            ep.ssq_in = ctx->ssq[0]; ep.ssq_in_parts = parts0; ep.norm_d = d; ep.eps = c.rms_eps;
+            if ((rc = run_gemm(ctx, packed, l, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+
+            if ((rc = run_attention(ctx, ctx->q, kl, vl, S, P, n, ctx->att, status, st)) != LLMCAD_OK) return rc;
+
+            ep = EpiParams{}; ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
+            ep.xg_out = ctx->xn; ep.gain_next = lb + ctx->lay.ffn_norm; ep.ssq_out = ctx->ssq[1];
+            if ((rc = run_gemm(ctx, packed, l, 1, 1, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+
+            ep = EpiParams{}; ep.n = n; ep.mode = EPI_SWIGLU; ep.n_out = f; ep.h = ctx->h;
+            ep.ssq_in = ctx->ssq[1]; ep.ssq_in_parts = tiles4; ep.norm_d = d; ep.eps = c.rms_eps;
+            if ((rc = run_gemm(ctx, packed, l, 2, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+
+            ep = EpiParams{}; ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
+            ep.xg_out = ctx->xn; ep.gain_next = next_attn_gain; ep.ssq_out = ctx->ssq[0];
+            if ((rc = run_gemm(ctx, packed, l, 3, 2, f, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+            parts0 = tiles4;
+        }
+        if (logits != nullptr) {
+            EpiParams ep{};
+            ep.n = n; ep.mode = EPI_PLAIN; ep.n_out = c.vocab; ep.y = logits; ep.ldy = c.vocab;
+            ep.ssq_in = ctx->ssq[0]; ep.ssq_in_parts = parts0; ep.norm_d = d; ep.eps = c.rms_eps;
+            if ((rc = run_gemm(ctx, packed, -1, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+        }
+        return LLMCAD_OK;
+    }
+
+    CUDA_TRY(launch_embed(base + ctx->lay.tok_embed, c.dtype, tokens, n, d, ctx->x, status, st));
     for (int l = 0; l < c.n_layers; ++l) {
         const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
         char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)l;
@@ -371,7 +419,10 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ok = ok && alloc((void **)&ctx->tb.rope_cs, 128 * (hd / 2) * sizeof(float2));
     ok = ok && alloc((void **)&ctx->ibuf, (520 + 128) * 4);
     ok = ok && alloc((void **)&ctx->partials, gemm_tc_partial_floats(ctx->n_sms, 128) * 4);
-    ok = ok && alloc((void **)&ctx->flags, (size_t)ctx->n_sms * 4);
+    ok = ok && alloc((void **)&ctx->flags, (size_t)4096 * 4 * 4);   // ticket counters of up to 4096 tiles
+    const size_t ssq_floats = (size_t)4 * ((d + 127) / 128) * LLMCAD_MAX_TREE;
+    ok = ok && alloc((void **)&ctx->ssq[0], ssq_floats * 4);
+    ok = ok && alloc((void **)&ctx->ssq[1], ssq_floats * 4);
     ok = ok && alloc((void **)&ctx->attn_ws, attention_tc_workspace_bytes(cfg->n_heads, ctx->n_sms));
     ok = ok && alloc((void **)&ctx->attn_counters, (size_t)cfg->n_heads * 8 * 4);
     if (ok) {
@@ -391,7 +442,8 @@ void llmcad_destroy(llmcad_ctx *ctx)
 {
     if (ctx == nullptr) return;
     void *ptrs[] = {ctx->x, ctx->xn, ctx->q, ctx->att, ctx->h, ctx->logits, ctx->tb.depth, ctx->tb.pos, ctx->tb.anc,
-                    ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->flags, ctx->attn_ws, ctx->attn_counters};
+                    ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->flags, ctx->attn_ws, ctx->attn_counters, ctx->ssq[0],
+                    ctx->ssq[1]};
     for (void *p : ptrs)
         if (p != nullptr) cudaFree(p);
     for (auto &t : ctx->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
@@ -586,7 +638,8 @@ int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, 
             return LLMCAD_ERR_CUDA;
         }
         ctx->epoch++;
-        CUDA_TRY(launch_gemm_tc(mw, mx, n_in, n_pad, ctx->n_sms, ctx->partials, ctx->flags, ctx->epoch, status, ep, st));
+        CUDA_TRY(launch_gemm_tc(mw, mx, n_in, n_pad, ctx->n_sms, ctx->partials, ctx->flags, ctx->epoch, status, ep, st,
+                                ctx->trace));
         return LLMCAD_OK;
     }
     CUDA_TRY(launch_gemm_simt(w, x, ctx->cfg.dtype, n_in, ep, status, st));
@@ -619,6 +672,13 @@ int llmcad_get_kernel_timing(llmcad_ctx *ctx, int32_t kind, double *total_ms, in
     ctx->timed.swap(rest);
     *total_ms = ms;
     *n_launches = cnt;
+    return LLMCAD_OK;
+}
+
+int llmcad_set_gemm_trace(llmcad_ctx *ctx, uint64_t *trace)
+{
+    if (ctx == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    ctx->trace = reinterpret_cast<unsigned long long *>(trace);
     return LLMCAD_OK;
 }
 

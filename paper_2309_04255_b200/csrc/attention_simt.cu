@@ -14,6 +14,8 @@ __global__ void __launch_bounds__(kAttnThreads)
 attention_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, int n_heads, int hd,
                       int kv_stride, int P, int n, const uint32_t *__restrict__ anc, T *o, const int32_t *status)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (*status) return;
     extern __shared__ float smem[];
     float *s_q = smem;              // [hd]
@@ -90,16 +92,17 @@ cudaError_t launch_attention_simt(const void *q, const void *k, const void *v, i
     if (dtype == LLMCAD_F32) {
         if (smem > 48 * 1024)
             cudaFuncSetAttribute(attention_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attention_simt_kernel<float><<<grid, kAttnThreads, smem, st>>>((const float *)q, (const float *)k, (const float *)v,
-                                                                      n_heads, hd, kv_stride, P, n, anc, (float *)o, status);
+        LaunchCfg lc(grid, kAttnThreads, smem, st);
+        return cudaLaunchKernelEx(&lc.cfg, attention_simt_kernel<float>, (const float *)q, (const float *)k,
+                                  (const float *)v, n_heads, hd, kv_stride, P, n, anc, (float *)o, status);
     } else {
         if (smem > 48 * 1024)
             cudaFuncSetAttribute(attention_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attention_simt_kernel<__nv_bfloat16><<<grid, kAttnThreads, smem, st>>>(
-            (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, n_heads, hd, kv_stride, P, n, anc,
-            (__nv_bfloat16 *)o, status);
+        LaunchCfg lc(grid, kAttnThreads, smem, st);
+        return cudaLaunchKernelEx(&lc.cfg, attention_simt_kernel<__nv_bfloat16>, (const __nv_bfloat16 *)q,
+                                  (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, n_heads, hd, kv_stride, P, n, anc,
+                                  (__nv_bfloat16 *)o, status);
     }
-    return cudaGetLastError();
 }
 
 }  // namespace llmcad

@@ -75,6 +75,8 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
                     const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
                     const int32_t *status)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (*status) return;   // uniform over the grid: set only by kernels that ran before this one
     extern __shared__ __align__(128) uint8_t sm[];
     uint8_t *s_q = sm;                                      // [n_pad][256 B]
@@ -319,20 +321,9 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(splits, n_heads);
-    cfg.blockDim = dim3(kAtThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = splits;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    LaunchCfg lc(dim3(splits, n_heads), dim3(kAtThreads), smem, st, splits);
     if (launched) *launched = 1;
-    return cudaLaunchKernelEx(&cfg, attention_tc_kernel, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
+    return cudaLaunchKernelEx(&lc.cfg, attention_tc_kernel, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                               (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc, (__nv_bfloat16 *)o, splits,
                               tiles_per_split, status);
 }

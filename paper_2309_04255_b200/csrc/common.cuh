@@ -44,6 +44,16 @@ struct EpiParams {
     void *v_cache;
     const float2 *rope_cs;  // [n][hd/2] (cos, sin) of pos[i] * base^(-2t/hd)
     int d, hd, S, P;
+    // RMSNorm folded into the tensor-core GEMM. Input side (any mode): the accumulator of node i
+    // is multiplied by rsqrt(sum_t ssq_in[t][i] / norm_d + eps); the GEMM input then is gain * x.
+    const float *ssq_in;    // [ssq_in_parts][128] partial sums of squares per node, or nullptr
+    int ssq_in_parts, norm_d;
+    float eps;
+    // Output side (EPI_RESID): besides x += acc, emit gain_next * x in the activation dtype and
+    // this tile's partial sums of squares (4 per tile, one per 32 rows) for the next norm.
+    void *xg_out;           // [n][n_out] or nullptr
+    const void *gain_next;  // [n_out]
+    float *ssq_out;         // [4 * n_tiles][128]
 };
 
 // (v0, v1) are the accumulators of output rows (r0, r0+1), r0 even, of node i; for
@@ -93,6 +103,37 @@ __device__ __forceinline__ uint64_t global_timer_ns()
 }
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every device-side wait gives up after 2 s
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of the pass is launched with programmatic stream serialization: it lets its
+// successor start (launch latency, prologue, weight prefetch) while it is still running, and it
+// calls pdl_wait() before it touches anything an earlier kernel wrote or still reads.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+struct LaunchCfg {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attrs[2];
+    LaunchCfg(dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_x = 0)
+    {
+        cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = block;
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attrs[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs = 1;
+        if (cluster_x > 0) {
+            attrs[1].id = cudaLaunchAttributeClusterDimension;
+            attrs[1].val.clusterDim.x = cluster_x;
+            attrs[1].val.clusterDim.y = 1;
+            attrs[1].val.clusterDim.z = 1;
+            cfg.numAttrs = 2;
+        }
+        cfg.attrs = attrs;
+    }
+};
+
 // ---------------------------------------------------------------- launchers (host)
 struct TreeBuffers {
     int32_t *depth, *pos;
@@ -104,6 +145,8 @@ cudaError_t launch_tree_prep(const int32_t *parent, const int32_t *tokens, int n
                              float rope_base, TreeBuffers tb, int32_t *status, cudaStream_t st);
 cudaError_t launch_embed(const void *E, int dtype, const int32_t *tokens, int n, int d, float *x, const int32_t *status,
                          cudaStream_t st);
+cudaError_t launch_embed_norm(const void *E, const int32_t *tokens, int n, int d, const void *gain, float *x, void *xg,
+                              float *ssq, const int32_t *status, cudaStream_t st);
 cudaError_t launch_rmsnorm(const float *x, const void *g, int dtype, int n, int d, float eps, void *out,
                            const int32_t *status, cudaStream_t st);
 cudaError_t launch_argmax(const float *logits, int n, int vocab, int32_t *argmax, int32_t *status, cudaStream_t st);

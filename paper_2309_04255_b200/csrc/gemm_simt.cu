@@ -30,6 +30,8 @@ template <typename T>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 gemm_simt_kernel(const T *__restrict__ W, const T *__restrict__ x, int n_in, EpiParams ep, const int32_t *status)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (*status) return;
     const int lane = threadIdx.x & 31;
     const int pair = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
@@ -81,12 +83,11 @@ cudaError_t launch_gemm_simt(const void *W, const void *x, int dtype, int n_in, 
 {
     const int n_pairs = ep.mode == EPI_SWIGLU ? ep.n_out : (ep.n_out + 1) / 2;
     const int blocks = (n_pairs + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    LaunchCfg lc(blocks, kWarpsPerBlock * 32, 0, st);
     if (dtype == LLMCAD_F32)
-        gemm_simt_kernel<float><<<blocks, kWarpsPerBlock * 32, 0, st>>>((const float *)W, (const float *)x, n_in, ep, status);
-    else
-        gemm_simt_kernel<__nv_bfloat16><<<blocks, kWarpsPerBlock * 32, 0, st>>>((const __nv_bfloat16 *)W,
-                                                                               (const __nv_bfloat16 *)x, n_in, ep, status);
-    return cudaGetLastError();
+        return cudaLaunchKernelEx(&lc.cfg, gemm_simt_kernel<float>, (const float *)W, (const float *)x, n_in, ep, status);
+    return cudaLaunchKernelEx(&lc.cfg, gemm_simt_kernel<__nv_bfloat16>, (const __nv_bfloat16 *)W, (const __nv_bfloat16 *)x,
+                              n_in, ep, status);
 }
 
 }  // namespace llmcad

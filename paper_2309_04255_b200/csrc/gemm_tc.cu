@@ -6,12 +6,21 @@
 // rows per tile = the 128 TMEM lanes) and the tree nodes on the N side (padded to a multiple of
 // 16), streams W exactly once through a deep TMA -> shared-memory ring, and keeps all SMs pulling
 // by splitting the (tile, k-block) work evenly over a persistent grid (stream-K): a CTA's range
-// may start and end inside a tile; partial tiles go through an fp32 workspace and the CTA that
-// holds a tile's last k-block adds them in a fixed order and runs the fused epilogue.
+// may start and end inside a tile; the sharers of a tile leave their partial accumulators in an
+// fp32 workspace and whichever warp arrives last at the tile's ticket counter adds them in a
+// fixed (CTA) order and runs the fused epilogue, so the result does not depend on timing and
+// no CTA ever waits for another.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer,
 // warps 2..5 = epilogue (tcgen05.ld of their 32 lanes each). Accumulators are double-buffered in
 // TMEM so that the epilogue of one tile overlaps the MMAs of the next.
+//
+// The kernel is launched with programmatic stream serialization: its producer fills the whole
+// ring with weight tiles (which no kernel ever writes) while the previous kernel of the pass is
+// still running, and only the activation tiles, the workspace and the outputs wait for the grid
+// dependency. A status word left by an earlier phase is not looked at here: the GEMM then
+// works on stale but finite activations and writes only scratch (slots >= prefix_len, the
+// context's buffers), and the search/rollback kernels at the end of the pass report the error.
 //
 // Every wait (mbarrier, workspace flag) is bounded; on expiry the kernel sets the status word to
 // LLMCAD_ERR_TIMEOUT, lets every role fall out of its loop, frees TMEM and returns.
@@ -147,8 +156,7 @@ struct SharedCtl {
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
-    int status_in;
-    int contrib_arrivals;
+    float rs[LLMCAD_MAX_TREE]; // per-node rsqrt(mean(x^2) + eps) of the folded input RMSNorm
 };
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
@@ -161,6 +169,28 @@ __device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v)
 {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+
+// Walks the (tile, k-block) units of one CTA's range [u0, u1) segment by segment, last segment
+// first (see the kernel comment for why), k-blocks ascending inside a segment.
+struct UnitWalk {
+    long long u0, hi;
+    int kb_per_tile;
+    int tile, kb, kb1;
+    __device__ UnitWalk(long long u0_, long long u1_, int kbpt) : u0(u0_), hi(u1_), kb_per_tile(kbpt), tile(0), kb(0), kb1(0) {}
+    // advance to the next unit; false when the range is exhausted
+    __device__ bool next()
+    {
+        if (kb + 1 < kb1) { ++kb; return true; }
+        if (hi <= u0) return false;
+        tile = (int)((hi - 1) / kb_per_tile);
+        const long long t0 = (long long)tile * kb_per_tile;
+        const long long lo = u0 > t0 ? u0 : t0;
+        kb = (int)(lo - t0);
+        kb1 = (int)(hi - t0);
+        hi = lo;
+        return true;
+    }
+};
 
 }  // namespace
 
@@ -177,10 +207,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     const uint32_t stage_bytes = n_acc * kATileBytes + b_tile_bytes;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
 
-    // an earlier phase of the pass failed: nothing to do (one read per CTA keeps the exit uniform)
-    if (threadIdx.x == 0) ctl.status_in = *p.status;
-    __syncthreads();
-    if (ctl.status_in) return;
+    // Let the next kernel of the stream start its own prologue and weight prefetch early. This
+    // kernel in turn must not read activations, the status word or the workspace, nor write
+    // anything, before pdl_wait(): until then it only prefetches weights, which no kernel writes.
+    pdl_launch_dependents();
+#define LLMCAD_TRACE(slot) do { if (p.trace) p.trace[(size_t)blockIdx.x * 16 + (slot)] = global_timer_ns(); } while (0)
+    if (threadIdx.x == 0) LLMCAD_TRACE(0);
 
     // ---- work range of this CTA
     const long long total_units = (long long)p.n_tiles * p.kb_per_tile;
@@ -197,7 +229,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             mbar_init(smem_u32(&ctl.tmem_empty[b]), 4);
         }
         ctl.abort_flag = 0;
-        ctl.contrib_arrivals = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -213,6 +244,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     const uint32_t tmem_base = ctl.tmem_base;
     volatile int *abort_flag = &ctl.abort_flag;
     bool timed_out = false;
+    if (threadIdx.x == 0) LLMCAD_TRACE(1);
 
     if (warp == 0) {
         // ================================================= TMA producer
@@ -220,24 +252,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             uint64_t pol_stream, pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-            uint32_t it = 0;
-            for (long long hi = u1; hi > u0 && !timed_out;) {
-                const int tile = (int)((hi - 1) / p.kb_per_tile);
-                const long long lo = max(u0, (long long)tile * p.kb_per_tile);
-                const int kb0 = (int)(lo - (long long)tile * p.kb_per_tile), kb1 = (int)(hi - (long long)tile * p.kb_per_tile);
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                    const int s = it % p.stages;
+            // Phase 1, before the grid dependency resolves: fill the ring with weight tiles only.
+            int pre = 0;
+            {
+                UnitWalk w(u0, u1, p.kb_per_tile);
+                for (; pre < p.stages && w.next(); ++pre) {
+                    const uint32_t full = smem_u32(&ctl.full[pre]);
+                    const uint32_t dst = smem_base + pre * stage_bytes;
+                    mbar_expect_tx(full, stage_bytes);
+                    tma_load_2d(dst, &tm_w, w.kb * kBlockK, w.tile * kTileM, full, pol_stream);
+                    if (p.dual) tma_load_2d(dst + kATileBytes, &tm_w, w.kb * kBlockK, p.up_row_offset + w.tile * kTileM, full, pol_stream);
+                }
+            }
+            LLMCAD_TRACE(2);
+            pdl_wait();
+            LLMCAD_TRACE(3);
+            // Phase 2: the activation tiles of the prefetched stages, then the steady state.
+            UnitWalk w(u0, u1, p.kb_per_tile);
+            for (uint32_t it = 0; w.next(); ++it) {
+                const int s = it % p.stages;
+                const uint32_t full = smem_u32(&ctl.full[s]);
+                const uint32_t dst = smem_base + s * stage_bytes;
+                if ((int)it >= pre) {
                     const uint32_t par = ((it / p.stages) & 1u) ^ 1u;
                     if (!mbar_wait(smem_u32(&ctl.empty[s]), par, abort_flag)) { timed_out = true; break; }
-                    const uint32_t full = smem_u32(&ctl.full[s]);
-                    const uint32_t dst = smem_base + s * stage_bytes;
                     mbar_expect_tx(full, stage_bytes);
-                    tma_load_2d(dst, &tm_w, kb * kBlockK, tile * kTileM, full, pol_stream);
-                    if (p.dual) tma_load_2d(dst + kATileBytes, &tm_w, kb * kBlockK, p.up_row_offset + tile * kTileM, full, pol_stream);
-                    tma_load_2d(dst + n_acc * kATileBytes, &tm_x, kb * kBlockK, 0, full, pol_keep);
+                    tma_load_2d(dst, &tm_w, w.kb * kBlockK, w.tile * kTileM, full, pol_stream);
+                    if (p.dual) tma_load_2d(dst + kATileBytes, &tm_w, w.kb * kBlockK, p.up_row_offset + w.tile * kTileM, full, pol_stream);
                 }
-                hi = lo;
+                tma_load_2d(dst + n_acc * kATileBytes, &tm_x, w.kb * kBlockK, 0, full, pol_keep);
             }
+            LLMCAD_TRACE(4);
         }
     } else if (warp == 1) {
         // ================================================= MMA issuer
@@ -255,6 +300,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int s = it % p.stages;
                     if (!mbar_wait(smem_u32(&ctl.full[s]), (it / p.stages) & 1u, abort_flag)) { timed_out = true; break; }
+                    if (it == 0) LLMCAD_TRACE(5);
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * stage_bytes;
                     const uint64_t a_desc = make_smem_desc(a_addr);
@@ -275,12 +321,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
                 tc_commit(smem_u32(&ctl.tmem_full[buf]));
                 hi = lo;
             }
+            LLMCAD_TRACE(6);
         }
     } else {
         // ================================================= epilogue (warps 2..5)
         const int lane_grp = warp & 3;                 // TMEM lanes 32*lane_grp .. +31 belong to this warp
         const int row_in_tile = lane_grp * 32 + lane;
+        const int et = (warp - 2) * 32 + lane;         // 0..127 among the epilogue threads
         const EpiParams &ep = p.ep;
+        pdl_wait();
+        // RMSNorm of the GEMM input folded into the epilogue: the producer of the residual stream
+        // left partial sums of squares per node; acc * rsqrt(mean(x^2) + eps) is applied to the
+        // complete sums below. Done once per CTA while the main loop is still filling the pipe.
+        if (ep.ssq_in != nullptr) {
+            float ss = 0.f;
+            for (int t = 0; t < ep.ssq_in_parts; ++t) ss += __ldcg(ep.ssq_in + (size_t)t * LLMCAD_MAX_TREE + et);
+            ctl.rs[et] = rsqrtf(ss / (float)ep.norm_d + ep.eps);
+            asm volatile("bar.sync 1, 128;" ::: "memory");   // all four epilogue warps get here unconditionally
+        }
         uint32_t seg = 0;
         for (long long hi = u1; hi > u0 && !timed_out; ++seg) {
             const int tile = (int)((hi - 1) / p.kb_per_tile);
@@ -288,124 +346,165 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             const long long lo = max(u0, tile_u0);
             const int kb0 = (int)(lo - tile_u0), kb1 = (int)(hi - tile_u0);
             const int buf = seg & 1;
-            const bool owner = (kb1 == p.kb_per_tile);
+            const bool sole = (kb0 == 0 && kb1 == p.kb_per_tile);      // this CTA holds the whole tile
             const int first_cta = (int)(tile_u0 / p.units_per_cta);
-            const int n_contrib = owner ? ((int)blockIdx.x - first_cta) : 0;   // kb0 > 0 <=> n_contrib > 0
+            const int last_cta = (int)((tile_u0 + p.kb_per_tile - 1) / p.units_per_cta);
+            const int n_parts = last_cta - first_cta + 1;
+            const size_t part_stride = (size_t)n_acc * p.n_pad * kTileM;  // floats per partial slot
 
             if (!mbar_wait(smem_u32(&ctl.tmem_full[buf]), (seg >> 1) & 1u, abort_flag)) { timed_out = true; break; }
             tc_fence_after();
-
-            // partial tiles of lower-numbered CTAs must have landed before this tile is finished
-            if (n_contrib > 0) {
-                const uint64_t t0 = global_timer_ns();
-                for (int c = first_cta; c < (int)blockIdx.x && !timed_out; ++c) {
-                    for (uint32_t spin = 0; (int32_t)(ld_acquire_u32(p.flags + c) - p.epoch) < 0; ++spin) {
-                        if ((spin & 63u) == 63u) {
-                            __nanosleep(64);
-                            if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) { timed_out = true; break; }
-                        }
-                    }
-                }
-                // the warp must stay convergent for tcgen05.ld: agree on the outcome
-                timed_out = __any_sync(0xffffffffu, timed_out);
-                if (timed_out) break;
-            }
+            if (threadIdx.x == 64) LLMCAD_TRACE(lo == u0 ? 8 : 7);   // 7: first segments, 8: the last one
 
             const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(buf * n_acc * p.n_pad);
             const int row = tile * kTileM + row_in_tile;           // output feature (weight row)
             const bool row_ok = row < ep.n_out;
-            const size_t part_stride = (size_t)n_acc * p.n_pad * kTileM;  // floats per CTA slot
+            bool finish = sole;
 
-            for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
-                float v[16], w[16];
-                tc_ld16(t_lane + c0, v);
-                if (p.dual) tc_ld16(t_lane + p.n_pad + c0, w);
-                if (!owner) {
-                    float *dst = p.partials + (size_t)blockIdx.x * part_stride + (size_t)c0 * kTileM + row_in_tile;
+            if (!sole) {
+                // A tile shared by several CTAs: every sharer leaves its partial accumulator in the
+                // workspace; the rows of a tile are independent per warp (32 rows each), so each
+                // warp takes a ticket for its own row group and the last warp to arrive adds all
+                // partials in CTA order and finishes those rows. Nobody waits for anybody.
+                // Slot 0 of a CTA holds the segment that contains its range start, slot 1 the other.
+                float *dst = p.partials + ((size_t)blockIdx.x * 2 + (lo == u0 ? 0 : 1)) * part_stride + row_in_tile;
+                for (int c0 = 0; c0 < n_acc * p.n_pad; c0 += 16) {
+                    float v[16];
+                    tc_ld16(t_lane + c0, v);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) dst[(size_t)j * kTileM] = v[j];
-                    if (p.dual) {
-                        dst += (size_t)p.n_pad * kTileM;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) dst[(size_t)j * kTileM] = w[j];
-                    }
-                    continue;
+                    for (int j = 0; j < 16; ++j) dst[(size_t)(c0 + j) * kTileM] = v[j];
                 }
-                for (int c = first_cta; c < first_cta + n_contrib; ++c) {
-                    const float *src = p.partials + (size_t)c * part_stride + (size_t)c0 * kTileM + row_in_tile;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] += __ldcg(src + (size_t)j * kTileM);
-                    if (p.dual) {
-                        src += (size_t)p.n_pad * kTileM;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) w[j] += __ldcg(src + (size_t)j * kTileM);
-                    }
-                }
-                // fused epilogue on complete sums; all loads of a 16-column chunk are issued before
-                // any dependent store so that they overlap instead of queueing behind each other
-                if (ep.mode == EPI_SWIGLU) {
-                    T *hrow = reinterpret_cast<T *>(ep.h) + row;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        if (row_ok && c0 + j < ep.n) {
-                            const float sg = v[j] / (1.0f + __expf(-v[j]));
-                            hrow[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(sg * w[j]);
-                        }
-                    }
-                } else if (ep.mode == EPI_QKV) {
-                    const int sec = row / ep.d, cidx = row - sec * ep.d;
-                    const int head = cidx / ep.hd, e = cidx - head * ep.hd;
-                    float2 cs[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        cs[j] = (sec < 2 && row_ok && c0 + j < ep.n) ? __ldg(ep.rope_cs + (size_t)(c0 + j) * (ep.hd >> 1) + (e >> 1))
-                                                                      : make_float2(1.f, 0.f);
-                    T *dst;
-                    size_t node_stride;
-                    if (sec == 0) { dst = reinterpret_cast<T *>(ep.q_out) + cidx; node_stride = ep.d; }
-                    else { dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P) * ep.hd + e; node_stride = ep.hd; }
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        // the rotary partner (2t <-> 2t+1) lives in the neighbouring lane
-                        const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
-                        const float rot = (lane & 1) ? (other * cs[j].y + v[j] * cs[j].x) : (v[j] * cs[j].x - other * cs[j].y);
-                        if (row_ok && c0 + j < ep.n) dst[(size_t)(c0 + j) * node_stride] = from_f32<T>(rot);
-                    }
-                } else if (ep.mode == EPI_RESID) {
-                    float *xr = ep.x + row;
-                    float xo[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) xo[j] = (row_ok && c0 + j < ep.n) ? __ldcg(xr + (size_t)(c0 + j) * ep.n_out) : 0.f;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (row_ok && c0 + j < ep.n) xr[(size_t)(c0 + j) * ep.n_out] = xo[j] + v[j];
-                } else {
-                    float *yr = ep.y + row;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (row_ok && c0 + j < ep.n) yr[(size_t)(c0 + j) * ep.ldy] = v[j];
-                }
-            }
-            // accumulator buffer drained: hand it back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
-            if (!owner) {
-                // publish this CTA's partial tile (a CTA has at most one such segment): the last of
-                // the four epilogue warps to get here raises the flag; nobody waits
                 __threadfence();
                 __syncwarp();
+                int last = 0;
                 if (lane == 0) {
-                    __threadfence();
-                    if (atomicAdd(&ctl.contrib_arrivals, 1) == 3) {
-                        __threadfence();
-                        st_release_u32(p.flags + blockIdx.x, p.epoch);
+                    uint32_t *ctr = p.tickets + (size_t)tile * 4 + lane_grp;
+                    last = (atomicAdd(ctr, 1u) == (uint32_t)n_parts - 1u);
+                    if (last) { *ctr = 0; __threadfence(); }
+                }
+                finish = __shfl_sync(0xffffffffu, last, 0) != 0;
+                // the accumulator is in the workspace now: hand the TMEM buffer back early
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+                if (threadIdx.x == 64) LLMCAD_TRACE(9);
+            }
+
+            if (finish) {
+                float gain = 0.f;
+                if (ep.mode == EPI_RESID && ep.xg_out != nullptr && row_ok)
+                    gain = to_f32<T>(reinterpret_cast<const T *>(ep.gain_next)[row]);
+                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                    float v[16], w[16];
+                    if (sole) {
+                        tc_ld16(t_lane + c0, v);
+                        if (p.dual) tc_ld16(t_lane + p.n_pad + c0, w);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] = w[j] = 0.f;
+                        // partial tiles in CTA order, two CTAs' loads in flight at a time
+                        for (int c = first_cta; c <= last_cta; c += 2) {
+                            const bool two = c + 1 <= last_cta;
+                            const int slot0 = ((long long)c * p.units_per_cta >= tile_u0) ? 0 : 1;
+                            const int slot1 = ((long long)(c + 1) * p.units_per_cta >= tile_u0) ? 0 : 1;
+                            const float *s0 = p.partials + ((size_t)c * 2 + slot0) * part_stride + (size_t)c0 * kTileM + row_in_tile;
+                            const float *s1 = two ? p.partials + ((size_t)(c + 1) * 2 + slot1) * part_stride + (size_t)c0 * kTileM + row_in_tile : s0;
+                            float a0[16], a1[16];
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) { a0[j] = __ldcg(s0 + (size_t)j * kTileM); a1[j] = __ldcg(s1 + (size_t)j * kTileM); }
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) { v[j] += a0[j]; if (two) v[j] += a1[j]; }
+                            if (p.dual) {
+                                s0 += (size_t)p.n_pad * kTileM;
+                                s1 += (size_t)p.n_pad * kTileM;
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) { a0[j] = __ldcg(s0 + (size_t)j * kTileM); a1[j] = __ldcg(s1 + (size_t)j * kTileM); }
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) { w[j] += a0[j]; if (two) w[j] += a1[j]; }
+                            }
+                        }
+                    }
+                    if (ep.ssq_in != nullptr) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) { const float r = ctl.rs[c0 + j]; v[j] *= r; w[j] *= r; }
+                    }
+                    // fused epilogue on complete sums; all loads of a 16-column chunk are issued before
+                    // any dependent store so that they overlap instead of queueing behind each other
+                    if (ep.mode == EPI_SWIGLU) {
+                        T *hrow = reinterpret_cast<T *>(ep.h) + row;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            if (row_ok && c0 + j < ep.n) {
+                                const float sg = v[j] / (1.0f + __expf(-v[j]));
+                                hrow[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(sg * w[j]);
+                            }
+                        }
+                    } else if (ep.mode == EPI_QKV) {
+                        const int sec = row / ep.d, cidx = row - sec * ep.d;
+                        const int head = cidx / ep.hd, e = cidx - head * ep.hd;
+                        float2 cs[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            cs[j] = (sec < 2 && row_ok && c0 + j < ep.n) ? __ldg(ep.rope_cs + (size_t)(c0 + j) * (ep.hd >> 1) + (e >> 1))
+                                                                          : make_float2(1.f, 0.f);
+                        T *dst;
+                        size_t node_stride;
+                        if (sec == 0) { dst = reinterpret_cast<T *>(ep.q_out) + cidx; node_stride = ep.d; }
+                        else { dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P) * ep.hd + e; node_stride = ep.hd; }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            // the rotary partner (2t <-> 2t+1) lives in the neighbouring lane
+                            const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
+                            const float rot = (lane & 1) ? (other * cs[j].y + v[j] * cs[j].x) : (v[j] * cs[j].x - other * cs[j].y);
+                            if (row_ok && c0 + j < ep.n) dst[(size_t)(c0 + j) * node_stride] = from_f32<T>(rot);
+                        }
+                    } else if (ep.mode == EPI_RESID) {
+                        float *xr = ep.x + row;
+                        float xo[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) xo[j] = (row_ok && c0 + j < ep.n) ? __ldcg(xr + (size_t)(c0 + j) * ep.n_out) : 0.f;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            xo[j] = (row_ok && c0 + j < ep.n) ? xo[j] + v[j] : 0.f;
+                            if (row_ok && c0 + j < ep.n) xr[(size_t)(c0 + j) * ep.n_out] = xo[j];
+                        }
+                        if (ep.xg_out != nullptr) {
+                            // what the next RMSNorm needs: gain * x in the GEMM input dtype, and this
+                            // warp's share (32 rows) of every node's sum of squares
+                            T *gr = reinterpret_cast<T *>(ep.xg_out) + row;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (row_ok && c0 + j < ep.n) gr[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(xo[j] * gain);
+                            float mine = 0.f;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                float sq = xo[j] * xo[j];
+#pragma unroll
+                                for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                                if (lane == j) mine = sq;
+                            }
+                            if (lane < 16)
+                                ep.ssq_out[(size_t)(tile * 4 + lane_grp) * LLMCAD_MAX_TREE + c0 + lane] = mine;
+                        }
+                    } else {
+                        float *yr = ep.y + row;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (row_ok && c0 + j < ep.n) yr[(size_t)(c0 + j) * ep.ldy] = v[j];
                     }
                 }
+            }
+            if (sole) {
+                // accumulator buffer drained: hand it back to the MMA warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
             }
             hi = lo;
         }
+        if (threadIdx.x == 64) LLMCAD_TRACE(10);
     }
+    __syncwarp();   // lanes that skipped their role's single-thread section rejoin their warp here
 
     if (timed_out) {
         *abort_flag = 1;
@@ -416,6 +515,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     }
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) LLMCAD_TRACE(11);
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
     }
@@ -455,15 +555,16 @@ bool make_tensor_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uin
     return r == CUDA_SUCCESS;
 }
 
-size_t gemm_tc_partial_floats(int n_sms, int max_n_pad) { return (size_t)n_sms * 2 * max_n_pad * kTileM; }
+size_t gemm_tc_partial_floats(int n_sms, int max_n_pad) { return (size_t)n_sms * 2 /*slots*/ * 2 /*gate+up*/ * max_n_pad * kTileM; }
 
 cudaError_t launch_gemm_tc(const CUtensorMap &tm_w, const CUtensorMap &tm_x, int n_in, int n_pad, int n_sms,
                            float *partials, uint32_t *flags, uint32_t epoch, int32_t *status, const EpiParams &ep,
-                           cudaStream_t st)
+                           cudaStream_t st, unsigned long long *trace)
 {
     TcGemmParams p;
     p.dual = ep.mode == EPI_SWIGLU;
     p.n_tiles = (ep.n_out + kTileM - 1) / kTileM;
+    if (p.n_tiles > 4096) return cudaErrorInvalidValue;   // size of the ticket array
     p.kb_per_tile = (n_in + kBlockK - 1) / kBlockK;
     p.n_pad = n_pad;
     p.up_row_offset = ep.n_out;
@@ -482,9 +583,10 @@ cudaError_t launch_gemm_tc(const CUtensorMap &tm_w, const CUtensorMap &tm_x, int
     while (pow2 < cols) pow2 <<= 1;
     p.tmem_cols = pow2;
     p.partials = partials;
-    p.flags = flags;
-    p.epoch = epoch;
+    p.tickets = flags;
+    (void)epoch;
     p.status = status;
+    p.trace = trace;
     p.ep = ep;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     static bool attr_set = false;
@@ -494,8 +596,8 @@ cudaError_t launch_gemm_tc(const CUtensorMap &tm_w, const CUtensorMap &tm_x, int
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    gemm_tc_kernel<__nv_bfloat16><<<grid, kThreads, smem, st>>>(tm_w, tm_x, p);
-    return cudaGetLastError();
+    LaunchCfg lc(grid, kThreads, smem, st);
+    return cudaLaunchKernelEx(&lc.cfg, gemm_tc_kernel<__nv_bfloat16>, tm_w, tm_x, p);
 }
 
 }  // namespace llmcad

@@ -16,10 +16,10 @@ struct TcGemmParams {
     int units_per_cta;  // (tile, k-block) units per CTA of the persistent grid
     int stages;         // depth of the shared-memory ring
     int tmem_cols;      // allocated TMEM columns (power of two)
-    float *partials;    // [grid][n_acc][n_pad][128] fp32 partial tiles
-    uint32_t *flags;    // [grid] "partial of launch `epoch` is complete"
-    uint32_t epoch;
+    float *partials;    // [grid][2 slots][n_acc][n_pad][128] fp32 partial tiles
+    uint32_t *tickets;  // [n_tiles][4] arrivals per (tile, 32-row group); zero between launches
     int32_t *status;
+    unsigned long long *trace;  // optional [grid][16] timeline in ns (nullptr: off)
     EpiParams ep;
 };
 
@@ -31,6 +31,6 @@ size_t gemm_tc_partial_floats(int n_sms, int max_n_pad);
 
 cudaError_t launch_gemm_tc(const CUtensorMap &tm_w, const CUtensorMap &tm_x, int n_in, int n_pad, int n_sms,
                            float *partials, uint32_t *flags, uint32_t epoch, int32_t *status, const EpiParams &ep,
-                           cudaStream_t st);
+                           cudaStream_t st, unsigned long long *trace = nullptr);
 
 }  // namespace llmcad

@@ -15,6 +15,8 @@ __global__ void tree_prep_kernel(const int32_t *__restrict__ parent, const int32
 {
     __shared__ int s_depth;
     const int i = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     if (threadIdx.x == 0) {
         uint32_t bits[4] = {0, 0, 0, 0};
         int d = 0, cur = i, err = 0;
@@ -52,9 +54,9 @@ __global__ void tree_prep_kernel(const int32_t *__restrict__ parent, const int32
 cudaError_t launch_tree_prep(const int32_t *parent, const int32_t *tokens, int n, int P, int vocab, int hd,
                              float rope_base, TreeBuffers tb, int32_t *status, cudaStream_t st)
 {
-    tree_prep_kernel<<<n, 64, 0, st>>>(parent, tokens, n, P, vocab, hd, (double)rope_base, tb.depth, tb.pos, tb.anc,
-                                       tb.rope_cs, status);
-    return cudaGetLastError();
+    LaunchCfg lc(n, 64, 0, st);
+    return cudaLaunchKernelEx(&lc.cfg, tree_prep_kernel, parent, tokens, n, P, vocab, hd, (double)rope_base, tb.depth,
+                              tb.pos, tb.anc, tb.rope_cs, status);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -62,6 +64,8 @@ template <typename T>
 __global__ void embed_kernel(const T *__restrict__ E, const int32_t *__restrict__ tokens, int d, float *x,
                              const int32_t *status)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (*status) return;
     const int i = blockIdx.x;
     const T *row = E + (size_t)tokens[i] * d;
@@ -71,9 +75,47 @@ __global__ void embed_kernel(const T *__restrict__ E, const int32_t *__restrict_
 cudaError_t launch_embed(const void *E, int dtype, const int32_t *tokens, int n, int d, float *x, const int32_t *status,
                          cudaStream_t st)
 {
-    if (dtype == LLMCAD_F32) embed_kernel<float><<<n, 256, 0, st>>>((const float *)E, tokens, d, x, status);
-    else embed_kernel<__nv_bfloat16><<<n, 256, 0, st>>>((const __nv_bfloat16 *)E, tokens, d, x, status);
-    return cudaGetLastError();
+    LaunchCfg lc(n, 256, 0, st);
+    if (dtype == LLMCAD_F32) return cudaLaunchKernelEx(&lc.cfg, embed_kernel<float>, (const float *)E, tokens, d, x, status);
+    return cudaLaunchKernelEx(&lc.cfg, embed_kernel<__nv_bfloat16>, (const __nv_bfloat16 *)E, tokens, d, x, status);
+}
+
+// Embedding gather for the tensor-core path, where the first RMSNorm is folded into the QKV GEMM:
+// besides x it writes gain * x in the GEMM input dtype and the row's sum of squares.
+template <typename T>
+__global__ void __launch_bounds__(256)
+embed_norm_kernel(const T *__restrict__ E, const int32_t *__restrict__ tokens, int d, const T *__restrict__ gain, float *x,
+                  T *xg, float *ssq, const int32_t *status)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    if (*status) return;
+    __shared__ float red[8];
+    const int i = blockIdx.x;
+    const T *row = E + (size_t)tokens[i] * d;
+    float ss = 0.f;
+    for (int k = threadIdx.x; k < d; k += 256) {
+        const float v = to_f32<T>(row[k]);
+        x[(size_t)i * d + k] = v;
+        xg[(size_t)i * d + k] = from_f32<T>(v * to_f32<T>(gain[k]));
+        ss += v * v;
+    }
+    for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < 8; ++w) t += red[w];
+        ssq[i] = t;
+    }
+}
+
+cudaError_t launch_embed_norm(const void *E, const int32_t *tokens, int n, int d, const void *gain, float *x, void *xg,
+                              float *ssq, const int32_t *status, cudaStream_t st)
+{
+    LaunchCfg lc(n, 256, 0, st);
+    return cudaLaunchKernelEx(&lc.cfg, embed_norm_kernel<__nv_bfloat16>, (const __nv_bfloat16 *)E, tokens, d,
+                              (const __nv_bfloat16 *)gain, x, (__nv_bfloat16 *)xg, ssq, status);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -102,6 +144,8 @@ __global__ void __launch_bounds__(kNormThreads)
 rmsnorm_kernel(const float *__restrict__ x, const T *__restrict__ g, int d, float eps, T *__restrict__ out,
                const int32_t *status)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (*status) return;
     __shared__ float red[kNormThreads / 32];
     const int i = blockIdx.x, tid = threadIdx.x;
@@ -147,9 +191,11 @@ rmsnorm_kernel(const float *__restrict__ x, const T *__restrict__ g, int d, floa
 cudaError_t launch_rmsnorm(const float *x, const void *g, int dtype, int n, int d, float eps, void *out,
                            const int32_t *status, cudaStream_t st)
 {
-    if (dtype == LLMCAD_F32) rmsnorm_kernel<float><<<n, kNormThreads, 0, st>>>(x, (const float *)g, d, eps, (float *)out, status);
-    else rmsnorm_kernel<__nv_bfloat16><<<n, kNormThreads, 0, st>>>(x, (const __nv_bfloat16 *)g, d, eps, (__nv_bfloat16 *)out, status);
-    return cudaGetLastError();
+    LaunchCfg lc(n, kNormThreads, 0, st);
+    if (dtype == LLMCAD_F32)
+        return cudaLaunchKernelEx(&lc.cfg, rmsnorm_kernel<float>, x, (const float *)g, d, eps, (float *)out, status);
+    return cudaLaunchKernelEx(&lc.cfg, rmsnorm_kernel<__nv_bfloat16>, x, (const __nv_bfloat16 *)g, d, eps,
+                              (__nv_bfloat16 *)out, status);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -165,6 +211,8 @@ __device__ __forceinline__ void argmax_take(float v, int t, float &best, int &bi
 __global__ void __launch_bounds__(kArgmaxThreads)
 argmax_kernel(const float *__restrict__ logits, int vocab, int32_t *argmax, int32_t *status)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (*status) return;
     __shared__ float s_v[32];
     __shared__ int s_i[32];
@@ -207,8 +255,8 @@ argmax_kernel(const float *__restrict__ logits, int vocab, int32_t *argmax, int3
 
 cudaError_t launch_argmax(const float *logits, int n, int vocab, int32_t *argmax, int32_t *status, cudaStream_t st)
 {
-    argmax_kernel<<<n, kArgmaxThreads, 0, st>>>(logits, vocab, argmax, status);
-    return cudaGetLastError();
+    LaunchCfg lc(n, kArgmaxThreads, 0, st);
+    return cudaLaunchKernelEx(&lc.cfg, argmax_kernel, logits, vocab, argmax, status);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -224,6 +272,8 @@ __global__ void accept_kernel(const int32_t *__restrict__ parent, const int32_t 
     __shared__ int s_key[4];
     __shared__ int s_best, s_haschild;
     const int c = threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     const int status = scalars[LLMCAD_S_STATUS];
     if (status) {  // an earlier phase failed: report an empty result, leave the cache as it was
         if (c == 0) {
@@ -291,8 +341,8 @@ __global__ void accept_kernel(const int32_t *__restrict__ parent, const int32_t 
 cudaError_t launch_accept(const int32_t *parent, const int32_t *tokens, const int32_t *argmax, int n, int P,
                           int32_t *path, int32_t *scalars, cudaStream_t st)
 {
-    accept_kernel<<<1, LLMCAD_MAX_TREE, 0, st>>>(parent, tokens, argmax, n, P, path, scalars);
-    return cudaGetLastError();
+    LaunchCfg lc(1, LLMCAD_MAX_TREE, 0, st);
+    return cudaLaunchKernelEx(&lc.cfg, accept_kernel, parent, tokens, argmax, n, P, path, scalars);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -303,6 +353,8 @@ cudaError_t launch_accept(const int32_t *parent, const int32_t *tokens, const in
 __global__ void compact_kernel(uint4 *kv, int n_lkh, int S, int chunks, int P, const int32_t *__restrict__ path,
                                const int32_t *__restrict__ scalars)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (scalars[LLMCAD_S_STATUS]) return;
     const int len = scalars[LLMCAD_S_ACCEPTED_LEN];
     const long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -330,8 +382,8 @@ cudaError_t launch_compact(void *kv, int dtype, int n_layers, int n_heads, int S
     const int n_lkh = n_layers * 2 * n_heads;
     const long long total = (long long)n_lkh * chunks;
     const int block = 128;
-    compact_kernel<<<(unsigned)((total + block - 1) / block), block, 0, st>>>((uint4 *)kv, n_lkh, S, chunks, P, path, scalars);
-    return cudaGetLastError();
+    LaunchCfg lc((unsigned)((total + block - 1) / block), block, 0, st);
+    return cudaLaunchKernelEx(&lc.cfg, compact_kernel, (uint4 *)kv, n_lkh, S, chunks, P, path, scalars);
 }
 
 }  // namespace llmcad
