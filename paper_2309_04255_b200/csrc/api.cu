@@ -629,6 +629,7 @@ int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, 
     EpiParams ep{};
     ep.mode = EPI_PLAIN; ep.n = n; ep.n_out = n_out; ep.y = y; ep.ldy = n_out;
     ctx->launches++;
+    TimedLaunch tl(ctx, 0, st);
     if (ctx->tc_gemm) {
         const int n_pad = (n + 15) / 16 * 16;
         CUtensorMap mw, mx;
