@@ -285,7 +285,8 @@ def run_gpu(args, w, cfg):
         ms_per = ms / args.steps
         value = world * args.steps / (ms * 1e-3)
         gemm_avg_ms = gemm_ms / max(gemm_cnt, 1)
-        gemm_gbs = (gb / gcount) / (gemm_avg_ms * 1e-3) / 1e9
+        gb_launch = gb * args.steps / max(gemm_cnt, 1)          # a launch may chain several GEMMs
+        gemm_gbs = gb_launch / (gemm_avg_ms * 1e-3) / 1e9
         fl = flops(cfg, P, n)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -299,11 +300,11 @@ def run_gpu(args, w, cfg):
                               "frac_of_measured_hbm": ab["total"] / (ms_per * 1e-3) / 1e9 / hbm_peak,
                               "frac_of_8TBs": ab["total"] / (ms_per * 1e-3) / 8e12,
                               "tensor_frac": fl / (ms_per * 1e-3) / 1e12 / tf_peak, "peaks": peak_kind},
-            "roofline": {"kernel": "gemm_tc_kernel", "bound": "hbm", "achieved": gemm_gbs, "peak": hbm_peak,
+            "roofline": {"kernel": "gemm_chain_kernel", "bound": "hbm", "achieved": gemm_gbs, "peak": hbm_peak,
                          "unit": "GB/s", "frac": gemm_gbs / hbm_peak,
-                         "traffic": (GEMM_TRAFFIC_RATIO * gb / gcount) if GEMM_TRAFFIC_RATIO else None,
+                         "traffic": (GEMM_TRAFFIC_RATIO * gb_launch) if GEMM_TRAFFIC_RATIO else None,
                          "launches_timed": gemm_cnt, "avg_launch_ms": gemm_avg_ms,
-                         "algorithmic_bytes_per_launch": gb / gcount, "of": peak_kind,
+                         "algorithmic_bytes_per_launch": gb_launch, "of": peak_kind,
                          "ms_per_step_with_kernel_events": ms_events / args.steps,
                          "attention_ms_per_step": attn_ms / args.steps, "gemm_ms_per_step": gemm_ms / args.steps},
             "e2e": {"value": world * args.steps / (e2e_ms * 1e-3), "unit": UNIT,

@@ -142,8 +142,10 @@ size_t llmcad_packed_weight_bytes(const llmcad_config *cfg);
 
 /* One-time packing into the layout the kernels stream: per layer attn_norm,
  * [wq;wk;wv] as one [3d][d] matrix, wo, ffn_norm, [w_gate;w_up] as one [2f][d]
- * matrix, w_down; then tok_embed, final_norm, lm_head. Device-to-device copies on
- * `stream`; the sources may be freed once the stream has run them.
+ * matrix, w_down; then tok_embed, final_norm, lm_head. In bf16 contexts every matrix
+ * is stored as pre-swizzled 16 KB tiles (see llmcad_tile_weight below), in fp32
+ * contexts row-major. Device-to-device work on `stream`; the sources may be freed
+ * once the stream has run it.
  * llmcad_pack_layer packs layer `layer`; llmcad_pack_globals the three shared
  * tensors. All of them must have been called before the first pass. */
 int llmcad_pack_layer(llmcad_ctx *ctx, int32_t layer, const llmcad_layer_weights *src /*HOST struct of DEVICE ptrs*/,
@@ -219,12 +221,24 @@ int llmcad_last_status(llmcad_ctx *ctx, void *stream);
 int llmcad_set_kernel_timing(llmcad_ctx *ctx, int32_t enable);
 int llmcad_get_kernel_timing(llmcad_ctx *ctx, int32_t kind, double *total_ms /*HOST*/, int64_t *n_launches /*HOST*/);
 
-/* Tracing aid: while `trace` (DEVICE, [number of SMs][16] uint64, or NULL to stop) is set, every
- * CTA of every tensor-core GEMM launch writes nanosecond timestamps of its phases there (entry,
- * set-up done, weight prefetch issued, grid dependency resolved, last load issued, first tile
- * landed, last MMA issued, accumulator ready, partial tiles ready, epilogue done, exit). The
- * buffer holds the most recent launch. */
-int llmcad_set_gemm_trace(llmcad_ctx *ctx, uint64_t *trace);
+/* Tracing aid: while `trace` (DEVICE, [capacity][256][16] uint64, or NULL to stop) is set, the
+ * next `capacity` tensor-core GEMM and attention launches of this context each fill one
+ * [256][16] slice: per CTA, nanosecond timestamps (%globaltimer) of entry (0), set-up done (1),
+ * grid dependency resolved (3), per chained GEMM g first accumulator ready (4+2g) and epilogue
+ * done (5+2g), exit (12). */
+int llmcad_set_gemm_trace(llmcad_ctx *ctx, uint64_t *trace, int32_t capacity);
+
+/* The tensor-core path streams each weight matrix as a sequence of 16 KB tiles (128 rows x 64
+ * columns, tile-row major then k-block, 128-byte rows with the 16-byte chunk c of row r stored
+ * at position c ^ (r & 7)), so that one bulk copy moves a tile from HBM into shared memory in
+ * the form the MMA reads. llmcad_pack_layer / llmcad_pack_globals produce this layout inside the
+ * packed buffer; these two calls expose it for a single row-major bf16 matrix [n_out][n_in]
+ * (DEVICE), n_in a multiple of 8. */
+size_t llmcad_tiled_weight_bytes(int32_t n_out, int32_t n_in);
+int llmcad_tile_weight(const void *w, int32_t n_out, int32_t n_in, void *tiled /*DEVICE*/, void *stream);
+/* llmcad_skinny_gemm on a matrix in that layout (bf16 contexts only). */
+int llmcad_skinny_gemm_tiled(llmcad_ctx *ctx, const void *w_tiled, const void *x, float *y, int32_t n_out, int32_t n_in,
+                             int32_t n, void *stream);
 
 /* Number of kernels this library has launched through this context so far. */
 int64_t llmcad_launch_count(const llmcad_ctx *ctx);

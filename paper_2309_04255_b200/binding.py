@@ -29,7 +29,7 @@ EXPORTS = [
     "llmcad_kv_cache_bytes", "llmcad_packed_weight_bytes", "llmcad_pack_layer", "llmcad_pack_globals",
     "llmcad_verify_tree", "llmcad_verify_tree_host", "llmcad_prefill", "llmcad_tree_prep",
     "llmcad_accept_compact", "llmcad_tree_attention", "llmcad_skinny_gemm", "llmcad_launch_count",
-    "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace",
+    "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace", "llmcad_tiled_weight_bytes", "llmcad_tile_weight", "llmcad_skinny_gemm_tiled",
 ]
 
 
@@ -96,7 +96,11 @@ def lib():
         L.llmcad_launch_count.argtypes = [vp]
         L.llmcad_launch_count.restype = C.c_int64
         L.llmcad_last_status.argtypes = [vp, vp]
-        L.llmcad_set_gemm_trace.argtypes = [vp, vp]
+        L.llmcad_set_gemm_trace.argtypes = [vp, vp, i32]
+        L.llmcad_tiled_weight_bytes.argtypes = [i32, i32]
+        L.llmcad_tiled_weight_bytes.restype = sz
+        L.llmcad_tile_weight.argtypes = [vp, i32, i32, vp, vp]
+        L.llmcad_skinny_gemm_tiled.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
         L.llmcad_set_kernel_timing.argtypes = [vp, i32]
         L.llmcad_get_kernel_timing.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         _lib = L
@@ -233,12 +237,27 @@ class Verifier:
         _check(lib().llmcad_skinny_gemm(self.ctx, _ptr(w), _ptr(x), _ptr(y), n_out, n_in, n, _stream()), "llmcad_skinny_gemm")
         return y
 
+    def tile_weight(self, w):
+        """Row-major bf16 [n_out][n_in] -> the tiled layout the tensor-core GEMM streams."""
+        n_out, n_in = w.shape
+        t = torch.empty(lib().llmcad_tiled_weight_bytes(n_out, n_in), dtype=torch.uint8, device=self.device)
+        _check(lib().llmcad_tile_weight(_ptr(w), n_out, n_in, _ptr(t), _stream()), "llmcad_tile_weight")
+        return t
+
+    def skinny_gemm_tiled(self, w_tiled, n_out, x):
+        n, n_in = x.shape
+        y = torch.empty((n, n_out), dtype=torch.float32, device=self.device)
+        _check(lib().llmcad_skinny_gemm_tiled(self.ctx, _ptr(w_tiled), _ptr(x), _ptr(y), n_out, n_in, n, _stream()),
+               "llmcad_skinny_gemm_tiled")
+        return y
+
     def last_status(self) -> int:
         return lib().llmcad_last_status(self.ctx, _stream())
 
     def set_gemm_trace(self, buf: Optional[torch.Tensor]):
-        """buf: int64 cuda tensor [n_sms][16] or None."""
-        _check(lib().llmcad_set_gemm_trace(self.ctx, _ptr(buf)), "llmcad_set_gemm_trace")
+        """buf: int64 cuda tensor [capacity][256][16] or None."""
+        _check(lib().llmcad_set_gemm_trace(self.ctx, _ptr(buf), buf.shape[0] if buf is not None else 0),
+               "llmcad_set_gemm_trace")
 
     def set_kernel_timing(self, on: bool):
         _check(lib().llmcad_set_kernel_timing(self.ctx, 1 if on else 0), "llmcad_set_kernel_timing")

@@ -4,6 +4,7 @@
 #include <cuda.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -37,23 +38,32 @@ struct PackedLayout {
     size_t tok_embed, final_norm, lm_head, total;                   // offsets from the start of the buffer
 };
 
+// The tensor-core path streams weights as pre-swizzled 16 KB tiles (pack.cu); the plain-ALU
+// path reads them row-major.
+bool want_tiled(const llmcad_config &c)
+{
+    return c.dtype == LLMCAD_BF16 && !(c.flags & LLMCAD_FLAG_SIMT_GEMM) && c.d_model % 128 == 0;
+}
+
 PackedLayout packed_layout(const llmcad_config &c)
 {
     const size_t e = c.dtype == LLMCAD_F32 ? 4 : 2;
     const size_t d = c.d_model, f = c.d_ffn, v = c.vocab;
+    const bool tiled = want_tiled(c);
+    auto mat = [&](size_t n_out, size_t n_in) { return tiled ? tiled_weight_bytes((int)n_out, (int)n_in) : n_out * n_in * e; };
     PackedLayout L{};
     size_t o = 0;
-    L.attn_norm = o; o = align_up(o + d * e, 256);
-    L.wqkv = o;      o = align_up(o + 3 * d * d * e, 256);
-    L.wo = o;        o = align_up(o + d * d * e, 256);
-    L.ffn_norm = o;  o = align_up(o + d * e, 256);
-    L.wgu = o;       o = align_up(o + 2 * f * d * e, 256);
-    L.wdown = o;     o = align_up(o + d * f * e, 256);
+    L.attn_norm = o; o = align_up(o + d * e, 1024);
+    L.wqkv = o;      o = align_up(o + 3 * mat(d, d), 1024);
+    L.wo = o;        o = align_up(o + mat(d, d), 1024);
+    L.ffn_norm = o;  o = align_up(o + d * e, 1024);
+    L.wgu = o;       o = align_up(o + 2 * mat(f, d), 1024);
+    L.wdown = o;     o = align_up(o + mat(d, f), 1024);
     L.layer_bytes = o;
     o = L.layer_bytes * (size_t)c.n_layers;
-    L.tok_embed = o;  o = align_up(o + v * d * e, 256);
-    L.final_norm = o; o = align_up(o + d * e, 256);
-    L.lm_head = o;    o = align_up(o + v * d * e, 256);
+    L.tok_embed = o;  o = align_up(o + v * d * e, 1024);
+    L.final_norm = o; o = align_up(o + d * e, 1024);
+    L.lm_head = o;    o = align_up(o + mat(v, d), 1024);
     L.total = o;
     return L;
 }
@@ -94,12 +104,17 @@ struct llmcad_ctx {
     float *ssq[2] = {nullptr, nullptr};   // partial sums of squares for the folded attention / FFN norms
     float *attn_ws = nullptr;
     uint32_t *attn_counters = nullptr;
-    uint32_t epoch = 0;
+    uint32_t *grid_counter = nullptr;   // grid barrier of the GEMM chains
+    uint32_t barrier_base = 0;          // its value once everything enqueued so far has run
     int64_t launches = 0;
-    unsigned long long *trace = nullptr;   // optional GEMM timeline buffer (llmcad_set_gemm_trace)
-    // tensor maps
-    const void *maps_for = nullptr;
-    std::vector<CUtensorMap> w_maps;   // [L][4] (qkv, o, gate/up, down) + lm_head
+    unsigned long long *trace = nullptr;   // optional timeline buffer (llmcad_set_gemm_trace): [launch][256][16]
+    int trace_launch = 0, trace_capacity = 0;
+    unsigned long long *next_trace()
+    {
+        if (trace == nullptr || trace_launch >= trace_capacity) return nullptr;
+        return trace + (size_t)(trace_launch++) * 256 * 16;
+    }
+    const void *maps_for = nullptr;    // packed weight buffer of the current call
     CUtensorMap act_maps[9][3];        // [n_pad/16][xn, att, h]
     bool act_ready[9] = {false, false, false, false, false, false, false, false, false};
     // optional per-launch timing (events around every GEMM / attention launch)
@@ -152,24 +167,8 @@ struct TimedLaunch {
 
 int ensure_weight_maps(llmcad_ctx *ctx, const void *packed)
 {
-    if (!ctx->tc_gemm || ctx->maps_for == packed) return LLMCAD_OK;
-    const llmcad_config &c = ctx->cfg;
-    const uint64_t d = c.d_model, f = c.d_ffn;
-    ctx->w_maps.assign((size_t)c.n_layers * 4 + 1, CUtensorMap{});
-    const char *base = static_cast<const char *>(packed);
-    bool ok = true;
-    for (int l = 0; l < c.n_layers; ++l) {
-        const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
-        ok &= make_tensor_map_bf16(&ctx->w_maps[l * 4 + 0], lb + ctx->lay.wqkv, 3 * d, d, 128);
-        ok &= make_tensor_map_bf16(&ctx->w_maps[l * 4 + 1], lb + ctx->lay.wo, d, d, 128);
-        ok &= make_tensor_map_bf16(&ctx->w_maps[l * 4 + 2], lb + ctx->lay.wgu, 2 * f, d, 128);
-        ok &= make_tensor_map_bf16(&ctx->w_maps[l * 4 + 3], lb + ctx->lay.wdown, d, f, 128);
-    }
-    ok &= make_tensor_map_bf16(&ctx->w_maps[(size_t)c.n_layers * 4], base + ctx->lay.lm_head, c.vocab, d, 128);
-    if (!ok) {
-        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed for a weight matrix");
-        return LLMCAD_ERR_CUDA;
-    }
+    // the pass reads its weights as pre-swizzled tiles through plain bulk copies, so there is no
+    // tensor map to encode for them: remember which packed buffer the chains address
     ctx->maps_for = packed;
     return LLMCAD_OK;
 }
@@ -191,21 +190,63 @@ int ensure_act_maps(llmcad_ctx *ctx, int n_pad)
     return LLMCAD_OK;
 }
 
-// One GEMM of the pass: W is `which` of layer l (or the lm_head when l < 0).
+// A chain of dependent tensor-core GEMMs that goes out as one persistent kernel.
+struct Chain {
+    ChainMaps maps;
+    ChainParams p;
+    Chain() { p = ChainParams{}; }
+    // W is `which` (0 qkv, 1 o, 2 gate/up, 3 down) of layer l, or the lm_head when l < 0;
+    // act selects the activation buffer it multiplies (0 normalised stream, 1 attention output, 2 SwiGLU output)
+    bool has_next = false;
+    GemmDesc next{};
+    static const char *weight_ptr(llmcad_ctx *ctx, int l, int which)
+    {
+        const char *base = static_cast<const char *>(ctx->maps_for);
+        if (l < 0) return base + ctx->lay.lm_head;
+        const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
+        return lb + (which == 0 ? ctx->lay.wqkv : which == 1 ? ctx->lay.wo : which == 2 ? ctx->lay.wgu : ctx->lay.wdown);
+    }
+    // the GEMM that the launch after this one will run: its first tiles get prefetched into L2
+    void set_next(llmcad_ctx *ctx, int l, int which, int n_in, const EpiParams &ep)
+    {
+        next = make_gemm_desc(n_in, ep, weight_ptr(ctx, l, which));
+        has_next = true;
+    }
+    void add(llmcad_ctx *ctx, int l, int which, int act, int n_in, const EpiParams &ep, int n_pad)
+    {
+        const char *w = weight_ptr(ctx, l, which);
+        maps.x[p.n_gemms] = ctx->act_maps[n_pad / 16][act];
+        p.g[p.n_gemms] = make_gemm_desc(n_in, ep, w);
+        p.n_pad = n_pad;
+        ++p.n_gemms;
+    }
+    int launch(llmcad_ctx *ctx, int32_t *status, cudaStream_t st)
+    {
+        if (p.n_gemms == 0) return LLMCAD_OK;
+        p.partials = ctx->partials;
+        p.tickets = ctx->flags;
+        p.grid_counter = ctx->grid_counter;
+        p.barrier_base = ctx->barrier_base;
+        p.status = status;
+        p.trace = ctx->next_trace();
+        uint32_t arrivals = 0;
+        ctx->launches++;
+        TimedLaunch tl(ctx, 0, st);
+        CUDA_TRY(launch_gemm_chain(maps, p, ctx->n_sms, st, &arrivals, has_next ? &next : nullptr));
+        ctx->barrier_base += arrivals;
+        return LLMCAD_OK;
+    }
+};
+
+// One GEMM of the plain-ALU path: W is `which` of layer l (or the lm_head when l < 0).
 int run_gemm(llmcad_ctx *ctx, const void *packed, int l, int which, int act, int n_in, const EpiParams &ep, int n_pad,
              int32_t *status, cudaStream_t st)
 {
+    (void)n_pad;
     const char *base = static_cast<const char *>(packed);
     const void *xin = act == 0 ? ctx->xn : act == 1 ? ctx->att : ctx->h;
     ctx->launches++;
     TimedLaunch tl(ctx, 0, st);
-    if (ctx->tc_gemm) {
-        const size_t mi = l < 0 ? (size_t)ctx->cfg.n_layers * 4 : (size_t)l * 4 + which;
-        ctx->epoch++;
-        CUDA_TRY(launch_gemm_tc(ctx->w_maps[mi], ctx->act_maps[n_pad / 16][act], n_in, n_pad, ctx->n_sms, ctx->partials,
-                                ctx->flags, ctx->epoch, status, ep, st, ctx->trace));
-        return LLMCAD_OK;
-    }
     const void *W;
     if (l < 0) W = base + ctx->lay.lm_head;
     else {
@@ -224,7 +265,7 @@ int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, 
     if (ctx->tc_attn) {
         int launched = 0;
         CUDA_TRY(launch_attention_tc(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->attn_ws,
-                                     ctx->attn_counters, ctx->n_sms, status, st, &launched));
+                                     ctx->attn_counters, ctx->n_sms, status, st, &launched, ctx->next_trace()));
         ctx->launches += launched;
         return LLMCAD_OK;
     }
@@ -252,47 +293,73 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
     const size_t kv_layer = (size_t)2 * H * S * hd * ctx->elem;
 
     if (ctx->tc_gemm) {
-        // Tensor-core path: the RMSNorms are folded into the GEMMs. Whoever produces the residual
+        // Tensor-core path. The RMSNorms are folded into the GEMMs: whoever produces the residual
         // stream (the embedding gather, the O and down GEMMs) also writes gain * x in bf16 and
         // partial sums of squares; the consuming GEMM scales its accumulators by the per-node
-        // rsqrt(mean(x^2) + eps). Five kernels per layer.
+        // rsqrt(mean(x^2) + eps). The GEMMs between two attention calls (O, gate/up, down and the
+        // next layer's QKV, or the lm_head at the end) go out as one persistent chain kernel, so a
+        // layer is two launches.
         const int tiles4 = 4 * ((d + 127) / 128);
         CUDA_TRY(launch_embed_norm(base + ctx->lay.tok_embed, tokens, n, d,
                                    c.n_layers > 0 ? base + ctx->lay.attn_norm : base + ctx->lay.final_norm, ctx->x, ctx->xn,
                                    ctx->ssq[0], status, st));
-        int parts0 = 1;   // how many partials the next attention-norm consumer must add up
+        auto qkv_ep = [&](int l, int parts) {
+            char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)l;
+            EpiParams ep{};
+            ep.n = n; ep.mode = EPI_QKV; ep.n_out = 3 * d; ep.q_out = ctx->q; ep.k_cache = kl; ep.v_cache = kl + kv_layer / 2;
+            ep.rope_cs = ctx->tb.rope_cs; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P;
+            ep.ssq_in = ctx->ssq[0]; ep.ssq_in_parts = parts; ep.norm_d = d; ep.eps = c.rms_eps;
+            return ep;
+        };
+        auto head_ep = [&](int parts) {
+            EpiParams ep{};
+            ep.n = n; ep.mode = EPI_PLAIN; ep.n_out = c.vocab; ep.y = logits; ep.ldy = c.vocab;
+            ep.ssq_in = ctx->ssq[0]; ep.ssq_in_parts = parts; ep.norm_d = d; ep.eps = c.rms_eps;
+            return ep;
+        };
+        // the GEMMs of the pass in order; attention runs before the O GEMM of every layer
+        struct Spec { int l, which, act, n_in; EpiParams ep; bool attention_first; };
+        std::vector<Spec> specs;
+        if (c.n_layers > 0) specs.push_back({0, 0, 0, d, qkv_ep(0, 1), false});
+        else if (logits != nullptr) specs.push_back({-1, 0, 0, d, head_ep(1), false});
         for (int l = 0; l < c.n_layers; ++l) {
             const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
-            const char *next_attn_gain = (l + 1 < c.n_layers) ? lb + ctx->lay.layer_bytes + ctx->lay.attn_norm
-                                                              : base + ctx->lay.final_norm;
-            char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)l;
-            char *vl = kl + kv_layer / 2;
+            const bool last = l + 1 == c.n_layers;
+            const char *next_gain = last ? base + ctx->lay.final_norm : lb + ctx->lay.layer_bytes + ctx->lay.attn_norm;
             EpiParams ep{};
-            ep.n = n; ep.mode = EPI_QKV; ep.n_out = 3 * d; ep.q_out = ctx->q; ep.k_cache = kl; ep.v_cache = vl;
-            ep.rope_cs = ctx->tb.rope_cs; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P;
-            ep.ssq_in = ctx->ssq[0]; ep.ssq_in_parts = parts0; ep.norm_d = d; ep.eps = c.rms_eps;
-            if ((rc = run_gemm(ctx, packed, l, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
-
-            if ((rc = run_attention(ctx, ctx->q, kl, vl, S, P, n, ctx->att, status, st)) != LLMCAD_OK) return rc;
-
-            ep = EpiParams{}; ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
+            ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
             ep.xg_out = ctx->xn; ep.gain_next = lb + ctx->lay.ffn_norm; ep.ssq_out = ctx->ssq[1];
-            if ((rc = run_gemm(ctx, packed, l, 1, 1, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+            specs.push_back({l, 1, 1, d, ep, true});
 
             ep = EpiParams{}; ep.n = n; ep.mode = EPI_SWIGLU; ep.n_out = f; ep.h = ctx->h;
             ep.ssq_in = ctx->ssq[1]; ep.ssq_in_parts = tiles4; ep.norm_d = d; ep.eps = c.rms_eps;
-            if ((rc = run_gemm(ctx, packed, l, 2, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+            specs.push_back({l, 2, 0, d, ep, false});
 
             ep = EpiParams{}; ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
-            ep.xg_out = ctx->xn; ep.gain_next = next_attn_gain; ep.ssq_out = ctx->ssq[0];
-            if ((rc = run_gemm(ctx, packed, l, 3, 2, f, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
-            parts0 = tiles4;
+            ep.xg_out = ctx->xn; ep.gain_next = next_gain; ep.ssq_out = ctx->ssq[0];
+            specs.push_back({l, 3, 2, f, ep, false});
+
+            if (!last) specs.push_back({l + 1, 0, 0, d, qkv_ep(l + 1, tiles4), false});
+            else if (logits != nullptr) specs.push_back({-1, 0, 0, d, head_ep(tiles4), false});
         }
-        if (logits != nullptr) {
-            EpiParams ep{};
-            ep.n = n; ep.mode = EPI_PLAIN; ep.n_out = c.vocab; ep.y = logits; ep.ldy = c.vocab;
-            ep.ssq_in = ctx->ssq[0]; ep.ssq_in_parts = parts0; ep.norm_d = d; ep.eps = c.rms_eps;
-            if ((rc = run_gemm(ctx, packed, -1, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
+        // Dependent GEMMs may share a launch (grid barriers between them, see gemm_tc.cu); measured
+        // on B200 one GEMM per launch, chained by programmatic dependent launch, is faster, so that
+        // is the default. LLMCAD_CHAIN_MAX is a tuning aid.
+        static const int chain_max = [] { const char *e = getenv("LLMCAD_CHAIN_MAX"); int v = e ? atoi(e) : 1; return v < 1 ? 1 : (v > kMaxChain ? kMaxChain : v); }();
+        for (size_t i = 0; i < specs.size();) {
+            if (specs[i].attention_first) {
+                char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)specs[i].l;
+                if ((rc = run_attention(ctx, ctx->q, kl, kl + kv_layer / 2, S, P, n, ctx->att, status, st)) != LLMCAD_OK) return rc;
+            }
+            Chain ch;
+            size_t j = i;
+            do {
+                ch.add(ctx, specs[j].l, specs[j].which, specs[j].act, specs[j].n_in, specs[j].ep, n_pad);
+                ++j;
+            } while (j < specs.size() && ch.p.n_gemms < chain_max && !specs[j].attention_first);
+            if (j < specs.size()) ch.set_next(ctx, specs[j].l, specs[j].which, specs[j].n_in, specs[j].ep);
+            if ((rc = ch.launch(ctx, status, st)) != LLMCAD_OK) return rc;
+            i = j;
         }
         return LLMCAD_OK;
     }
@@ -331,6 +398,17 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
         ep.n = n; ep.mode = EPI_PLAIN; ep.n_out = c.vocab; ep.y = logits; ep.ldy = c.vocab;
         if ((rc = run_gemm(ctx, packed, -1, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
     }
+    return LLMCAD_OK;
+}
+
+// The chain kernels synchronise through a grid counter and per-tile tickets. Both return to a
+// known state by themselves, but not when a wait ran out: start every call from zero.
+int reset_chain_sync(llmcad_ctx *ctx, cudaStream_t st)
+{
+    if (!ctx->tc_gemm) return LLMCAD_OK;
+    CUDA_TRY(cudaMemsetAsync(ctx->grid_counter, 0, sizeof(uint32_t), st));
+    CUDA_TRY(cudaMemsetAsync(ctx->flags, 0, (size_t)kMaxChain * kTicketsPerGemm * sizeof(uint32_t), st));
+    ctx->barrier_base = 0;
     return LLMCAD_OK;
 }
 
@@ -398,7 +476,12 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ctx->n_sms = prop.multiProcessorCount;
     ctx->elem = cfg->dtype == LLMCAD_F32 ? 4 : 2;
     const bool sm100 = prop.major == 10;
-    ctx->tc_gemm = sm100 && cfg->dtype == LLMCAD_BF16 && !(cfg->flags & LLMCAD_FLAG_SIMT_GEMM);
+    ctx->tc_gemm = want_tiled(*cfg);
+    if (ctx->tc_gemm && !sm100) {   // the tensor-core kernels are sm_100a only
+        delete ctx;
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "device is not sm_100");
+        return LLMCAD_ERR_CUDA;
+    }
     ctx->tc_attn = cfg->dtype == LLMCAD_BF16 && cfg->head_dim == 128 && !(cfg->flags & LLMCAD_FLAG_SIMT_ATTN);
 
     const size_t d = cfg->d_model, f = cfg->d_ffn, hd = cfg->head_dim;
@@ -418,8 +501,9 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ok = ok && alloc((void **)&ctx->tb.anc, 128 * 16);
     ok = ok && alloc((void **)&ctx->tb.rope_cs, 128 * (hd / 2) * sizeof(float2));
     ok = ok && alloc((void **)&ctx->ibuf, (520 + 128) * 4);
-    ok = ok && alloc((void **)&ctx->partials, gemm_tc_partial_floats(ctx->n_sms, 128) * 4);
-    ok = ok && alloc((void **)&ctx->flags, (size_t)4096 * 4 * 4);   // ticket counters of up to 4096 tiles
+    ok = ok && alloc((void **)&ctx->partials, gemm_tc_partial_floats(2 * ctx->n_sms, 128) * 4);
+    ok = ok && alloc((void **)&ctx->flags, (size_t)kMaxChain * kTicketsPerGemm * 4);   // ticket counters
+    ok = ok && alloc((void **)&ctx->grid_counter, 256);
     const size_t ssq_floats = (size_t)4 * ((d + 127) / 128) * LLMCAD_MAX_TREE;
     ok = ok && alloc((void **)&ctx->ssq[0], ssq_floats * 4);
     ok = ok && alloc((void **)&ctx->ssq[1], ssq_floats * 4);
@@ -443,7 +527,7 @@ void llmcad_destroy(llmcad_ctx *ctx)
     if (ctx == nullptr) return;
     void *ptrs[] = {ctx->x, ctx->xn, ctx->q, ctx->att, ctx->h, ctx->logits, ctx->tb.depth, ctx->tb.pos, ctx->tb.anc,
                     ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->flags, ctx->attn_ws, ctx->attn_counters, ctx->ssq[0],
-                    ctx->ssq[1]};
+                    ctx->ssq[1], ctx->grid_counter};
     for (void *p : ptrs)
         if (p != nullptr) cudaFree(p);
     for (auto &t : ctx->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
@@ -464,6 +548,19 @@ int llmcad_pack_layer(llmcad_ctx *ctx, int32_t layer, const llmcad_layer_weights
     auto cp = [&](size_t off, const void *s, size_t bytes) {
         return cudaMemcpyAsync(lb + off, s, bytes, cudaMemcpyDeviceToDevice, st);
     };
+    if (ctx->tc_gemm) {
+        const size_t t_dd = tiled_weight_bytes((int)d, (int)d), t_fd = tiled_weight_bytes((int)f, (int)d);
+        CUDA_TRY(cp(ctx->lay.attn_norm, src->attn_norm, d * e));
+        CUDA_TRY(cp(ctx->lay.ffn_norm, src->ffn_norm, d * e));
+        CUDA_TRY(launch_tile_weight(src->wq, (int)d, (int)d, lb + ctx->lay.wqkv, st));
+        CUDA_TRY(launch_tile_weight(src->wk, (int)d, (int)d, lb + ctx->lay.wqkv + t_dd, st));
+        CUDA_TRY(launch_tile_weight(src->wv, (int)d, (int)d, lb + ctx->lay.wqkv + 2 * t_dd, st));
+        CUDA_TRY(launch_tile_weight(src->wo, (int)d, (int)d, lb + ctx->lay.wo, st));
+        CUDA_TRY(launch_tile_weight(src->w_gate, (int)f, (int)d, lb + ctx->lay.wgu, st));
+        CUDA_TRY(launch_tile_weight(src->w_up, (int)f, (int)d, lb + ctx->lay.wgu + t_fd, st));
+        CUDA_TRY(launch_tile_weight(src->w_down, (int)d, (int)f, lb + ctx->lay.wdown, st));
+        return LLMCAD_OK;
+    }
     CUDA_TRY(cp(ctx->lay.attn_norm, src->attn_norm, d * e));
     CUDA_TRY(cp(ctx->lay.wqkv, src->wq, d * d * e));
     CUDA_TRY(cp(ctx->lay.wqkv + d * d * e, src->wk, d * d * e));
@@ -485,7 +582,8 @@ int llmcad_pack_globals(llmcad_ctx *ctx, const llmcad_global_weights *src, void 
     char *b = static_cast<char *>(packed);
     CUDA_TRY(cudaMemcpyAsync(b + ctx->lay.tok_embed, src->tok_embed, v * d * e, cudaMemcpyDeviceToDevice, st));
     CUDA_TRY(cudaMemcpyAsync(b + ctx->lay.final_norm, src->final_norm, d * e, cudaMemcpyDeviceToDevice, st));
-    CUDA_TRY(cudaMemcpyAsync(b + ctx->lay.lm_head, src->lm_head, v * d * e, cudaMemcpyDeviceToDevice, st));
+    if (ctx->tc_gemm) CUDA_TRY(launch_tile_weight(src->lm_head, (int)v, (int)d, b + ctx->lay.lm_head, st));
+    else CUDA_TRY(cudaMemcpyAsync(b + ctx->lay.lm_head, src->lm_head, v * d * e, cudaMemcpyDeviceToDevice, st));
     return LLMCAD_OK;
 }
 
@@ -502,6 +600,7 @@ int llmcad_verify_tree(llmcad_ctx *ctx, const void *packed, void *kv_cache, int3
     int32_t *status = out->scalars + LLMCAD_S_STATUS;
     float *logits = out->logits != nullptr ? out->logits : ctx->logits;
     CUDA_TRY(cudaMemsetAsync(out->scalars, 0, 8 * sizeof(int32_t), st));
+    if ((rc = reset_chain_sync(ctx, st)) != LLMCAD_OK) return rc;
     if ((rc = run_forward(ctx, packed, kv_cache, prefix_len, tree_tokens, parent_idx, n, logits, status, st)) != LLMCAD_OK)
         return rc;
     CUDA_TRY(launch_argmax(logits, n, c.vocab, out->argmax, status, st));
@@ -549,6 +648,10 @@ int llmcad_prefill(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
     CUDA_TRY(cudaMemsetAsync(ctx->scalars_dev(), 0, 8 * sizeof(int32_t), st));
+    {
+        int rc0 = reset_chain_sync(ctx, st);
+        if (rc0 != LLMCAD_OK) return rc0;
+    }
     const int chunk = ctx->cfg.max_tree;
     for (int done = 0; done < n; done += chunk) {
         const int m = n - done < chunk ? n - done : chunk;
@@ -628,23 +731,67 @@ int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, 
     CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
     EpiParams ep{};
     ep.mode = EPI_PLAIN; ep.n = n; ep.n_out = n_out; ep.y = y; ep.ldy = n_out;
-    ctx->launches++;
-    TimedLaunch tl(ctx, 0, st);
+    {
+        int rc0 = reset_chain_sync(ctx, st);
+        if (rc0 != LLMCAD_OK) return rc0;
+    }
     if (ctx->tc_gemm) {
         const int n_pad = (n + 15) / 16 * 16;
-        CUtensorMap mw, mx;
+        Chain ch;
         // rows of x beyond n are outside the tensor: the copy engine fills them with zeros
-        if (!make_tensor_map_bf16(&mw, w, n_out, n_in, 128) || !make_tensor_map_bf16(&mx, x, n, n_in, n_pad)) {
+        if (!make_tensor_map_bf16(&ch.maps.w[0], w, n_out, n_in, 128) || !make_tensor_map_bf16(&ch.maps.x[0], x, n, n_in, n_pad)) {
             snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
             return LLMCAD_ERR_CUDA;
         }
-        ctx->epoch++;
-        CUDA_TRY(launch_gemm_tc(mw, mx, n_in, n_pad, ctx->n_sms, ctx->partials, ctx->flags, ctx->epoch, status, ep, st,
-                                ctx->trace));
-        return LLMCAD_OK;
+        ch.p.g[0] = make_gemm_desc(n_in, ep);
+        ch.p.n_pad = n_pad;
+        ch.p.n_gemms = 1;
+        return ch.launch(ctx, status, st);
     }
+    ctx->launches++;
+    TimedLaunch tl(ctx, 0, st);
     CUDA_TRY(launch_gemm_simt(w, x, ctx->cfg.dtype, n_in, ep, status, st));
     return LLMCAD_OK;
+}
+
+size_t llmcad_tiled_weight_bytes(int32_t n_out, int32_t n_in)
+{
+    if (n_out < 1 || n_in < 1) return 0;
+    return tiled_weight_bytes(n_out, n_in);
+}
+
+int llmcad_tile_weight(const void *w, int32_t n_out, int32_t n_in, void *tiled, void *stream)
+{
+    if (!w || !tiled) return LLMCAD_ERR_INVALID_ARG;
+    if (n_out < 1 || n_in < 1) return LLMCAD_ERR_INVALID_ARG;
+    if (n_in % 8) return LLMCAD_ERR_UNSUPPORTED;
+    CUDA_TRY(launch_tile_weight(w, n_out, n_in, tiled, static_cast<cudaStream_t>(stream)));
+    return LLMCAD_OK;
+}
+
+int llmcad_skinny_gemm_tiled(llmcad_ctx *ctx, const void *w_tiled, const void *x, float *y, int32_t n_out, int32_t n_in,
+                             int32_t n, void *stream)
+{
+    if (!ctx || !w_tiled || !x || !y) return LLMCAD_ERR_INVALID_ARG;
+    if (n_out < 1 || n_in < 1 || n < 1) return LLMCAD_ERR_INVALID_ARG;
+    if (n > ctx->cfg.max_tree || n_in % 8 || !ctx->tc_gemm) return LLMCAD_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
+    CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    int rc = reset_chain_sync(ctx, st);
+    if (rc != LLMCAD_OK) return rc;
+    EpiParams ep{};
+    ep.mode = EPI_PLAIN; ep.n = n; ep.n_out = n_out; ep.y = y; ep.ldy = n_out;
+    const int n_pad = (n + 15) / 16 * 16;
+    Chain ch;
+    if (!make_tensor_map_bf16(&ch.maps.x[0], x, n, n_in, n_pad)) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
+        return LLMCAD_ERR_CUDA;
+    }
+    ch.p.g[0] = make_gemm_desc(n_in, ep, w_tiled);
+    ch.p.n_pad = n_pad;
+    ch.p.n_gemms = 1;
+    return ch.launch(ctx, status, st);
 }
 
 int llmcad_set_kernel_timing(llmcad_ctx *ctx, int32_t enable)
@@ -676,10 +823,12 @@ int llmcad_get_kernel_timing(llmcad_ctx *ctx, int32_t kind, double *total_ms, in
     return LLMCAD_OK;
 }
 
-int llmcad_set_gemm_trace(llmcad_ctx *ctx, uint64_t *trace)
+int llmcad_set_gemm_trace(llmcad_ctx *ctx, uint64_t *trace, int32_t capacity)
 {
     if (ctx == nullptr) return LLMCAD_ERR_INVALID_ARG;
     ctx->trace = reinterpret_cast<unsigned long long *>(trace);
+    ctx->trace_launch = 0;
+    ctx->trace_capacity = trace ? capacity : 0;
     return LLMCAD_OK;
 }
 

@@ -73,10 +73,13 @@ __global__ void __launch_bounds__(kAtThreads)
 attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
                     const __nv_bfloat16 *__restrict__ v, int n_heads, int kv_stride, int P, int n, int n_pad,
                     const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
-                    const int32_t *status)
+                    const int32_t *status, unsigned long long *trace)
 {
+    const int cta = blockIdx.y * gridDim.x + blockIdx.x;
+    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 0] = global_timer_ns();
     pdl_launch_dependents();
     pdl_wait();
+    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 1] = global_timer_ns();
     if (*status) return;   // uniform over the grid: set only by kernels that ran before this one
     extern __shared__ __align__(128) uint8_t sm[];
     uint8_t *s_q = sm;                                      // [n_pad][256 B]
@@ -237,6 +240,7 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
                 if (row1 < n) *reinterpret_cast<uint32_t *>(o + ((size_t)row1 * n_heads + head) * kHd + dim) = pack_bf16(oacc[j][2] * i1, oacc[j][3] * i1);
             }
         }
+        if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
         return;
     }
 
@@ -288,6 +292,7 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         *reinterpret_cast<uint32_t *>(o + ((size_t)row * n_heads + head) * kHd + dim) = pack_bf16(a0 * inv, a1 * inv);
     }
     cluster.sync();                                          // peers may still be reading this CTA's partial
+    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
 }
 
 size_t attention_tc_workspace_bytes(int n_heads, int n_sms)
@@ -298,7 +303,7 @@ size_t attention_tc_workspace_bytes(int n_heads, int n_sms)
 
 cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, float *ws, uint32_t *counters, int n_sms,
-                                int32_t *status, cudaStream_t st, int *launched)
+                                int32_t *status, cudaStream_t st, int *launched, unsigned long long *trace)
 {
     (void)ws; (void)counters;
     if (hd != kHd) return cudaErrorInvalidValue;
@@ -325,7 +330,7 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     if (launched) *launched = 1;
     return cudaLaunchKernelEx(&lc.cfg, attention_tc_kernel, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                               (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc, (__nv_bfloat16 *)o, splits,
-                              tiles_per_split, status);
+                              tiles_per_split, status, trace);
 }
 
 }  // namespace llmcad

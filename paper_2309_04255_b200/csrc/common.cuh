@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include "../../include/llmcad.h"
 
@@ -98,7 +99,7 @@ __device__ __forceinline__ void epilogue_pair(const EpiParams &ep, int r0, int i
 __device__ __forceinline__ uint64_t global_timer_ns()
 {
     uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t) :: "memory");   // the clobber keeps the read where it is written
     return t;
 }
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every device-side wait gives up after 2 s
@@ -120,8 +121,9 @@ struct LaunchCfg {
         cfg.blockDim = block;
         cfg.dynamicSmemBytes = smem;
         cfg.stream = st;
+        static const int pdl = [] { const char *e = getenv("LLMCAD_PDL"); return e ? atoi(e) : 1; }();   // tuning aid
         attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attrs[0].val.programmaticStreamSerializationAllowed = 1;
+        attrs[0].val.programmaticStreamSerializationAllowed = pdl;
         cfg.numAttrs = 1;
         if (cluster_x > 0) {
             attrs[1].id = cudaLaunchAttributeClusterDimension;
@@ -154,6 +156,8 @@ cudaError_t launch_accept(const int32_t *parent, const int32_t *tokens, const in
                           int32_t *path, int32_t *scalars, cudaStream_t st);
 cudaError_t launch_compact(void *kv, int dtype, int n_layers, int n_heads, int S, int hd, int P, const int32_t *path,
                            const int32_t *scalars, cudaStream_t st);
+size_t tiled_weight_bytes(int n_out, int n_in);
+cudaError_t launch_tile_weight(const void *w, int n_out, int n_in, void *dst, cudaStream_t st);
 cudaError_t launch_gemm_simt(const void *W, const void *x, int dtype, int n_in, const EpiParams &ep,
                              const int32_t *status, cudaStream_t st);
 cudaError_t launch_attention_simt(const void *q, const void *k, const void *v, int dtype, int n_heads, int hd,

@@ -1,30 +1,36 @@
-// Weight-streaming skinny GEMM on the sm_100a tensor cores.
+// Weight-streaming skinny GEMMs on the sm_100a tensor cores, run as a chain.
 //
 // The one-shot verification of Sec. 3.2 visits every parameter once for all N <= 128 tree nodes,
 // so each GEMM is D[n_out][N] = W[n_out][K] * X[N][K]^T with a tiny N: it is bound by the bytes
 // of W coming from HBM. The kernel therefore puts W on the M side of tcgen05.mma (128 weight
 // rows per tile = the 128 TMEM lanes) and the tree nodes on the N side (padded to a multiple of
-// 16), streams W exactly once through a deep TMA -> shared-memory ring, and keeps all SMs pulling
-// by splitting the (tile, k-block) work evenly over a persistent grid (stream-K): a CTA's range
-// may start and end inside a tile; the sharers of a tile leave their partial accumulators in an
-// fp32 workspace and whichever warp arrives last at the tile's ticket counter adds them in a
-// fixed (CTA) order and runs the fused epilogue, so the result does not depend on timing and
-// no CTA ever waits for another.
+// 16), and streams W exactly once through a deep TMA -> shared-memory ring.
+//
+// One launch runs up to four *dependent* GEMMs (e.g. O -> gate/up -> down -> next layer's QKV) on a
+// persistent grid of one CTA per SM. The weights do not depend on the activations, so the producer
+// warp keeps streaming the next GEMM's weight tiles into the ring while the current GEMM's tail
+// (partial-tile reduction, epilogue) and the grid barrier between the two are still in progress;
+// only the small activation tiles and the epilogues wait for the barrier. Within a GEMM the (tile,
+// k-block) items are split evenly over the CTAs (stream-K): a CTA's range may start and end inside
+// a tile; the sharers of a tile leave their partial accumulators in an fp32 workspace and whichever
+// warp arrives last at the tile's ticket counter adds them in a fixed (CTA) order and runs the fused
+// epilogue, so the result does not depend on timing and no CTA waits for another inside a GEMM.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer,
 // warps 2..5 = epilogue (tcgen05.ld of their 32 lanes each). Accumulators are double-buffered in
 // TMEM so that the epilogue of one tile overlaps the MMAs of the next.
 //
-// The kernel is launched with programmatic stream serialization: its producer fills the whole
-// ring with weight tiles (which no kernel ever writes) while the previous kernel of the pass is
-// still running, and only the activation tiles, the workspace and the outputs wait for the grid
-// dependency. A status word left by an earlier phase is not looked at here: the GEMM then
-// works on stale but finite activations and writes only scratch (slots >= prefix_len, the
-// context's buffers), and the search/rollback kernels at the end of the pass report the error.
+// The kernel is launched with programmatic stream serialization: the ring is filled with weight
+// tiles while the previous kernel of the pass is still running; activations, workspace and outputs
+// wait for the grid dependency. A status word left by an earlier phase is not looked at here: the
+// GEMMs then work on stale but finite activations and write only scratch, and the search/rollback
+// kernels at the end of the pass report the error.
 //
-// Every wait (mbarrier, workspace flag) is bounded; on expiry the kernel sets the status word to
-// LLMCAD_ERR_TIMEOUT, lets every role fall out of its loop, frees TMEM and returns.
+// Every wait (mbarrier, grid barrier) is bounded by a deadline; on expiry the kernel sets the status
+// word to LLMCAD_ERR_TIMEOUT, lets every role fall out of its loop, frees TMEM and returns.
 #include <cuda.h>
+
+#include <cstdlib>
 
 #include "common.cuh"
 #include "gemm_tc.cuh"
@@ -35,8 +41,10 @@ namespace {
 
 constexpr int kTileM = 128;     // weight rows per tile
 constexpr int kBlockK = 64;     // bf16 elements per k-block = one 128-byte swizzle row
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;   // producer, MMA, 4 epilogue warps, activation loader
 constexpr int kATileBytes = kTileM * kBlockK * 2;  // 16 KB
+constexpr int kMaxStages = 16;
+constexpr int kPairK = 2;        // k-blocks per ring item: one 32 KB weight copy feeds 8 MMAs
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -69,14 +77,35 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
     if (mbar_try(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
+    uint64_t t0 = 0;
     for (uint32_t it = 1;; ++it) {
+        // a hot poller would take issue slots from the epilogue warp that shares its scheduler
+        __nanosleep(32);
         if (mbar_try(bar, parity)) return true;
         if ((it & 255u) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+            if (t0 == 0) t0 = global_timer_ns();
+            else if (global_timer_ns() - t0 > kWaitLimitNs) return false;
         }
     }
+}
+
+// Whole-warp wait for roles that are not on the critical path of the weight stream: one lane
+// polls, with a short sleep between polls, and the warp follows. A warp of 32 hot pollers per
+// barrier would saturate the shared-memory pipeline that the producer's copies and barrier
+// operations also go through.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane)
+{
+    int ok = 1;
+    if (lane == 0 && !mbar_try(bar, parity)) {
+        const uint64_t t0 = global_timer_ns();
+        for (uint32_t it = 1;; ++it) {
+            __nanosleep(40);
+            if (mbar_try(bar, parity)) break;
+            if ((it & 63u) == 0 && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) { ok = 0; break; }
+        }
+    }
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 // ---------------------------------------------------------------- TMA
@@ -87,6 +116,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
         " [%0], [%1, {%2, %3}], [%4], %5;"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
+        : "memory");
+}
+
+// One contiguous run of global memory into shared memory (both 16-byte aligned, size a multiple of 16).
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
         : "memory");
 }
 
@@ -150,13 +188,14 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n)
 }
 
 struct SharedCtl {
-    uint64_t full[16];
-    uint64_t empty[16];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
-    float rs[LLMCAD_MAX_TREE]; // per-node rsqrt(mean(x^2) + eps) of the folded input RMSNorm
+    volatile uint32_t a_issued;     // ring items whose weight copy (and expect_tx) has been issued
+    float rs[4][LLMCAD_MAX_TREE];   // per epilogue warp: rsqrt(mean(x^2) + eps) of the folded input RMSNorm
 };
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
@@ -165,59 +204,185 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v)
+
+// A ring item is (tile, k-block pair, half): up to two consecutive 64-wide k-blocks of one
+// 128-row weight tile (32 KB, contiguous in the tiled layout) and the matching activation tiles.
+__device__ __forceinline__ int pairs_per_tile(const GemmDesc &g) { return (g.kb_per_tile + kPairK - 1) / kPairK; }
+
+// This CTA's share of GEMM g: items [begin, end) of its item list.
+struct Range {
+    int begin, end;
+};
+__device__ __forceinline__ Range cta_range(const GemmDesc &g)
 {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+    const int total = g.n_tiles * pairs_per_tile(g) * g.halves;
+    Range r;
+    r.begin = min(total, (int)blockIdx.x * g.items_per_cta);
+    r.end = min(total, r.begin + g.items_per_cta);
+    return r;
 }
 
-// Walks the (tile, k-block) units of one CTA's range [u0, u1) segment by segment, last segment
-// first (see the kernel comment for why), k-blocks ascending inside a segment.
-struct UnitWalk {
-    long long u0, hi;
-    int kb_per_tile;
-    int tile, kb, kb1;
-    __device__ UnitWalk(long long u0_, long long u1_, int kbpt) : u0(u0_), hi(u1_), kb_per_tile(kbpt), tile(0), kb(0), kb1(0) {}
-    // advance to the next unit; false when the range is exhausted
-    __device__ bool next()
+// Cursor over the concatenated item stream of the chain (all GEMMs, this CTA's ranges, in order).
+// Coordinates are kept incrementally: the single-thread roles have well under a microsecond per item.
+struct Cursor {
+    int g;                 // current GEMM, == n_gemms when exhausted
+    int tile, kp, half;    // coordinates of the current item (kp: k-block pair)
+    int left;              // items left in this CTA's range of GEMM g, the current one included
+    int ppt, halves, kbpt;
+    __device__ void init(const ChainParams &p)
     {
-        if (kb + 1 < kb1) { ++kb; return true; }
-        if (hi <= u0) return false;
-        tile = (int)((hi - 1) / kb_per_tile);
-        const long long t0 = (long long)tile * kb_per_tile;
-        const long long lo = u0 > t0 ? u0 : t0;
-        kb = (int)(lo - t0);
-        kb1 = (int)(hi - t0);
-        hi = lo;
-        return true;
+        g = -1;
+        left = 0;
+        next_gemm(p);
+    }
+    __device__ void next_gemm(const ChainParams &p)
+    {
+        while (true) {
+            if (++g >= p.n_gemms) { g = p.n_gemms; left = 0; return; }
+            const GemmDesc &d = p.g[g];
+            const Range r = cta_range(d);
+            left = r.end - r.begin;
+            if (left <= 0) continue;
+            kbpt = d.kb_per_tile;
+            ppt = pairs_per_tile(d);
+            halves = d.halves;
+            const int ipt = ppt * halves;
+            tile = r.begin / ipt;
+            const int q = r.begin - tile * ipt;
+            kp = q / halves;
+            half = q - kp * halves;
+            return;
+        }
+    }
+    __device__ bool done(const ChainParams &p) const { return g >= p.n_gemms; }
+    __device__ int kb0() const { return kp * kPairK; }
+    __device__ int nk() const { return min(kPairK, kbpt - kp * kPairK); }   // k-blocks in this item
+    __device__ void advance(const ChainParams &p)
+    {
+        if (--left <= 0) { next_gemm(p); return; }
+        if (++half == halves) {
+            half = 0;
+            if (++kp == ppt) { kp = 0; ++tile; }
+        }
     }
 };
+
+// ------------------------------------------------------------------------------------------------
+// Fused epilogue of 16 columns (tree nodes c0..c0+15) of one thread's output row. v/w hold the
+// complete sums (w: the up-projection half of a SwiGLU tile).
+template <typename T>
+__device__ __forceinline__ void epilogue_chunk(const EpiParams &ep, const float *rs, int tile, int lane_grp, int lane, int row,
+                                               bool row_ok, float gain, int c0, float (&v)[16], float (&w)[16], float (&xo)[16])
+{
+    if (ep.ssq_in != nullptr) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) { const float r = rs[c0 + j]; v[j] *= r; w[j] *= r; }
+    }
+    // all loads of the chunk are issued before any dependent store so that they overlap
+    if (ep.mode == EPI_SWIGLU) {
+        T *hrow = reinterpret_cast<T *>(ep.h) + row;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            if (row_ok && c0 + j < ep.n) {
+                const float sg = v[j] / (1.0f + __expf(-v[j]));
+                hrow[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(sg * w[j]);
+            }
+        }
+    } else if (ep.mode == EPI_QKV) {
+        const int sec = row / ep.d, cidx = row - sec * ep.d;
+        const int head = cidx / ep.hd, e = cidx - head * ep.hd;
+        float2 cs[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            cs[j] = (sec < 2 && row_ok && c0 + j < ep.n) ? __ldg(ep.rope_cs + (size_t)(c0 + j) * (ep.hd >> 1) + (e >> 1))
+                                                          : make_float2(1.f, 0.f);
+        T *dst;
+        size_t node_stride;
+        if (sec == 0) { dst = reinterpret_cast<T *>(ep.q_out) + cidx; node_stride = ep.d; }
+        else { dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P) * ep.hd + e; node_stride = ep.hd; }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            // the rotary partner (2t <-> 2t+1) lives in the neighbouring lane
+            const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
+            const float rot = (lane & 1) ? (other * cs[j].y + v[j] * cs[j].x) : (v[j] * cs[j].x - other * cs[j].y);
+            if (row_ok && c0 + j < ep.n) dst[(size_t)(c0 + j) * node_stride] = from_f32<T>(rot);
+        }
+    } else if (ep.mode == EPI_RESID) {
+        // xo: the residual values of this chunk, loaded by the caller together with the partial tiles
+        float *xr = ep.x + row;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            xo[j] = (row_ok && c0 + j < ep.n) ? xo[j] + v[j] : 0.f;
+            if (row_ok && c0 + j < ep.n) xr[(size_t)(c0 + j) * ep.n_out] = xo[j];
+        }
+        if (ep.xg_out != nullptr) {
+            // what the next RMSNorm needs: gain * x in the GEMM input dtype, and this warp's share
+            // (32 rows) of every node's sum of squares
+            T *gr = reinterpret_cast<T *>(ep.xg_out) + row;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (row_ok && c0 + j < ep.n) gr[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(xo[j] * gain);
+            // column sums over the warp's 32 rows by recursive halving: after exchanging with
+            // lane^16, ^8, ^4, ^2 a lane is left with one column, after lane^1 with its full sum
+            // (16 shuffles instead of 80). Column held by a lane: bits 4..1 of the lane, msb first.
+            float s8[8], s4[4], s2[2], s1;
+            {
+                const bool up = lane & 16;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float keep = up ? xo[8 + j] * xo[8 + j] : xo[j] * xo[j];
+                    const float give = up ? xo[j] * xo[j] : xo[8 + j] * xo[8 + j];
+                    s8[j] = keep + __shfl_xor_sync(0xffffffffu, give, 16);
+                }
+            }
+            {
+                const bool up = lane & 8;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) s4[j] = (up ? s8[4 + j] : s8[j]) + __shfl_xor_sync(0xffffffffu, up ? s8[j] : s8[4 + j], 8);
+            }
+            {
+                const bool up = lane & 4;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) s2[j] = (up ? s4[2 + j] : s4[j]) + __shfl_xor_sync(0xffffffffu, up ? s4[j] : s4[2 + j], 4);
+            }
+            {
+                const bool up = lane & 2;
+                s1 = (up ? s2[1] : s2[0]) + __shfl_xor_sync(0xffffffffu, up ? s2[0] : s2[1], 2);
+            }
+            s1 += __shfl_xor_sync(0xffffffffu, s1, 1);
+            if (!(lane & 1)) ep.ssq_out[(size_t)(tile * 4 + lane_grp) * LLMCAD_MAX_TREE + c0 + (lane >> 1)] = s1;
+        }
+    } else {
+        float *yr = ep.y + row;
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (row_ok && c0 + j < ep.n) yr[(size_t)(c0 + j) * ep.ldy] = v[j];
+    }
+}
 
 }  // namespace
 
 template <typename T>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, TcGemmParams p)
+gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ SharedCtl ctl;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_acc = p.dual ? 2 : 1;
     const uint32_t b_tile_bytes = (uint32_t)p.n_pad * kBlockK * 2;
-    const uint32_t stage_bytes = n_acc * kATileBytes + b_tile_bytes;
+    // stage: [weights k-block 0 | weights k-block 1 | activations k-block 0 | activations k-block 1]
+    const uint32_t stage_bytes = kPairK * (kATileBytes + b_tile_bytes);
+    const uint32_t b_off = kPairK * kATileBytes;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t acc_cols = 2u * (uint32_t)p.n_pad;     // TMEM columns of one accumulator buffer (gate | up)
 
-    // Let the next kernel of the stream start its own prologue and weight prefetch early. This
-    // kernel in turn must not read activations, the status word or the workspace, nor write
-    // anything, before pdl_wait(): until then it only prefetches weights, which no kernel writes.
+    // Let the next kernel of the stream start early. This kernel in turn must not read activations,
+    // the status word or the workspace, nor write anything, before pdl_wait(): until then it only
+    // prefetches weights, which no kernel writes.
     pdl_launch_dependents();
 #define LLMCAD_TRACE(slot) do { if (p.trace) p.trace[(size_t)blockIdx.x * 16 + (slot)] = global_timer_ns(); } while (0)
     if (threadIdx.x == 0) LLMCAD_TRACE(0);
-
-    // ---- work range of this CTA
-    const long long total_units = (long long)p.n_tiles * p.kb_per_tile;
-    const long long u0 = min(total_units, (long long)blockIdx.x * p.units_per_cta);
-    const long long u1 = min(total_units, u0 + p.units_per_cta);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -229,6 +394,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             mbar_init(smem_u32(&ctl.tmem_empty[b]), 4);
         }
         ctl.abort_flag = 0;
+        ctl.a_issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -245,266 +411,365 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     volatile int *abort_flag = &ctl.abort_flag;
     bool timed_out = false;
     if (threadIdx.x == 0) LLMCAD_TRACE(1);
+    // "GEMM g of this launch is complete on every CTA": 4 epilogue warps x gridDim arrivals each.
+    const uint32_t arrivals_per_gemm = 4u * gridDim.x;
 
     if (warp == 0) {
-        // ================================================= TMA producer
+        // ================================================= weight producer
+        // Streams this CTA's weight tiles of the whole chain, in order, as fast as ring slots
+        // free up; it never looks at activations or barriers between GEMMs.
         if (lane == 0) {
-            uint64_t pol_stream, pol_keep;
+            uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            Cursor c, cpf;                   // next item to copy into the ring / to prefetch into L2
+            c.init(p);
+            cpf.init(p);
+            int s = 0;
+            uint32_t par = 1, issued = 0, prefetched = 0;   // a fresh barrier passes a wait on parity 1: no special first lap
+            uint64_t t_idle = 0;
+            while (!c.done(p)) {
+                if (mbar_try(smem_u32(&ctl.empty[s]), par)) {
+                    const GemmDesc &d = p.g[c.g];
+                    const int nk = c.nk();
+                    const uint32_t full = smem_u32(&ctl.full[s]);
+                    const uint32_t dst = smem_base + s * stage_bytes;
+                    mbar_expect_tx(full, (uint32_t)nk * (kATileBytes + b_tile_bytes));
+                    if (d.w_tiled != nullptr) {
+                        // consecutive k-blocks of a tile are contiguous in the tiled layout: one copy
+                        const size_t t = (size_t)(c.tile + (c.half ? d.up_tile_offset : 0)) * d.kb_per_tile + c.kb0();
+                        bulk_load_1d(dst, d.w_tiled + t * kATileBytes, (uint32_t)nk * kATileBytes, full, pol_stream);
+                    } else {
+                        for (int k = 0; k < nk; ++k)
+                            tma_load_2d(dst + k * kATileBytes, &maps.w[c.g], (c.kb0() + k) * kBlockK,
+                                        (c.half ? d.up_row_offset : 0) + c.tile * kTileM, full, pol_stream);
+                    }
+                    __threadfence_block();
+                    ctl.a_issued = ++issued;     // the activation loader may now add its bytes to this stage
+                    c.advance(p);
+                    if (++s == p.stages) { s = 0; par ^= 1u; }
+                    t_idle = 0;
+                    continue;
+                }
+                // The ring is full: the consumers are busy with a tail or a barrier between two GEMMs.
+                // Weights do not depend on any of that, so pull the next ones from HBM into L2 now;
+                // when the ring moves again it refills at L2 speed.
+                if (prefetched < issued) {       // the ring overtook the prefetch cursor: catch up
+                    while (prefetched < issued && !cpf.done(p)) { cpf.advance(p); ++prefetched; }
+                }
+                if (!cpf.done(p) && prefetched < issued + (uint32_t)p.stages + (uint32_t)p.l2_ahead) {
+                    const GemmDesc &d = p.g[cpf.g];
+                    if (prefetched >= issued + (uint32_t)p.stages && d.w_tiled != nullptr) {
+                        const size_t t = (size_t)(cpf.tile + (cpf.half ? d.up_tile_offset : 0)) * d.kb_per_tile + cpf.kb0();
+                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(d.w_tiled + t * kATileBytes),
+                                     "r"((uint32_t)cpf.nk() * kATileBytes) : "memory");
+                    }
+                    cpf.advance(p);
+                    ++prefetched;
+                    continue;
+                }
+                __nanosleep(32);
+                if (t_idle == 0) t_idle = global_timer_ns();
+                else if (*abort_flag || global_timer_ns() - t_idle > kWaitLimitNs) { timed_out = true; break; }
+            }
+            // This CTA's weight stream has ended; its tail (partial-tile reduction, epilogue) and the
+            // hand-over to the next kernel leave HBM idle. Pull the first tiles that the CTA with this
+            // index will want in the next launch into L2 meanwhile.
+            if (p.next_items > 0 && p.next.w_tiled != nullptr && !timed_out) {
+                const GemmDesc &d = p.next;
+                const int ppt = pairs_per_tile(d), ipt = ppt * d.halves;
+                const Range r = cta_range(d);
+                const int end = min(r.end, r.begin + p.next_items);
+                for (int it = r.begin; it < end; ++it) {
+                    const int tile = it / ipt, q = it - tile * ipt, kp = q / d.halves, half = q - kp * d.halves;
+                    const int kb0 = kp * kPairK, nk = min(kPairK, d.kb_per_tile - kb0);
+                    const size_t t = (size_t)(tile + (half ? d.up_tile_offset : 0)) * d.kb_per_tile + kb0;
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(d.w_tiled + t * kATileBytes),
+                                 "r"((uint32_t)nk * kATileBytes) : "memory");
+                }
+            }
+        }
+    } else if (warp == 6) {
+        // ================================================= activation loader
+        // Follows the weight producer item by item and adds the (small, L2-resident) activation
+        // tiles of each item, but only once the GEMM that the item belongs to may read its input:
+        // after the grid dependency for the first GEMM, after the grid barrier for the others.
+        if (lane == 0) {
+            uint64_t pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-            // Phase 1, before the grid dependency resolves: fill the ring with weight tiles only.
-            int pre = 0;
-            {
-                UnitWalk w(u0, u1, p.kb_per_tile);
-                for (; pre < p.stages && w.next(); ++pre) {
-                    const uint32_t full = smem_u32(&ctl.full[pre]);
-                    const uint32_t dst = smem_base + pre * stage_bytes;
-                    mbar_expect_tx(full, stage_bytes);
-                    tma_load_2d(dst, &tm_w, w.kb * kBlockK, w.tile * kTileM, full, pol_stream);
-                    if (p.dual) tma_load_2d(dst + kATileBytes, &tm_w, w.kb * kBlockK, p.up_row_offset + w.tile * kTileM, full, pol_stream);
-                }
-            }
-            LLMCAD_TRACE(2);
+            Cursor c;
+            c.init(p);
+            int s = 0, ready = 0, traced_g = 0;
+            uint32_t i = 0;
             pdl_wait();
-            LLMCAD_TRACE(3);
-            // Phase 2: the activation tiles of the prefetched stages, then the steady state.
-            UnitWalk w(u0, u1, p.kb_per_tile);
-            for (uint32_t it = 0; w.next(); ++it) {
-                const int s = it % p.stages;
-                const uint32_t full = smem_u32(&ctl.full[s]);
-                const uint32_t dst = smem_base + s * stage_bytes;
-                if ((int)it >= pre) {
-                    const uint32_t par = ((it / p.stages) & 1u) ^ 1u;
-                    if (!mbar_wait(smem_u32(&ctl.empty[s]), par, abort_flag)) { timed_out = true; break; }
-                    mbar_expect_tx(full, stage_bytes);
-                    tma_load_2d(dst, &tm_w, w.kb * kBlockK, w.tile * kTileM, full, pol_stream);
-                    if (p.dual) tma_load_2d(dst + kATileBytes, &tm_w, w.kb * kBlockK, p.up_row_offset + w.tile * kTileM, full, pol_stream);
+            while (!c.done(p) && !timed_out) {
+                uint64_t t0 = 0;
+                // (1) the stage is ours: the producer has passed its "empty" wait and armed the barrier
+                for (uint32_t spin = 0; (int32_t)(ctl.a_issued - (i + 1)) < 0; ++spin) {
+                    __nanosleep(32);
+                    if ((spin & 255u) == 255u) {
+                        if (t0 == 0) t0 = global_timer_ns();
+                        if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) { timed_out = true; break; }
+                    }
                 }
-                tma_load_2d(dst + n_acc * kATileBytes, &tm_x, w.kb * kBlockK, 0, full, pol_keep);
+                // (2) the GEMM's input is final on every CTA
+                while (!timed_out && c.g > ready) {
+                    const uint32_t have = ld_acquire_u32(p.grid_counter) - p.barrier_base;
+                    ready = (int)(have / arrivals_per_gemm);       // GEMMs 0..ready-1 are complete everywhere
+                    if (c.g > ready) {
+                        __nanosleep(100);
+                        if (t0 == 0) t0 = global_timer_ns();
+                        if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) timed_out = true;
+                    }
+                }
+                if (timed_out) break;
+                if (c.g != traced_g) { traced_g = c.g; if (c.g >= 1 && c.g <= 3) LLMCAD_TRACE(12 + c.g); }
+                const uint32_t full = smem_u32(&ctl.full[s]);
+                const uint32_t dst = smem_base + s * stage_bytes + b_off;
+                const int nk = c.nk();
+                for (int k = 0; k < nk; ++k)
+                    tma_load_2d(dst + k * b_tile_bytes, &maps.x[c.g], (c.kb0() + k) * kBlockK, 0, full, pol_keep);
+                c.advance(p);
+                ++i;
+                if (++s == p.stages) s = 0;
             }
-            LLMCAD_TRACE(4);
+        } else {
+            pdl_wait();
         }
     } else if (warp == 1) {
         // ================================================= MMA issuer
         if (lane == 0) {
             const uint32_t idesc = make_idesc(kTileM, p.n_pad);
-            uint32_t it = 0, seg = 0;
-            for (long long hi = u1; hi > u0 && !timed_out; ++seg) {
-                const int tile = (int)((hi - 1) / p.kb_per_tile);
-                const long long lo = max(u0, (long long)tile * p.kb_per_tile);
-                const int kb0 = (int)(lo - (long long)tile * p.kb_per_tile), kb1 = (int)(hi - (long long)tile * p.kb_per_tile);
+            Cursor c;
+            c.init(p);
+            uint32_t seg = 0, ph = 0;   // ph: parity the MMA warp waits for on its stage's "full" barrier
+            int s = 0;
+            while (!c.done(p) && !timed_out) {
+                // one segment: the items of one tile that belong to this CTA
+                const int cg = c.g, tile = c.tile, halves = c.halves;
                 const int buf = seg & 1;
                 if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), ((seg >> 1) & 1u) ^ 1u, abort_flag)) { timed_out = true; break; }
                 tc_fence_after();
-                const uint32_t d0 = tmem_base + (uint32_t)(buf * n_acc * p.n_pad);
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                    const int s = it % p.stages;
-                    if (!mbar_wait(smem_u32(&ctl.full[s]), (it / p.stages) & 1u, abort_flag)) { timed_out = true; break; }
-                    if (it == 0) LLMCAD_TRACE(5);
+                const uint32_t d0 = tmem_base + buf * acc_cols;
+                for (int q = 0; c.g == cg && c.tile == tile; ++q) {
+                    if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) { timed_out = true; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * stage_bytes;
-                    const uint64_t a_desc = make_smem_desc(a_addr);
-                    const uint64_t b_desc = make_smem_desc(a_addr + n_acc * kATileBytes);
+                    // segments of a two-half GEMM start on a gate item, so the first `halves` items
+                    // of a segment are the ones that must overwrite their accumulator
+                    const uint32_t dcol = d0 + c.half * p.n_pad;
+                    const int nk = c.nk();
+                    for (int k = 0; k < nk; ++k) {
+                        const uint64_t a_desc = make_smem_desc(a_addr + k * kATileBytes);
+                        const uint64_t b_desc = make_smem_desc(a_addr + b_off + k * b_tile_bytes);
 #pragma unroll
-                    for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
-                        const uint32_t acc = (kb > kb0 || k4 > 0) ? 1u : 0u;
-                        // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the >>4 address field
-                        tc_mma_bf16(d0, a_desc + 2 * k4, b_desc + 2 * k4, idesc, acc);
-                        if (p.dual) {
-                            const uint64_t a2_desc = make_smem_desc(a_addr + kATileBytes);
-                            tc_mma_bf16(d0 + p.n_pad, a2_desc + 2 * k4, b_desc + 2 * k4, idesc, acc);
+                        for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
+                            // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the >>4 address field
+                            tc_mma_bf16(dcol, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (q >= halves || k > 0 || k4 > 0) ? 1u : 0u);
                         }
                     }
                     tc_commit(smem_u32(&ctl.empty[s]));  // frees the stage when these MMAs have read it
+                    c.advance(p);
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
                 if (timed_out) break;
                 tc_commit(smem_u32(&ctl.tmem_full[buf]));
-                hi = lo;
+                ++seg;
             }
-            LLMCAD_TRACE(6);
         }
     } else {
         // ================================================= epilogue (warps 2..5)
         const int lane_grp = warp & 3;                 // TMEM lanes 32*lane_grp .. +31 belong to this warp
         const int row_in_tile = lane_grp * 32 + lane;
-        const int et = (warp - 2) * 32 + lane;         // 0..127 among the epilogue threads
-        const EpiParams &ep = p.ep;
+        float *my_rs = ctl.rs[warp - 2];
         pdl_wait();
-        // RMSNorm of the GEMM input folded into the epilogue: the producer of the residual stream
-        // left partial sums of squares per node; acc * rsqrt(mean(x^2) + eps) is applied to the
-        // complete sums below. Done once per CTA while the main loop is still filling the pipe.
-        if (ep.ssq_in != nullptr) {
-            float ss = 0.f;
-            for (int t = 0; t < ep.ssq_in_parts; ++t) ss += __ldcg(ep.ssq_in + (size_t)t * LLMCAD_MAX_TREE + et);
-            ctl.rs[et] = rsqrtf(ss / (float)ep.norm_d + ep.eps);
-            asm volatile("bar.sync 1, 128;" ::: "memory");   // all four epilogue warps get here unconditionally
-        }
+        if (threadIdx.x == 64) LLMCAD_TRACE(3);
         uint32_t seg = 0;
-        for (long long hi = u1; hi > u0 && !timed_out; ++seg) {
-            const int tile = (int)((hi - 1) / p.kb_per_tile);
-            const long long tile_u0 = (long long)tile * p.kb_per_tile;
-            const long long lo = max(u0, tile_u0);
-            const int kb0 = (int)(lo - tile_u0), kb1 = (int)(hi - tile_u0);
-            const int buf = seg & 1;
-            const bool sole = (kb0 == 0 && kb1 == p.kb_per_tile);      // this CTA holds the whole tile
-            const int first_cta = (int)(tile_u0 / p.units_per_cta);
-            const int last_cta = (int)((tile_u0 + p.kb_per_tile - 1) / p.units_per_cta);
-            const int n_parts = last_cta - first_cta + 1;
-            const size_t part_stride = (size_t)n_acc * p.n_pad * kTileM;  // floats per partial slot
-
-            if (!mbar_wait(smem_u32(&ctl.tmem_full[buf]), (seg >> 1) & 1u, abort_flag)) { timed_out = true; break; }
-            tc_fence_after();
-            if (threadIdx.x == 64) LLMCAD_TRACE(lo == u0 ? 8 : 7);   // 7: first segments, 8: the last one
-
-            const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(buf * n_acc * p.n_pad);
-            const int row = tile * kTileM + row_in_tile;           // output feature (weight row)
-            const bool row_ok = row < ep.n_out;
-            bool finish = sole;
-
-            if (!sole) {
-                // A tile shared by several CTAs: every sharer leaves its partial accumulator in the
-                // workspace; the rows of a tile are independent per warp (32 rows each), so each
-                // warp takes a ticket for its own row group and the last warp to arrive adds all
-                // partials in CTA order and finishes those rows. Nobody waits for anybody.
-                // Slot 0 of a CTA holds the segment that contains its range start, slot 1 the other.
-                float *dst = p.partials + ((size_t)blockIdx.x * 2 + (lo == u0 ? 0 : 1)) * part_stride + row_in_tile;
-                for (int c0 = 0; c0 < n_acc * p.n_pad; c0 += 16) {
-                    float v[16];
-                    tc_ld16(t_lane + c0, v);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) dst[(size_t)(c0 + j) * kTileM] = v[j];
-                }
-                __threadfence();
-                __syncwarp();
-                int last = 0;
+        for (int g = 0; g < p.n_gemms && !timed_out; ++g) {
+            const GemmDesc &d = p.g[g];
+            const EpiParams &ep = d.ep;
+            // ---- grid barrier: everything GEMM g-1 wrote (activations, residual, norm sums) is final
+            if (g > 0) {
+                int bad = 0;
                 if (lane == 0) {
-                    uint32_t *ctr = p.tickets + (size_t)tile * 4 + lane_grp;
-                    last = (atomicAdd(ctr, 1u) == (uint32_t)n_parts - 1u);
-                    if (last) { *ctr = 0; __threadfence(); }
+                    const uint32_t target = arrivals_per_gemm * (uint32_t)g;
+                    const uint64_t t0 = global_timer_ns();
+                    for (uint32_t spin = 0; (int32_t)(ld_acquire_u32(p.grid_counter) - p.barrier_base - target) < 0; ++spin) {
+                        __nanosleep(100);
+                        if ((spin & 15u) == 15u && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) { bad = 1; break; }
+                    }
+                    __threadfence();
                 }
-                finish = __shfl_sync(0xffffffffu, last, 0) != 0;
-                // the accumulator is in the workspace now: hand the TMEM buffer back early
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
-                if (threadIdx.x == 64) LLMCAD_TRACE(9);
+                if (__shfl_sync(0xffffffffu, bad, 0)) { timed_out = true; break; }
             }
+            // ---- RMSNorm of the GEMM input folded into the epilogue: the producer of the residual
+            // stream left partial sums of squares per node; every warp keeps its own copy of the
+            // per-node factors (no block-level barrier among the epilogue warps)
+            if (ep.ssq_in != nullptr) {
+                // rows of ssq_in hold 128 floats (one per node); read them as float4 "quads". A lane
+                // owns one quad and every (32 / quads)-th partial row, eight loads in flight at a time;
+                // the lane groups are then added in a fixed order, so the sum does not depend on timing.
+                int qp = 4;
+                while (qp * 4 < p.n_pad) qp <<= 1;                 // quads, rounded up to 4, 8, 16 or 32
+                const int groups = 32 / qp, quad = lane & (qp - 1), slice = lane / qp;
+                const float4 *rows = reinterpret_cast<const float4 *>(ep.ssq_in) + quad;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                int t = slice;
+                for (; t + 7 * groups < ep.ssq_in_parts; t += 8 * groups) {
+                    float4 v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v[u] = __ldcg(rows + (size_t)(t + u * groups) * (LLMCAD_MAX_TREE / 4));
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+                }
+                for (; t < ep.ssq_in_parts; t += groups) {
+                    const float4 v = __ldcg(rows + (size_t)t * (LLMCAD_MAX_TREE / 4));
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
+                for (int off = qp; off < 32; off <<= 1) {
+                    acc.x += __shfl_xor_sync(0xffffffffu, acc.x, off);
+                    acc.y += __shfl_xor_sync(0xffffffffu, acc.y, off);
+                    acc.z += __shfl_xor_sync(0xffffffffu, acc.z, off);
+                    acc.w += __shfl_xor_sync(0xffffffffu, acc.w, off);
+                }
+                if (lane < qp) {
+                    const float inv_d = 1.0f / (float)ep.norm_d;
+                    my_rs[4 * quad + 0] = rsqrtf(acc.x * inv_d + ep.eps);
+                    my_rs[4 * quad + 1] = rsqrtf(acc.y * inv_d + ep.eps);
+                    my_rs[4 * quad + 2] = rsqrtf(acc.z * inv_d + ep.eps);
+                    my_rs[4 * quad + 3] = rsqrtf(acc.w * inv_d + ep.eps);
+                }
+                __syncwarp();
+            }
+            const Range r = cta_range(d);
+            const int ipt = pairs_per_tile(d) * d.halves;
+            const bool dual = d.halves == 2;
+            const size_t part_stride = (size_t)2 * p.n_pad * kTileM;   // floats per partial slot (gate | up)
+            const int quads = p.n_pad >> 2;                            // column quads per accumulator
+            uint32_t *tickets = p.tickets + (size_t)g * kTicketsPerGemm;
+            for (int seg_begin = r.begin; seg_begin < r.end && !timed_out; ++seg) {
+                const int tile = seg_begin / ipt;
+                const int tile_i0 = tile * ipt;
+                const int seg_end = min(r.end, tile_i0 + ipt);
+                const int buf = seg & 1;
+                const bool sole = (seg_begin == tile_i0 && seg_end == tile_i0 + ipt);   // this CTA holds the whole tile
+                const int first_cta = tile_i0 / d.items_per_cta;
+                const int last_cta = (tile_i0 + ipt - 1) / d.items_per_cta;
+                const int n_parts = last_cta - first_cta + 1;
 
-            if (finish) {
-                float gain = 0.f;
-                if (ep.mode == EPI_RESID && ep.xg_out != nullptr && row_ok)
-                    gain = to_f32<T>(reinterpret_cast<const T *>(ep.gain_next)[row]);
-                for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
-                    float v[16], w[16];
-                    if (sole) {
+                if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), (seg >> 1) & 1u, abort_flag, lane)) { timed_out = true; break; }
+                tc_fence_after();
+                if (threadIdx.x == 64 && g < 4 && seg_begin == r.begin) LLMCAD_TRACE(4 + 2 * g);
+
+                const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * acc_cols;
+                const int row = tile * kTileM + row_in_tile;           // output feature (weight row)
+                const bool row_ok = row < ep.n_out;
+                bool finish = sole;
+
+                if (!sole) {
+                    // A tile shared by several CTAs: every sharer leaves its partial accumulator in the
+                    // workspace; the rows of a tile are independent per warp (32 rows each), so each
+                    // warp takes a ticket for its own row group and the last warp to arrive adds all
+                    // partials in CTA order and finishes those rows. Nobody waits for anybody.
+                    // Slot 0 of a CTA holds the segment that contains its range start, slot 1 the other.
+                    // Slot layout: [row group][gate|up][column quad][row 0..31][4 columns], so a lane
+                    // moves 16 bytes per access and a warp 512 contiguous bytes.
+                    float4 *dst = reinterpret_cast<float4 *>(p.partials + ((size_t)blockIdx.x * 2 + (seg_begin == r.begin ? 0 : 1)) * part_stride) +
+                                  (size_t)lane_grp * 2 * quads * 32 + lane;
+                    const int ncol = dual ? 2 * p.n_pad : p.n_pad;
+                    for (int c0 = 0; c0 < ncol; c0 += 16) {
+                        float v[16];
                         tc_ld16(t_lane + c0, v);
-                        if (p.dual) tc_ld16(t_lane + p.n_pad + c0, w);
-                    } else {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) v[j] = w[j] = 0.f;
-                        // partial tiles in CTA order, two CTAs' loads in flight at a time
-                        for (int c = first_cta; c <= last_cta; c += 2) {
-                            const bool two = c + 1 <= last_cta;
-                            const int slot0 = ((long long)c * p.units_per_cta >= tile_u0) ? 0 : 1;
-                            const int slot1 = ((long long)(c + 1) * p.units_per_cta >= tile_u0) ? 0 : 1;
-                            const float *s0 = p.partials + ((size_t)c * 2 + slot0) * part_stride + (size_t)c0 * kTileM + row_in_tile;
-                            const float *s1 = two ? p.partials + ((size_t)(c + 1) * 2 + slot1) * part_stride + (size_t)c0 * kTileM + row_in_tile : s0;
-                            float a0[16], a1[16];
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) { a0[j] = __ldcg(s0 + (size_t)j * kTileM); a1[j] = __ldcg(s1 + (size_t)j * kTileM); }
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) { v[j] += a0[j]; if (two) v[j] += a1[j]; }
-                            if (p.dual) {
-                                s0 += (size_t)p.n_pad * kTileM;
-                                s1 += (size_t)p.n_pad * kTileM;
-#pragma unroll
-                                for (int j = 0; j < 16; ++j) { a0[j] = __ldcg(s0 + (size_t)j * kTileM); a1[j] = __ldcg(s1 + (size_t)j * kTileM); }
-#pragma unroll
-                                for (int j = 0; j < 16; ++j) { w[j] += a0[j]; if (two) w[j] += a1[j]; }
-                            }
-                        }
+                        for (int k = 0; k < 4; ++k)
+                            dst[(size_t)((c0 >> 2) + k) * 32] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
                     }
-                    if (ep.ssq_in != nullptr) {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) { const float r = ctl.rs[c0 + j]; v[j] *= r; w[j] *= r; }
+                    __threadfence();
+                    __syncwarp();
+                    int last = 0;
+                    if (lane == 0) {
+                        uint32_t *ctr = tickets + (size_t)tile * 4 + lane_grp;
+                        last = (atomicAdd(ctr, 1u) == (uint32_t)n_parts - 1u);
+                        if (last) { __threadfence(); *ctr = 0; }   // acquire side; the counter is ready for the next launch
                     }
-                    // fused epilogue on complete sums; all loads of a 16-column chunk are issued before
-                    // any dependent store so that they overlap instead of queueing behind each other
-                    if (ep.mode == EPI_SWIGLU) {
-                        T *hrow = reinterpret_cast<T *>(ep.h) + row;
+                    finish = __shfl_sync(0xffffffffu, last, 0) != 0;
+                    // the accumulator is in the workspace now: hand the TMEM buffer back early
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+                }
+
+                if (finish) {
+                    float gain = 0.f;
+                    if (ep.mode == EPI_RESID && ep.xg_out != nullptr && row_ok)
+                        gain = to_f32<T>(reinterpret_cast<const T *>(ep.gain_next)[row]);
+                    for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                        float v[16], w[16], xo[16];
+                        if (ep.mode == EPI_RESID) {
+                            // issued first so that it overlaps the partial-tile loads below
+                            const float *xr = ep.x + row;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            if (row_ok && c0 + j < ep.n) {
-                                const float sg = v[j] / (1.0f + __expf(-v[j]));
-                                hrow[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(sg * w[j]);
+                            for (int j = 0; j < 16; ++j) xo[j] = (row_ok && c0 + j < ep.n) ? __ldcg(xr + (size_t)(c0 + j) * ep.n_out) : 0.f;
+                        }
+                        if (sole) {
+                            tc_ld16(t_lane + c0, v);
+                            if (dual) tc_ld16(t_lane + p.n_pad + c0, w);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) v[j] = w[j] = 0.f;
+                            // partial tiles added in CTA order; the loads of several CTAs are in flight at a time
+                            const size_t lane_off = (size_t)lane_grp * 2 * quads * 32 + (size_t)(c0 >> 2) * 32 + lane;
+                            for (int hf = 0; hf < (dual ? 2 : 1); ++hf) {
+                                float *acc = hf ? w : v;
+                                constexpr int kBatch = 6;
+                                for (int c = first_cta; c <= last_cta; c += kBatch) {
+                                    float4 t[kBatch][4];
+#pragma unroll
+                                    for (int u = 0; u < kBatch; ++u) {
+                                        const int cc = min(c + u, last_cta);
+                                        const int slot = (cc * d.items_per_cta >= tile_i0) ? 0 : 1;
+                                        const float4 *src = reinterpret_cast<const float4 *>(p.partials + ((size_t)cc * 2 + slot) * part_stride) +
+                                                            lane_off + (size_t)hf * quads * 32;
+#pragma unroll
+                                        for (int k = 0; k < 4; ++k) t[u][k] = __ldcg(src + (size_t)k * 32);
+                                    }
+#pragma unroll
+                                    for (int u = 0; u < kBatch; ++u) {
+                                        if (c + u <= last_cta) {
+#pragma unroll
+                                            for (int k = 0; k < 4; ++k) {
+                                                acc[4 * k] += t[u][k].x; acc[4 * k + 1] += t[u][k].y;
+                                                acc[4 * k + 2] += t[u][k].z; acc[4 * k + 3] += t[u][k].w;
+                                            }
+                                        }
+                                    }
+                                }
                             }
                         }
-                    } else if (ep.mode == EPI_QKV) {
-                        const int sec = row / ep.d, cidx = row - sec * ep.d;
-                        const int head = cidx / ep.hd, e = cidx - head * ep.hd;
-                        float2 cs[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            cs[j] = (sec < 2 && row_ok && c0 + j < ep.n) ? __ldg(ep.rope_cs + (size_t)(c0 + j) * (ep.hd >> 1) + (e >> 1))
-                                                                          : make_float2(1.f, 0.f);
-                        T *dst;
-                        size_t node_stride;
-                        if (sec == 0) { dst = reinterpret_cast<T *>(ep.q_out) + cidx; node_stride = ep.d; }
-                        else { dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P) * ep.hd + e; node_stride = ep.hd; }
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            // the rotary partner (2t <-> 2t+1) lives in the neighbouring lane
-                            const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
-                            const float rot = (lane & 1) ? (other * cs[j].y + v[j] * cs[j].x) : (v[j] * cs[j].x - other * cs[j].y);
-                            if (row_ok && c0 + j < ep.n) dst[(size_t)(c0 + j) * node_stride] = from_f32<T>(rot);
-                        }
-                    } else if (ep.mode == EPI_RESID) {
-                        float *xr = ep.x + row;
-                        float xo[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) xo[j] = (row_ok && c0 + j < ep.n) ? __ldcg(xr + (size_t)(c0 + j) * ep.n_out) : 0.f;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            xo[j] = (row_ok && c0 + j < ep.n) ? xo[j] + v[j] : 0.f;
-                            if (row_ok && c0 + j < ep.n) xr[(size_t)(c0 + j) * ep.n_out] = xo[j];
-                        }
-                        if (ep.xg_out != nullptr) {
-                            // what the next RMSNorm needs: gain * x in the GEMM input dtype, and this
-                            // warp's share (32 rows) of every node's sum of squares
-                            T *gr = reinterpret_cast<T *>(ep.xg_out) + row;
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (row_ok && c0 + j < ep.n) gr[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(xo[j] * gain);
-                            float mine = 0.f;
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                float sq = xo[j] * xo[j];
-#pragma unroll
-                                for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-                                if (lane == j) mine = sq;
-                            }
-                            if (lane < 16)
-                                ep.ssq_out[(size_t)(tile * 4 + lane_grp) * LLMCAD_MAX_TREE + c0 + lane] = mine;
-                        }
-                    } else {
-                        float *yr = ep.y + row;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (row_ok && c0 + j < ep.n) yr[(size_t)(c0 + j) * ep.ldy] = v[j];
+                        epilogue_chunk<T>(ep, my_rs, tile, lane_grp, lane, row, row_ok, gain, c0, v, w, xo);
                     }
                 }
+                if (sole) {
+                    // accumulator buffer drained: hand it back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+                }
+                seg_begin = seg_end;
             }
-            if (sole) {
-                // accumulator buffer drained: hand it back to the MMA warp
-                tc_fence_before();
+            if (timed_out) break;
+            if (threadIdx.x == 64 && g < 4) LLMCAD_TRACE(5 + 2 * g);
+            // ---- this warp is done with GEMM g: arrive at the grid barrier that gates GEMM g+1
+            if (g + 1 < p.n_gemms) {
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(p.grid_counter, 1u);
+                }
             }
-            hi = lo;
         }
-        if (threadIdx.x == 64) LLMCAD_TRACE(10);
     }
     __syncwarp();   // lanes that skipped their role's single-thread section rejoin their warp here
+    timed_out = __any_sync(0xffffffffu, timed_out);   // keep the warp together on the way out
 
     if (timed_out) {
         *abort_flag = 1;
@@ -515,9 +780,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     }
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) LLMCAD_TRACE(11);
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+        if (lane == 0) LLMCAD_TRACE(12);
     }
 }
 
@@ -555,49 +820,86 @@ bool make_tensor_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uin
     return r == CUDA_SUCCESS;
 }
 
-size_t gemm_tc_partial_floats(int n_sms, int max_n_pad) { return (size_t)n_sms * 2 /*slots*/ * 2 /*gate+up*/ * max_n_pad * kTileM; }
+size_t gemm_tc_partial_floats(int n_sms, int max_n_pad) { return (size_t)n_sms * 2 /*slots*/ * 2 /*gate|up*/ * max_n_pad * kTileM; }
 
-cudaError_t launch_gemm_tc(const CUtensorMap &tm_w, const CUtensorMap &tm_x, int n_in, int n_pad, int n_sms,
-                           float *partials, uint32_t *flags, uint32_t epoch, int32_t *status, const EpiParams &ep,
-                           cudaStream_t st, unsigned long long *trace)
+GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)
 {
-    TcGemmParams p;
-    p.dual = ep.mode == EPI_SWIGLU;
-    p.n_tiles = (ep.n_out + kTileM - 1) / kTileM;
-    if (p.n_tiles > 4096) return cudaErrorInvalidValue;   // size of the ticket array
-    p.kb_per_tile = (n_in + kBlockK - 1) / kBlockK;
-    p.n_pad = n_pad;
-    p.up_row_offset = ep.n_out;
-    const long long total = (long long)p.n_tiles * p.kb_per_tile;
-    int grid = (int)(total < n_sms ? total : n_sms);
-    p.units_per_cta = (int)((total + grid - 1) / grid);
-    grid = (int)((total + p.units_per_cta - 1) / p.units_per_cta);
-    const int n_acc = p.dual ? 2 : 1;
-    const size_t stage_bytes = (size_t)n_acc * kATileBytes + (size_t)n_pad * kBlockK * 2;
-    const size_t smem_limit = 227 * 1024 - 1024 /*alignment slack*/ - 2048 /*static*/;
-    int stages = (int)(smem_limit / stage_bytes);
-    if (stages > 16) stages = 16;
-    if (stages < 2) return cudaErrorInvalidConfiguration;
-    p.stages = stages;
-    int cols = 2 * n_acc * n_pad, pow2 = 32;
+    GemmDesc d{};
+    d.halves = ep.mode == EPI_SWIGLU ? 2 : 1;
+    d.n_tiles = (ep.n_out + kTileM - 1) / kTileM;
+    d.kb_per_tile = (n_in + kBlockK - 1) / kBlockK;
+    d.up_row_offset = ep.n_out;
+    d.items_per_cta = 0;
+    d.w_tiled = static_cast<const uint8_t *>(w_tiled);
+    d.up_tile_offset = d.n_tiles;
+    d.ep = ep;
+    return d;
+}
+
+cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, cudaStream_t st, uint32_t *barrier_arrivals,
+                              const GemmDesc *next)
+{
+    if (p.n_gemms < 1 || p.n_gemms > kMaxChain) return cudaErrorInvalidValue;
+    // a chain needs every CTA at every barrier: the grid is the SM count; a single GEMM may use fewer
+    long long max_items = 0;
+    auto items_of = [](const GemmDesc &d) { return (long long)d.n_tiles * ((d.kb_per_tile + kPairK - 1) / kPairK) * d.halves; };
+    for (int g = 0; g < p.n_gemms; ++g) {
+        if (p.g[g].n_tiles > 4096) return cudaErrorInvalidValue;   // size of the ticket array
+        const long long total = items_of(p.g[g]);
+        if (total > max_items) max_items = total;
+    }
+    int grid = n_sms;
+    if (p.n_gemms == 1 && max_items < grid) grid = (int)max_items;
+    for (int g = 0; g < p.n_gemms; ++g) {
+        const long long total = items_of(p.g[g]);
+        long long ipc = (total + grid - 1) / grid;
+        if (p.g[g].halves == 2) ipc += ipc & 1;   // ranges of a two-half GEMM start on a gate item
+        p.g[g].items_per_cta = (int)ipc;
+    }
+    if (p.n_gemms == 1) {
+        const long long total = items_of(p.g[0]);
+        grid = (int)((total + p.g[0].items_per_cta - 1) / p.g[0].items_per_cta);
+    }
+    const size_t stage_bytes = (size_t)kPairK * ((size_t)kATileBytes + (size_t)p.n_pad * kBlockK * 2);
+    // One CTA per SM with the whole shared memory as the ring. (Two CTAs per SM with half-size rings,
+    // so that the next kernel is resident during this one's tail, measured slower on B200.)
+    int cols = 4 * p.n_pad, pow2 = 32;
     while (pow2 < cols) pow2 <<= 1;
     p.tmem_cols = pow2;
-    p.partials = partials;
-    p.tickets = flags;
-    (void)epoch;
-    p.status = status;
-    p.trace = trace;
-    p.ep = ep;
+    const size_t full_limit = 227 * 1024 - 1024 /*alignment slack*/ - 4096 /*static*/;
+    int stages = (int)(full_limit / stage_bytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (const char *e = getenv("LLMCAD_GEMM_STAGES")) {   // tuning aid: cap the ring depth
+        const int cap = atoi(e);
+        if (cap >= 2 && cap < stages) stages = cap;
+    }
+    if (stages < 2) return cudaErrorInvalidConfiguration;
+    p.stages = stages;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             227 * 1024 - 2048);
+        cudaError_t e = cudaFuncSetAttribute(gemm_chain_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             227 * 1024 - 4096);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
+    // weight tiles pulled into L2 beyond the ring while the ring is blocked
+    p.l2_ahead = 8;
+    if (const char *e = getenv("LLMCAD_GEMM_L2_AHEAD")) p.l2_ahead = atoi(e);
+    // what the following launch will stream first (it uses the same grid and the same split)
+    p.next_items = 0;
+    if (next != nullptr && next->w_tiled != nullptr && grid == n_sms) {
+        p.next = *next;
+        const long long total = items_of(p.next);
+        long long ipc = (total + grid - 1) / grid;
+        if (p.next.halves == 2) ipc += ipc & 1;
+        p.next.items_per_cta = (int)ipc;
+        p.next_items = 12;                      // x 32 KB x 148 CTAs = 57 MB, under half of L2
+        if (const char *e = getenv("LLMCAD_GEMM_NEXT_ITEMS")) p.next_items = atoi(e);
+    }
+    if (barrier_arrivals) *barrier_arrivals = 4u * (uint32_t)grid * (uint32_t)(p.n_gemms - 1);
     LaunchCfg lc(grid, kThreads, smem, st);
-    return cudaLaunchKernelEx(&lc.cfg, gemm_tc_kernel<__nv_bfloat16>, tm_w, tm_x, p);
+    return cudaLaunchKernelEx(&lc.cfg, gemm_chain_kernel<__nv_bfloat16>, maps, p);
 }
 
 }  // namespace llmcad

@@ -1,4 +1,4 @@
-// Host-visible interface of the tensor-core skinny GEMM (gemm_tc.cu).
+// Host-visible interface of the tensor-core skinny-GEMM chain kernel (gemm_tc.cu).
 #pragma once
 
 #include <cuda.h>
@@ -7,20 +7,41 @@
 
 namespace llmcad {
 
-struct TcGemmParams {
+constexpr int kMaxChain = 4;
+
+// One GEMM of a chain: D[n_out][n] = W[n_out][n_in] X[n][n_in]^T followed by its fused epilogue.
+struct GemmDesc {
     int n_tiles;        // tiles of 128 output features
     int kb_per_tile;    // 64-wide k-blocks per tile
-    int n_pad;          // tree nodes padded to a multiple of 16 (the MMA N)
-    int dual;           // 1: every tile carries a gate and an up accumulator (SwiGLU)
+    int halves;         // 2: every tile carries a gate and an up accumulator (SwiGLU), else 1
     int up_row_offset;  // row of the first up-projection row in the packed [2f][d] matrix
-    int units_per_cta;  // (tile, k-block) units per CTA of the persistent grid
+    int items_per_cta;  // ring items ((tile, k-block, half) triples) per CTA of the persistent grid
+    const uint8_t *w_tiled;  // weights as a sequence of pre-swizzled 16 KB tiles [tile][k-block] (see pack.cu),
+                             // or nullptr: row-major weights through the tensor map
+    int up_tile_offset;      // first tile of the up projection in the tiled sequence
+    EpiParams ep;
+};
+
+struct ChainMaps {
+    CUtensorMap w[kMaxChain];  // weight matrices, box 64 x 128 rows
+    CUtensorMap x[kMaxChain];  // the activation matrix each GEMM multiplies, box 64 x n_pad rows
+};
+
+struct ChainParams {
+    int n_gemms;
+    int n_pad;          // tree nodes padded to a multiple of 16 (the MMA N)
     int stages;         // depth of the shared-memory ring
     int tmem_cols;      // allocated TMEM columns (power of two)
-    float *partials;    // [grid][2 slots][n_acc][n_pad][128] fp32 partial tiles
-    uint32_t *tickets;  // [n_tiles][4] arrivals per (tile, 32-row group); zero between launches
+    float *partials;    // [grid][2 slots][2 halves][n_pad][128] fp32 partial tiles
+    uint32_t *tickets;  // [kMaxChain][4096][4] arrivals per (GEMM, tile, 32-row group); zero between launches
+    uint32_t *grid_counter;   // grid barrier between the GEMMs of a chain (monotonic)
+    uint32_t barrier_base;    // value of the counter when this launch starts
     int32_t *status;
     unsigned long long *trace;  // optional [grid][16] timeline in ns (nullptr: off)
-    EpiParams ep;
+    int l2_ahead;       // ring items the producer may prefetch into L2 beyond the ring
+    int next_items;     // leading items of `next` (the GEMM of the following launch) each CTA pulls into L2 when its own stream ends
+    GemmDesc next;
+    GemmDesc g[kMaxChain];
 };
 
 // Tensor map over a row-major bf16 matrix [rows][cols] with a box of 64 columns x box_rows rows
@@ -28,9 +49,14 @@ struct TcGemmParams {
 bool make_tensor_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
 size_t gemm_tc_partial_floats(int n_sms, int max_n_pad);
+constexpr size_t kTicketsPerGemm = 4096 * 4;
 
-cudaError_t launch_gemm_tc(const CUtensorMap &tm_w, const CUtensorMap &tm_x, int n_in, int n_pad, int n_sms,
-                           float *partials, uint32_t *flags, uint32_t epoch, int32_t *status, const EpiParams &ep,
-                           cudaStream_t st, unsigned long long *trace = nullptr);
+// Describes one GEMM for a chain (fills everything but items_per_cta, which the launcher sets).
+GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled = nullptr);
+
+// Launches a chain of 1..kMaxChain dependent GEMMs as one persistent kernel. Returns in
+// *barrier_arrivals how far the grid counter advances (the caller adds it to its running base).
+cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, cudaStream_t st, uint32_t *barrier_arrivals,
+                              const GemmDesc *next = nullptr);
 
 }  // namespace llmcad

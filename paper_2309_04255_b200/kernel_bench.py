@@ -104,13 +104,15 @@ def bench_gemm(args):
         nbuf = max(2, int(2 * L2_BYTES // wbytes) + 1)
         g = torch.Generator(device=dev)
         g.manual_seed(gen.MASTER_SEED + n_out)
-        Ws = [(torch.randn((n_out, n_in), generator=g, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16) for _ in range(nbuf)]
+        Ws = []
+        for _ in range(nbuf):   # the layout the pass streams: pre-swizzled 16 KB tiles
+            Ws.append(v.tile_weight((torch.randn((n_out, n_in), generator=g, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)))
         x = torch.randn((n, n_in), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
-        us = time_launches(lambda i: v.skinny_gemm(Ws[i], x), nbuf, args.reps, args.warmup)
+        us = time_launches(lambda i: v.skinny_gemm_tiled(Ws[i], n_out, x), nbuf, args.reps, args.warmup)
         assert v.last_status() == 0
         v.set_kernel_timing(True)
         for i in range(args.reps):
-            v.skinny_gemm(Ws[i % nbuf], x)
+            v.skinny_gemm_tiled(Ws[i % nbuf], n_out, x)
         ms, cnt = v.get_kernel_timing(0)
         v.set_kernel_timing(False)
         k_us = ms * 1e3 / max(cnt, 1)

@@ -135,7 +135,7 @@ GEMM_SHAPES = [
 
 
 @pytest.mark.parametrize("shape", GEMM_SHAPES)
-@pytest.mark.parametrize("mode", ["f32", "bf16_simt", "bf16_tc"])
+@pytest.mark.parametrize("mode", ["f32", "bf16_simt", "bf16_tc", "bf16_tc_tiled"])
 def test_skinny_gemm(shape, mode):
     n_out, n_in, n = shape
     g = np.random.default_rng(n_out + n_in + n)
@@ -145,7 +145,10 @@ def test_skinny_gemm(shape, mode):
     td = torch.float32 if dtype == "f32" else torch.bfloat16
     W = torch.from_numpy(g.standard_normal((n_out, n_in), dtype=np.float32)).to(td)
     x = torch.from_numpy(g.standard_normal((n, n_in), dtype=np.float32)).to(td)
-    y = v.skinny_gemm(W.to(DEV), x.to(DEV))
+    if mode == "bf16_tc_tiled":     # the layout the pass itself streams (pre-swizzled 16 KB tiles)
+        y = v.skinny_gemm_tiled(v.tile_weight(W.to(DEV)), n_out, x.to(DEV))
+    else:
+        y = v.skinny_gemm(W.to(DEV), x.to(DEV))
     assert v.last_status() == 0
     ref = orc.linear(W, x.double())
     # inputs are identical on both sides and products are exact in fp32; only the order of the
