@@ -69,12 +69,21 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 
 }  // namespace
 
+// GROUPS key groups per CTA: warp w works on query tile w % q_tiles and on the keys
+// [g * 64/GROUPS, (g+1) * 64/GROUPS) of every 64-key tile, g = w / q_tiles. With few tree nodes
+// (n <= 32: two query tiles) a single warp per query tile would leave most of the SM idle and its
+// dependent mma chain would set the pace; splitting the keys of a tile over four warps cuts the
+// per-tile latency four-fold. Each warp keeps its own running softmax; the groups are merged in
+// shared memory at the end, then the cluster merges the splits.
+template <int GROUPS>
 __global__ void __launch_bounds__(kAtThreads)
 attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
                     const __nv_bfloat16 *__restrict__ v, int n_heads, int kv_stride, int P, int n, int n_pad,
                     const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
                     const int32_t *status, unsigned long long *trace)
 {
+    constexpr int KW = kKeyTile / GROUPS;     // keys per warp per tile: 64, 32 or 16
+    constexpr int NT = KW / 8;                // 8-key score tiles per warp per tile
     const int cta = blockIdx.y * gridDim.x + blockIdx.x;
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 0] = global_timer_ns();
     pdl_launch_dependents();
@@ -108,7 +117,7 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         }
     };
 
-    // queries of this head (rows >= n are zero) and the first key tile
+    // queries of this head (rows >= n are zero) and the first key tiles
     for (int c = tid; c < n_pad * 16; c += kAtThreads) {
         const int r = c >> 4, ch = c & 15;
         const bool ok = r < n;
@@ -120,8 +129,9 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     }
 
     const int q_tiles = n_pad >> 4;
-    const bool active = warp < q_tiles;
-    const int row0 = warp * 16 + (lane >> 2), row1 = row0 + 8;   // the two query rows this thread holds
+    const int qt = warp % q_tiles, kg = warp / q_tiles;
+    const bool active = kg < GROUPS;
+    const int row0 = qt * 16 + (lane >> 2), row1 = row0 + 8;   // the two query rows this thread holds
     uint32_t anc0[4] = {0, 0, 0, 0}, anc1[4] = {0, 0, 0, 0};
     if (active) {
         for (int w = 0; w < 4; ++w) {
@@ -141,38 +151,40 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         const int buf = (t - t_begin) % kStages;
         cp_wait<kStages - 2>();
         __syncthreads();                       // tile t (and Q) visible; everyone is done with tile t-1's buffer
+        if (trace && threadIdx.x == 0 && cta < 256 && t == t_begin) trace[(size_t)cta * 16 + 2] = global_timer_ns();
         if (t + kStages - 1 < t_end) load_tile(t + kStages - 1, (t + kStages - 1 - t_begin) % kStages);
         cp_commit();
         if (t == t_begin && active) {
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-                ldsm4(smem_u32(s_q) + swz(warp * 16 + (lane & 15), ks * 2 + (lane >> 4)), qf[ks]);
+                ldsm4(smem_u32(s_q) + swz(qt * 16 + (lane & 15), ks * 2 + (lane >> 4)), qf[ks]);
         }
         if (!active) continue;
         const uint32_t kb = smem_u32(s_k) + buf * kKeyTile * kRowBytes;
         const uint32_t vb = smem_u32(s_v) + buf * kKeyTile * kRowBytes;
+        const int key_off = kg * KW;           // this warp's keys inside the tile
 
-        // ---- S = Q K^T for 64 keys: 8 n-tiles of 8 keys
-        float s[8][4];
+        // ---- S = Q K^T for this warp's KW keys: NT score tiles of 8 keys
+        float s[NT][4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+        for (int j = 0; j < NT; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
 #pragma unroll
-            for (int np = 0; np < 4; ++np) {
+            for (int np = 0; np < NT / 2; ++np) {
                 uint32_t b[4];
-                const int key = np * 16 + (lane & 7) + ((lane >> 4) << 3);
+                const int key = key_off + np * 16 + (lane & 7) + ((lane >> 4) << 3);
                 ldsm4(kb + swz(key, ks * 2 + ((lane >> 3) & 1)), b);
                 mma_bf16(s[2 * np], qf[ks], b[0], b[1]);
                 mma_bf16(s[2 * np + 1], qf[ks], b[2], b[3]);
             }
         }
         // ---- scale, mask (tree region and the ragged end only), online softmax
-        const int key_base = t * kKeyTile;
-        const bool needs_mask = key_base + kKeyTile > P;
+        const int key_base = t * kKeyTile + key_off;
+        const bool needs_mask = key_base + KW > P;
         float tmax0 = -INFINITY, tmax1 = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < NT; ++j) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 float val = s[j][e] * scale_log2;
@@ -199,9 +211,9 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         const float alpha0 = exp2f(m0 - ref0), alpha1 = exp2f(m1 - ref1);
         m0 = mn0; m1 = mn1;
         float rs0 = 0.f, rs1 = 0.f;
-        uint32_t pa[4][4];
+        uint32_t pa[NT / 2][4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < NT; ++j) {
             const float p0 = exp2f(s[j][0] - ref0), p1 = exp2f(s[j][1] - ref0);
             const float p2 = exp2f(s[j][2] - ref1), p3 = exp2f(s[j][3] - ref1);
             rs0 += p0 + p1; rs1 += p2 + p3;
@@ -211,13 +223,13 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         l0 = l0 * alpha0 + rs0; l1 = l1 * alpha1 + rs1;
 #pragma unroll
         for (int j = 0; j < 16; ++j) { oacc[j][0] *= alpha0; oacc[j][1] *= alpha0; oacc[j][2] *= alpha1; oacc[j][3] *= alpha1; }
-        // ---- O += P V: k = 64 keys (4 steps of 16), n = 128 dims (8 pairs of n-tiles)
+        // ---- O += P V: k = KW keys (steps of 16), n = 128 dims (8 pairs of n-tiles)
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
+        for (int kk = 0; kk < NT / 2; ++kk) {
 #pragma unroll
             for (int dp = 0; dp < 8; ++dp) {
                 uint32_t b[4];
-                const int key = kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                const int key = key_off + kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
                 ldsm4_t(vb + swz(key, dp * 2 + (lane >> 4)), b);
                 mma_bf16(oacc[2 * dp], pa[kk], b[0], b[1]);
                 mma_bf16(oacc[2 * dp + 1], pa[kk], b[2], b[3]);
@@ -225,42 +237,78 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         }
     }
     cp_wait<0>();
+    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 3] = global_timer_ns();
 
     // ---- row sums over the four threads of a row
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
 
-    if (splits == 1) {
-        if (active) {
-            const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+    // ---- every warp leaves its unnormalised partial (outputs, max, sum) in shared memory (the
+    // K/V ring is done): wpart[kg][row][130]; the merged partial of the CTA goes to part[row][130]
+    __syncthreads();
+    float *wpart = reinterpret_cast<float *>(sm);
+    float *part = (GROUPS > 1) ? wpart + (size_t)GROUPS * n_pad * kWsRow : wpart;
+    if (active) {
+        float *wp = wpart + (size_t)kg * n_pad * kWsRow;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int dim = j * 8 + ((lane & 3) << 1);
-                if (row0 < n) *reinterpret_cast<uint32_t *>(o + ((size_t)row0 * n_heads + head) * kHd + dim) = pack_bf16(oacc[j][0] * i0, oacc[j][1] * i0);
-                if (row1 < n) *reinterpret_cast<uint32_t *>(o + ((size_t)row1 * n_heads + head) * kHd + dim) = pack_bf16(oacc[j][2] * i1, oacc[j][3] * i1);
+        for (int j = 0; j < 16; ++j) {
+            const int dim = j * 8 + ((lane & 3) << 1);
+            *reinterpret_cast<float2 *>(wp + (size_t)row0 * kWsRow + dim) = make_float2(oacc[j][0], oacc[j][1]);
+            *reinterpret_cast<float2 *>(wp + (size_t)row1 * kWsRow + dim) = make_float2(oacc[j][2], oacc[j][3]);
+        }
+        if ((lane & 3) == 0) {
+            *reinterpret_cast<float2 *>(wp + (size_t)row0 * kWsRow + kHd) = make_float2(m0, l0);
+            *reinterpret_cast<float2 *>(wp + (size_t)row1 * kWsRow + kHd) = make_float2(m1, l1);
+        }
+    }
+    if (GROUPS > 1) {
+        __syncthreads();
+        // merge the key groups of this CTA: out = sum_g O_g 2^(m_g - M), l = sum_g l_g 2^(m_g - M).
+        // First the per-(row, group) weights, once; then every thread combines float4 columns.
+        float *wgt = part + (size_t)n_pad * kWsRow;           // [n_pad][GROUPS]
+        for (int row = tid; row < n_pad; row += kAtThreads) {
+            float mg[GROUPS], M = -INFINITY, L = 0.f;
+#pragma unroll
+            for (int g = 0; g < GROUPS; ++g) { mg[g] = wpart[((size_t)g * n_pad + row) * kWsRow + kHd]; M = fmaxf(M, mg[g]); }
+#pragma unroll
+            for (int g = 0; g < GROUPS; ++g) {
+                const float w = (mg[g] == -INFINITY) ? 0.f : exp2f(mg[g] - M);
+                wgt[row * GROUPS + g] = w;
+                L += wpart[((size_t)g * n_pad + row) * kWsRow + kHd + 1] * w;
             }
+            *reinterpret_cast<float2 *>(part + (size_t)row * kWsRow + kHd) = make_float2(M, L);
+        }
+        __syncthreads();
+        for (int idx = tid; idx < n_pad * (kHd / 2); idx += kAtThreads) {
+            const int row = idx / (kHd / 2), c = (idx % (kHd / 2)) * 2;    // rows are 520 bytes: 8-byte accesses
+            float2 a = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int g = 0; g < GROUPS; ++g) {
+                const float2 vv = *reinterpret_cast<const float2 *>(wpart + ((size_t)g * n_pad + row) * kWsRow + c);
+                const float w = wgt[row * GROUPS + g];
+                a.x += vv.x * w; a.y += vv.y * w;
+            }
+            *reinterpret_cast<float2 *>(part + (size_t)row * kWsRow + c) = a;
+        }
+    }
+
+    if (splits == 1) {
+        __syncthreads();
+        for (int idx = tid; idx < n * (kHd / 2); idx += kAtThreads) {
+            const int row = idx / (kHd / 2), dim = (idx % (kHd / 2)) * 2;
+            const float L = part[(size_t)row * kWsRow + kHd + 1];
+            const float inv = L > 0.f ? 1.f / L : 0.f;
+            const float2 ov = *reinterpret_cast<const float2 *>(part + (size_t)row * kWsRow + dim);
+            *reinterpret_cast<uint32_t *>(o + ((size_t)row * n_heads + head) * kHd + dim) = pack_bf16(ov.x * inv, ov.y * inv);
         }
         if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
         return;
     }
 
-    // ---- partial result of this split, left in this CTA's shared memory (the K/V ring is done)
-    __syncthreads();
-    float *part = reinterpret_cast<float *>(sm);            // [n_pad][kWsRow]
-    if (active) {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int dim = j * 8 + ((lane & 3) << 1);
-            *reinterpret_cast<float2 *>(part + (size_t)row0 * kWsRow + dim) = make_float2(oacc[j][0], oacc[j][1]);
-            *reinterpret_cast<float2 *>(part + (size_t)row1 * kWsRow + dim) = make_float2(oacc[j][2], oacc[j][3]);
-        }
-        if ((lane & 3) == 0) {
-            *reinterpret_cast<float2 *>(part + (size_t)row0 * kWsRow + kHd) = make_float2(m0, l0);
-            *reinterpret_cast<float2 *>(part + (size_t)row1 * kWsRow + kHd) = make_float2(m1, l1);
-        }
-    }
+    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 4] = global_timer_ns();
     cg::cluster_group cluster = cg::this_cluster();
     cluster.sync();                                          // all partials of this head are written
+    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 5] = global_timer_ns();
     // ---- merge rows split, split + splits, ...: out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M)
     const float *peer[kMaxSplits];
 #pragma unroll
@@ -291,6 +339,7 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         const float inv = L > 0.f ? 1.f / L : 0.f;
         *reinterpret_cast<uint32_t *>(o + ((size_t)row * n_heads + head) * kHd + dim) = pack_bf16(a0 * inv, a1 * inv);
     }
+    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 6] = global_timer_ns();
     cluster.sync();                                          // peers may still be reading this CTA's partial
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
 }
@@ -316,19 +365,24 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     if (splits < 1) splits = 1;
     const int tiles_per_split = (n_tiles + splits - 1) / splits;
     splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
+    const int q_tiles = n_pad / 16;
+    const int groups = q_tiles <= 2 ? 4 : (q_tiles <= 4 ? 2 : 1);
     const size_t ring = (size_t)n_pad * kRowBytes + 2 * kStages * kKeyTile * kRowBytes;
-    const size_t part = (size_t)n_pad * kWsRow * sizeof(float);
+    const size_t part = (size_t)(groups > 1 ? groups + 1 : 1) * n_pad * kWsRow * sizeof(float) + (size_t)n_pad * groups * sizeof(float);
     const size_t smem = ring > part ? ring : part;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             128 * kRowBytes + 2 * kStages * kKeyTile * kRowBytes);
+        const int max_smem = 128 * kRowBytes + 2 * kStages * kKeyTile * kRowBytes;
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     LaunchCfg lc(dim3(splits, n_heads), dim3(kAtThreads), smem, st, splits);
     if (launched) *launched = 1;
-    return cudaLaunchKernelEx(&lc.cfg, attention_tc_kernel, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
+    auto kern = groups == 4 ? attention_tc_kernel<4> : (groups == 2 ? attention_tc_kernel<2> : attention_tc_kernel<1>);
+    return cudaLaunchKernelEx(&lc.cfg, kern, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                               (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc, (__nv_bfloat16 *)o, splits,
                               tiles_per_split, status, trace);
 }
