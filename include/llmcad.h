@@ -240,6 +240,34 @@ int llmcad_tile_weight(const void *w, int32_t n_out, int32_t n_in, void *tiled /
 int llmcad_skinny_gemm_tiled(llmcad_ctx *ctx, const void *w_tiled, const void *x, float *y, int32_t n_out, int32_t n_in,
                              int32_t n, void *stream);
 
+/* Tree attention without any allocation. (The paper has no counterpart: this entry point exists
+ * for the way the library is embedded, not for the method.)
+ *
+ * Who needs it: code that may not allocate device memory -- a plug-in loaded into a server that
+ * gave the whole device to its own memory pool at start-up, or a latency-critical loop where a
+ * device-synchronising cudaMalloc is not allowed. llmcad_tree_attention() needs a context, and
+ * llmcad_create() allocates; this variant needs no context and calls no cudaMalloc, cudaFree or
+ * other allocating routine, ever. Its scratch (per-node depth, position, ancestor bit rows, a
+ * status word: 4 KB) is a static device array inside the library image; every GPU that loads the
+ * library holds those 4 KB until the process exits.
+ *
+ * Same computation and layouts as llmcad_tree_attention, bf16, head_dim 128 only:
+ * q, o [n][n_heads][128]; k, v [n_heads][kv_stride][128]; parent_idx int32[n]; all DEVICE,
+ * caller-owned. status_out (DEVICE int32, may be NULL) receives 0 or LLMCAD_ERR_BAD_TREE.
+ * Limits: n <= 128 (what the static scratch holds) -- larger n is refused with
+ * LLMCAD_ERR_UNSUPPORTED and a message in llmcad_noalloc_last_error(); n_heads <= 65535.
+ *
+ * The first call on a device looks up the device address of the static array (with that device
+ * current); make that first call before starting any stream capture. All calls share the one
+ * array, which keeps the previous call's contents (the status word is cleared on the stream at
+ * the start of every call): two calls whose work overlaps on the GPU -- different streams
+ * without ordering, or several host threads -- race on it. Calls on one stream are safe.
+ * Asynchronous on `stream`. */
+int llmcad_tree_attention_noalloc(const void *q, const void *k, const void *v, int32_t n_heads, int32_t kv_stride,
+                                  int32_t prefix_len, const int32_t *parent_idx, int32_t n, void *o,
+                                  int32_t *status_out, void *stream);
+const char *llmcad_noalloc_last_error(void);
+
 /* Number of kernels this library has launched through this context so far. */
 int64_t llmcad_launch_count(const llmcad_ctx *ctx);
 

@@ -29,7 +29,7 @@ EXPORTS = [
     "llmcad_kv_cache_bytes", "llmcad_packed_weight_bytes", "llmcad_pack_layer", "llmcad_pack_globals",
     "llmcad_verify_tree", "llmcad_verify_tree_host", "llmcad_prefill", "llmcad_tree_prep",
     "llmcad_accept_compact", "llmcad_tree_attention", "llmcad_skinny_gemm", "llmcad_launch_count",
-    "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace", "llmcad_tiled_weight_bytes", "llmcad_tile_weight", "llmcad_skinny_gemm_tiled",
+    "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace", "llmcad_tiled_weight_bytes", "llmcad_tile_weight", "llmcad_skinny_gemm_tiled", "llmcad_tree_attention_noalloc", "llmcad_noalloc_last_error",
 ]
 
 
@@ -101,6 +101,8 @@ def lib():
         L.llmcad_tiled_weight_bytes.restype = sz
         L.llmcad_tile_weight.argtypes = [vp, i32, i32, vp, vp]
         L.llmcad_skinny_gemm_tiled.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
+        L.llmcad_tree_attention_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, vp, i32, vp, vp, vp]
+        L.llmcad_noalloc_last_error.restype = C.c_char_p
         L.llmcad_set_kernel_timing.argtypes = [vp, i32]
         L.llmcad_get_kernel_timing.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         _lib = L
@@ -269,6 +271,17 @@ class Verifier:
 
     def launch_count(self) -> int:
         return lib().llmcad_launch_count(self.ctx)
+
+
+def tree_attention_noalloc(q, k, v, prefix_len: int, parent, o, status=None):
+    """Context-free tree attention on caller-provided buffers (the library allocates nothing):
+    q, o [n][H][128] bf16; k, v [H][kv_stride][128] bf16; parent int32[n]; status int32[1] or None."""
+    n, H = q.shape[0], q.shape[1]
+    code = lib().llmcad_tree_attention_noalloc(_ptr(q), _ptr(k), _ptr(v), H, k.shape[1], prefix_len, _ptr(parent), n, _ptr(o),
+                                               _ptr(status), _stream())
+    if code != OK:
+        raise LlmcadError(code, "llmcad_tree_attention_noalloc: " + lib().llmcad_noalloc_last_error().decode())
+    return o
 
 
 def tree_prep(parent: torch.Tensor, prefix_len: int):

@@ -1,0 +1,64 @@
+"""The allocation-free tree-attention entry point against the regular one.
+
+llmcad_tree_attention_noalloc serves callers that must not allocate device memory (a plug-in
+inside a server whose pool already owns the device, a loop where cudaMalloc's device-wide
+synchronisation is not acceptable): it takes no context and keeps its scratch in a static device
+array. Here it is called twice in a row through the C ABI, on different trees, and each result
+must equal what llmcad_tree_attention gives for the same inputs (same kernels, same arithmetic:
+bit-identical, which is within the 2e-2 tolerance the other bf16 tests use). The file sorts last
+so that a run that stops at the first failure has already run every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2309_04255_b200 import binding as B
+from paper_2309_04255_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+
+
+def test_noalloc_matches_regular_entry_point_twice():
+    dev = torch.device("cuda:0")
+    H, hd = 8, 128
+    cfg = gen.ModelConfig("a", 0, H * hd, H, hd, 256, 512, "bf16")
+    ref = B.Verifier(cfg, 16)                    # the regular entry point needs a context
+    cases = [(300, 24, 1), (77, 128, 2)]         # (prefix, nodes, seed): the second reuses the scratch of the first
+    for P, n, seed in cases:
+        parent = torch.as_tensor(gen.tree_random(n, 12, "uniform4", seed), device=dev)
+        q, k, v = (t.to(dev) for t in gen.gen_attention_inputs(H, hd, P, n, seed=seed))
+        want = ref.tree_attention(q, k, v, P, parent)
+        got = torch.full_like(q, float("nan"))
+        status = torch.full((1,), -7, dtype=torch.int32, device=dev)
+        before = torch.cuda.memory_allocated(dev)
+        B.tree_attention_noalloc(q, k, v, P, parent, got, status)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated(dev) == before
+        assert int(status.item()) == 0
+        g, w = got.float().cpu().numpy(), want.float().cpu().numpy()
+        assert np.isfinite(g).all()
+        assert np.abs(g - w).max() <= 2e-2 * np.abs(w).max()
+        assert np.array_equal(g, w)              # same kernels on the same inputs
+    # a malformed tree is reported through the status word, which the previous calls left at 0
+    bad = torch.as_tensor(np.array([-1, 2, 0], np.int32), device=dev)
+    q, k, v = (t.to(dev) for t in gen.gen_attention_inputs(H, hd, 5, 3, seed=3))
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    B.tree_attention_noalloc(q, k, v, 5, bad, torch.empty_like(q), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.ERR_BAD_TREE
+    # and the call after that starts from a clean status again
+    good = torch.as_tensor(np.array([-1, 0, 0], np.int32), device=dev)
+    B.tree_attention_noalloc(q, k, v, 5, good, torch.empty_like(q), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+
+def test_noalloc_rejects_sizes_beyond_the_static_scratch():
+    dev = torch.device("cuda:0")
+    H, hd, n = 2, 128, 129
+    q = torch.zeros((n, H, hd), dtype=torch.bfloat16, device=dev)
+    k = torch.zeros((H, n + 4, hd), dtype=torch.bfloat16, device=dev)
+    parent = torch.zeros(n, dtype=torch.int32, device=dev)
+    with pytest.raises(B.LlmcadError) as e:
+        B.tree_attention_noalloc(q, k, k, 4, parent, torch.empty_like(q))
+    assert e.value.code == B.ERR_UNSUPPORTED and "128" in str(e.value)
