@@ -90,12 +90,15 @@ struct llmcad_ctx {
     int n_sms = 0;
     size_t elem = 2;
     bool tc_gemm = false, tc_attn = false;
-    // activations of up to 128 nodes
+    // Tensor-core path: activations travel as bf16 hi + lo planes (common.cuh); a tuning aid
+    // (LLMCAD_COMP=0) turns the lo planes off.
+    bool comp = false;
+    // activations of up to 128 nodes; xn, q, att and h hold two planes of 128 rows (hi, lo)
     float *x = nullptr;       // residual stream [128][d] fp32
-    void *xn = nullptr;       // normalised GEMM input [128][d]
-    void *q = nullptr;        // rotated queries [128][d]
-    void *att = nullptr;      // attention output [128][d]
-    void *h = nullptr;        // SwiGLU output [128][f]
+    void *xn = nullptr;       // normalised GEMM input [2][128][d]
+    void *q = nullptr;        // rotated queries [2][128][d]
+    void *att = nullptr;      // attention output [2][128][d]
+    void *h = nullptr;        // SwiGLU output [2][128][f]
     float *logits = nullptr;  // [128][V], used when the caller does not want logits
     TreeBuffers tb{};
     int32_t *ibuf = nullptr;  // tokens[128], parent[128], argmax[128], path[128], scalars[8], chain[128]
@@ -179,9 +182,10 @@ int ensure_act_maps(llmcad_ctx *ctx, int n_pad)
     if (!ctx->tc_gemm || ctx->act_ready[slot]) return LLMCAD_OK;
     const llmcad_config &c = ctx->cfg;
     bool ok = true;
-    ok &= make_tensor_map_bf16(&ctx->act_maps[slot][0], ctx->xn, 128, c.d_model, n_pad);
-    ok &= make_tensor_map_bf16(&ctx->act_maps[slot][1], ctx->att, 128, c.d_model, n_pad);
-    ok &= make_tensor_map_bf16(&ctx->act_maps[slot][2], ctx->h, 128, c.d_ffn, n_pad);
+    const uint32_t planes = ctx->comp ? 2 : 1;
+    ok &= make_act_map_bf16(&ctx->act_maps[slot][0], ctx->xn, 128, c.d_model, n_pad, planes, kLoRows);
+    ok &= make_act_map_bf16(&ctx->act_maps[slot][1], ctx->att, 128, c.d_model, n_pad, planes, kLoRows);
+    ok &= make_act_map_bf16(&ctx->act_maps[slot][2], ctx->h, 128, c.d_ffn, n_pad, planes, kLoRows);
     if (!ok) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed for an activation buffer");
         return LLMCAD_ERR_CUDA;
@@ -218,6 +222,7 @@ struct Chain {
         maps.x[p.n_gemms] = ctx->act_maps[n_pad / 16][act];
         p.g[p.n_gemms] = make_gemm_desc(n_in, ep, w);
         p.n_pad = n_pad;
+        p.comp = ctx->comp ? 1 : 0;
         ++p.n_gemms;
     }
     int launch(llmcad_ctx *ctx, int32_t *status, cudaStream_t st)
@@ -257,15 +262,17 @@ int run_gemm(llmcad_ctx *ctx, const void *packed, int l, int which, int act, int
     return LLMCAD_OK;
 }
 
+// comp: q carries a lo plane kLoRows rows after the hi plane, and o gets one too (the pass);
+// the single-step entry points work on plain bf16 buffers.
 int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, int kv_stride, int P, int n, void *o,
-                  int32_t *status, cudaStream_t st)
+                  bool comp, int32_t *status, cudaStream_t st)
 {
     const llmcad_config &c = ctx->cfg;
     TimedLaunch tl(ctx, 1, st);
     if (ctx->tc_attn) {
         int launched = 0;
         CUDA_TRY(launch_attention_tc(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->attn_ws,
-                                     ctx->attn_counters, ctx->n_sms, status, st, &launched, ctx->next_trace()));
+                                     ctx->attn_counters, ctx->n_sms, status, st, &launched, ctx->next_trace(), comp ? 1 : 0));
         ctx->launches += launched;
         return LLMCAD_OK;
     }
@@ -302,13 +309,14 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
         const int tiles4 = 4 * ((d + 127) / 128);
         CUDA_TRY(launch_embed_norm(base + ctx->lay.tok_embed, tokens, n, d,
                                    c.n_layers > 0 ? base + ctx->lay.attn_norm : base + ctx->lay.final_norm, ctx->x, ctx->xn,
-                                   ctx->ssq[0], status, st));
+                                   ctx->ssq[0], ctx->comp ? 1 : 0, status, st));
         auto qkv_ep = [&](int l, int parts) {
             char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)l;
             EpiParams ep{};
             ep.n = n; ep.mode = EPI_QKV; ep.n_out = 3 * d; ep.q_out = ctx->q; ep.k_cache = kl; ep.v_cache = kl + kv_layer / 2;
             ep.rope_cs = ctx->tb.rope_cs; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P;
             ep.ssq_in = ctx->ssq[0]; ep.ssq_in_parts = parts; ep.norm_d = d; ep.eps = c.rms_eps;
+            ep.comp = ctx->comp ? 1 : 0;
             return ep;
         };
         auto head_ep = [&](int parts) {
@@ -329,14 +337,17 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
             EpiParams ep{};
             ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
             ep.xg_out = ctx->xn; ep.gain_next = lb + ctx->lay.ffn_norm; ep.ssq_out = ctx->ssq[1];
+            ep.comp = ctx->comp ? 1 : 0;
             specs.push_back({l, 1, 1, d, ep, true});
 
             ep = EpiParams{}; ep.n = n; ep.mode = EPI_SWIGLU; ep.n_out = f; ep.h = ctx->h;
             ep.ssq_in = ctx->ssq[1]; ep.ssq_in_parts = tiles4; ep.norm_d = d; ep.eps = c.rms_eps;
+            ep.comp = ctx->comp ? 1 : 0;
             specs.push_back({l, 2, 0, d, ep, false});
 
             ep = EpiParams{}; ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
             ep.xg_out = ctx->xn; ep.gain_next = next_gain; ep.ssq_out = ctx->ssq[0];
+            ep.comp = ctx->comp ? 1 : 0;
             specs.push_back({l, 3, 2, f, ep, false});
 
             if (!last) specs.push_back({l + 1, 0, 0, d, qkv_ep(l + 1, tiles4), false});
@@ -349,7 +360,8 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
         for (size_t i = 0; i < specs.size();) {
             if (specs[i].attention_first) {
                 char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)specs[i].l;
-                if ((rc = run_attention(ctx, ctx->q, kl, kl + kv_layer / 2, S, P, n, ctx->att, status, st)) != LLMCAD_OK) return rc;
+                // without the tensor-core attention kernel the lo plane of att stays zero, as allocated
+                if ((rc = run_attention(ctx, ctx->q, kl, kl + kv_layer / 2, S, P, n, ctx->att, ctx->comp && ctx->tc_attn, status, st)) != LLMCAD_OK) return rc;
             }
             Chain ch;
             size_t j = i;
@@ -378,7 +390,7 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
         ep.rope_cs = ctx->tb.rope_cs; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P;
         if ((rc = run_gemm(ctx, packed, l, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
 
-        if ((rc = run_attention(ctx, ctx->q, kl, vl, S, P, n, ctx->att, status, st)) != LLMCAD_OK) return rc;
+        if ((rc = run_attention(ctx, ctx->q, kl, vl, S, P, n, ctx->att, false, status, st)) != LLMCAD_OK) return rc;
 
         ep = EpiParams{}; ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
         if ((rc = run_gemm(ctx, packed, l, 1, 1, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
@@ -483,6 +495,10 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
         return LLMCAD_ERR_CUDA;
     }
     ctx->tc_attn = cfg->dtype == LLMCAD_BF16 && cfg->head_dim == 128 && !(cfg->flags & LLMCAD_FLAG_SIMT_ATTN);
+    {
+        const char *e = getenv("LLMCAD_COMP");
+        ctx->comp = ctx->tc_gemm && !(e != nullptr && atoi(e) == 0);
+    }
 
     const size_t d = cfg->d_model, f = cfg->d_ffn, hd = cfg->head_dim;
     auto alloc = [&](void **p, size_t bytes) {
@@ -491,10 +507,10 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     };
     bool ok = true;
     ok = ok && alloc((void **)&ctx->x, 128 * d * 4);
-    ok = ok && alloc(&ctx->xn, 128 * d * ctx->elem);
-    ok = ok && alloc(&ctx->q, 128 * d * ctx->elem);
-    ok = ok && alloc(&ctx->att, 128 * d * ctx->elem);
-    ok = ok && alloc(&ctx->h, 128 * f * ctx->elem);
+    ok = ok && alloc(&ctx->xn, 2 * kLoRows * d * ctx->elem);
+    ok = ok && alloc(&ctx->q, 2 * kLoRows * d * ctx->elem);
+    ok = ok && alloc(&ctx->att, 2 * kLoRows * d * ctx->elem);
+    ok = ok && alloc(&ctx->h, 2 * kLoRows * f * ctx->elem);
     ok = ok && alloc((void **)&ctx->logits, (size_t)128 * cfg->vocab * 4);
     ok = ok && alloc((void **)&ctx->tb.depth, 128 * 4);
     ok = ok && alloc((void **)&ctx->tb.pos, 128 * 4);
@@ -717,7 +733,7 @@ int llmcad_tree_attention(llmcad_ctx *ctx, const void *q, const void *k, const v
     tb.rope_cs = nullptr;
     CUDA_TRY(launch_tree_prep(parent_idx, nullptr, n, prefix_len, 0, 0, 0.f, tb, status, st));
     ctx->launches++;
-    return run_attention(ctx, q, k, v, kv_stride, prefix_len, n, o, status, st);
+    return run_attention(ctx, q, k, v, kv_stride, prefix_len, n, o, false, status, st);
 }
 
 int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, int32_t n_out, int32_t n_in, int32_t n,
@@ -739,7 +755,7 @@ int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, 
         const int n_pad = (n + 15) / 16 * 16;
         Chain ch;
         // rows of x beyond n are outside the tensor: the copy engine fills them with zeros
-        if (!make_tensor_map_bf16(&ch.maps.w[0], w, n_out, n_in, 128) || !make_tensor_map_bf16(&ch.maps.x[0], x, n, n_in, n_pad)) {
+        if (!make_tensor_map_bf16(&ch.maps.w[0], w, n_out, n_in, 128) || !make_act_map_bf16(&ch.maps.x[0], x, n, n_in, n_pad, 1, n)) {
             snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
             return LLMCAD_ERR_CUDA;
         }
@@ -784,7 +800,7 @@ int llmcad_skinny_gemm_tiled(llmcad_ctx *ctx, const void *w_tiled, const void *x
     ep.mode = EPI_PLAIN; ep.n = n; ep.n_out = n_out; ep.y = y; ep.ldy = n_out;
     const int n_pad = (n + 15) / 16 * 16;
     Chain ch;
-    if (!make_tensor_map_bf16(&ch.maps.x[0], x, n, n_in, n_pad)) {
+    if (!make_act_map_bf16(&ch.maps.x[0], x, n, n_in, n_pad, 1, n)) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
         return LLMCAD_ERR_CUDA;
     }

@@ -67,6 +67,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
+// (a, b) as two bf16 pairs: hi = bf16(value), lo = bf16(value - hi).
+__device__ __forceinline__ void pack_split(float a, float b, uint32_t &hi, uint32_t &lo)
+{
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    const float2 hf = __bfloat1622float2(h);
+    __nv_bfloat162 l = __floats2bfloat162_rn(a - hf.x, b - hf.y);
+    hi = *reinterpret_cast<uint32_t *>(&h);
+    lo = *reinterpret_cast<uint32_t *>(&l);
+}
+
 }  // namespace
 
 // GROUPS key groups per CTA: warp w works on query tile w % q_tiles and on the keys
@@ -75,7 +85,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 // dependent mma chain would set the pace; splitting the keys of a tile over four warps cuts the
 // per-tile latency four-fold. Each warp keeps its own running softmax; the groups are merged in
 // shared memory at the end, then the cluster merges the splits.
-template <int GROUPS>
+//
+// COMP (the verification pass): queries arrive as bf16 hi + lo planes and the output leaves as hi +
+// lo planes (kLoRows rows apart, see common.cuh), and the softmax weights are split into hi + lo as
+// well, so that Q K^T and P V each take two MMAs per fragment and only the cached K/V themselves
+// carry bf16 rounding.
+template <int GROUPS, bool COMP>
 __global__ void __launch_bounds__(kAtThreads)
 attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
                     const __nv_bfloat16 *__restrict__ v, int n_heads, int kv_stride, int P, int n, int n_pad,
@@ -91,10 +106,11 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 1] = global_timer_ns();
     if (*status) return;   // uniform over the grid: set only by kernels that ran before this one
     extern __shared__ __align__(128) uint8_t sm[];
-    uint8_t *s_q = sm;                                      // [n_pad][256 B]
-    uint8_t *s_k = s_q + (size_t)n_pad * kRowBytes;         // [kStages][64][256 B]
+    uint8_t *s_q = sm;                                      // [n_pad][256 B], with COMP followed by the lo plane
+    uint8_t *s_k = s_q + (size_t)(COMP ? 2 : 1) * n_pad * kRowBytes;   // [kStages][64][256 B]
     uint8_t *s_v = s_k + kStages * kKeyTile * kRowBytes;    // [kStages][64][256 B]
 
+    const size_t lo_off = (size_t)kLoRows * n_heads * kHd;  // elements from a hi plane of q / o to its lo plane
     const int split = blockIdx.x, head = blockIdx.y;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_keys = P + n;
@@ -121,7 +137,9 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     for (int c = tid; c < n_pad * 16; c += kAtThreads) {
         const int r = c >> 4, ch = c & 15;
         const bool ok = r < n;
-        cp_async16(smem_u32(s_q) + swz(r, ch), q + ((size_t)(ok ? r : 0) * n_heads + head) * kHd + ch * 8, ok);
+        const size_t off = ((size_t)(ok ? r : 0) * n_heads + head) * kHd + ch * 8;
+        cp_async16(smem_u32(s_q) + swz(r, ch), q + off, ok);
+        if (COMP) cp_async16(smem_u32(s_q) + n_pad * kRowBytes + swz(r, ch), q + lo_off + off, ok);
     }
     for (int st = 0; st < kStages - 1; ++st) {
         if (t_begin + st < t_end) load_tile(t_begin + st, st);
@@ -170,6 +188,8 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         for (int j = 0; j < NT; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
+            uint32_t ql[4];
+            if (COMP) ldsm4(smem_u32(s_q) + n_pad * kRowBytes + swz(qt * 16 + (lane & 15), ks * 2 + (lane >> 4)), ql);
 #pragma unroll
             for (int np = 0; np < NT / 2; ++np) {
                 uint32_t b[4];
@@ -177,6 +197,10 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
                 ldsm4(kb + swz(key, ks * 2 + ((lane >> 3) & 1)), b);
                 mma_bf16(s[2 * np], qf[ks], b[0], b[1]);
                 mma_bf16(s[2 * np + 1], qf[ks], b[2], b[3]);
+                if (COMP) {
+                    mma_bf16(s[2 * np], ql, b[0], b[1]);
+                    mma_bf16(s[2 * np + 1], ql, b[2], b[3]);
+                }
             }
         }
         // ---- scale, mask (tree region and the ragged end only), online softmax
@@ -211,14 +235,19 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         const float alpha0 = exp2f(m0 - ref0), alpha1 = exp2f(m1 - ref1);
         m0 = mn0; m1 = mn1;
         float rs0 = 0.f, rs1 = 0.f;
-        uint32_t pa[NT / 2][4];
+        uint32_t pa[NT / 2][4], pl[COMP ? NT / 2 : 1][4];
 #pragma unroll
         for (int j = 0; j < NT; ++j) {
             const float p0 = exp2f(s[j][0] - ref0), p1 = exp2f(s[j][1] - ref0);
             const float p2 = exp2f(s[j][2] - ref1), p3 = exp2f(s[j][3] - ref1);
             rs0 += p0 + p1; rs1 += p2 + p3;
-            pa[j >> 1][(j & 1) * 2 + 0] = pack_bf16(p0, p1);
-            pa[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
+            if (COMP) {
+                pack_split(p0, p1, pa[j >> 1][(j & 1) * 2 + 0], pl[COMP ? j >> 1 : 0][(j & 1) * 2 + 0]);
+                pack_split(p2, p3, pa[j >> 1][(j & 1) * 2 + 1], pl[COMP ? j >> 1 : 0][(j & 1) * 2 + 1]);
+            } else {
+                pa[j >> 1][(j & 1) * 2 + 0] = pack_bf16(p0, p1);
+                pa[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
+            }
         }
         l0 = l0 * alpha0 + rs0; l1 = l1 * alpha1 + rs1;
 #pragma unroll
@@ -233,6 +262,10 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
                 ldsm4_t(vb + swz(key, dp * 2 + (lane >> 4)), b);
                 mma_bf16(oacc[2 * dp], pa[kk], b[0], b[1]);
                 mma_bf16(oacc[2 * dp + 1], pa[kk], b[2], b[3]);
+                if (COMP) {
+                    mma_bf16(oacc[2 * dp], pl[COMP ? kk : 0], b[0], b[1]);
+                    mma_bf16(oacc[2 * dp + 1], pl[COMP ? kk : 0], b[2], b[3]);
+                }
             }
         }
     }
@@ -299,7 +332,11 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
             const float L = part[(size_t)row * kWsRow + kHd + 1];
             const float inv = L > 0.f ? 1.f / L : 0.f;
             const float2 ov = *reinterpret_cast<const float2 *>(part + (size_t)row * kWsRow + dim);
-            *reinterpret_cast<uint32_t *>(o + ((size_t)row * n_heads + head) * kHd + dim) = pack_bf16(ov.x * inv, ov.y * inv);
+            uint32_t hi, lo;
+            pack_split(ov.x * inv, ov.y * inv, hi, lo);
+            __nv_bfloat16 *dst = o + ((size_t)row * n_heads + head) * kHd + dim;
+            *reinterpret_cast<uint32_t *>(dst) = hi;
+            if (COMP) *reinterpret_cast<uint32_t *>(dst + lo_off) = lo;
         }
         if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
         return;
@@ -337,7 +374,11 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
             L += ml[sp].y * wgt; a0 += ov[sp].x * wgt; a1 += ov[sp].y * wgt;
         }
         const float inv = L > 0.f ? 1.f / L : 0.f;
-        *reinterpret_cast<uint32_t *>(o + ((size_t)row * n_heads + head) * kHd + dim) = pack_bf16(a0 * inv, a1 * inv);
+        uint32_t hi, lo;
+        pack_split(a0 * inv, a1 * inv, hi, lo);
+        __nv_bfloat16 *dst = o + ((size_t)row * n_heads + head) * kHd + dim;
+        *reinterpret_cast<uint32_t *>(dst) = hi;
+        if (COMP) *reinterpret_cast<uint32_t *>(dst + lo_off) = lo;
     }
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 6] = global_timer_ns();
     cluster.sync();                                          // peers may still be reading this CTA's partial
@@ -352,7 +393,7 @@ size_t attention_tc_workspace_bytes(int n_heads, int n_sms)
 
 cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, float *ws, uint32_t *counters, int n_sms,
-                                int32_t *status, cudaStream_t st, int *launched, unsigned long long *trace)
+                                int32_t *status, cudaStream_t st, int *launched, unsigned long long *trace, int comp)
 {
     (void)ws; (void)counters;
     if (hd != kHd) return cudaErrorInvalidValue;
@@ -367,24 +408,29 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
     const int q_tiles = n_pad / 16;
     const int groups = q_tiles <= 2 ? 4 : (q_tiles <= 4 ? 2 : 1);
-    const size_t ring = (size_t)n_pad * kRowBytes + 2 * kStages * kKeyTile * kRowBytes;
+    const size_t ring = (size_t)(comp ? 2 : 1) * n_pad * kRowBytes + 2 * kStages * kKeyTile * kRowBytes;
     const size_t part = (size_t)(groups > 1 ? groups + 1 : 1) * n_pad * kWsRow * sizeof(float) + (size_t)n_pad * groups * sizeof(float);
     const size_t smem = ring > part ? ring : part;
+    typedef void (*Kern)(const __nv_bfloat16 *, const __nv_bfloat16 *, const __nv_bfloat16 *, int, int, int, int, int,
+                         const uint32_t *, __nv_bfloat16 *, int, int, const int32_t *, unsigned long long *);
+    static const Kern kerns[2][3] = {{attention_tc_kernel<1, false>, attention_tc_kernel<2, false>, attention_tc_kernel<4, false>},
+                                     {attention_tc_kernel<1, true>, attention_tc_kernel<2, true>, attention_tc_kernel<4, true>}};
     static bool attr_set = false;
     if (!attr_set) {
-        const int max_smem = 128 * kRowBytes + 2 * kStages * kKeyTile * kRowBytes;
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        if (e != cudaSuccess) return e;
+        const int max_smem = 2 * 128 * kRowBytes + 2 * kStages * kKeyTile * kRowBytes;
+        for (int c = 0; c < 2; ++c)
+            for (int g = 0; g < 3; ++g) {
+                cudaError_t e = cudaFuncSetAttribute(kerns[c][g], cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+                if (e != cudaSuccess) return e;
+            }
         attr_set = true;
     }
     LaunchCfg lc(dim3(splits, n_heads), dim3(kAtThreads), smem, st, splits);
     if (launched) *launched = 1;
-    auto kern = groups == 4 ? attention_tc_kernel<4> : (groups == 2 ? attention_tc_kernel<2> : attention_tc_kernel<1>);
+    Kern kern = kerns[comp ? 1 : 0][groups == 4 ? 2 : (groups == 2 ? 1 : 0)];
     return cudaLaunchKernelEx(&lc.cfg, kern, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                               (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc, (__nv_bfloat16 *)o, splits,
-                              tiles_per_split, status, trace);
+                              tiles_per_split, (const int32_t *)status, trace);
 }
 
 }  // namespace llmcad

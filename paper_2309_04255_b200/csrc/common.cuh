@@ -19,6 +19,31 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+// ---------------------------------------------------------------- compensated bf16 activations
+// A bf16 keeps 8 significant bits; rounding every activation to it at every GEMM and attention
+// input adds up, over tens of layers, to logit errors beyond 2e-2 of the largest logit. The
+// tensor-core path therefore carries each activation as hi + lo, hi = bf16(v), lo = bf16(v - hi)
+// (16 significant bits together), in two planes of the same buffer: the lo plane of a [128][len]
+// activation buffer starts kLoRows rows after the hi plane. The weights stream once either way;
+// the MMAs see the nodes twice (N = 2 * n_pad) and the epilogue adds the two accumulator columns.
+constexpr int kLoRows = LLMCAD_MAX_TREE;
+
+__device__ __forceinline__ void split_bf16(float v, __nv_bfloat16 &hi, __nv_bfloat16 &lo)
+{
+    hi = __float2bfloat16_rn(v);
+    lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+// Stores v at p[0] and, if comp, its remainder at p[lo_off]. For fp32 buffers there is no remainder.
+template <typename T> __device__ __forceinline__ void store_split(T *p, size_t lo_off, float v, bool comp);
+template <> __device__ __forceinline__ void store_split<float>(float *p, size_t, float v, bool) { *p = v; }
+template <> __device__ __forceinline__ void store_split<__nv_bfloat16>(__nv_bfloat16 *p, size_t lo_off, float v, bool comp)
+{
+    __nv_bfloat16 hi, lo;
+    split_bf16(v, hi, lo);
+    p[0] = hi;
+    if (comp) p[lo_off] = lo;
+}
+
 // ---------------------------------------------------------------- GEMM epilogues
 // What a GEMM does with a finished pair of output values of one tree node.
 enum EpiMode : int {
@@ -55,6 +80,8 @@ struct EpiParams {
     void *xg_out;           // [n][n_out] or nullptr
     const void *gain_next;  // [n_out]
     float *ssq_out;         // [4 * n_tiles][128]
+    // Tensor-core path: q_out, h and xg_out also get their lo plane (see kLoRows).
+    int comp;
 };
 
 // (v0, v1) are the accumulators of output rows (r0, r0+1), r0 even, of node i; for
@@ -148,7 +175,7 @@ cudaError_t launch_tree_prep(const int32_t *parent, const int32_t *tokens, int n
 cudaError_t launch_embed(const void *E, int dtype, const int32_t *tokens, int n, int d, float *x, const int32_t *status,
                          cudaStream_t st);
 cudaError_t launch_embed_norm(const void *E, const int32_t *tokens, int n, int d, const void *gain, float *x, void *xg,
-                              float *ssq, const int32_t *status, cudaStream_t st);
+                              float *ssq, int comp, const int32_t *status, cudaStream_t st);
 cudaError_t launch_rmsnorm(const float *x, const void *g, int dtype, int n, int d, float eps, void *out,
                            const int32_t *status, cudaStream_t st);
 cudaError_t launch_argmax(const float *logits, int n, int vocab, int32_t *argmax, int32_t *status, cudaStream_t st);

@@ -119,6 +119,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// Activation box (64 columns x rows x planes) at column c0, row 0, plane 0.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, uint32_t bar, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(0), "r"(bar), "l"(policy)
+        : "memory");
+}
+
 // One contiguous run of global memory into shared memory (both 16-byte aligned, size a multiple of 16).
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint64_t policy)
 {
@@ -285,7 +295,7 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &ep, const float 
         for (int j = 0; j < 16; ++j) {
             if (row_ok && c0 + j < ep.n) {
                 const float sg = v[j] / (1.0f + __expf(-v[j]));
-                hrow[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(sg * w[j]);
+                store_split<T>(hrow + (size_t)(c0 + j) * ep.n_out, (size_t)kLoRows * ep.n_out, sg * w[j], ep.comp != 0);
             }
         }
     } else if (ep.mode == EPI_QKV) {
@@ -305,7 +315,8 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &ep, const float 
             // the rotary partner (2t <-> 2t+1) lives in the neighbouring lane
             const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
             const float rot = (lane & 1) ? (other * cs[j].y + v[j] * cs[j].x) : (v[j] * cs[j].x - other * cs[j].y);
-            if (row_ok && c0 + j < ep.n) dst[(size_t)(c0 + j) * node_stride] = from_f32<T>(rot);
+            // queries also get their lo plane; keys and values are stored once, in the cache's dtype
+            if (row_ok && c0 + j < ep.n) store_split<T>(dst + (size_t)(c0 + j) * node_stride, (size_t)kLoRows * ep.d, rot, ep.comp != 0 && sec == 0);
         }
     } else if (ep.mode == EPI_RESID) {
         // xo: the residual values of this chunk, loaded by the caller together with the partial tiles
@@ -321,7 +332,7 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &ep, const float 
             T *gr = reinterpret_cast<T *>(ep.xg_out) + row;
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-                if (row_ok && c0 + j < ep.n) gr[(size_t)(c0 + j) * ep.n_out] = from_f32<T>(xo[j] * gain);
+                if (row_ok && c0 + j < ep.n) store_split<T>(gr + (size_t)(c0 + j) * ep.n_out, (size_t)kLoRows * ep.n_out, xo[j] * gain, ep.comp != 0);
             // column sums over the warp's 32 rows by recursive halving: after exchanging with
             // lane^16, ^8, ^4, ^2 a lane is left with one column, after lane^1 with its full sum
             // (16 shuffles instead of 80). Column held by a lane: bits 4..1 of the lane, msb first.
@@ -370,12 +381,14 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
     __shared__ SharedCtl ctl;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t b_tile_bytes = (uint32_t)p.n_pad * kBlockK * 2;
+    const uint32_t nb = (uint32_t)p.n_pad * (p.comp ? 2u : 1u);   // activation rows per k-block = the MMA N: nodes (hi | lo)
+    const uint32_t b_tile_bytes = nb * kBlockK * 2;
     // stage: [weights k-block 0 | weights k-block 1 | activations k-block 0 | activations k-block 1]
     const uint32_t stage_bytes = kPairK * (kATileBytes + b_tile_bytes);
     const uint32_t b_off = kPairK * kATileBytes;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t acc_cols = 2u * (uint32_t)p.n_pad;     // TMEM columns of one accumulator buffer (gate | up)
+    const uint32_t acc_cols = 2u * nb;                    // TMEM columns of one accumulator buffer (gate | up)
+    const bool two_bufs = p.acc_bufs == 2;
 
     // Let the next kernel of the stream start early. This kernel in turn must not read activations,
     // the status word or the workspace, nor write anything, before pdl_wait(): until then it only
@@ -527,7 +540,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 const uint32_t dst = smem_base + s * stage_bytes + b_off;
                 const int nk = c.nk();
                 for (int k = 0; k < nk; ++k)
-                    tma_load_2d(dst + k * b_tile_bytes, &maps.x[c.g], (c.kb0() + k) * kBlockK, 0, full, pol_keep);
+                    tma_load_3d(dst + k * b_tile_bytes, &maps.x[c.g], (c.kb0() + k) * kBlockK, full, pol_keep);
                 c.advance(p);
                 ++i;
                 if (++s == p.stages) s = 0;
@@ -538,7 +551,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
     } else if (warp == 1) {
         // ================================================= MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = make_idesc(kTileM, p.n_pad);
+            const uint32_t idesc = make_idesc(kTileM, (int)nb);
             Cursor c;
             c.init(p);
             uint32_t seg = 0, ph = 0;   // ph: parity the MMA warp waits for on its stage's "full" barrier
@@ -546,8 +559,9 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             while (!c.done(p) && !timed_out) {
                 // one segment: the items of one tile that belong to this CTA
                 const int cg = c.g, tile = c.tile, halves = c.halves;
-                const int buf = seg & 1;
-                if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), ((seg >> 1) & 1u) ^ 1u, abort_flag)) { timed_out = true; break; }
+                const int buf = two_bufs ? (seg & 1) : 0;
+                const uint32_t use = two_bufs ? (seg >> 1) : seg;     // how often this buffer has been used before
+                if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, abort_flag)) { timed_out = true; break; }
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + buf * acc_cols;
                 for (int q = 0; c.g == cg && c.tile == tile; ++q) {
@@ -556,7 +570,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     const uint32_t a_addr = smem_base + s * stage_bytes;
                     // segments of a two-half GEMM start on a gate item, so the first `halves` items
                     // of a segment are the ones that must overwrite their accumulator
-                    const uint32_t dcol = d0 + c.half * p.n_pad;
+                    const uint32_t dcol = d0 + c.half * nb;
                     const int nk = c.nk();
                     for (int k = 0; k < nk; ++k) {
                         const uint64_t a_desc = make_smem_desc(a_addr + k * kATileBytes);
@@ -650,13 +664,14 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 const int tile = seg_begin / ipt;
                 const int tile_i0 = tile * ipt;
                 const int seg_end = min(r.end, tile_i0 + ipt);
-                const int buf = seg & 1;
+                const int buf = two_bufs ? (seg & 1) : 0;
+                const uint32_t use = two_bufs ? (seg >> 1) : seg;
                 const bool sole = (seg_begin == tile_i0 && seg_end == tile_i0 + ipt);   // this CTA holds the whole tile
                 const int first_cta = tile_i0 / d.items_per_cta;
                 const int last_cta = (tile_i0 + ipt - 1) / d.items_per_cta;
                 const int n_parts = last_cta - first_cta + 1;
 
-                if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), (seg >> 1) & 1u, abort_flag, lane)) { timed_out = true; break; }
+                if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), use & 1u, abort_flag, lane)) { timed_out = true; break; }
                 tc_fence_after();
                 if (threadIdx.x == 64 && g < 4 && seg_begin == r.begin) LLMCAD_TRACE(4 + 2 * g);
 
@@ -664,6 +679,17 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 const int row = tile * kTileM + row_in_tile;           // output feature (weight row)
                 const bool row_ok = row < ep.n_out;
                 bool finish = sole;
+                // 16 nodes of accumulator `hf` (0 gate or the only one, 1 up); with hi + lo activations
+                // the node's two columns are added here, before anything else sees them
+                auto ld_acc = [&](int hf, int c0, float (&v)[16]) {
+                    tc_ld16(t_lane + hf * nb + c0, v);
+                    if (p.comp) {
+                        float t[16];
+                        tc_ld16(t_lane + hf * nb + p.n_pad + c0, t);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] += t[j];
+                    }
+                };
 
                 if (!sole) {
                     // A tile shared by several CTAs: every sharer leaves its partial accumulator in the
@@ -675,13 +701,14 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     // moves 16 bytes per access and a warp 512 contiguous bytes.
                     float4 *dst = reinterpret_cast<float4 *>(p.partials + ((size_t)blockIdx.x * 2 + (seg_begin == r.begin ? 0 : 1)) * part_stride) +
                                   (size_t)lane_grp * 2 * quads * 32 + lane;
-                    const int ncol = dual ? 2 * p.n_pad : p.n_pad;
-                    for (int c0 = 0; c0 < ncol; c0 += 16) {
-                        float v[16];
-                        tc_ld16(t_lane + c0, v);
+                    for (int hf = 0; hf < (dual ? 2 : 1); ++hf) {
+                        for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                            float v[16];
+                            ld_acc(hf, c0, v);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            dst[(size_t)((c0 >> 2) + k) * 32] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+                            for (int k = 0; k < 4; ++k)
+                                dst[(size_t)(hf * quads + (c0 >> 2) + k) * 32] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+                        }
                     }
                     __threadfence();
                     __syncwarp();
@@ -711,8 +738,8 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                             for (int j = 0; j < 16; ++j) xo[j] = (row_ok && c0 + j < ep.n) ? __ldcg(xr + (size_t)(c0 + j) * ep.n_out) : 0.f;
                         }
                         if (sole) {
-                            tc_ld16(t_lane + c0, v);
-                            if (dual) tc_ld16(t_lane + p.n_pad + c0, w);
+                            ld_acc(0, c0, v);
+                            if (dual) ld_acc(1, c0, w);
                         } else {
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = w[j] = 0.f;
@@ -820,6 +847,21 @@ bool make_tensor_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uin
     return r == CUDA_SUCCESS;
 }
 
+bool make_act_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t planes,
+                       uint64_t plane_rows)
+{
+    auto fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[3] = {cols, rows, planes};
+    cuuint64_t strides[2] = {cols * 2, plane_rows * cols * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kBlockK, box_rows, planes};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 size_t gemm_tc_partial_floats(int n_sms, int max_n_pad) { return (size_t)n_sms * 2 /*slots*/ * 2 /*gate|up*/ * max_n_pad * kTileM; }
 
 GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)
@@ -860,10 +902,14 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
         const long long total = items_of(p.g[0]);
         grid = (int)((total + p.g[0].items_per_cta - 1) / p.g[0].items_per_cta);
     }
-    const size_t stage_bytes = (size_t)kPairK * ((size_t)kATileBytes + (size_t)p.n_pad * kBlockK * 2);
+    const int nb = p.n_pad * (p.comp ? 2 : 1);       // MMA N
+    if (nb > 256) return cudaErrorInvalidValue;
+    const size_t stage_bytes = (size_t)kPairK * ((size_t)kATileBytes + (size_t)nb * kBlockK * 2);
     // One CTA per SM with the whole shared memory as the ring. (Two CTAs per SM with half-size rings,
     // so that the next kernel is resident during this one's tail, measured slower on B200.)
-    int cols = 4 * p.n_pad, pow2 = 32;
+    // accumulators: (gate | up) x MMA N columns each, double-buffered when two of them fit
+    p.acc_bufs = 4 * nb <= 512 ? 2 : 1;
+    int cols = p.acc_bufs * 2 * nb, pow2 = 32;
     while (pow2 < cols) pow2 <<= 1;
     p.tmem_cols = pow2;
     const size_t full_limit = 227 * 1024 - 1024 /*alignment slack*/ - 4096 /*static*/;

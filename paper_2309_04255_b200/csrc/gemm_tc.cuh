@@ -24,12 +24,14 @@ struct GemmDesc {
 
 struct ChainMaps {
     CUtensorMap w[kMaxChain];  // weight matrices, box 64 x 128 rows
-    CUtensorMap x[kMaxChain];  // the activation matrix each GEMM multiplies, box 64 x n_pad rows
+    CUtensorMap x[kMaxChain];  // the activation matrix each GEMM multiplies, box 64 x n_pad rows x planes (hi, lo)
 };
 
 struct ChainParams {
     int n_gemms;
-    int n_pad;          // tree nodes padded to a multiple of 16 (the MMA N)
+    int n_pad;          // tree nodes padded to a multiple of 16
+    int comp;           // 1: activations come as hi + lo planes; the MMA N is 2 * n_pad and the epilogue adds the two
+    int acc_bufs;       // accumulator buffers in TMEM: 2, or 1 when 2 x (gate | up) x MMA N exceeds the 512 columns
     int stages;         // depth of the shared-memory ring
     int tmem_cols;      // allocated TMEM columns (power of two)
     float *partials;    // [grid][2 slots][2 halves][n_pad][128] fp32 partial tiles
@@ -47,6 +49,12 @@ struct ChainParams {
 // Tensor map over a row-major bf16 matrix [rows][cols] with a box of 64 columns x box_rows rows
 // and 128-byte swizzle. cols must be a multiple of 8 and base 16-byte aligned.
 bool make_tensor_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+
+// Tensor map over `planes` (1 or 2) row-major bf16 matrices [rows][cols] that lie plane_rows rows
+// apart, with a box of 64 columns x box_rows rows x planes: one copy brings the hi and the lo tile
+// of an activation k-block, one after the other, into shared memory. Rows beyond `rows` read as zero.
+bool make_act_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t planes,
+                       uint64_t plane_rows);
 
 size_t gemm_tc_partial_floats(int n_sms, int max_n_pad);
 constexpr size_t kTicketsPerGemm = 4096 * 4;

@@ -81,11 +81,12 @@ cudaError_t launch_embed(const void *E, int dtype, const int32_t *tokens, int n,
 }
 
 // Embedding gather for the tensor-core path, where the first RMSNorm is folded into the QKV GEMM:
-// besides x it writes gain * x in the GEMM input dtype and the row's sum of squares.
+// besides x it writes gain * x in the GEMM input dtype (hi and, if comp, lo plane) and the row's
+// sum of squares.
 template <typename T>
 __global__ void __launch_bounds__(256)
 embed_norm_kernel(const T *__restrict__ E, const int32_t *__restrict__ tokens, int d, const T *__restrict__ gain, float *x,
-                  T *xg, float *ssq, const int32_t *status)
+                  T *xg, float *ssq, int comp, const int32_t *status)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -97,7 +98,7 @@ embed_norm_kernel(const T *__restrict__ E, const int32_t *__restrict__ tokens, i
     for (int k = threadIdx.x; k < d; k += 256) {
         const float v = to_f32<T>(row[k]);
         x[(size_t)i * d + k] = v;
-        xg[(size_t)i * d + k] = from_f32<T>(v * to_f32<T>(gain[k]));
+        store_split<T>(xg + (size_t)i * d + k, (size_t)kLoRows * d, v * to_f32<T>(gain[k]), comp != 0);
         ss += v * v;
     }
     for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -111,11 +112,11 @@ embed_norm_kernel(const T *__restrict__ E, const int32_t *__restrict__ tokens, i
 }
 
 cudaError_t launch_embed_norm(const void *E, const int32_t *tokens, int n, int d, const void *gain, float *x, void *xg,
-                              float *ssq, const int32_t *status, cudaStream_t st)
+                              float *ssq, int comp, const int32_t *status, cudaStream_t st)
 {
     LaunchCfg lc(n, 256, 0, st);
     return cudaLaunchKernelEx(&lc.cfg, embed_norm_kernel<__nv_bfloat16>, (const __nv_bfloat16 *)E, tokens, d,
-                              (const __nv_bfloat16 *)gain, x, (__nv_bfloat16 *)xg, ssq, status);
+                              (const __nv_bfloat16 *)gain, x, (__nv_bfloat16 *)xg, ssq, comp, status);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -1,0 +1,96 @@
+"""Full-size parity: the 7B workload at its full depth (the launch configuration bench.py times),
+and the 30B width at N = 128 (the widest MMA, the shallowest ring) on one layer, each against the
+CPU oracle on the same seeded bytes. Weights are generated once per layer and handed to both sides."""
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2309_04255_b200 import binding as B
+from paper_2309_04255_b200 import inputs as gen
+
+from gpu_util import BF16_TOL, argmax_agrees_where_decided, check_acceptance_against_oracle, logits_close
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def gen_layer_parallel(cfg, l, pool):
+    futs = {name: pool.submit(gen.gen_tensor, cfg, name, l) for name in gen.LAYER_TENSORS}
+    return {k: f.result() for k, f in futs.items()}
+
+
+def run_streamed(cfg, P, n, parent, tokens):
+    """One generation of every layer feeds the GPU (packed on arrival) and the oracle (layer-streamed)."""
+    v = B.Verifier(cfg, P + n + 8)
+    glob = gen.gen_globals(cfg)
+    v.pack_globals(glob)
+    kvv = v.kv_view()
+    pool = ThreadPoolExecutor(9)
+    nxt = [pool.submit(gen_layer_parallel, cfg, 0, pool)] if cfg.n_layers else []
+
+    def layer_fn(l):
+        w = nxt.pop(0).result()
+        if l + 1 < cfg.n_layers:
+            nxt.append(pool.submit(gen_layer_parallel, cfg, l + 1, pool))
+        v.pack_layer(l, w)
+        return w
+
+    def prefix_fn(l):
+        k, vv = gen.gen_prefix_kv(cfg, l, P)
+        kvv[l, 0, :, :P] = k.to(DEV)
+        kvv[l, 1, :, :P] = vv.to(DEV)
+        return k, vv
+
+    ref = orc.verify_tree(cfg, glob, layer_fn, prefix_fn, P, tokens, parent, keep_kv=False)
+    pool.shutdown()
+    dev_t = torch.as_tensor(tokens, device=DEV)
+    dev_p = torch.as_tensor(parent, device=DEV)
+    out = v.verify_tree(P, dev_t, dev_p)
+    torch.cuda.synchronize()
+    out = {k: t.cpu().numpy() for k, t in out.items()}
+    return v, ref, out
+
+
+def test_c2_full_depth_parity():
+    """Config 2 as benchmarked: LLaMA-7B shape, 32 layers, prefix 512, random tree of 32 nodes."""
+    w = gen.WORKLOADS["C2"]
+    cfg = gen.MODELS[w.model]
+    parent = gen.gen_tree(w)
+    tokens = gen.gen_tokens(cfg, w.n_nodes)
+    v, ref, out = run_streamed(cfg, w.prefix_len, w.n_nodes, parent, tokens)
+    logits_close(out["logits"], ref.logits, BF16_TOL)
+    argmax_agrees_where_decided(out["argmax"], ref.logits, BF16_TOL)
+    acc = check_acceptance_against_oracle(out, tokens, parent)
+    assert out["scalars"][B.S_NEW_PREFIX_LEN] == w.prefix_len + acc.accepted_len
+    # a second pass on the same inputs gives the same bits (fixed summation orders everywhere)
+    again = v.verify_tree(w.prefix_len, torch.as_tensor(tokens, device=DEV), torch.as_tensor(parent, device=DEV))
+    torch.cuda.synchronize()
+    assert np.array_equal(again["logits"].cpu().numpy(), out["logits"])
+    # planted variant: the GPU's own argmax along branches gives a non-trivial verified path; the
+    # search and the rollback layout are then checked bit-exactly (oracle search on the GPU argmax)
+    tok = gen.plant_tokens(parent, tokens, out["argmax"], seed=1, prob=0.9)
+    before = v.kv_view()[:, :, :, : w.prefix_len + w.n_nodes].clone()
+    o2 = v.verify_tree(w.prefix_len, torch.as_tensor(tok, device=DEV), torch.as_tensor(parent, device=DEV))
+    torch.cuda.synchronize()
+    o2 = {k: t.cpu().numpy() for k, t in o2.items()}
+    acc2 = check_acceptance_against_oracle(o2, tok, parent)
+    assert acc2.accepted_len >= 2
+    after = v.kv_view()
+    assert torch.equal(after[:, :, :, : w.prefix_len], before[:, :, :, : w.prefix_len])
+
+
+def test_30b_width_128_nodes_one_layer():
+    """Config 5's widths (d 6656, 52 heads, FFN 17920) and tree size (128 nodes, 12 levels) on one
+    layer: every tile count, the N = 128 accumulators and the three-stage ring."""
+    w = gen.WORKLOADS["C5"]
+    cfg = gen.shrink(gen.MODELS[w.model], 1)
+    P = 300
+    parent = gen.gen_tree(w)
+    tokens = gen.gen_tokens(cfg, w.n_nodes)
+    v, ref, out = run_streamed(cfg, P, w.n_nodes, parent, tokens)
+    logits_close(out["logits"], ref.logits, BF16_TOL)
+    argmax_agrees_where_decided(out["argmax"], ref.logits, BF16_TOL)
+    check_acceptance_against_oracle(out, tokens, parent)
