@@ -99,6 +99,7 @@ struct llmcad_ctx {
     void *q = nullptr;        // rotated queries [2][128][d]
     void *att = nullptr;      // attention output [2][128][d]
     void *h = nullptr;        // SwiGLU output [2][128][f]
+    void *kv_lo = nullptr;    // bf16 remainders of the current layer's tree keys and values [2][H][128][hd]
     float *logits = nullptr;  // [128][V], used when the caller does not want logits
     TreeBuffers tb{};
     int32_t *ibuf = nullptr;  // tokens[128], parent[128], argmax[128], path[128], scalars[8], chain[128]
@@ -272,7 +273,8 @@ int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, 
     if (ctx->tc_attn) {
         int launched = 0;
         CUDA_TRY(launch_attention_tc(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->attn_ws,
-                                     ctx->attn_counters, ctx->n_sms, status, st, &launched, ctx->next_trace(), comp ? 1 : 0));
+                                     ctx->attn_counters, ctx->n_sms, status, st, &launched, ctx->next_trace(), comp ? 1 : 0,
+                                     ctx->kv_lo));
         ctx->launches += launched;
         return LLMCAD_OK;
     }
@@ -316,7 +318,7 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
             ep.n = n; ep.mode = EPI_QKV; ep.n_out = 3 * d; ep.q_out = ctx->q; ep.k_cache = kl; ep.v_cache = kl + kv_layer / 2;
             ep.rope_cs = ctx->tb.rope_cs; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P;
             ep.ssq_in = ctx->ssq[0]; ep.ssq_in_parts = parts; ep.norm_d = d; ep.eps = c.rms_eps;
-            ep.comp = ctx->comp ? 1 : 0;
+            ep.comp = ctx->comp ? 1 : 0; ep.kv_lo = ctx->kv_lo;
             return ep;
         };
         auto head_ep = [&](int parts) {
@@ -511,6 +513,7 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ok = ok && alloc(&ctx->q, 2 * kLoRows * d * ctx->elem);
     ok = ok && alloc(&ctx->att, 2 * kLoRows * d * ctx->elem);
     ok = ok && alloc(&ctx->h, 2 * kLoRows * f * ctx->elem);
+    ok = ok && alloc(&ctx->kv_lo, 2 * kLoRows * d * ctx->elem);
     ok = ok && alloc((void **)&ctx->logits, (size_t)128 * cfg->vocab * 4);
     ok = ok && alloc((void **)&ctx->tb.depth, 128 * 4);
     ok = ok && alloc((void **)&ctx->tb.pos, 128 * 4);
@@ -541,7 +544,7 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
 void llmcad_destroy(llmcad_ctx *ctx)
 {
     if (ctx == nullptr) return;
-    void *ptrs[] = {ctx->x, ctx->xn, ctx->q, ctx->att, ctx->h, ctx->logits, ctx->tb.depth, ctx->tb.pos, ctx->tb.anc,
+    void *ptrs[] = {ctx->x, ctx->xn, ctx->q, ctx->att, ctx->h, ctx->kv_lo, ctx->logits, ctx->tb.depth, ctx->tb.pos, ctx->tb.anc,
                     ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->flags, ctx->attn_ws, ctx->attn_counters, ctx->ssq[0],
                     ctx->ssq[1], ctx->grid_counter};
     for (void *p : ptrs)

@@ -29,7 +29,7 @@ constexpr int kAtThreads = 256;
 constexpr int kRowBytes = kHd * 2;            // 256-byte rows = 16 chunks of 16 bytes
 constexpr int kWsRow = kHd + 2;               // partial row: 128 outputs, max, sum
 constexpr int kMaxSplits = 8;                 // portable cluster size
-constexpr int kStages = 4;
+constexpr int kMaxStages = 4;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -88,15 +88,19 @@ __device__ __forceinline__ void pack_split(float a, float b, uint32_t &hi, uint3
 //
 // COMP (the verification pass): queries arrive as bf16 hi + lo planes and the output leaves as hi +
 // lo planes (kLoRows rows apart, see common.cuh), and the softmax weights are split into hi + lo as
-// well, so that Q K^T and P V each take two MMAs per fragment and only the cached K/V themselves
-// carry bf16 rounding.
+// well, so that Q K^T and P V each take two MMAs per fragment. The keys and values of the tree nodes
+// themselves, which the QKV GEMM has just rounded into the cache, come with their remainders in a
+// side buffer kv_lo ([2][H][kLoRows][128]: K then V, indexed by node); the tiles that contain tree
+// keys add Q K_lo^T and P V_lo. Only the prefix K/V, which are bf16 by definition, stay as they are.
 template <int GROUPS, bool COMP>
 __global__ void __launch_bounds__(kAtThreads)
 attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
                     const __nv_bfloat16 *__restrict__ v, int n_heads, int kv_stride, int P, int n, int n_pad,
                     const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
-                    const int32_t *status, unsigned long long *trace)
+                    const int32_t *status, unsigned long long *trace, const __nv_bfloat16 *__restrict__ kv_lo)
 {
+    // ring depth: with 128 nodes and the lo planes three stages are what fits in shared memory
+    constexpr int kStages = (COMP && GROUPS == 1) ? 3 : kMaxStages;
     constexpr int KW = kKeyTile / GROUPS;     // keys per warp per tile: 64, 32 or 16
     constexpr int NT = KW / 8;                // 8-key score tiles per warp per tile
     const int cta = blockIdx.y * gridDim.x + blockIdx.x;
@@ -109,6 +113,9 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     uint8_t *s_q = sm;                                      // [n_pad][256 B], with COMP followed by the lo plane
     uint8_t *s_k = s_q + (size_t)(COMP ? 2 : 1) * n_pad * kRowBytes;   // [kStages][64][256 B]
     uint8_t *s_v = s_k + kStages * kKeyTile * kRowBytes;    // [kStages][64][256 B]
+    // COMP: remainders of the tree nodes' K and V, [n_pad + 1][256 B] each, row = node; the extra row is zero
+    uint8_t *s_kl = s_v + kStages * kKeyTile * kRowBytes;
+    uint8_t *s_vl = s_kl + (size_t)(n_pad + 1) * kRowBytes;
 
     const size_t lo_off = (size_t)kLoRows * n_heads * kHd;  // elements from a hi plane of q / o to its lo plane
     const int split = blockIdx.x, head = blockIdx.y;
@@ -140,6 +147,17 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         const size_t off = ((size_t)(ok ? r : 0) * n_heads + head) * kHd + ch * 8;
         cp_async16(smem_u32(s_q) + swz(r, ch), q + off, ok);
         if (COMP) cp_async16(smem_u32(s_q) + n_pad * kRowBytes + swz(r, ch), q + lo_off + off, ok);
+    }
+    if (COMP && t_end * kKeyTile > P) {         // this CTA's key range reaches the tree nodes
+        const __nv_bfloat16 *kl = kv_lo + (size_t)head * kLoRows * kHd;
+        const __nv_bfloat16 *vl = kl + (size_t)n_heads * kLoRows * kHd;
+        for (int c = tid; c < (n_pad + 1) * 16; c += kAtThreads) {
+            const int r = c >> 4, ch = c & 15;
+            const bool ok = r < n;
+            const size_t off = (size_t)(ok ? r : 0) * kHd + ch * 8;
+            cp_async16(smem_u32(s_kl) + swz(r, ch), kl + off, ok);
+            cp_async16(smem_u32(s_vl) + swz(r, ch), vl + off, ok);
+        }
     }
     for (int st = 0; st < kStages - 1; ++st) {
         if (t_begin + st < t_end) load_tile(t_begin + st, st);
@@ -203,9 +221,24 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
                 }
             }
         }
-        // ---- scale, mask (tree region and the ragged end only), online softmax
         const int key_base = t * kKeyTile + key_off;
-        const bool needs_mask = key_base + KW > P;
+        const bool needs_mask = key_base + KW > P;          // this warp's keys reach into the tree nodes
+        // row of the lo buffers that holds the remainder of key `key` (the zero row for prefix keys)
+        auto lo_row = [&](int key) { const int node = key - P; return (node >= 0 && node < n) ? node : n_pad; };
+        if (COMP && needs_mask) {
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+#pragma unroll
+                for (int np = 0; np < NT / 2; ++np) {
+                    uint32_t b[4];
+                    const int row = lo_row(key_base + np * 16 + (lane & 7) + ((lane >> 4) << 3));
+                    ldsm4(smem_u32(s_kl) + swz(row, ks * 2 + ((lane >> 3) & 1)), b);
+                    mma_bf16(s[2 * np], qf[ks], b[0], b[1]);
+                    mma_bf16(s[2 * np + 1], qf[ks], b[2], b[3]);
+                }
+            }
+        }
+        // ---- scale, mask (tree region and the ragged end only), online softmax
         float tmax0 = -INFINITY, tmax1 = -INFINITY;
 #pragma unroll
         for (int j = 0; j < NT; ++j) {
@@ -265,6 +298,19 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
                 if (COMP) {
                     mma_bf16(oacc[2 * dp], pl[COMP ? kk : 0], b[0], b[1]);
                     mma_bf16(oacc[2 * dp + 1], pl[COMP ? kk : 0], b[2], b[3]);
+                }
+            }
+        }
+        if (COMP && needs_mask) {
+#pragma unroll
+            for (int kk = 0; kk < NT / 2; ++kk) {
+#pragma unroll
+                for (int dp = 0; dp < 8; ++dp) {
+                    uint32_t b[4];
+                    const int row = lo_row(key_base + kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3));
+                    ldsm4_t(smem_u32(s_vl) + swz(row, dp * 2 + (lane >> 4)), b);
+                    mma_bf16(oacc[2 * dp], pa[kk], b[0], b[1]);
+                    mma_bf16(oacc[2 * dp + 1], pa[kk], b[2], b[3]);
                 }
             }
         }
@@ -393,7 +439,8 @@ size_t attention_tc_workspace_bytes(int n_heads, int n_sms)
 
 cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, float *ws, uint32_t *counters, int n_sms,
-                                int32_t *status, cudaStream_t st, int *launched, unsigned long long *trace, int comp)
+                                int32_t *status, cudaStream_t st, int *launched, unsigned long long *trace, int comp,
+                                const void *kv_lo)
 {
     (void)ws; (void)counters;
     if (hd != kHd) return cudaErrorInvalidValue;
@@ -408,16 +455,20 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
     const int q_tiles = n_pad / 16;
     const int groups = q_tiles <= 2 ? 4 : (q_tiles <= 4 ? 2 : 1);
-    const size_t ring = (size_t)(comp ? 2 : 1) * n_pad * kRowBytes + 2 * kStages * kKeyTile * kRowBytes;
+    if (comp && kv_lo == nullptr) return cudaErrorInvalidValue;
+    const int stages = (comp && groups == 1) ? 3 : kMaxStages;
+    const size_t ring = (size_t)(comp ? 2 : 1) * n_pad * kRowBytes + (size_t)2 * stages * kKeyTile * kRowBytes +
+                        (comp ? (size_t)2 * (n_pad + 1) * kRowBytes : 0);
     const size_t part = (size_t)(groups > 1 ? groups + 1 : 1) * n_pad * kWsRow * sizeof(float) + (size_t)n_pad * groups * sizeof(float);
     const size_t smem = ring > part ? ring : part;
     typedef void (*Kern)(const __nv_bfloat16 *, const __nv_bfloat16 *, const __nv_bfloat16 *, int, int, int, int, int,
-                         const uint32_t *, __nv_bfloat16 *, int, int, const int32_t *, unsigned long long *);
+                         const uint32_t *, __nv_bfloat16 *, int, int, const int32_t *, unsigned long long *,
+                         const __nv_bfloat16 *);
     static const Kern kerns[2][3] = {{attention_tc_kernel<1, false>, attention_tc_kernel<2, false>, attention_tc_kernel<4, false>},
                                      {attention_tc_kernel<1, true>, attention_tc_kernel<2, true>, attention_tc_kernel<4, true>}};
     static bool attr_set = false;
     if (!attr_set) {
-        const int max_smem = 2 * 128 * kRowBytes + 2 * kStages * kKeyTile * kRowBytes;
+        const int max_smem = 2 * 128 * kRowBytes + 2 * 3 * kKeyTile * kRowBytes + 2 * 129 * kRowBytes;   // 128 nodes, hi + lo
         for (int c = 0; c < 2; ++c)
             for (int g = 0; g < 3; ++g) {
                 cudaError_t e = cudaFuncSetAttribute(kerns[c][g], cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
@@ -430,7 +481,7 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     Kern kern = kerns[comp ? 1 : 0][groups == 4 ? 2 : (groups == 2 ? 1 : 0)];
     return cudaLaunchKernelEx(&lc.cfg, kern, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                               (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc, (__nv_bfloat16 *)o, splits,
-                              tiles_per_split, (const int32_t *)status, trace);
+                              tiles_per_split, (const int32_t *)status, trace, (const __nv_bfloat16 *)kv_lo);
 }
 
 }  // namespace llmcad

@@ -33,6 +33,13 @@ __device__ __forceinline__ void split_bf16(float v, __nv_bfloat16 &hi, __nv_bflo
     hi = __float2bfloat16_rn(v);
     lo = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
+// Stores v at *p and its remainder at *p_lo.
+template <typename T> __device__ __forceinline__ void store_split(T *p, T *p_lo, float v);
+template <> __device__ __forceinline__ void store_split<float>(float *p, float *, float v) { *p = v; }
+template <> __device__ __forceinline__ void store_split<__nv_bfloat16>(__nv_bfloat16 *p, __nv_bfloat16 *p_lo, float v)
+{
+    split_bf16(v, *p, *p_lo);
+}
 // Stores v at p[0] and, if comp, its remainder at p[lo_off]. For fp32 buffers there is no remainder.
 template <typename T> __device__ __forceinline__ void store_split(T *p, size_t lo_off, float v, bool comp);
 template <> __device__ __forceinline__ void store_split<float>(float *p, size_t, float v, bool) { *p = v; }
@@ -80,8 +87,10 @@ struct EpiParams {
     void *xg_out;           // [n][n_out] or nullptr
     const void *gain_next;  // [n_out]
     float *ssq_out;         // [4 * n_tiles][128]
-    // Tensor-core path: q_out, h and xg_out also get their lo plane (see kLoRows).
+    // Tensor-core path: q_out, h and xg_out also get their lo plane (see kLoRows), and the bf16
+    // remainders of the keys and values go to kv_lo, [2][H][kLoRows][hd] (K then V, row = node).
     int comp;
+    void *kv_lo;
 };
 
 // (v0, v1) are the accumulators of output rows (r0, r0+1), r0 even, of node i; for

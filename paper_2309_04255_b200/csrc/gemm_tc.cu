@@ -306,17 +306,28 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &ep, const float 
         for (int j = 0; j < 16; ++j)
             cs[j] = (sec < 2 && row_ok && c0 + j < ep.n) ? __ldg(ep.rope_cs + (size_t)(c0 + j) * (ep.hd >> 1) + (e >> 1))
                                                           : make_float2(1.f, 0.f);
-        T *dst;
+        T *dst, *dst_lo;               // where a value goes, and where its remainder goes
         size_t node_stride;
-        if (sec == 0) { dst = reinterpret_cast<T *>(ep.q_out) + cidx; node_stride = ep.d; }
-        else { dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P) * ep.hd + e; node_stride = ep.hd; }
+        if (sec == 0) {
+            dst = reinterpret_cast<T *>(ep.q_out) + cidx;
+            dst_lo = dst + (size_t)kLoRows * ep.d;
+            node_stride = ep.d;
+        } else {
+            dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P) * ep.hd + e;
+            dst_lo = reinterpret_cast<T *>(ep.kv_lo) + ((size_t)((sec - 1) * (ep.d / ep.hd) + head) * kLoRows) * ep.hd + e;
+            node_stride = ep.hd;
+        }
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
             // the rotary partner (2t <-> 2t+1) lives in the neighbouring lane
             const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
             const float rot = (lane & 1) ? (other * cs[j].y + v[j] * cs[j].x) : (v[j] * cs[j].x - other * cs[j].y);
-            // queries also get their lo plane; keys and values are stored once, in the cache's dtype
-            if (row_ok && c0 + j < ep.n) store_split<T>(dst + (size_t)(c0 + j) * node_stride, (size_t)kLoRows * ep.d, rot, ep.comp != 0 && sec == 0);
+            // queries get their lo plane; keys and values go to the cache rounded, their remainders to kv_lo
+            if (row_ok && c0 + j < ep.n) {
+                const size_t at = (size_t)(c0 + j) * node_stride;
+                if (ep.comp) store_split<T>(dst + at, dst_lo + at, rot);
+                else dst[at] = from_f32<T>(rot);
+            }
         }
     } else if (ep.mode == EPI_RESID) {
         // xo: the residual values of this chunk, loaded by the caller together with the partial tiles

@@ -15,6 +15,7 @@ from gpu_util import BF16_TOL, argmax_agrees_where_decided, check_acceptance_aga
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
+HI_LO_TOL = 1e-3    # measured 7e-5 at 32 layers; one uncompensated bf16 rounding site costs 5e-3 or more
 
 
 def gen_layer_parallel(cfg, l, pool):
@@ -62,6 +63,9 @@ def test_c2_full_depth_parity():
     tokens = gen.gen_tokens(cfg, w.n_nodes)
     v, ref, out = run_streamed(cfg, w.prefix_len, w.n_nodes, parent, tokens)
     logits_close(out["logits"], ref.logits, BF16_TOL)
+    # the pass carries its activations as bf16 hi + lo pairs, which leaves it far inside the bound;
+    # a lost lo plane anywhere (GEMM inputs, queries, softmax weights, tree K/V) shows up here
+    logits_close(out["logits"], ref.logits, HI_LO_TOL)
     argmax_agrees_where_decided(out["argmax"], ref.logits, BF16_TOL)
     acc = check_acceptance_against_oracle(out, tokens, parent)
     assert out["scalars"][B.S_NEW_PREFIX_LEN] == w.prefix_len + acc.accepted_len
@@ -84,7 +88,8 @@ def test_c2_full_depth_parity():
 
 def test_30b_width_128_nodes_one_layer():
     """Config 5's widths (d 6656, 52 heads, FFN 17920) and tree size (128 nodes, 12 levels) on one
-    layer: every tile count, the N = 128 accumulators and the three-stage ring."""
+    layer: every tile count, the widest MMA (N = 256: 128 nodes, hi and lo), the single accumulator
+    buffer and the two-stage ring."""
     w = gen.WORKLOADS["C5"]
     cfg = gen.shrink(gen.MODELS[w.model], 1)
     P = 300
@@ -92,5 +97,6 @@ def test_30b_width_128_nodes_one_layer():
     tokens = gen.gen_tokens(cfg, w.n_nodes)
     v, ref, out = run_streamed(cfg, P, w.n_nodes, parent, tokens)
     logits_close(out["logits"], ref.logits, BF16_TOL)
+    logits_close(out["logits"], ref.logits, HI_LO_TOL)
     argmax_agrees_where_decided(out["argmax"], ref.logits, BF16_TOL)
     check_acceptance_against_oracle(out, tokens, parent)
