@@ -278,107 +278,165 @@ struct Cursor {
 };
 
 // ------------------------------------------------------------------------------------------------
-// Fused epilogue of 16 columns (tree nodes c0..c0+15) of one thread's output row. v/w hold the
-// complete sums (w: the up-projection half of a SwiGLU tile).
-template <typename T>
-__device__ __forceinline__ void epilogue_chunk(const EpiParams &ep, const float *rs, int tile, int lane_grp, int lane, int row,
-                                               bool row_ok, float gain, int c0, float (&v)[16], float (&w)[16], float (&xo)[16])
+// Finishing a 32-row group of an output tile. Every CTA that holds a share of a tile leaves its
+// accumulators in the workspace as [row group][gate|up][node][32 rows] fp32; the warp that arrives
+// last at the group's ticket (or the only holder) adds the shares in CTA order and applies the fused
+// epilogue. It works on four output rows at a time: lane = (node sub-index ns = lane / 8, row quad
+// r4 = lane % 8) and iteration `it` handles node 4 * it + ns, so that the shares, the residual stream
+// and every output move as 16- or 8-byte vectors, a rotary pair sits in one thread, and the loads of
+// several nodes and several shares are in flight together (this warp is alone on its scheduler:
+// what it costs is the number of dependent round trips, not the bytes).
+__device__ __forceinline__ uint2 pack4_bf16(const __nv_bfloat16 (&h)[4])
 {
-    if (ep.ssq_in != nullptr) {
+    uint2 r;
+    r.x = (uint32_t)__bfloat16_as_ushort(h[0]) | ((uint32_t)__bfloat16_as_ushort(h[1]) << 16);
+    r.y = (uint32_t)__bfloat16_as_ushort(h[2]) | ((uint32_t)__bfloat16_as_ushort(h[3]) << 16);
+    return r;
+}
+
+// Four consecutive bf16 values at dst (8-byte aligned) and, if dst_lo is not null, their remainders.
+__device__ __forceinline__ void store4_split(__nv_bfloat16 *dst, __nv_bfloat16 *dst_lo, const float (&v)[4])
+{
+    __nv_bfloat16 hi[4], lo[4];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) { const float r = rs[c0 + j]; v[j] *= r; w[j] *= r; }
-    }
-    // all loads of the chunk are issued before any dependent store so that they overlap
-    if (ep.mode == EPI_SWIGLU) {
-        T *hrow = reinterpret_cast<T *>(ep.h) + row;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            if (row_ok && c0 + j < ep.n) {
-                const float sg = v[j] / (1.0f + __expf(-v[j]));
-                store_split<T>(hrow + (size_t)(c0 + j) * ep.n_out, (size_t)kLoRows * ep.n_out, sg * w[j], ep.comp != 0);
-            }
-        }
+    for (int k = 0; k < 4; ++k) split_bf16(v[k], hi[k], lo[k]);
+    *reinterpret_cast<uint2 *>(dst) = pack4_bf16(hi);
+    if (dst_lo != nullptr) *reinterpret_cast<uint2 *>(dst_lo) = pack4_bf16(lo);
+}
+
+template <bool DUAL>
+__device__ __forceinline__ void finish_rows(const ChainParams &p, const GemmDesc &d, const float *rs, int tile, int tile_i0,
+                                            int first_cta, int last_cta, int lane_grp, int lane)
+{
+    constexpr int G = 4;                    // nodes per lane whose loads are in flight together
+    constexpr int kBatch = DUAL ? 3 : 6;    // shares in flight together
+    typedef __nv_bfloat16 T;
+    const EpiParams &ep = d.ep;
+    const int ns = lane >> 3, r4 = lane & 7;
+    const int row0 = tile * kTileM + lane_grp * 32 + 4 * r4;   // first of this lane's four output rows
+    const int n_valid = min(4, ep.n_out - row0);               // how many of them exist
+    const bool rows_ok = n_valid == 4;                         // all modes but PLAIN have n_out % 4 == 0
+    const bool comp = ep.comp != 0;
+    const size_t part_stride = (size_t)2 * p.n_pad * kTileM;
+    const size_t lane_off = (size_t)lane_grp * 2 * p.n_pad * 32 + 4 * r4;
+
+    // per-lane constants of the mode
+    float gain[4] = {0.f, 0.f, 0.f, 0.f};
+    int sec = 0, head = 0, e = 0, cidx = 0;
+    if (ep.mode == EPI_RESID && ep.xg_out != nullptr && rows_ok) {
+        const uint2 g4 = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const T *>(ep.gain_next) + row0));
+        gain[0] = __uint_as_float(g4.x << 16); gain[1] = __uint_as_float(g4.x & 0xffff0000u);
+        gain[2] = __uint_as_float(g4.y << 16); gain[3] = __uint_as_float(g4.y & 0xffff0000u);
     } else if (ep.mode == EPI_QKV) {
-        const int sec = row / ep.d, cidx = row - sec * ep.d;
-        const int head = cidx / ep.hd, e = cidx - head * ep.hd;
-        float2 cs[16];
+        sec = row0 / ep.d; cidx = row0 - sec * ep.d;
+        head = cidx / ep.hd; e = cidx - head * ep.hd;
+    }
+
+    for (int it0 = 0; it0 < (p.n_pad >> 2); it0 += G) {
+        float4 a[G], b[G], xr[G], cs[G];
+        // loads that do not depend on the shares go first
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-            cs[j] = (sec < 2 && row_ok && c0 + j < ep.n) ? __ldg(ep.rope_cs + (size_t)(c0 + j) * (ep.hd >> 1) + (e >> 1))
-                                                          : make_float2(1.f, 0.f);
-        T *dst, *dst_lo;               // where a value goes, and where its remainder goes
-        size_t node_stride;
-        if (sec == 0) {
-            dst = reinterpret_cast<T *>(ep.q_out) + cidx;
-            dst_lo = dst + (size_t)kLoRows * ep.d;
-            node_stride = ep.d;
-        } else {
-            dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P) * ep.hd + e;
-            dst_lo = reinterpret_cast<T *>(ep.kv_lo) + ((size_t)((sec - 1) * (ep.d / ep.hd) + head) * kLoRows) * ep.hd + e;
-            node_stride = ep.hd;
+        for (int g = 0; g < G; ++g) {
+            const int node = (it0 + g) * 4 + ns;
+            const bool ok = rows_ok && node < ep.n;
+            a[g] = b[g] = xr[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+            cs[g] = make_float4(1.f, 0.f, 1.f, 0.f);
+            if (ep.mode == EPI_RESID && ok) xr[g] = __ldcg(reinterpret_cast<const float4 *>(ep.x + (size_t)node * ep.n_out + row0));
+            if (ep.mode == EPI_QKV && ok && sec < 2)
+                cs[g] = __ldg(reinterpret_cast<const float4 *>(ep.rope_cs + (size_t)node * (ep.hd >> 1) + (e >> 1)));
         }
+        // the shares, added in CTA order
+        for (int c = first_cta; c <= last_cta; c += kBatch) {
+            float4 t[kBatch][G], u[DUAL ? kBatch : 1][G];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            // the rotary partner (2t <-> 2t+1) lives in the neighbouring lane
-            const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
-            const float rot = (lane & 1) ? (other * cs[j].y + v[j] * cs[j].x) : (v[j] * cs[j].x - other * cs[j].y);
-            // queries get their lo plane; keys and values go to the cache rounded, their remainders to kv_lo
-            if (row_ok && c0 + j < ep.n) {
-                const size_t at = (size_t)(c0 + j) * node_stride;
-                if (ep.comp) store_split<T>(dst + at, dst_lo + at, rot);
-                else dst[at] = from_f32<T>(rot);
-            }
-        }
-    } else if (ep.mode == EPI_RESID) {
-        // xo: the residual values of this chunk, loaded by the caller together with the partial tiles
-        float *xr = ep.x + row;
+            for (int k = 0; k < kBatch; ++k) {
+                const int cc = min(c + k, last_cta);
+                // slot 0 of a CTA holds the tile in which its range starts, slot 1 any later one
+                const int slot = (cc * d.items_per_cta >= tile_i0) ? 0 : 1;
+                const float *src = p.partials + ((size_t)cc * 2 + slot) * part_stride + lane_off;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            xo[j] = (row_ok && c0 + j < ep.n) ? xo[j] + v[j] : 0.f;
-            if (row_ok && c0 + j < ep.n) xr[(size_t)(c0 + j) * ep.n_out] = xo[j];
-        }
-        if (ep.xg_out != nullptr) {
-            // what the next RMSNorm needs: gain * x in the GEMM input dtype, and this warp's share
-            // (32 rows) of every node's sum of squares
-            T *gr = reinterpret_cast<T *>(ep.xg_out) + row;
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-                if (row_ok && c0 + j < ep.n) store_split<T>(gr + (size_t)(c0 + j) * ep.n_out, (size_t)kLoRows * ep.n_out, xo[j] * gain, ep.comp != 0);
-            // column sums over the warp's 32 rows by recursive halving: after exchanging with
-            // lane^16, ^8, ^4, ^2 a lane is left with one column, after lane^1 with its full sum
-            // (16 shuffles instead of 80). Column held by a lane: bits 4..1 of the lane, msb first.
-            float s8[8], s4[4], s2[2], s1;
-            {
-                const bool up = lane & 16;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float keep = up ? xo[8 + j] * xo[8 + j] : xo[j] * xo[j];
-                    const float give = up ? xo[j] * xo[j] : xo[8 + j] * xo[8 + j];
-                    s8[j] = keep + __shfl_xor_sync(0xffffffffu, give, 16);
+                for (int g = 0; g < G; ++g) {
+                    const int node = (it0 + g) * 4 + ns;
+                    t[k][g] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)node * 32));
+                    if (DUAL) u[k][g] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(p.n_pad + node) * 32));
                 }
             }
-            {
-                const bool up = lane & 8;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) s4[j] = (up ? s8[4 + j] : s8[j]) + __shfl_xor_sync(0xffffffffu, up ? s8[j] : s8[4 + j], 8);
-            }
-            {
-                const bool up = lane & 4;
+            for (int k = 0; k < kBatch; ++k) {
+                if (c + k <= last_cta) {
 #pragma unroll
-                for (int j = 0; j < 2; ++j) s2[j] = (up ? s4[2 + j] : s4[j]) + __shfl_xor_sync(0xffffffffu, up ? s4[j] : s4[2 + j], 4);
+                    for (int g = 0; g < G; ++g) {
+                        a[g].x += t[k][g].x; a[g].y += t[k][g].y; a[g].z += t[k][g].z; a[g].w += t[k][g].w;
+                        if (DUAL) { b[g].x += u[k][g].x; b[g].y += u[k][g].y; b[g].z += u[k][g].z; b[g].w += u[k][g].w; }
+                    }
+                }
             }
-            {
-                const bool up = lane & 2;
-                s1 = (up ? s2[1] : s2[0]) + __shfl_xor_sync(0xffffffffu, up ? s2[0] : s2[1], 2);
-            }
-            s1 += __shfl_xor_sync(0xffffffffu, s1, 1);
-            if (!(lane & 1)) ep.ssq_out[(size_t)(tile * 4 + lane_grp) * LLMCAD_MAX_TREE + c0 + (lane >> 1)] = s1;
         }
-    } else {
-        float *yr = ep.y + row;
+        // fused epilogue
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-            if (row_ok && c0 + j < ep.n) yr[(size_t)(c0 + j) * ep.ldy] = v[j];
+        for (int g = 0; g < G; ++g) {
+            const int node = (it0 + g) * 4 + ns;
+            const bool ok = rows_ok && node < ep.n;
+            float v[4] = {a[g].x, a[g].y, a[g].z, a[g].w};
+            if (ep.ssq_in != nullptr) {
+                const float r = rs[node];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) v[k] *= r;
+                if (DUAL) { b[g].x *= r; b[g].y *= r; b[g].z *= r; b[g].w *= r; }
+            }
+            if (ep.mode == EPI_SWIGLU) {
+                if (ok) {
+                    const float w[4] = {b[g].x, b[g].y, b[g].z, b[g].w};
+                    float hv[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) hv[k] = v[k] / (1.0f + __expf(-v[k])) * w[k];
+                    T *dst = reinterpret_cast<T *>(ep.h) + (size_t)node * ep.n_out + row0;
+                    store4_split(dst, comp ? dst + (size_t)kLoRows * ep.n_out : nullptr, hv);
+                }
+            } else if (ep.mode == EPI_QKV) {
+                if (ok) {
+                    // rotary pairs (2t, 2t+1) = (v0, v1), (v2, v3); values pass through with (cos, sin) = (1, 0)
+                    const float rot[4] = {v[0] * cs[g].x - v[1] * cs[g].y, v[0] * cs[g].y + v[1] * cs[g].x,
+                                          v[2] * cs[g].z - v[3] * cs[g].w, v[2] * cs[g].w + v[3] * cs[g].z};
+                    T *dst, *dst_lo;   // queries get a lo plane; keys and values go to the cache rounded, their remainders to kv_lo
+                    if (sec == 0) {
+                        dst = reinterpret_cast<T *>(ep.q_out) + (size_t)node * ep.d + cidx;
+                        dst_lo = dst + (size_t)kLoRows * ep.d;
+                    } else {
+                        dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P + node) * ep.hd + e;
+                        dst_lo = reinterpret_cast<T *>(ep.kv_lo) + ((size_t)((sec - 1) * (ep.d / ep.hd) + head) * kLoRows + node) * ep.hd + e;
+                    }
+                    store4_split(dst, comp ? dst_lo : nullptr, rot);
+                }
+            } else if (ep.mode == EPI_RESID) {
+                float xo[4] = {xr[g].x + v[0], xr[g].y + v[1], xr[g].z + v[2], xr[g].w + v[3]};
+                if (!ok) xo[0] = xo[1] = xo[2] = xo[3] = 0.f;
+                if (ok) *reinterpret_cast<float4 *>(ep.x + (size_t)node * ep.n_out + row0) = make_float4(xo[0], xo[1], xo[2], xo[3]);
+                if (ep.xg_out != nullptr) {
+                    // what the next RMSNorm needs: gain * x in the GEMM input format, and this row
+                    // group's share of every node's sum of squares
+                    if (ok) {
+                        const float xg[4] = {xo[0] * gain[0], xo[1] * gain[1], xo[2] * gain[2], xo[3] * gain[3]};
+                        T *dst = reinterpret_cast<T *>(ep.xg_out) + (size_t)node * ep.n_out + row0;
+                        store4_split(dst, comp ? dst + (size_t)kLoRows * ep.n_out : nullptr, xg);
+                    }
+                    float ss = xo[0] * xo[0] + xo[1] * xo[1] + xo[2] * xo[2] + xo[3] * xo[3];
+                    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+                    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+                    ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+                    if (r4 == 0) ep.ssq_out[(size_t)(tile * 4 + lane_grp) * LLMCAD_MAX_TREE + node] = ss;
+                }
+            } else if (node < ep.n) {
+                float *yr = ep.y + (size_t)node * ep.ldy + row0;
+                if (rows_ok && (ep.ldy & 3) == 0 && (reinterpret_cast<uintptr_t>(ep.y) & 15) == 0)
+                    *reinterpret_cast<float4 *>(yr) = make_float4(v[0], v[1], v[2], v[3]);
+                else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (k < n_valid) yr[k] = v[k];
+                }
+            }
+        }
     }
 }
 
@@ -468,6 +526,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                                         (c.half ? d.up_row_offset : 0) + c.tile * kTileM, full, pol_stream);
                     }
                     __threadfence_block();
+                    if (issued == 0) LLMCAD_TRACE(2);
                     ctl.a_issued = ++issued;     // the activation loader may now add its bytes to this stage
                     c.advance(p);
                     if (++s == p.stages) { s = 0; par ^= 1u; }
@@ -495,6 +554,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 if (t_idle == 0) t_idle = global_timer_ns();
                 else if (*abort_flag || global_timer_ns() - t_idle > kWaitLimitNs) { timed_out = true; break; }
             }
+            if (p.n_gemms == 1) LLMCAD_TRACE(6);
             // This CTA's weight stream has ended; its tail (partial-tile reduction, epilogue) and the
             // hand-over to the next kernel leave HBM idle. Pull the first tiles that the CTA with this
             // index will want in the next launch into L2 meanwhile.
@@ -600,11 +660,11 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 tc_commit(smem_u32(&ctl.tmem_full[buf]));
                 ++seg;
             }
+            if (p.n_gemms == 1) LLMCAD_TRACE(7);
         }
     } else {
         // ================================================= epilogue (warps 2..5)
         const int lane_grp = warp & 3;                 // TMEM lanes 32*lane_grp .. +31 belong to this warp
-        const int row_in_tile = lane_grp * 32 + lane;
         float *my_rs = ctl.rs[warp - 2];
         pdl_wait();
         if (threadIdx.x == 64) LLMCAD_TRACE(3);
@@ -668,8 +728,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             const Range r = cta_range(d);
             const int ipt = pairs_per_tile(d) * d.halves;
             const bool dual = d.halves == 2;
-            const size_t part_stride = (size_t)2 * p.n_pad * kTileM;   // floats per partial slot (gate | up)
-            const int quads = p.n_pad >> 2;                            // column quads per accumulator
+            const size_t part_stride = (size_t)2 * p.n_pad * kTileM;   // floats per workspace slot (gate | up)
             uint32_t *tickets = p.tickets + (size_t)g * kTicketsPerGemm;
             for (int seg_begin = r.begin; seg_begin < r.end && !timed_out; ++seg) {
                 const int tile = seg_begin / ipt;
@@ -677,52 +736,51 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 const int seg_end = min(r.end, tile_i0 + ipt);
                 const int buf = two_bufs ? (seg & 1) : 0;
                 const uint32_t use = two_bufs ? (seg >> 1) : seg;
-                const bool sole = (seg_begin == tile_i0 && seg_end == tile_i0 + ipt);   // this CTA holds the whole tile
                 const int first_cta = tile_i0 / d.items_per_cta;
                 const int last_cta = (tile_i0 + ipt - 1) / d.items_per_cta;
-                const int n_parts = last_cta - first_cta + 1;
+                const int n_parts = last_cta - first_cta + 1;           // CTAs that hold a share of this tile
+                const bool tail = p.n_gemms == 1 && seg_end == r.end;   // (tracing) the segment that ends this CTA's work
 
                 if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), use & 1u, abort_flag, lane)) { timed_out = true; break; }
                 tc_fence_after();
                 if (threadIdx.x == 64 && g < 4 && seg_begin == r.begin) LLMCAD_TRACE(4 + 2 * g);
+                if (threadIdx.x == 64 && tail) LLMCAD_TRACE(14);
 
+                // ---- this CTA's share of the tile goes to the workspace, lane = row of the 32-row group.
+                // With hi + lo activations a node's two accumulator columns are added first. Slot 0 of a
+                // CTA holds the tile in which its range starts, slot 1 any later one (a later tile is
+                // finished, by this same warp, before the next one is written).
                 const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * acc_cols;
-                const int row = tile * kTileM + row_in_tile;           // output feature (weight row)
-                const bool row_ok = row < ep.n_out;
-                bool finish = sole;
-                // 16 nodes of accumulator `hf` (0 gate or the only one, 1 up); with hi + lo activations
-                // the node's two columns are added here, before anything else sees them
-                auto ld_acc = [&](int hf, int c0, float (&v)[16]) {
-                    tc_ld16(t_lane + hf * nb + c0, v);
-                    if (p.comp) {
-                        float t[16];
-                        tc_ld16(t_lane + hf * nb + p.n_pad + c0, t);
+                float *dst = p.partials + ((size_t)blockIdx.x * 2 + (seg_begin == r.begin ? 0 : 1)) * part_stride +
+                             (size_t)lane_grp * 2 * p.n_pad * 32 + lane;
+                for (int hf = 0; hf < (dual ? 2 : 1); ++hf) {
+                    for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                        float v[16];
+                        tc_ld16(t_lane + hf * nb + c0, v);
+                        if (p.comp) {
+                            float t[16];
+                            tc_ld16(t_lane + hf * nb + p.n_pad + c0, t);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) v[j] += t[j];
-                    }
-                };
-
-                if (!sole) {
-                    // A tile shared by several CTAs: every sharer leaves its partial accumulator in the
-                    // workspace; the rows of a tile are independent per warp (32 rows each), so each
-                    // warp takes a ticket for its own row group and the last warp to arrive adds all
-                    // partials in CTA order and finishes those rows. Nobody waits for anybody.
-                    // Slot 0 of a CTA holds the segment that contains its range start, slot 1 the other.
-                    // Slot layout: [row group][gate|up][column quad][row 0..31][4 columns], so a lane
-                    // moves 16 bytes per access and a warp 512 contiguous bytes.
-                    float4 *dst = reinterpret_cast<float4 *>(p.partials + ((size_t)blockIdx.x * 2 + (seg_begin == r.begin ? 0 : 1)) * part_stride) +
-                                  (size_t)lane_grp * 2 * quads * 32 + lane;
-                    for (int hf = 0; hf < (dual ? 2 : 1); ++hf) {
-                        for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
-                            float v[16];
-                            ld_acc(hf, c0, v);
-#pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                dst[(size_t)(hf * quads + (c0 >> 2) + k) * 32] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+                            for (int j = 0; j < 16; ++j) v[j] += t[j];
                         }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) dst[(size_t)(hf * p.n_pad + c0 + j) * 32] = v[j];
                     }
+                }
+                if (threadIdx.x == 64 && tail) LLMCAD_TRACE(8);
+                // the accumulator has left TMEM: hand the buffer back to the MMA warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+
+                // ---- the rows of a tile are independent per warp (32 rows each): each warp takes a
+                // ticket for its own row group, and whoever arrives last adds all shares in CTA order
+                // and finishes those rows. Nobody waits for anybody.
+                bool finish = true;
+                if (n_parts > 1) {
                     __threadfence();
                     __syncwarp();
+                    if (threadIdx.x == 64 && tail) LLMCAD_TRACE(9);
                     int last = 0;
                     if (lane == 0) {
                         uint32_t *ctr = tickets + (size_t)tile * 4 + lane_grp;
@@ -730,67 +788,12 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                         if (last) { __threadfence(); *ctr = 0; }   // acquire side; the counter is ready for the next launch
                     }
                     finish = __shfl_sync(0xffffffffu, last, 0) != 0;
-                    // the accumulator is in the workspace now: hand the TMEM buffer back early
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+                    if (threadIdx.x == 64 && tail) LLMCAD_TRACE(10);
                 }
-
                 if (finish) {
-                    float gain = 0.f;
-                    if (ep.mode == EPI_RESID && ep.xg_out != nullptr && row_ok)
-                        gain = to_f32<T>(reinterpret_cast<const T *>(ep.gain_next)[row]);
-                    for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
-                        float v[16], w[16], xo[16];
-                        if (ep.mode == EPI_RESID) {
-                            // issued first so that it overlaps the partial-tile loads below
-                            const float *xr = ep.x + row;
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) xo[j] = (row_ok && c0 + j < ep.n) ? __ldcg(xr + (size_t)(c0 + j) * ep.n_out) : 0.f;
-                        }
-                        if (sole) {
-                            ld_acc(0, c0, v);
-                            if (dual) ld_acc(1, c0, w);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) v[j] = w[j] = 0.f;
-                            // partial tiles added in CTA order; the loads of several CTAs are in flight at a time
-                            const size_t lane_off = (size_t)lane_grp * 2 * quads * 32 + (size_t)(c0 >> 2) * 32 + lane;
-                            for (int hf = 0; hf < (dual ? 2 : 1); ++hf) {
-                                float *acc = hf ? w : v;
-                                constexpr int kBatch = 6;
-                                for (int c = first_cta; c <= last_cta; c += kBatch) {
-                                    float4 t[kBatch][4];
-#pragma unroll
-                                    for (int u = 0; u < kBatch; ++u) {
-                                        const int cc = min(c + u, last_cta);
-                                        const int slot = (cc * d.items_per_cta >= tile_i0) ? 0 : 1;
-                                        const float4 *src = reinterpret_cast<const float4 *>(p.partials + ((size_t)cc * 2 + slot) * part_stride) +
-                                                            lane_off + (size_t)hf * quads * 32;
-#pragma unroll
-                                        for (int k = 0; k < 4; ++k) t[u][k] = __ldcg(src + (size_t)k * 32);
-                                    }
-#pragma unroll
-                                    for (int u = 0; u < kBatch; ++u) {
-                                        if (c + u <= last_cta) {
-#pragma unroll
-                                            for (int k = 0; k < 4; ++k) {
-                                                acc[4 * k] += t[u][k].x; acc[4 * k + 1] += t[u][k].y;
-                                                acc[4 * k + 2] += t[u][k].z; acc[4 * k + 3] += t[u][k].w;
-                                            }
-                                        }
-                                    }
-                                }
-                            }
-                        }
-                        epilogue_chunk<T>(ep, my_rs, tile, lane_grp, lane, row, row_ok, gain, c0, v, w, xo);
-                    }
-                }
-                if (sole) {
-                    // accumulator buffer drained: hand it back to the MMA warp
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+                    if (dual) finish_rows<true>(p, d, my_rs, tile, tile_i0, first_cta, last_cta, lane_grp, lane);
+                    else finish_rows<false>(p, d, my_rs, tile, tile_i0, first_cta, last_cta, lane_grp, lane);
+                    if (threadIdx.x == 64 && tail) LLMCAD_TRACE(13);
                 }
                 seg_begin = seg_end;
             }
