@@ -205,6 +205,7 @@ struct SharedCtl {
     uint32_t tmem_base;
     volatile int abort_flag;
     volatile uint32_t a_issued;     // ring items whose weight copy (and expect_tx) has been issued
+    volatile uint32_t dep_ok;       // the grid dependency is resolved: the previous kernel of the stream is complete
     float rs[4][LLMCAD_MAX_TREE];   // per epilogue warp: rsqrt(mean(x^2) + eps) of the folded input RMSNorm
 };
 
@@ -304,138 +305,169 @@ __device__ __forceinline__ void store4_split(__nv_bfloat16 *dst, __nv_bfloat16 *
     if (dst_lo != nullptr) *reinterpret_cast<uint2 *>(dst_lo) = pack4_bf16(lo);
 }
 
-template <bool DUAL>
-__device__ __forceinline__ void finish_rows(const ChainParams &p, const GemmDesc &d, const float *rs, int tile, int tile_i0,
-                                            int first_cta, int last_cta, int lane_grp, int lane)
+// Which workspace slot of CTA cc holds its share of the tile whose first item is tile_i0: slot 0
+// holds the tile in which the CTA's range starts, slot 1 any later one.
+__device__ __forceinline__ const float *share_ptr(const ChainParams &p, const GemmDesc &d, int cc, int tile_i0, int lane_grp)
 {
-    constexpr int G = 4;                    // nodes per lane whose loads are in flight together
-    constexpr int kBatch = DUAL ? 3 : 6;    // shares in flight together
+    const int slot = (cc * d.items_per_cta >= tile_i0) ? 0 : 1;
+    return p.partials + ((size_t)cc * 2 + slot) * ((size_t)2 * p.n_pad * kTileM) + (size_t)lane_grp * 2 * p.n_pad * 32;
+}
+
+// Everything the finishing code needs, gathered in one place so that the function below can be a
+// real call (one copy of its code in the kernel).
+struct FinishArgs {
+    const ChainParams *p;
+    const GemmDesc *d;              // in shared memory
+    const float *rs;                // per-node factors of the folded input norm (shared memory)
+    int tile, tile_i0, first_cta, last_cta, lane_grp;
+    int it_first, it_step;          // this warp finishes node groups it_first, it_first + it_step, ...
+};
+
+// Finishing a 32-row group of an output tile: add the shares of all CTAs that hold part of the
+// tile, in CTA order, and apply the fused epilogue. This is the one stretch of the kernel that runs
+// with nothing to hide behind: a warp alone on its scheduler, once per launch, after the weight
+// stream has ended. What it costs is the length of its dependent chain: round trips to L2 (a lone
+// warp gets a global load or store through only every 50 to 150 ns) and plain instruction latency;
+// and, the code being cold every time, instruction-cache misses, so it is kept small (one copy,
+// rolled loops, no specialisation per mode or shape). Hence: lane = (node sub-index ns = lane / 8,
+// row quad r4 = lane % 8), iteration `it` handles the four output rows 4 * r4 .. + 3 of node
+// 4 * it + ns, everything moves as 16- or 8-byte vectors, a rotary pair sits in one thread; and the
+// iterations of a group are dealt out to all the CTAs that end their work on this tile (it_first,
+// it_step), each of which would otherwise idle while one of them did everything.
+__device__ __noinline__ void finish_rows(const FinishArgs &fa, int lane)
+{
     typedef __nv_bfloat16 T;
+    const ChainParams &p = *fa.p;
+    const GemmDesc &d = *fa.d;
     const EpiParams &ep = d.ep;
+    const int mode = ep.mode, n_nodes = ep.n, n_out = ep.n_out, n_pad = p.n_pad;
+    const bool dual = d.halves == 2, comp = ep.comp != 0, has_rs = ep.ssq_in != nullptr, has_xg = ep.xg_out != nullptr;
+    const bool resid = mode == EPI_RESID;
+    const int tile = fa.tile, lane_grp = fa.lane_grp;
     const int ns = lane >> 3, r4 = lane & 7;
     const int row0 = tile * kTileM + lane_grp * 32 + 4 * r4;   // first of this lane's four output rows
-    const int n_valid = min(4, ep.n_out - row0);               // how many of them exist
-    const bool rows_ok = n_valid == 4;                         // all modes but PLAIN have n_out % 4 == 0
-    const bool comp = ep.comp != 0;
-    const size_t part_stride = (size_t)2 * p.n_pad * kTileM;
-    const size_t lane_off = (size_t)lane_grp * 2 * p.n_pad * 32 + 4 * r4;
+    const int n_valid = min(4, n_out - row0);                  // how many of them exist
+    const bool rows_ok = n_valid == 4;                         // all modes but EPI_PLAIN have n_out % 4 == 0
+    const int n_parts = fa.last_cta - fa.first_cta + 1;
 
     // per-lane constants of the mode
     float gain[4] = {0.f, 0.f, 0.f, 0.f};
     int sec = 0, head = 0, e = 0, cidx = 0;
-    if (ep.mode == EPI_RESID && ep.xg_out != nullptr && rows_ok) {
+    if (resid && has_xg && rows_ok) {
         const uint2 g4 = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const T *>(ep.gain_next) + row0));
         gain[0] = __uint_as_float(g4.x << 16); gain[1] = __uint_as_float(g4.x & 0xffff0000u);
         gain[2] = __uint_as_float(g4.y << 16); gain[3] = __uint_as_float(g4.y & 0xffff0000u);
-    } else if (ep.mode == EPI_QKV) {
+    } else if (mode == EPI_QKV) {
         sec = row0 / ep.d; cidx = row0 - sec * ep.d;
         head = cidx / ep.hd; e = cidx - head * ep.hd;
     }
+    // what a node's epilogue reads besides the shares: the residual (EPI_RESID) or the rotary
+    // (cos, sin) of the lane's two pairs (EPI_QKV, q and k sections)
+    const float *aux = nullptr;
+    size_t aux_stride = 0;
+    if (rows_ok && resid) { aux = ep.x + row0; aux_stride = (size_t)n_out; }
+    if (rows_ok && mode == EPI_QKV && sec < 2) { aux = reinterpret_cast<const float *>(ep.rope_cs) + 2 * (e >> 1); aux_stride = (size_t)ep.hd; }
+    const float4 aux_none = resid ? make_float4(0.f, 0.f, 0.f, 0.f) : make_float4(1.f, 0.f, 1.f, 0.f);
 
-    for (int it0 = 0; it0 < (p.n_pad >> 2); it0 += G) {
-        float4 a[G], b[G], xr[G], cs[G];
-        // loads that do not depend on the shares go first
+    const int iters = n_pad >> 2;
+    constexpr int G = 2;          // node groups whose loads travel together (one round trip per G iterations)
+    constexpr int kB = 4;         // shares in flight together, per node group
+    for (int itg = fa.it_first; itg < iters; itg += G * fa.it_step) {
+        // every load of the G iterations is issued before the first use
+        float4 axs[G], as[G], bs[G];
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-            const int node = (it0 + g) * 4 + ns;
-            const bool ok = rows_ok && node < ep.n;
-            a[g] = b[g] = xr[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-            cs[g] = make_float4(1.f, 0.f, 1.f, 0.f);
-            if (ep.mode == EPI_RESID && ok) xr[g] = __ldcg(reinterpret_cast<const float4 *>(ep.x + (size_t)node * ep.n_out + row0));
-            if (ep.mode == EPI_QKV && ok && sec < 2)
-                cs[g] = __ldg(reinterpret_cast<const float4 *>(ep.rope_cs + (size_t)node * (ep.hd >> 1) + (e >> 1)));
+            const int node = min(itg + g * fa.it_step, iters - 1) * 4 + ns;
+            axs[g] = aux_none;
+            if (aux != nullptr && node < n_nodes) axs[g] = __ldcg(reinterpret_cast<const float4 *>(aux + (size_t)node * aux_stride));
+            as[g] = bs[g] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        // the shares, added in CTA order
-        for (int c = first_cta; c <= last_cta; c += kBatch) {
-            float4 t[kBatch][G], u[DUAL ? kBatch : 1][G];
+        for (int k0 = 0; k0 < n_parts; k0 += kB) {
+            float4 t[G][kB], u[G][kB];
 #pragma unroll
-            for (int k = 0; k < kBatch; ++k) {
-                const int cc = min(c + k, last_cta);
-                // slot 0 of a CTA holds the tile in which its range starts, slot 1 any later one
-                const int slot = (cc * d.items_per_cta >= tile_i0) ? 0 : 1;
-                const float *src = p.partials + ((size_t)cc * 2 + slot) * part_stride + lane_off;
+            for (int k = 0; k < kB; ++k) {
+                const float *sk = share_ptr(p, d, fa.first_cta + min(k0 + k, n_parts - 1), fa.tile_i0, lane_grp) + 4 * r4;
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    const int node = (it0 + g) * 4 + ns;
-                    t[k][g] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)node * 32));
-                    if (DUAL) u[k][g] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(p.n_pad + node) * 32));
+                    const int node = min(itg + g * fa.it_step, iters - 1) * 4 + ns;
+                    t[g][k] = __ldcg(reinterpret_cast<const float4 *>(sk + (size_t)node * 32));
+                    if (dual) u[g][k] = __ldcg(reinterpret_cast<const float4 *>(sk + (size_t)(n_pad + node) * 32));
                 }
             }
 #pragma unroll
-            for (int k = 0; k < kBatch; ++k) {
-                if (c + k <= last_cta) {
+            for (int k = 0; k < kB; ++k) {
+                if (k0 + k < n_parts) {          // CTA order
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
-                        a[g].x += t[k][g].x; a[g].y += t[k][g].y; a[g].z += t[k][g].z; a[g].w += t[k][g].w;
-                        if (DUAL) { b[g].x += u[k][g].x; b[g].y += u[k][g].y; b[g].z += u[k][g].z; b[g].w += u[k][g].w; }
+                        as[g].x += t[g][k].x; as[g].y += t[g][k].y; as[g].z += t[g][k].z; as[g].w += t[g][k].w;
+                        if (dual) { bs[g].x += u[g][k].x; bs[g].y += u[g][k].y; bs[g].z += u[g][k].z; bs[g].w += u[g][k].w; }
                     }
                 }
             }
         }
-        // fused epilogue
-#pragma unroll
         for (int g = 0; g < G; ++g) {
-            const int node = (it0 + g) * 4 + ns;
-            const bool ok = rows_ok && node < ep.n;
-            float v[4] = {a[g].x, a[g].y, a[g].z, a[g].w};
-            if (ep.ssq_in != nullptr) {
-                const float r = rs[node];
+        const int it = itg + g * fa.it_step;
+        if (it >= iters) break;
+        const int node = it * 4 + ns;
+        const bool ok = rows_ok && node < n_nodes;
+        float4 ax = axs[0], a = as[0], b = bs[0];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) v[k] *= r;
-                if (DUAL) { b[g].x *= r; b[g].y *= r; b[g].z *= r; b[g].w *= r; }
+        for (int q = 1; q < G; ++q) if (q == g) { ax = axs[q]; a = as[q]; b = bs[q]; }
+        const float r = has_rs ? fa.rs[node] : 1.f;
+        float v[4] = {a.x * r, a.y * r, a.z * r, a.w * r};
+        float out[4];                 // what goes out in the activation format (hi and lo plane)
+        T *dst = nullptr, *dst_lo = nullptr;
+        if (resid) {
+            const float xo[4] = {ok ? ax.x + v[0] : 0.f, ok ? ax.y + v[1] : 0.f, ok ? ax.z + v[2] : 0.f, ok ? ax.w + v[3] : 0.f};
+            if (ok) *reinterpret_cast<float4 *>(ep.x + (size_t)node * n_out + row0) = make_float4(xo[0], xo[1], xo[2], xo[3]);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) out[k] = xo[k] * gain[k];
+            if (has_xg) {
+                // what the next RMSNorm needs: gain * x in the GEMM input format, and this row
+                // group's share of every node's sum of squares
+                dst = reinterpret_cast<T *>(ep.xg_out) + (size_t)node * n_out + row0;
+                dst_lo = dst + (size_t)kLoRows * n_out;
+                float ss = xo[0] * xo[0] + xo[1] * xo[1] + xo[2] * xo[2] + xo[3] * xo[3];
+                ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+                ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+                ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+                if (r4 == 0) ep.ssq_out[(size_t)(tile * 4 + lane_grp) * LLMCAD_MAX_TREE + node] = ss;
             }
-            if (ep.mode == EPI_SWIGLU) {
-                if (ok) {
-                    const float w[4] = {b[g].x, b[g].y, b[g].z, b[g].w};
-                    float hv[4];
+        } else if (mode == EPI_SWIGLU) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) hv[k] = v[k] / (1.0f + __expf(-v[k])) * w[k];
-                    T *dst = reinterpret_cast<T *>(ep.h) + (size_t)node * ep.n_out + row0;
-                    store4_split(dst, comp ? dst + (size_t)kLoRows * ep.n_out : nullptr, hv);
-                }
-            } else if (ep.mode == EPI_QKV) {
-                if (ok) {
-                    // rotary pairs (2t, 2t+1) = (v0, v1), (v2, v3); values pass through with (cos, sin) = (1, 0)
-                    const float rot[4] = {v[0] * cs[g].x - v[1] * cs[g].y, v[0] * cs[g].y + v[1] * cs[g].x,
-                                          v[2] * cs[g].z - v[3] * cs[g].w, v[2] * cs[g].w + v[3] * cs[g].z};
-                    T *dst, *dst_lo;   // queries get a lo plane; keys and values go to the cache rounded, their remainders to kv_lo
-                    if (sec == 0) {
-                        dst = reinterpret_cast<T *>(ep.q_out) + (size_t)node * ep.d + cidx;
-                        dst_lo = dst + (size_t)kLoRows * ep.d;
-                    } else {
-                        dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P + node) * ep.hd + e;
-                        dst_lo = reinterpret_cast<T *>(ep.kv_lo) + ((size_t)((sec - 1) * (ep.d / ep.hd) + head) * kLoRows + node) * ep.hd + e;
-                    }
-                    store4_split(dst, comp ? dst_lo : nullptr, rot);
-                }
-            } else if (ep.mode == EPI_RESID) {
-                float xo[4] = {xr[g].x + v[0], xr[g].y + v[1], xr[g].z + v[2], xr[g].w + v[3]};
-                if (!ok) xo[0] = xo[1] = xo[2] = xo[3] = 0.f;
-                if (ok) *reinterpret_cast<float4 *>(ep.x + (size_t)node * ep.n_out + row0) = make_float4(xo[0], xo[1], xo[2], xo[3]);
-                if (ep.xg_out != nullptr) {
-                    // what the next RMSNorm needs: gain * x in the GEMM input format, and this row
-                    // group's share of every node's sum of squares
-                    if (ok) {
-                        const float xg[4] = {xo[0] * gain[0], xo[1] * gain[1], xo[2] * gain[2], xo[3] * gain[3]};
-                        T *dst = reinterpret_cast<T *>(ep.xg_out) + (size_t)node * ep.n_out + row0;
-                        store4_split(dst, comp ? dst + (size_t)kLoRows * ep.n_out : nullptr, xg);
-                    }
-                    float ss = xo[0] * xo[0] + xo[1] * xo[1] + xo[2] * xo[2] + xo[3] * xo[3];
-                    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
-                    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-                    ss += __shfl_xor_sync(0xffffffffu, ss, 4);
-                    if (r4 == 0) ep.ssq_out[(size_t)(tile * 4 + lane_grp) * LLMCAD_MAX_TREE + node] = ss;
-                }
-            } else if (node < ep.n) {
-                float *yr = ep.y + (size_t)node * ep.ldy + row0;
-                if (rows_ok && (ep.ldy & 3) == 0 && (reinterpret_cast<uintptr_t>(ep.y) & 15) == 0)
-                    *reinterpret_cast<float4 *>(yr) = make_float4(v[0], v[1], v[2], v[3]);
-                else {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (k < n_valid) yr[k] = v[k];
-                }
+            for (int k = 0; k < 4; ++k) out[k] = v[k] / (1.0f + __expf(-v[k]));
+            out[0] *= b.x * r; out[1] *= b.y * r; out[2] *= b.z * r; out[3] *= b.w * r;
+            dst = reinterpret_cast<T *>(ep.h) + (size_t)node * n_out + row0;
+            dst_lo = dst + (size_t)kLoRows * n_out;
+        } else if (mode == EPI_QKV) {
+            // rotary pairs (2t, 2t+1) = (v0, v1), (v2, v3); values pass through with (cos, sin) = (1, 0)
+            out[0] = v[0] * ax.x - v[1] * ax.y; out[1] = v[0] * ax.y + v[1] * ax.x;
+            out[2] = v[2] * ax.z - v[3] * ax.w; out[3] = v[2] * ax.w + v[3] * ax.z;
+            // queries get a lo plane; keys and values go to the cache rounded, their remainders to kv_lo
+            if (sec == 0) {
+                dst = reinterpret_cast<T *>(ep.q_out) + (size_t)node * ep.d + cidx;
+                dst_lo = dst + (size_t)kLoRows * ep.d;
+            } else {
+                dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P + node) * ep.hd + e;
+                dst_lo = reinterpret_cast<T *>(ep.kv_lo) + ((size_t)((sec - 1) * (ep.d / ep.hd) + head) * kLoRows + node) * ep.hd + e;
             }
+        } else if (node < n_nodes) {
+            float *yr = ep.y + (size_t)node * ep.ldy + row0;
+            if (rows_ok && (ep.ldy & 3) == 0 && (reinterpret_cast<uintptr_t>(ep.y) & 15) == 0)
+                *reinterpret_cast<float4 *>(yr) = make_float4(v[0], v[1], v[2], v[3]);
+            else {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (k < n_valid) yr[k] = v[k];
+            }
+        }
+        if (dst != nullptr && ok) {
+            T hi[4], lo[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) split_bf16(out[k], hi[k], lo[k]);
+            *reinterpret_cast<uint2 *>(dst) = pack4_bf16(hi);
+            if (comp) *reinterpret_cast<uint2 *>(dst_lo) = pack4_bf16(lo);
+        }
         }
     }
 }
@@ -448,6 +480,17 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ SharedCtl ctl;
+    // The epilogue reads its GEMM's description (pointers, sizes, mode) all over the finishing code.
+    // From the kernel parameters, indexed by the GEMM's number, every first touch of a constant-cache
+    // line is a miss that stalls the lone finishing warp for most of a microsecond; a copy in shared
+    // memory, made while the first weights are still on their way, costs nothing to read.
+    __shared__ __align__(16) GemmDesc s_desc[kMaxChain];
+    {
+        static_assert(sizeof(GemmDesc) % 4 == 0, "GemmDesc is copied word by word");
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(&p.g[0]);
+        uint32_t *dst = reinterpret_cast<uint32_t *>(&s_desc[0]);
+        for (int i = threadIdx.x; i < (int)(sizeof(GemmDesc) / 4) * p.n_gemms; i += kThreads) dst[i] = src[i];
+    }
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t nb = (uint32_t)p.n_pad * (p.comp ? 2u : 1u);   // activation rows per k-block = the MMA N: nodes (hi | lo)
@@ -477,6 +520,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         }
         ctl.abort_flag = 0;
         ctl.a_issued = 0;
+        ctl.dep_ok = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -510,6 +554,15 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             uint32_t par = 1, issued = 0, prefetched = 0;   // a fresh barrier passes a wait on parity 1: no special first lap
             uint64_t t_idle = 0;
             while (!c.done(p)) {
+                // While the previous kernel is still in its tail, a full-speed fill of every ring of the
+                // grid would sit in the memory system in front of that tail's few, latency-bound accesses
+                // and stretch it by more than the head start is worth: hold back after pre_items.
+                if (issued >= (uint32_t)p.pre_items && !ctl.dep_ok) {
+                    __nanosleep(64);
+                    if (t_idle == 0) t_idle = global_timer_ns();
+                    else if (*abort_flag || global_timer_ns() - t_idle > kWaitLimitNs) { timed_out = true; break; }
+                    continue;
+                }
                 if (mbar_try(smem_u32(&ctl.empty[s]), par)) {
                     const GemmDesc &d = p.g[c.g];
                     const int nk = c.nk();
@@ -585,6 +638,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             int s = 0, ready = 0, traced_g = 0;
             uint32_t i = 0;
             pdl_wait();
+            ctl.dep_ok = 1;
             while (!c.done(p) && !timed_out) {
                 uint64_t t0 = 0;
                 // (1) the stage is ours: the producer has passed its "empty" wait and armed the barrier
@@ -670,7 +724,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         if (threadIdx.x == 64) LLMCAD_TRACE(3);
         uint32_t seg = 0;
         for (int g = 0; g < p.n_gemms && !timed_out; ++g) {
-            const GemmDesc &d = p.g[g];
+            const GemmDesc &d = s_desc[g];
             const EpiParams &ep = d.ep;
             // ---- grid barrier: everything GEMM g-1 wrote (activations, residual, norm sums) is final
             if (g > 0) {
@@ -773,28 +827,51 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
 
-                // ---- the rows of a tile are independent per warp (32 rows each): each warp takes a
-                // ticket for its own row group, and whoever arrives last adds all shares in CTA order
-                // and finishes those rows. Nobody waits for anybody.
-                bool finish = true;
-                if (n_parts > 1) {
+                // ---- finishing. The rows of a tile are independent per warp (32 rows each), so each
+                // warp works with the same-numbered warps of the other CTAs that hold a share of the
+                // tile, through two counters per (tile, row group): arrivals (a share is in the
+                // workspace) and departures. The CTAs whose range ends in this tile (all sharers, except
+                // the last one when its range goes on into the next tile) have nothing left to do: each
+                // waits until every share has arrived and finishes its part of the nodes. A CTA that goes
+                // on only announces its share; it held the tile's last k-blocks first thing in the
+                // kernel, so nobody waits for it in practice, and it waits for nobody.
+                FinishArgs fa;
+                fa.p = &p; fa.d = &d; fa.rs = my_rs;
+                fa.tile = tile; fa.tile_i0 = tile_i0; fa.first_cta = first_cta; fa.last_cta = last_cta; fa.lane_grp = lane_grp;
+                if (n_parts == 1) {
+                    fa.it_first = 0; fa.it_step = 1;
+                    finish_rows(fa, lane);
+                } else {
+                    uint32_t *ctr = tickets + ((size_t)tile * 4 + lane_grp) * 2;
                     __threadfence();
                     __syncwarp();
                     if (threadIdx.x == 64 && tail) LLMCAD_TRACE(9);
-                    int last = 0;
-                    if (lane == 0) {
-                        uint32_t *ctr = tickets + (size_t)tile * 4 + lane_grp;
-                        last = (atomicAdd(ctr, 1u) == (uint32_t)n_parts - 1u);
-                        if (last) { __threadfence(); *ctr = 0; }   // acquire side; the counter is ready for the next launch
+                    if (lane == 0) atomicAdd(ctr, 1u);
+                    if (seg_end == r.end) {
+                        // (a range never goes beyond the last tile)
+                        const int n_fin = n_parts - ((min((last_cta + 1) * d.items_per_cta, d.n_tiles * ipt) > tile_i0 + ipt) ? 1 : 0);
+                        int bad = 0;
+                        if (lane == 0) {
+                            uint64_t t0 = 0;
+                            for (uint32_t spin = 0; ld_acquire_u32(ctr) < (uint32_t)n_parts; ++spin) {
+                                __nanosleep(64);
+                                if ((spin & 15u) == 15u) {
+                                    if (t0 == 0) t0 = global_timer_ns();
+                                    else if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) { bad = 1; break; }
+                                }
+                            }
+                            __threadfence();
+                        }
+                        if (__shfl_sync(0xffffffffu, bad, 0)) { timed_out = true; break; }
+                        if (threadIdx.x == 64 && tail) LLMCAD_TRACE(10);
+                        fa.it_first = (int)blockIdx.x - first_cta; fa.it_step = n_fin;
+                        finish_rows(fa, lane);
+                        __syncwarp();
+                        // the last one to leave puts the counters back for the next launch
+                        if (lane == 0 && atomicAdd(ctr + 1, 1u) == (uint32_t)n_fin - 1u) { ctr[0] = 0; ctr[1] = 0; }
                     }
-                    finish = __shfl_sync(0xffffffffu, last, 0) != 0;
-                    if (threadIdx.x == 64 && tail) LLMCAD_TRACE(10);
                 }
-                if (finish) {
-                    if (dual) finish_rows<true>(p, d, my_rs, tile, tile_i0, first_cta, last_cta, lane_grp, lane);
-                    else finish_rows<false>(p, d, my_rs, tile, tile_i0, first_cta, last_cta, lane_grp, lane);
-                    if (threadIdx.x == 64 && tail) LLMCAD_TRACE(13);
-                }
+                if (threadIdx.x == 64 && tail) LLMCAD_TRACE(13);
                 seg_begin = seg_end;
             }
             if (timed_out) break;
@@ -943,6 +1020,8 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
+    p.pre_items = 2;
+    if (const char *e = getenv("LLMCAD_GEMM_PRE_ITEMS")) p.pre_items = atoi(e);   // tuning aid
     // weight tiles pulled into L2 beyond the ring while the ring is blocked
     p.l2_ahead = 8;
     if (const char *e = getenv("LLMCAD_GEMM_L2_AHEAD")) p.l2_ahead = atoi(e);

@@ -35,11 +35,12 @@ struct ChainParams {
     int stages;         // depth of the shared-memory ring
     int tmem_cols;      // allocated TMEM columns (power of two)
     float *partials;    // [grid][2 slots][2 halves][n_pad][128] fp32 partial tiles
-    uint32_t *tickets;  // [kMaxChain][4096][4] arrivals per (GEMM, tile, 32-row group); zero between launches
+    uint32_t *tickets;  // [kMaxChain][4096][4][2] arrivals and departures per (GEMM, tile, 32-row group); zero between launches
     uint32_t *grid_counter;   // grid barrier between the GEMMs of a chain (monotonic)
     uint32_t barrier_base;    // value of the counter when this launch starts
     int32_t *status;
     unsigned long long *trace;  // optional [grid][16] timeline in ns (nullptr: off)
+    int pre_items;      // ring items a CTA may request before the previous kernel of the stream is complete
     int l2_ahead;       // ring items the producer may prefetch into L2 beyond the ring
     int next_items;     // leading items of `next` (the GEMM of the following launch) each CTA pulls into L2 when its own stream ends
     GemmDesc next;
@@ -57,7 +58,7 @@ bool make_act_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64
                        uint64_t plane_rows);
 
 size_t gemm_tc_partial_floats(int n_sms, int max_n_pad);
-constexpr size_t kTicketsPerGemm = 4096 * 4;
+constexpr size_t kTicketsPerGemm = 4096 * 4 * 2;
 
 // Describes one GEMM for a chain (fills everything but items_per_cta, which the launcher sets).
 GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled = nullptr);
