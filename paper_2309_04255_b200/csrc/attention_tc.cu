@@ -106,9 +106,6 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     const int cta = blockIdx.y * gridDim.x + blockIdx.x;
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 0] = global_timer_ns();
     pdl_launch_dependents();
-    pdl_wait();
-    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 1] = global_timer_ns();
-    if (*status) return;   // uniform over the grid: set only by kernels that ran before this one
     extern __shared__ __align__(128) uint8_t sm[];
     uint8_t *s_q = sm;                                      // [n_pad][256 B], with COMP followed by the lo plane
     uint8_t *s_k = s_q + (size_t)(COMP ? 2 : 1) * n_pad * kRowBytes;   // [kStages][64][256 B]
@@ -140,7 +137,23 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         }
     };
 
-    // queries of this head (rows >= n are zero) and the first key tiles
+    // The prefix keys and values were written by earlier passes: the first tiles that lie wholly in
+    // the prefix are requested before the grid dependency, while the QKV GEMM of this layer is still
+    // finishing; the queries, the tree nodes' K/V and the status word wait for it.
+    bool early[kStages - 1];
+#pragma unroll
+    for (int st = 0; st < kStages - 1; ++st) {
+        early[st] = t_begin + st < t_end && (t_begin + st + 1) * kKeyTile <= P;
+        if (early[st]) load_tile(t_begin + st, st);
+    }
+    pdl_wait();
+    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 1] = global_timer_ns();
+    if (*status) {             // uniform over the grid: set only by kernels that ran before this one
+        cp_commit();
+        cp_wait<0>();          // nothing may still be writing this CTA's shared memory when it exits
+        return;
+    }
+    // queries of this head (rows >= n are zero) and the remaining first key tiles
     for (int c = tid; c < n_pad * 16; c += kAtThreads) {
         const int r = c >> 4, ch = c & 15;
         const bool ok = r < n;
@@ -159,9 +172,10 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
             cp_async16(smem_u32(s_vl) + swz(r, ch), vl + off, ok);
         }
     }
+#pragma unroll
     for (int st = 0; st < kStages - 1; ++st) {
-        if (t_begin + st < t_end) load_tile(t_begin + st, st);
-        cp_commit();                            // group 0 also carries the queries
+        if (t_begin + st < t_end && !early[st]) load_tile(t_begin + st, st);
+        cp_commit();                            // group 0 also carries the queries and everything requested early
     }
 
     const int q_tiles = n_pad >> 4;
