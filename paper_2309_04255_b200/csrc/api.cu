@@ -305,9 +305,7 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
         // Tensor-core path. The RMSNorms are folded into the GEMMs: whoever produces the residual
         // stream (the embedding gather, the O and down GEMMs) also writes gain * x in bf16 and
         // partial sums of squares; the consuming GEMM scales its accumulators by the per-node
-        // rsqrt(mean(x^2) + eps). The GEMMs between two attention calls (O, gate/up, down and the
-        // next layer's QKV, or the lm_head at the end) go out as one persistent chain kernel, so a
-        // layer is two launches.
+        // rsqrt(mean(x^2) + eps). Activations travel as bf16 hi + lo planes (ctx->comp).
         const int tiles4 = 4 * ((d + 127) / 128);
         CUDA_TRY(launch_embed_norm(base + ctx->lay.tok_embed, tokens, n, d,
                                    c.n_layers > 0 ? base + ctx->lay.attn_norm : base + ctx->lay.final_norm, ctx->x, ctx->xn,

@@ -1,33 +1,35 @@
-// Weight-streaming skinny GEMMs on the sm_100a tensor cores, run as a chain.
+// Weight-streaming skinny GEMMs on the sm_100a tensor cores.
 //
 // The one-shot verification of Sec. 3.2 visits every parameter once for all N <= 128 tree nodes,
 // so each GEMM is D[n_out][N] = W[n_out][K] * X[N][K]^T with a tiny N: it is bound by the bytes
 // of W coming from HBM. The kernel therefore puts W on the M side of tcgen05.mma (128 weight
 // rows per tile = the 128 TMEM lanes) and the tree nodes on the N side (padded to a multiple of
-// 16), and streams W exactly once through a deep TMA -> shared-memory ring.
+// 16; with hi + lo activation planes the MMA sees every node twice), and streams W exactly once
+// through a ring in shared memory: the weights are stored as pre-swizzled 16 KB tiles (pack.cu), so
+// a ring item (one tile, two k-blocks) is one contiguous 32 KB bulk copy.
 //
-// One launch runs up to four *dependent* GEMMs (e.g. O -> gate/up -> down -> next layer's QKV) on a
-// persistent grid of one CTA per SM. The weights do not depend on the activations, so the producer
-// warp keeps streaming the next GEMM's weight tiles into the ring while the current GEMM's tail
-// (partial-tile reduction, epilogue) and the grid barrier between the two are still in progress;
-// only the small activation tiles and the epilogues wait for the barrier. Within a GEMM the (tile,
-// k-block) items are split evenly over the CTAs (stream-K): a CTA's range may start and end inside
-// a tile; the sharers of a tile leave their partial accumulators in an fp32 workspace and whichever
-// warp arrives last at the tile's ticket counter adds them in a fixed (CTA) order and runs the fused
-// epilogue, so the result does not depend on timing and no CTA waits for another inside a GEMM.
+// The grid is persistent, one CTA per SM. The (tile, k-block pair, half) items of a GEMM are split
+// evenly over the CTAs (stream-K): a CTA's range may start and end inside a tile; every holder of a
+// tile leaves its accumulators in an fp32 workspace, and the CTAs whose range ends in that tile add
+// all shares in a fixed (CTA) order and run the fused epilogue together (see finish_rows), so the
+// result does not depend on timing. A launch may run up to four *dependent* GEMMs with grid
+// barriers between them (the producer keeps streaming the next GEMM's weights meanwhile); one GEMM
+// per launch, chained by programmatic dependent launch, measured faster and is what the pass uses.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer,
-// warps 2..5 = epilogue (tcgen05.ld of their 32 lanes each). Accumulators are double-buffered in
-// TMEM so that the epilogue of one tile overlaps the MMAs of the next.
+// Warp roles (224 threads): warp 0 = weight producer, warp 1 = TMEM allocator + MMA issuer,
+// warps 2..5 = epilogue (tcgen05.ld of their 32 lanes each), warp 6 = activation loader (TMA).
+// Accumulators are double-buffered in TMEM when two buffers fit, so that the epilogue of one tile
+// overlaps the MMAs of the next.
 //
-// The kernel is launched with programmatic stream serialization: the ring is filled with weight
-// tiles while the previous kernel of the pass is still running; activations, workspace and outputs
-// wait for the grid dependency. A status word left by an earlier phase is not looked at here: the
-// GEMMs then work on stale but finite activations and write only scratch, and the search/rollback
-// kernels at the end of the pass report the error.
+// Programmatic stream serialization: the ring is filled with weight tiles while the previous
+// kernel of the pass is still running; activations, workspace and outputs wait for the grid
+// dependency. A status word left by an earlier phase is not looked at here: the GEMMs then work on
+// stale but finite activations and write only scratch, and the search/rollback kernels at the end
+// of the pass report the error.
 //
-// Every wait (mbarrier, grid barrier) is bounded by a deadline; on expiry the kernel sets the status
-// word to LLMCAD_ERR_TIMEOUT, lets every role fall out of its loop, frees TMEM and returns.
+// Every wait (mbarrier, arrival counter, grid barrier) is bounded by a deadline; on expiry the
+// kernel sets the status word to LLMCAD_ERR_TIMEOUT, lets every role fall out of its loop, frees
+// TMEM and returns. All CTAs of a launch are resident at once (grid <= SM count, one CTA per SM).
 #include <cuda.h>
 
 #include <cstdlib>
