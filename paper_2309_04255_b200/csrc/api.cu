@@ -110,6 +110,8 @@ struct llmcad_ctx {
     uint32_t *attn_counters = nullptr;
     uint32_t *grid_counter = nullptr;   // grid barrier of the GEMM chains
     uint32_t barrier_base = 0;          // its value once everything enqueued so far has run
+    int ticket_set = 0;                 // arrival-counter set of the next GEMM launch (launches alternate)
+    int prev_gemms = 0, prev_ticket_words = 0;   // what the last GEMM launch touched in its set
     int64_t launches = 0;
     unsigned long long *trace = nullptr;   // optional timeline buffer (llmcad_set_gemm_trace): [launch][256][16]
     int trace_launch = 0, trace_capacity = 0;
@@ -231,6 +233,14 @@ struct Chain {
         if (p.n_gemms == 0) return LLMCAD_OK;
         p.partials = ctx->partials;
         p.tickets = ctx->flags;
+        p.ticket_set = ctx->ticket_set;
+        p.prev_gemms = ctx->prev_gemms;
+        p.prev_ticket_words = ctx->prev_ticket_words;
+        ctx->ticket_set ^= 1;
+        ctx->prev_gemms = p.n_gemms;
+        ctx->prev_ticket_words = 0;
+        for (int g = 0; g < p.n_gemms; ++g)
+            if (p.g[g].n_tiles * 4 > ctx->prev_ticket_words) ctx->prev_ticket_words = p.g[g].n_tiles * 4;
         p.grid_counter = ctx->grid_counter;
         p.barrier_base = ctx->barrier_base;
         p.status = status;
@@ -419,8 +429,10 @@ int reset_chain_sync(llmcad_ctx *ctx, cudaStream_t st)
 {
     if (!ctx->tc_gemm) return LLMCAD_OK;
     CUDA_TRY(cudaMemsetAsync(ctx->grid_counter, 0, sizeof(uint32_t), st));
-    CUDA_TRY(cudaMemsetAsync(ctx->flags, 0, (size_t)kMaxChain * kTicketsPerGemm * sizeof(uint32_t), st));
+    CUDA_TRY(cudaMemsetAsync(ctx->flags, 0, kTicketWords * sizeof(uint32_t), st));
     ctx->barrier_base = 0;
+    ctx->ticket_set = 0;
+    ctx->prev_gemms = ctx->prev_ticket_words = 0;
     return LLMCAD_OK;
 }
 
@@ -519,7 +531,7 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ok = ok && alloc((void **)&ctx->tb.rope_cs, 128 * (hd / 2) * sizeof(float2));
     ok = ok && alloc((void **)&ctx->ibuf, (520 + 128) * 4);
     ok = ok && alloc((void **)&ctx->partials, gemm_tc_partial_floats(2 * ctx->n_sms, 128) * 4);
-    ok = ok && alloc((void **)&ctx->flags, (size_t)kMaxChain * kTicketsPerGemm * 4);   // ticket counters
+    ok = ok && alloc((void **)&ctx->flags, kTicketWords * 4);   // arrival counters
     ok = ok && alloc((void **)&ctx->grid_counter, 256);
     const size_t ssq_floats = (size_t)4 * ((d + 127) / 128) * LLMCAD_MAX_TREE;
     ok = ok && alloc((void **)&ctx->ssq[0], ssq_floats * 4);

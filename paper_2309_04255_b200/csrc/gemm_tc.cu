@@ -724,6 +724,12 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         float *my_rs = ctl.rs[warp - 2];
         pdl_wait();
         if (threadIdx.x == 64) LLMCAD_TRACE(3);
+        // The previous launch (complete now) counted arrivals in the other counter set; the launch
+        // after this one will use that set again: put the words it touched back to zero.
+        for (int g = 0; g < p.prev_gemms; ++g) {
+            uint32_t *old = p.tickets + ((size_t)(p.ticket_set ^ 1) * kMaxChain + g) * kTicketsPerGemm;
+            for (int i = (int)blockIdx.x * 128 + (int)threadIdx.x - 64; i < p.prev_ticket_words; i += (int)gridDim.x * 128) old[i] = 0;
+        }
         uint32_t seg = 0;
         for (int g = 0; g < p.n_gemms && !timed_out; ++g) {
             const GemmDesc &d = s_desc[g];
@@ -785,7 +791,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             const int ipt = pairs_per_tile(d) * d.halves;
             const bool dual = d.halves == 2;
             const size_t part_stride = (size_t)2 * p.n_pad * kTileM;   // floats per workspace slot (gate | up)
-            uint32_t *tickets = p.tickets + (size_t)g * kTicketsPerGemm;
+            uint32_t *tickets = p.tickets + ((size_t)p.ticket_set * kMaxChain + g) * kTicketsPerGemm;
             for (int seg_begin = r.begin; seg_begin < r.end && !timed_out; ++seg) {
                 const int tile = seg_begin / ipt;
                 const int tile_i0 = tile * ipt;
@@ -831,12 +837,12 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
 
                 // ---- finishing. The rows of a tile are independent per warp (32 rows each), so each
                 // warp works with the same-numbered warps of the other CTAs that hold a share of the
-                // tile, through two counters per (tile, row group): arrivals (a share is in the
-                // workspace) and departures. The CTAs whose range ends in this tile (all sharers, except
-                // the last one when its range goes on into the next tile) have nothing left to do: each
-                // waits until every share has arrived and finishes its part of the nodes. A CTA that goes
-                // on only announces its share; it held the tile's last k-blocks first thing in the
-                // kernel, so nobody waits for it in practice, and it waits for nobody.
+                // tile, through one arrival counter per (tile, row group). The CTAs whose range ends in
+                // this tile (all holders, except the last one when its range goes on into the next tile)
+                // have nothing left to do: each waits until every share has arrived and finishes its
+                // part of the nodes. A CTA that goes on only announces its share; it held the tile's
+                // last k-blocks first thing in the kernel, so nobody waits for it in practice, and it
+                // waits for nobody. The counters are put back to zero by the next launch.
                 FinishArgs fa;
                 fa.p = &p; fa.d = &d; fa.rs = my_rs;
                 fa.tile = tile; fa.tile_i0 = tile_i0; fa.first_cta = first_cta; fa.last_cta = last_cta; fa.lane_grp = lane_grp;
@@ -844,11 +850,11 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     fa.it_first = 0; fa.it_step = 1;
                     finish_rows(fa, lane);
                 } else {
-                    uint32_t *ctr = tickets + ((size_t)tile * 4 + lane_grp) * 2;
-                    __threadfence();
+                    uint32_t *ctr = tickets + (size_t)tile * 4 + lane_grp;
                     __syncwarp();
+                    // release: the share written by all lanes of this warp is visible to whoever sees the count
+                    if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
                     if (threadIdx.x == 64 && tail) LLMCAD_TRACE(9);
-                    if (lane == 0) atomicAdd(ctr, 1u);
                     if (seg_end == r.end) {
                         // (a range never goes beyond the last tile)
                         const int n_fin = n_parts - ((min((last_cta + 1) * d.items_per_cta, d.n_tiles * ipt) > tile_i0 + ipt) ? 1 : 0);
@@ -862,15 +868,11 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                                     else if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) { bad = 1; break; }
                                 }
                             }
-                            __threadfence();
                         }
                         if (__shfl_sync(0xffffffffu, bad, 0)) { timed_out = true; break; }
                         if (threadIdx.x == 64 && tail) LLMCAD_TRACE(10);
                         fa.it_first = (int)blockIdx.x - first_cta; fa.it_step = n_fin;
                         finish_rows(fa, lane);
-                        __syncwarp();
-                        // the last one to leave puts the counters back for the next launch
-                        if (lane == 0 && atomicAdd(ctr + 1, 1u) == (uint32_t)n_fin - 1u) { ctr[0] = 0; ctr[1] = 0; }
                     }
                 }
                 if (threadIdx.x == 64 && tail) LLMCAD_TRACE(13);
