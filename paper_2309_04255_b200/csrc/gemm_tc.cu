@@ -323,6 +323,7 @@ struct FinishArgs {
     const float *rs;                // per-node factors of the folded input norm (shared memory)
     int tile, tile_i0, first_cta, last_cta, lane_grp;
     int it_first, it_step;          // this warp finishes node groups it_first, it_first + it_step, ...
+    unsigned long long *trace;      // optional timeline slots of this CTA (tracing)
 };
 
 // Finishing a 32-row group of an output tile: add the shares of all CTAs that hold part of the
@@ -336,7 +337,11 @@ struct FinishArgs {
 // 4 * it + ns, everything moves as 16- or 8-byte vectors, a rotary pair sits in one thread; and the
 // iterations of a group are dealt out to all the CTAs that end their work on this tile (it_first,
 // it_step), each of which would otherwise idle while one of them did everything.
-__device__ __noinline__ void finish_rows(const FinishArgs &fa, int lane)
+// G node groups travel together (one round trip per G iterations), kB shares per node group at a
+// time: tiles held by many CTAs have many shares and few iterations per finisher (G = 2, kB = 4),
+// tiles held by one or two have few shares and many iterations (G = 4, kB = 2).
+template <int G, int kB>
+__device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
 {
     typedef __nv_bfloat16 T;
     const ChainParams &p = *fa.p;
@@ -372,8 +377,6 @@ __device__ __noinline__ void finish_rows(const FinishArgs &fa, int lane)
     const float4 aux_none = resid ? make_float4(0.f, 0.f, 0.f, 0.f) : make_float4(1.f, 0.f, 1.f, 0.f);
 
     const int iters = n_pad >> 2;
-    constexpr int G = 2;          // node groups whose loads travel together (one round trip per G iterations)
-    constexpr int kB = 4;         // shares in flight together, per node group
     for (int itg = fa.it_first; itg < iters; itg += G * fa.it_step) {
         // every load of the G iterations is issued before the first use
         float4 axs[G], as[G], bs[G];
@@ -407,9 +410,14 @@ __device__ __noinline__ void finish_rows(const FinishArgs &fa, int lane)
                 }
             }
         }
-        for (int g = 0; g < G; ++g) {
+        if (fa.trace && itg == fa.it_first) fa.trace[11] = (unsigned long long)(as[0].x + as[G - 1].w != 12345.f) * global_timer_ns();
+        // two at a time, unrolled: the warp is alone on its scheduler and the two chains overlap
+        for (int g2 = 0; g2 < G; g2 += 2) {
+#pragma unroll
+        for (int gq = 0; gq < 2; ++gq) {
+        const int g = g2 + gq;
         const int it = itg + g * fa.it_step;
-        if (it >= iters) break;
+        if (it >= iters) continue;
         const int node = it * 4 + ns;
         const bool ok = rows_ok && node < n_nodes;
         float4 ax = axs[0], a = as[0], b = bs[0];
@@ -471,7 +479,15 @@ __device__ __noinline__ void finish_rows(const FinishArgs &fa, int lane)
             if (comp) *reinterpret_cast<uint2 *>(dst_lo) = pack4_bf16(lo);
         }
         }
+        }
+        if (fa.trace && itg == fa.it_first) fa.trace[15] = global_timer_ns();
     }
+}
+
+__device__ __forceinline__ void finish_rows(const FinishArgs &fa, int lane)
+{
+    if (fa.last_cta - fa.first_cta + 1 > 3) finish_rows_t<2, 4>(fa, lane);
+    else finish_rows_t<4, 2>(fa, lane);
 }
 
 }  // namespace
@@ -846,6 +862,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 FinishArgs fa;
                 fa.p = &p; fa.d = &d; fa.rs = my_rs;
                 fa.tile = tile; fa.tile_i0 = tile_i0; fa.first_cta = first_cta; fa.last_cta = last_cta; fa.lane_grp = lane_grp;
+                fa.trace = (threadIdx.x == 64 && tail && p.trace) ? p.trace + (size_t)blockIdx.x * 16 : nullptr;
                 if (n_parts == 1) {
                     fa.it_first = 0; fa.it_step = 1;
                     finish_rows(fa, lane);
