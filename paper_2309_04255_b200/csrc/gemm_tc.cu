@@ -46,7 +46,8 @@ constexpr int kBlockK = 64;     // bf16 elements per k-block = one 128-byte swiz
 constexpr int kThreads = 224;   // producer, MMA, 4 epilogue warps, activation loader
 constexpr int kATileBytes = kTileM * kBlockK * 2;  // 16 KB
 constexpr int kMaxStages = 16;
-constexpr int kPairK = 2;        // k-blocks per ring item: one 32 KB weight copy feeds 8 MMAs
+constexpr int kMaxPairK = 2;     // k-blocks per ring item (GemmDesc::pair_k): 2 = one 32 KB weight copy feeds 8 MMAs;
+                                 // 1 for wide activation tiles, which would leave too few ring stages otherwise
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -220,15 +221,18 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
 
 // A ring item is (tile, k-block pair, half): up to two consecutive 64-wide k-blocks of one
 // 128-row weight tile (32 KB, contiguous in the tiled layout) and the matching activation tiles.
-__device__ __forceinline__ int pairs_per_tile(const GemmDesc &g) { return (g.kb_per_tile + kPairK - 1) / kPairK; }
+__host__ __device__ __forceinline__ int pairs_per_tile(const GemmDesc &g) { return (g.kb_per_tile + g.pair_k - 1) / g.pair_k; }
+// the same with the k-blocks per item as a compile-time constant (the kernel is instantiated for 1 and 2)
+template <int PK> __device__ __forceinline__ int pairs_per_tile_c(const GemmDesc &g) { return (g.kb_per_tile + PK - 1) / PK; }
 
 // This CTA's share of GEMM g: items [begin, end) of its item list.
 struct Range {
     int begin, end;
 };
+template <int PK>
 __device__ __forceinline__ Range cta_range(const GemmDesc &g)
 {
-    const int total = g.n_tiles * pairs_per_tile(g) * g.halves;
+    const int total = g.n_tiles * pairs_per_tile_c<PK>(g) * g.halves;
     Range r;
     r.begin = min(total, (int)blockIdx.x * g.items_per_cta);
     r.end = min(total, r.begin + g.items_per_cta);
@@ -237,6 +241,7 @@ __device__ __forceinline__ Range cta_range(const GemmDesc &g)
 
 // Cursor over the concatenated item stream of the chain (all GEMMs, this CTA's ranges, in order).
 // Coordinates are kept incrementally: the single-thread roles have well under a microsecond per item.
+template <int PK>
 struct Cursor {
     int g;                 // current GEMM, == n_gemms when exhausted
     int tile, kp, half;    // coordinates of the current item (kp: k-block pair)
@@ -253,11 +258,11 @@ struct Cursor {
         while (true) {
             if (++g >= p.n_gemms) { g = p.n_gemms; left = 0; return; }
             const GemmDesc &d = p.g[g];
-            const Range r = cta_range(d);
+            const Range r = cta_range<PK>(d);
             left = r.end - r.begin;
             if (left <= 0) continue;
             kbpt = d.kb_per_tile;
-            ppt = pairs_per_tile(d);
+            ppt = pairs_per_tile_c<PK>(d);
             halves = d.halves;
             const int ipt = ppt * halves;
             tile = r.begin / ipt;
@@ -268,8 +273,8 @@ struct Cursor {
         }
     }
     __device__ bool done(const ChainParams &p) const { return g >= p.n_gemms; }
-    __device__ int kb0() const { return kp * kPairK; }
-    __device__ int nk() const { return min(kPairK, kbpt - kp * kPairK); }   // k-blocks in this item
+    __device__ int kb0() const { return kp * PK; }
+    __device__ int nk() const { return min(PK, kbpt - kp * PK); }   // k-blocks in this item
     __device__ void advance(const ChainParams &p)
     {
         if (--left <= 0) { next_gemm(p); return; }
@@ -492,7 +497,7 @@ __device__ __forceinline__ void finish_rows(const FinishArgs &fa, int lane)
 
 }  // namespace
 
-template <typename T>
+template <typename T, int PK>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams p)
 {
@@ -514,8 +519,8 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
     const uint32_t nb = (uint32_t)p.n_pad * (p.comp ? 2u : 1u);   // activation rows per k-block = the MMA N: nodes (hi | lo)
     const uint32_t b_tile_bytes = nb * kBlockK * 2;
     // stage: [weights k-block 0 | weights k-block 1 | activations k-block 0 | activations k-block 1]
-    const uint32_t stage_bytes = kPairK * (kATileBytes + b_tile_bytes);
-    const uint32_t b_off = kPairK * kATileBytes;
+    const uint32_t stage_bytes = PK * (kATileBytes + b_tile_bytes);
+    const uint32_t b_off = PK * kATileBytes;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t acc_cols = 2u * nb;                    // TMEM columns of one accumulator buffer (gate | up)
     const bool two_bufs = p.acc_bufs == 2;
@@ -565,7 +570,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         if (lane == 0) {
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            Cursor c, cpf;                   // next item to copy into the ring / to prefetch into L2
+            Cursor<PK> c, cpf;                   // next item to copy into the ring / to prefetch into L2
             c.init(p);
             cpf.init(p);
             int s = 0;
@@ -631,12 +636,12 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             // index will want in the next launch into L2 meanwhile.
             if (p.next_items > 0 && p.next.w_tiled != nullptr && !timed_out) {
                 const GemmDesc &d = p.next;
-                const int ppt = pairs_per_tile(d), ipt = ppt * d.halves;
-                const Range r = cta_range(d);
+                const int ppt = pairs_per_tile_c<PK>(d), ipt = ppt * d.halves;
+                const Range r = cta_range<PK>(d);
                 const int end = min(r.end, r.begin + p.next_items);
                 for (int it = r.begin; it < end; ++it) {
                     const int tile = it / ipt, q = it - tile * ipt, kp = q / d.halves, half = q - kp * d.halves;
-                    const int kb0 = kp * kPairK, nk = min(kPairK, d.kb_per_tile - kb0);
+                    const int kb0 = kp * PK, nk = min(PK, d.kb_per_tile - kb0);
                     const size_t t = (size_t)(tile + (half ? d.up_tile_offset : 0)) * d.kb_per_tile + kb0;
                     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(d.w_tiled + t * kATileBytes),
                                  "r"((uint32_t)nk * kATileBytes) : "memory");
@@ -651,7 +656,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         if (lane == 0) {
             uint64_t pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-            Cursor c;
+            Cursor<PK> c;
             c.init(p);
             int s = 0, ready = 0, traced_g = 0;
             uint32_t i = 0;
@@ -695,7 +700,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         // ================================================= MMA issuer
         if (lane == 0) {
             const uint32_t idesc = make_idesc(kTileM, (int)nb);
-            Cursor c;
+            Cursor<PK> c;
             c.init(p);
             uint32_t seg = 0, ph = 0;   // ph: parity the MMA warp waits for on its stage's "full" barrier
             int s = 0;
@@ -803,8 +808,8 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 }
                 __syncwarp();
             }
-            const Range r = cta_range(d);
-            const int ipt = pairs_per_tile(d) * d.halves;
+            const Range r = cta_range<PK>(d);
+            const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
             const bool dual = d.halves == 2;
             const size_t part_stride = (size_t)2 * p.n_pad * kTileM;   // floats per workspace slot (gate | up)
             uint32_t *tickets = p.tickets + ((size_t)p.ticket_set * kMaxChain + g) * kTicketsPerGemm;
@@ -982,6 +987,7 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)
     d.halves = ep.mode == EPI_SWIGLU ? 2 : 1;
     d.n_tiles = (ep.n_out + kTileM - 1) / kTileM;
     d.kb_per_tile = (n_in + kBlockK - 1) / kBlockK;
+    d.pair_k = kMaxPairK;
     d.up_row_offset = ep.n_out;
     d.items_per_cta = 0;
     d.w_tiled = static_cast<const uint8_t *>(w_tiled);
@@ -996,7 +1002,15 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
     if (p.n_gemms < 1 || p.n_gemms > kMaxChain) return cudaErrorInvalidValue;
     // a chain needs every CTA at every barrier: the grid is the SM count; a single GEMM may use fewer
     long long max_items = 0;
-    auto items_of = [](const GemmDesc &d) { return (long long)d.n_tiles * ((d.kb_per_tile + kPairK - 1) / kPairK) * d.halves; };
+    // Ring items of two k-blocks (one 32 KB weight copy each) unless the activation tiles are so wide
+    // (hi | lo planes of more than 64 nodes) that only two stages would fit; measured on B200:
+    // single k-blocks cost 10-17 % up to 64 nodes and gain 6 % at 128.
+    const int nb = p.n_pad * (p.comp ? 2 : 1);       // MMA N
+    if (nb > 256) return cudaErrorInvalidValue;
+    int pair_k = nb > 128 ? 1 : kMaxPairK;
+    if (const char *e = getenv("LLMCAD_GEMM_PAIR_K")) { const int v = atoi(e); if (v == 1 || v == 2) pair_k = v; }   // tuning aid
+    for (int g = 0; g < p.n_gemms; ++g) p.g[g].pair_k = pair_k;
+    auto items_of = [](const GemmDesc &d) { return (long long)d.n_tiles * pairs_per_tile(d) * d.halves; };
     for (int g = 0; g < p.n_gemms; ++g) {
         if (p.g[g].n_tiles > 4096) return cudaErrorInvalidValue;   // size of the ticket array
         const long long total = items_of(p.g[g]);
@@ -1014,9 +1028,7 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
         const long long total = items_of(p.g[0]);
         grid = (int)((total + p.g[0].items_per_cta - 1) / p.g[0].items_per_cta);
     }
-    const int nb = p.n_pad * (p.comp ? 2 : 1);       // MMA N
-    if (nb > 256) return cudaErrorInvalidValue;
-    const size_t stage_bytes = (size_t)kPairK * ((size_t)kATileBytes + (size_t)nb * kBlockK * 2);
+    const size_t stage_bytes = (size_t)pair_k * ((size_t)kATileBytes + (size_t)nb * kBlockK * 2);
     // One CTA per SM with the whole shared memory as the ring. (Two CTAs per SM with half-size rings,
     // so that the next kernel is resident during this one's tail, measured slower on B200.)
     // accumulators: (gate | up) x MMA N columns each, double-buffered when two of them fit
@@ -1036,8 +1048,11 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_chain_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemm_chain_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              227 * 1024 - 4096);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(gemm_chain_kernel<__nv_bfloat16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     227 * 1024 - 4096);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -1050,16 +1065,18 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
     p.next_items = 0;
     if (next != nullptr && next->w_tiled != nullptr && grid == n_sms) {
         p.next = *next;
+        p.next.pair_k = pair_k;
         const long long total = items_of(p.next);
         long long ipc = (total + grid - 1) / grid;
         if (p.next.halves == 2) ipc += ipc & 1;
         p.next.items_per_cta = (int)ipc;
-        p.next_items = 12;                      // x 32 KB x 148 CTAs = 57 MB, under half of L2
+        p.next_items = 24 / pair_k;             // 12 x 32 KB x 148 CTAs = 57 MB, under half of L2
         if (const char *e = getenv("LLMCAD_GEMM_NEXT_ITEMS")) p.next_items = atoi(e);
     }
     if (barrier_arrivals) *barrier_arrivals = 4u * (uint32_t)grid * (uint32_t)(p.n_gemms - 1);
     LaunchCfg lc(grid, kThreads, smem, st);
-    return cudaLaunchKernelEx(&lc.cfg, gemm_chain_kernel<__nv_bfloat16>, maps, p);
+    if (pair_k == 1) return cudaLaunchKernelEx(&lc.cfg, gemm_chain_kernel<__nv_bfloat16, 1>, maps, p);
+    return cudaLaunchKernelEx(&lc.cfg, gemm_chain_kernel<__nv_bfloat16, 2>, maps, p);
 }
 
 }  // namespace llmcad

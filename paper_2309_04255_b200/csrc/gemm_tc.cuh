@@ -13,6 +13,7 @@ constexpr int kMaxChain = 4;
 struct GemmDesc {
     int n_tiles;        // tiles of 128 output features
     int kb_per_tile;    // 64-wide k-blocks per tile
+    int pair_k;         // k-blocks per ring item (1 or 2), set by the launcher
     int halves;         // 2: every tile carries a gate and an up accumulator (SwiGLU), else 1
     int up_row_offset;  // row of the first up-projection row in the packed [2f][d] matrix
     int items_per_cta;  // ring items ((tile, k-block, half) triples) per CTA of the persistent grid

@@ -3,6 +3,7 @@ reads its operands from HBM, not from L2).
 
     python -m paper_2309_04255_b200.kernel_bench attention            # prefix x tree-size sweep (config 4)
     python -m paper_2309_04255_b200.kernel_bench gemm [--n 32] [--model 7b] [--only qkv,o]
+    python -m paper_2309_04255_b200.kernel_bench avnav [--model 7b] [--prefix 512] [--nodes 2,4,...]
 
 Each line of output is one JSON object. `--reps` launches are timed per case after `--warmup`.
 """
@@ -124,6 +125,66 @@ def bench_gemm(args):
         del Ws
 
 
+def bench_avnav(args):
+    """Autoregressive against non-autoregressive verification (Sec. 3.2, the comparison of Fig. 6):
+    N tokens verified by N passes of one token each, the prefix growing by one per pass, against one
+    pass over a chain of N nodes and one pass over a bushy tree of N nodes. The one-token pass is
+    also the plain decoding step of the target model."""
+    cfg = gen.MODELS[args.model]
+    dev = torch.device("cuda:0")
+    P = args.prefix
+    sizes = [int(x) for x in args.nodes.split(",")]
+    v = B.Verifier(cfg, P + 2 * max(sizes) + 8, device=dev)
+    v.pack_globals({k: gen.gen_tensor_device(cfg, k, -1, dev) for k in ("tok_embed", "final_norm", "lm_head")})
+    for l in range(cfg.n_layers):
+        v.pack_layer(l, {k: gen.gen_tensor_device(cfg, k, l, dev) for k in gen.LAYER_TENSORS})
+    kvv = v.kv_view()
+    g = torch.Generator(device=dev)
+    g.manual_seed(gen.MASTER_SEED)
+    for l in range(cfg.n_layers):
+        kvv[l, :, :, :P] = torch.randn((2, cfg.n_heads, P, cfg.head_dim), generator=g, device=dev, dtype=torch.float32).to(kvv.dtype)
+    peak, kind = _peak()
+    wbytes = cfg.weight_bytes()
+    root = torch.as_tensor(np.array([-1], np.int32), device=dev)
+
+    def timed(fn, reps):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    for n in sizes:
+        tokens = torch.as_tensor(gen.gen_tokens(cfg, n, seed=n), device=dev)
+        chain = torch.as_tensor(gen.tree_chain(n), device=dev)
+        bushy = torch.as_tensor(gen.tree_random(n, 16, "uniform4", n), device=dev)
+        outs1 = [v.new_outputs(1, want_logits=True) for _ in range(n)]
+        outn = v.new_outputs(n, want_logits=True)
+
+        def av():
+            for i in range(n):
+                v.verify_tree(P + i, tokens[i:i + 1], root, out=outs1[i])
+
+        av_ms = timed(av, args.reps)
+        step_logits = torch.cat([o["logits"] for o in outs1]).float()
+        nav_chain_ms = timed(lambda: v.verify_tree(P, tokens, chain, out=outn), args.reps)
+        # the same tokens in one pass must give the same logits as the N one-token passes
+        diff = (outn["logits"].float() - step_logits).abs().max().item() / step_logits.abs().max().item()
+        nav_tree_ms = timed(lambda: v.verify_tree(P, tokens, bushy, out=outn), args.reps)
+        assert v.last_status() == 0
+        print(json.dumps({
+            "bench": "av_vs_nav", "model": cfg.name, "prefix": P, "nodes": n,
+            "av_ms": av_ms, "nav_chain_ms": nav_chain_ms, "nav_tree_ms": nav_tree_ms,
+            "speedup_chain": av_ms / nav_chain_ms, "speedup_tree": av_ms / nav_tree_ms,
+            "decode_step_ms": av_ms / n, "decode_step_gbs": wbytes / (av_ms / n) / 1e6,
+            "decode_step_frac": wbytes / (av_ms / n) / 1e6 / peak, "peak": kind,
+            "chain_vs_steps_max_rel_diff": diff}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -139,10 +200,15 @@ def main():
     g.add_argument("--only", default="")
     g.add_argument("--reps", type=int, default=30)
     g.add_argument("--warmup", type=int, default=5)
+    n = sub.add_parser("avnav")
+    n.add_argument("--model", default="7b")
+    n.add_argument("--prefix", type=int, default=512)
+    n.add_argument("--nodes", default="2,4,8,16,32,64,128")
+    n.add_argument("--reps", type=int, default=3)
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("kernel_bench needs a CUDA device")
-    (bench_attention if args.cmd == "attention" else bench_gemm)(args)
+    {"attention": bench_attention, "gemm": bench_gemm, "avnav": bench_avnav}[args.cmd](args)
 
 
 if __name__ == "__main__":
