@@ -1056,7 +1056,7 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    p.pre_items = 2;
+    p.pre_items = 1 << 30;   // no holding back: measured best on B200 (the knob stays as a tuning aid)
     if (const char *e = getenv("LLMCAD_GEMM_PRE_ITEMS")) p.pre_items = atoi(e);   // tuning aid
     // weight tiles pulled into L2 beyond the ring while the ring is blocked
     p.l2_ahead = 8;
