@@ -43,7 +43,8 @@ namespace {
 
 constexpr int kTileM = 128;     // weight rows per tile
 constexpr int kBlockK = 64;     // bf16 elements per k-block = one 128-byte swizzle row
-constexpr int kThreads = 224;   // producer, MMA, 4 epilogue warps, activation loader
+constexpr int kThreads = 256;   // producer, MMA, 4 epilogue warps, activation loader, one spare: the four
+                                // non-epilogue warps each help one epilogue warp with the launch's last tile
 constexpr int kATileBytes = kTileM * kBlockK * 2;  // 16 KB
 constexpr int kMaxStages = 16;
 constexpr int kMaxPairK = 2;     // k-blocks per ring item (GemmDesc::pair_k): 2 = one 32 KB weight copy feeds 8 MMAs;
@@ -209,6 +210,7 @@ struct SharedCtl {
     volatile int abort_flag;
     volatile uint32_t a_issued;     // ring items whose weight copy (and expect_tx) has been issued
     volatile uint32_t dep_ok;       // the grid dependency is resolved: the previous kernel of the stream is complete
+    volatile uint32_t dumped[4];    // per row group: this CTA's share of its last tile is in the workspace
     float rs[4][LLMCAD_MAX_TREE];   // per epilogue warp: rsqrt(mean(x^2) + eps) of the folded input RMSNorm
 };
 
@@ -544,6 +546,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         ctl.abort_flag = 0;
         ctl.a_issued = 0;
         ctl.dep_ok = 0;
+        for (int w = 0; w < 4; ++w) ctl.dumped[w] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -739,7 +742,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             }
             if (p.n_gemms == 1) LLMCAD_TRACE(7);
         }
-    } else {
+    } else if (warp < 6) {
         // ================================================= epilogue (warps 2..5)
         const int lane_grp = warp & 3;                 // TMEM lanes 32*lane_grp .. +31 belong to this warp
         float *my_rs = ctl.rs[warp - 2];
@@ -868,14 +871,25 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 fa.p = &p; fa.d = &d; fa.rs = my_rs;
                 fa.tile = tile; fa.tile_i0 = tile_i0; fa.first_cta = first_cta; fa.last_cta = last_cta; fa.lane_grp = lane_grp;
                 fa.trace = (threadIdx.x == 64 && tail && p.trace) ? p.trace + (size_t)blockIdx.x * 16 : nullptr;
+                // The segment that ends this CTA's work in the launch: the warp of another role with
+                // the same row group (idle by now) takes every other node group (see the helpers below).
+                const bool helped = g + 1 == p.n_gemms && seg_end == r.end;
                 if (n_parts == 1) {
-                    fa.it_first = 0; fa.it_step = 1;
+                    if (helped) {
+                        __threadfence_block();
+                        __syncwarp();
+                        if (lane == 0) ctl.dumped[lane_grp] = 1;
+                    }
+                    fa.it_first = 0; fa.it_step = helped ? 2 : 1;
                     finish_rows(fa, lane);
                 } else {
                     uint32_t *ctr = tickets + (size_t)tile * 4 + lane_grp;
                     __syncwarp();
                     // release: the share written by all lanes of this warp is visible to whoever sees the count
-                    if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
+                    if (lane == 0) {
+                        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
+                        if (helped) ctl.dumped[lane_grp] = 1;
+                    }
                     if (threadIdx.x == 64 && tail) LLMCAD_TRACE(9);
                     if (seg_end == r.end) {
                         // (a range never goes beyond the last tile)
@@ -893,7 +907,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                         }
                         if (__shfl_sync(0xffffffffu, bad, 0)) { timed_out = true; break; }
                         if (threadIdx.x == 64 && tail) LLMCAD_TRACE(10);
-                        fa.it_first = (int)blockIdx.x - first_cta; fa.it_step = n_fin;
+                        fa.it_first = ((int)blockIdx.x - first_cta) * (helped ? 2 : 1); fa.it_step = n_fin * (helped ? 2 : 1);
                         finish_rows(fa, lane);
                     }
                 }
@@ -914,6 +928,48 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
     }
     __syncwarp();   // lanes that skipped their role's single-thread section rejoin their warp here
     timed_out = __any_sync(0xffffffffu, timed_out);   // keep the warp together on the way out
+
+    // ================================================= helpers
+    // The producer, MMA, loader and spare warps have nothing left to do when the launch's last GEMM
+    // reaches its tail, which is exactly when the epilogue warps have the most: each takes the row
+    // group warp % 4 of this CTA's last tile and finishes every other node group of it, next to the
+    // epilogue warp that owns the group (which takes the others).
+    if (!timed_out && (warp < 2 || warp > 5)) {
+        const int g = p.n_gemms - 1;
+        const GemmDesc &d = s_desc[g];
+        const Range r = cta_range<PK>(d);
+        if (r.end > r.begin) {
+            const int lane_grp = warp & 3;
+            const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
+            const int tile = (r.end - 1) / ipt, tile_i0 = tile * ipt;
+            const int first_cta = tile_i0 / d.items_per_cta, last_cta = (tile_i0 + ipt - 1) / d.items_per_cta;
+            const int n_parts = last_cta - first_cta + 1;
+            const int n_fin = n_parts == 1 ? 1 : n_parts - ((min((last_cta + 1) * d.items_per_cta, d.n_tiles * ipt) > tile_i0 + ipt) ? 1 : 0);
+            const uint32_t *ctr = p.tickets + ((size_t)p.ticket_set * kMaxChain + g) * kTicketsPerGemm + (size_t)tile * 4 + lane_grp;
+            int bad = 0;
+            if (lane == 0) {
+                // this CTA's own share first (a flag in shared memory), then everybody's (the arrival counter)
+                uint64_t t0 = 0;
+                for (uint32_t spin = 0; ctl.dumped[lane_grp] == 0 || (n_parts > 1 && ld_acquire_u32(ctr) < (uint32_t)n_parts); ++spin) {
+                    __nanosleep(ctl.dumped[lane_grp] == 0 ? 200 : 64);
+                    if ((spin & 15u) == 15u) {
+                        if (t0 == 0) t0 = global_timer_ns();
+                        else if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) { bad = 1; break; }
+                    }
+                }
+                __threadfence_block();
+            }
+            if (__shfl_sync(0xffffffffu, bad, 0)) timed_out = true;
+            else {
+                FinishArgs fa;
+                fa.p = &p; fa.d = &d; fa.rs = ctl.rs[lane_grp < 2 ? lane_grp + 2 : lane_grp - 2];   // of the epilogue warp of this row group
+                fa.tile = tile; fa.tile_i0 = tile_i0; fa.first_cta = first_cta; fa.last_cta = last_cta; fa.lane_grp = lane_grp;
+                fa.trace = nullptr;
+                fa.it_first = ((int)blockIdx.x - first_cta) * 2 + 1; fa.it_step = n_fin * 2;
+                finish_rows(fa, lane);
+            }
+        }
+    }
 
     if (timed_out) {
         *abort_flag = 1;
