@@ -16,10 +16,11 @@
 // barriers between them (the producer keeps streaming the next GEMM's weights meanwhile); one GEMM
 // per launch, chained by programmatic dependent launch, measured faster and is what the pass uses.
 //
-// Warp roles (224 threads): warp 0 = weight producer, warp 1 = TMEM allocator + MMA issuer,
-// warps 2..5 = epilogue (tcgen05.ld of their 32 lanes each), warp 6 = activation loader (TMA).
-// Accumulators are double-buffered in TMEM when two buffers fit, so that the epilogue of one tile
-// overlaps the MMAs of the next.
+// Warp roles (256 threads): warp 0 = weight producer, warp 1 = TMEM allocator + MMA issuer,
+// warps 2..5 = epilogue (tcgen05.ld of their 32 lanes each), warp 6 = activation loader (TMA),
+// warp 7 = spare; when the launch's last tile is finished, warps 0, 1, 6 and 7 each take half of one
+// epilogue warp's work. Accumulators are double-buffered in TMEM when two buffers fit, so that the
+// epilogue of one tile overlaps the MMAs of the next.
 //
 // Programmatic stream serialization: the ring is filled with weight tiles while the previous
 // kernel of the pass is still running; activations, workspace and outputs wait for the grid
@@ -302,16 +303,6 @@ __device__ __forceinline__ uint2 pack4_bf16(const __nv_bfloat16 (&h)[4])
     r.x = (uint32_t)__bfloat16_as_ushort(h[0]) | ((uint32_t)__bfloat16_as_ushort(h[1]) << 16);
     r.y = (uint32_t)__bfloat16_as_ushort(h[2]) | ((uint32_t)__bfloat16_as_ushort(h[3]) << 16);
     return r;
-}
-
-// Four consecutive bf16 values at dst (8-byte aligned) and, if dst_lo is not null, their remainders.
-__device__ __forceinline__ void store4_split(__nv_bfloat16 *dst, __nv_bfloat16 *dst_lo, const float (&v)[4])
-{
-    __nv_bfloat16 hi[4], lo[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) split_bf16(v[k], hi[k], lo[k]);
-    *reinterpret_cast<uint2 *>(dst) = pack4_bf16(hi);
-    if (dst_lo != nullptr) *reinterpret_cast<uint2 *>(dst_lo) = pack4_bf16(lo);
 }
 
 // Which workspace slot of CTA cc holds its share of the tile whose first item is tile_i0: slot 0
