@@ -268,6 +268,17 @@ int llmcad_tree_attention_noalloc(const void *q, const void *k, const void *v, i
                                   int32_t *status_out, void *stream);
 const char *llmcad_noalloc_last_error(void);
 
+/* Host-side scalars of the fallback decision (Sec. 3.3); plain arithmetic, no device work.
+ * llmcad_tree_confidence: T_c = max_i C_i over the n_branches cumulative confidences of a token
+ * tree (host array, each in (0, 1]). llmcad_update_threshold: the self-adaptive threshold of
+ * Eq. 3 after one verification: n_correct = scalars[LLMCAD_S_N_CORRECT], n_all =
+ * scalars[LLMCAD_S_N_ALL] of that pass, tree_confidence = T_c of the verified tree;
+ * *alpha_next = alpha / 2 when n_correct == n_all, else alpha / T_c^((n_all - n_correct) / n_all);
+ * n_all == 0 (a tree of the root alone) leaves alpha unchanged. LLMCAD_ERR_INVALID_ARG for null
+ * pointers, n_branches < 1, alpha <= 0, n_correct outside [0, n_all] or a confidence outside (0, 1]. */
+int llmcad_tree_confidence(const double *branch_conf, int32_t n_branches, double *t_c);
+int llmcad_update_threshold(double alpha, int32_t n_correct, int32_t n_all, double tree_confidence, double *alpha_next);
+
 /* Number of kernels this library has launched through this context so far. */
 int64_t llmcad_launch_count(const llmcad_ctx *ctx);
 

@@ -283,3 +283,23 @@ void orc_compact(const double *prefix, const double *tree, int P, int n_heads, i
             memcpy(out + ((size_t)h * (P + len) + P + j) * hd, tree + (size_t)path[j] * d + (size_t)h * hd, sizeof(double) * hd);
     }
 }
+
+/* Fallback scalars (Sec. 3.3). Tree-cumulative confidence: the largest cumulative confidence over
+ * the branches of a token tree. */
+double orc_tree_confidence(const double *branch_conf, int n_branches)
+{
+    double t = branch_conf[0];
+    for (int i = 1; i < n_branches; ++i)
+        if (branch_conf[i] > t) t = branch_conf[i];
+    return t;
+}
+
+/* Self-adaptive threshold, Eq. 3: after a verification with n_correct correct draft tokens out of
+ * n_all on the most matching branch, alpha is halved when all were correct and otherwise divided
+ * by T_c^((n_all - n_correct) / n_all). A verification without draft tokens (n_all = 0) leaves it. */
+double orc_alpha_update(double alpha, int n_correct, int n_all, double t_c)
+{
+    if (n_all == 0) return alpha;
+    if (n_correct == n_all) return alpha * 0.5;
+    return alpha / pow(t_c, (double)(n_all - n_correct) / (double)n_all);
+}

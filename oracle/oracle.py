@@ -266,3 +266,19 @@ class SequentialDecoder:
         k = self.kc[layer, :upto].reshape(upto, H, hd).transpose(1, 0, 2)
         v = self.vc[layer, :upto].reshape(upto, H, hd).transpose(1, 0, 2)
         return np.ascontiguousarray(k), np.ascontiguousarray(v)
+
+
+def tree_confidence(branch_conf) -> float:
+    """Sec. 3.3: T_c = max over branches of the cumulative confidence."""
+    c = np.ascontiguousarray(branch_conf, dtype=np.float64)
+    f = lib().orc_tree_confidence
+    f.restype = C.c_double
+    return float(f(_p(c), C.c_int(len(c))))
+
+
+def alpha_update(alpha: float, n_correct: int, n_all: int, t_c: float) -> float:
+    """Eq. 3: the self-adaptive fallback threshold after one verification."""
+    f = lib().orc_alpha_update
+    f.restype = C.c_double
+    f.argtypes = [C.c_double, C.c_int, C.c_int, C.c_double]
+    return float(f(alpha, n_correct, n_all, t_c))

@@ -30,6 +30,7 @@ EXPORTS = [
     "llmcad_verify_tree", "llmcad_verify_tree_host", "llmcad_prefill", "llmcad_tree_prep",
     "llmcad_accept_compact", "llmcad_tree_attention", "llmcad_skinny_gemm", "llmcad_launch_count",
     "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace", "llmcad_tiled_weight_bytes", "llmcad_tile_weight", "llmcad_skinny_gemm_tiled", "llmcad_tree_attention_noalloc", "llmcad_noalloc_last_error",
+    "llmcad_tree_confidence", "llmcad_update_threshold",
 ]
 
 
@@ -282,6 +283,25 @@ def tree_attention_noalloc(q, k, v, prefix_len: int, parent, o, status=None):
     if code != OK:
         raise LlmcadError(code, "llmcad_tree_attention_noalloc: " + lib().llmcad_noalloc_last_error().decode())
     return o
+
+
+def tree_confidence(branch_conf) -> float:
+    """T_c of Sec. 3.3: the largest cumulative branch confidence (host arithmetic)."""
+    c = (C.c_double * len(branch_conf))(*[float(x) for x in branch_conf])
+    out = C.c_double(0.0)
+    f = lib().llmcad_tree_confidence
+    f.argtypes = [C.POINTER(C.c_double), C.c_int32, C.POINTER(C.c_double)]
+    _check(f(c, len(branch_conf), C.byref(out)), "llmcad_tree_confidence")
+    return out.value
+
+
+def update_threshold(alpha: float, n_correct: int, n_all: int, t_c: float) -> float:
+    """Eq. 3: the self-adaptive fallback threshold after one verification (host arithmetic)."""
+    out = C.c_double(0.0)
+    f = lib().llmcad_update_threshold
+    f.argtypes = [C.c_double, C.c_int32, C.c_int32, C.c_double, C.POINTER(C.c_double)]
+    _check(f(alpha, n_correct, n_all, t_c, C.byref(out)), "llmcad_update_threshold")
+    return out.value
 
 
 def tree_prep(parent: torch.Tensor, prefix_len: int):

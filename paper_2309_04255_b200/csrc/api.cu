@@ -3,6 +3,7 @@
 // other translation units; this file only validates arguments and enqueues them in order.
 #include <cuda.h>
 
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -869,6 +870,28 @@ int llmcad_last_status(llmcad_ctx *ctx, void *stream)
     CUDA_TRY(cudaMemcpyAsync(&v, ctx->scalars_dev() + LLMCAD_S_STATUS, sizeof(v), cudaMemcpyDeviceToHost, st));
     CUDA_TRY(cudaStreamSynchronize(st));
     return v;
+}
+
+int llmcad_tree_confidence(const double *branch_conf, int32_t n_branches, double *t_c)
+{
+    if (branch_conf == nullptr || t_c == nullptr || n_branches < 1) return LLMCAD_ERR_INVALID_ARG;
+    double best = 0.0;
+    for (int32_t i = 0; i < n_branches; ++i) {
+        if (!(branch_conf[i] > 0.0 && branch_conf[i] <= 1.0)) return LLMCAD_ERR_INVALID_ARG;
+        best = branch_conf[i] > best ? branch_conf[i] : best;
+    }
+    *t_c = best;
+    return LLMCAD_OK;
+}
+
+int llmcad_update_threshold(double alpha, int32_t n_correct, int32_t n_all, double tree_confidence, double *alpha_next)
+{
+    if (alpha_next == nullptr || !(alpha > 0.0) || n_all < 0 || n_correct < 0 || n_correct > n_all) return LLMCAD_ERR_INVALID_ARG;
+    if (!(tree_confidence > 0.0 && tree_confidence <= 1.0)) return LLMCAD_ERR_INVALID_ARG;
+    if (n_all == 0) *alpha_next = alpha;                       // nothing was verified
+    else if (n_correct == n_all) *alpha_next = 0.5 * alpha;    // no error: trust the draft model more
+    else *alpha_next = alpha * exp(-log(tree_confidence) * (double)(n_all - n_correct) / (double)n_all);
+    return LLMCAD_OK;
 }
 
 int64_t llmcad_launch_count(const llmcad_ctx *ctx) { return ctx ? ctx->launches : 0; }

@@ -142,3 +142,26 @@ def test_bench_reference_arm_runs_on_cpu():
     d = json.loads(out.stdout.strip().splitlines()[-1])
     assert d["impl"] == "reference" and d["value"] > 0 and d["cpu_baseline"]["kind"] == "oracle"
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["unit"] == "passes/s"
+
+
+def test_fallback_scalars_match_the_oracle():
+    """llmcad_update_threshold / llmcad_tree_confidence (host arithmetic of Eq. 3) against the oracle
+    on a grid of cases, and their argument checks."""
+    from oracle import oracle as orc
+    from paper_2309_04255_b200 import binding as B
+    rng = np.random.default_rng(11)
+    for _ in range(200):
+        n_all = int(rng.integers(0, 12))
+        n_correct = int(rng.integers(0, n_all + 1))
+        t_c = float(rng.uniform(1e-3, 1.0))
+        alpha = float(rng.uniform(1e-4, 0.5))
+        got = B.update_threshold(alpha, n_correct, n_all, t_c)
+        ref = orc.alpha_update(alpha, n_correct, n_all, t_c)
+        assert abs(got - ref) <= 1e-12 * abs(ref)
+    c = rng.uniform(0.01, 1.0, 9)
+    assert B.tree_confidence(c) == orc.tree_confidence(c)
+    for bad in [(0.0, 1, 2, 0.5), (0.01, 3, 2, 0.5), (0.01, -1, 2, 0.5), (0.01, 1, 2, 0.0), (0.01, 1, 2, 1.5)]:
+        with pytest.raises(B.LlmcadError):
+            B.update_threshold(*bad)
+    with pytest.raises(B.LlmcadError):
+        B.tree_confidence([0.5, 0.0])

@@ -428,3 +428,44 @@ def test_tiny_config_whole_pass_against_library():
         seq = list(prefix) + [tokens[j] for j in path_of(parent, i)]
         ref = hf_logits(m, seq)[-1]
         np.testing.assert_allclose(res.logits[i], ref, rtol=HF_TOL, atol=HF_TOL * np.abs(ref).max())
+
+
+# ------------------------------------------------------------------ fallback scalars (Sec. 3.3, Eq. 3)
+
+def test_alpha_update_closed_forms():
+    """The two branches of Eq. 3 on values that can be checked by hand."""
+    a = 0.01                                               # the paper's default threshold
+    assert orc.alpha_update(a, 5, 5, 0.3) == a * 0.5       # no error: halved, whatever T_c
+    # one of two draft tokens wrong, T_c = 1/4: alpha / (1/4)^(1/2) = 2 alpha
+    assert abs(orc.alpha_update(a, 1, 2, 0.25) - 2 * a) < 1e-15
+    # all wrong: alpha / T_c
+    assert abs(orc.alpha_update(a, 0, 4, 0.125) - a / 0.125) < 1e-15
+    # three of four wrong, T_c = 1/16: exponent 3/4 -> 16^(3/4) = 8
+    assert abs(orc.alpha_update(a, 1, 4, 1.0 / 16) - 8 * a) < 1e-14
+    # a fully confident tree does not move the threshold when there are errors
+    assert orc.alpha_update(a, 2, 7, 1.0) == a
+    # nothing verified
+    assert orc.alpha_update(a, 0, 0, 0.5) == a
+
+
+def test_alpha_update_monotonic():
+    """With errors the threshold never drops, and it grows with the share of wrong tokens and with
+    lower confidence; a run of k verifications without error divides it by 2^k."""
+    a = 0.01
+    prev = a
+    for wrong in range(1, 9):
+        cur = orc.alpha_update(a, 8 - wrong, 8, 0.4)
+        assert cur > prev
+        prev = cur
+    assert orc.alpha_update(a, 3, 8, 0.2) > orc.alpha_update(a, 3, 8, 0.6) > a
+    x = a
+    for _ in range(6):
+        x = orc.alpha_update(x, 4, 4, 0.9)
+    assert x == a / 64
+
+
+def test_tree_confidence_is_the_maximum():
+    rng = np.random.default_rng(5)
+    c = rng.uniform(0.01, 1.0, 17)
+    assert orc.tree_confidence(c) == c.max()
+    assert orc.tree_confidence([0.3]) == 0.3
