@@ -268,6 +268,25 @@ int llmcad_tree_attention_noalloc(const void *q, const void *k, const void *v, i
                                   int32_t *status_out, void *stream);
 const char *llmcad_noalloc_last_error(void);
 
+/* Tree extension: the tree decoder of Sec. 3.2 on the generating side. A token tree grows by a few
+ * nodes at a time; the K/V of its first n_old nodes are already in cache slots prefix_len ..
+ * prefix_len + n_old - 1 of every layer (from earlier calls of this function with the same prefix;
+ * llmcad_verify_tree moves the cache, so a tree is not extended across it). The call computes the
+ * decoder forward of the nodes n_old .. n_tree-1 only, each at position prefix_len + depth and
+ * attending to the prefix and its own ancestors among ALL n_tree nodes (same mask table), writes
+ * their K/V to slots prefix_len + n_old .. prefix_len + n_tree - 1, and returns per new node the
+ * fp32 logits (logits [n_tree - n_old][vocab], optional) and the top_k most probable next tokens
+ * with their softmax probabilities (topk_ids, topk_probs [n_tree - n_old][top_k], descending, ties
+ * to the lower id; top_k in 0..LLMCAD_MAX_TOPK): the confidences that the branch rule (a successor
+ * above a threshold opens a branch) and the cumulative branch confidences are made of. tree_tokens
+ * and parent_idx describe the whole tree (n_tree entries, parent_idx[i] < i, root -1); all pointers
+ * but ctx are device pointers; *status receives 0 or a device-detected error. n_old = 0 starts a
+ * tree. Asynchronous on `stream`. */
+#define LLMCAD_MAX_TOPK 8
+int llmcad_extend_tree(llmcad_ctx *ctx, const void *packed_weights, void *kv_cache, int32_t prefix_len,
+                       const int32_t *tree_tokens, const int32_t *parent_idx, int32_t n_old, int32_t n_tree, int32_t top_k,
+                       float *logits, int32_t *topk_ids, float *topk_probs, int32_t *status, void *stream);
+
 /* Host-side scalars of the fallback decision (Sec. 3.3); plain arithmetic, no device work.
  * llmcad_tree_confidence: T_c = max_i C_i over the n_branches cumulative confidences of a token
  * tree (host array, each in (0, 1]). llmcad_update_threshold: the self-adaptive threshold of

@@ -303,3 +303,29 @@ double orc_alpha_update(double alpha, int n_correct, int n_all, double t_c)
     if (n_correct == n_all) return alpha * 0.5;
     return alpha / pow(t_c, (double)(n_all - n_correct) / (double)n_all);
 }
+
+/* Confidences of the generating side (Sec. 3.2: a candidate whose confidence exceeds a threshold
+ * opens a branch): the softmax of a node's logits, and its k largest entries in descending order
+ * (ties: lower token id first). */
+void orc_topk_softmax(const double *logits, int n, int vocab, int k, int *ids, double *probs)
+{
+    double *p = (double *)malloc(sizeof(double) * (size_t)vocab);
+    for (int i = 0; i < n; ++i) {
+        const double *row = logits + (size_t)i * vocab;
+        double mx = row[0], sum = 0.0;
+        for (int t = 1; t < vocab; ++t) if (row[t] > mx) mx = row[t];
+        for (int t = 0; t < vocab; ++t) { p[t] = exp(row[t] - mx); sum += p[t]; }
+        for (int t = 0; t < vocab; ++t) p[t] /= sum;
+        for (int r = 0; r < k; ++r) {
+            int best = -1;
+            for (int t = 0; t < vocab; ++t) {
+                int taken = 0;
+                for (int q = 0; q < r; ++q) if (ids[(size_t)i * k + q] == t) taken = 1;
+                if (!taken && (best < 0 || row[t] > row[best])) best = t;
+            }
+            ids[(size_t)i * k + r] = best;
+            probs[(size_t)i * k + r] = p[best];
+        }
+    }
+    free(p);
+}

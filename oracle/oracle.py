@@ -282,3 +282,13 @@ def alpha_update(alpha: float, n_correct: int, n_all: int, t_c: float) -> float:
     f.restype = C.c_double
     f.argtypes = [C.c_double, C.c_int, C.c_int, C.c_double]
     return float(f(alpha, n_correct, n_all, t_c))
+
+
+def topk_softmax(logits: np.ndarray, k: int):
+    """Softmax of every row and its k largest entries (descending, ties to the lower id): (ids, probs)."""
+    lg = np.ascontiguousarray(logits, dtype=np.float64)
+    n, vocab = lg.shape
+    ids = np.zeros((n, k), np.int32)
+    probs = np.zeros((n, k), np.float64)
+    lib().orc_topk_softmax(_p(lg), C.c_int(n), C.c_int(vocab), C.c_int(k), _p(ids), _p(probs))
+    return ids, probs

@@ -30,7 +30,7 @@ EXPORTS = [
     "llmcad_verify_tree", "llmcad_verify_tree_host", "llmcad_prefill", "llmcad_tree_prep",
     "llmcad_accept_compact", "llmcad_tree_attention", "llmcad_skinny_gemm", "llmcad_launch_count",
     "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace", "llmcad_tiled_weight_bytes", "llmcad_tile_weight", "llmcad_skinny_gemm_tiled", "llmcad_tree_attention_noalloc", "llmcad_noalloc_last_error",
-    "llmcad_tree_confidence", "llmcad_update_threshold",
+    "llmcad_tree_confidence", "llmcad_update_threshold", "llmcad_extend_tree",
 ]
 
 
@@ -104,6 +104,7 @@ def lib():
         L.llmcad_skinny_gemm_tiled.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
         L.llmcad_tree_attention_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, vp, i32, vp, vp, vp]
         L.llmcad_noalloc_last_error.restype = C.c_char_p
+        L.llmcad_extend_tree.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
         L.llmcad_set_kernel_timing.argtypes = [vp, i32]
         L.llmcad_get_kernel_timing.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         _lib = L
@@ -196,6 +197,24 @@ class Verifier:
         r = Result(_ptr(out["logits"]), _ptr(out["argmax"]), _ptr(out["accepted_path"]), _ptr(out["scalars"]))
         _check(lib().llmcad_verify_tree(self.ctx, self.packed.data_ptr(), self.kv.data_ptr(), prefix_len, _ptr(tokens),
                                         _ptr(parent), n, C.byref(r), _stream()), "llmcad_verify_tree")
+        return out
+
+    def extend_tree(self, prefix_len: int, tokens: torch.Tensor, parent: torch.Tensor, n_old: int, top_k: int = 4,
+                    want_logits: bool = True):
+        """Decoder forward of the tree nodes n_old.. (the K/V of the first n_old nodes are in the cache):
+        returns logits [n_new][vocab] (or None), top-k ids and probabilities [n_new][top_k], status."""
+        n_tree = tokens.numel()
+        n_new = n_tree - n_old
+        dev = self.device
+        out = {
+            "logits": torch.empty((n_new, self.cfg.vocab), dtype=torch.float32, device=dev) if want_logits else None,
+            "topk_ids": torch.empty((n_new, max(top_k, 1)), dtype=torch.int32, device=dev),
+            "topk_probs": torch.empty((n_new, max(top_k, 1)), dtype=torch.float32, device=dev),
+            "status": torch.zeros(1, dtype=torch.int32, device=dev),
+        }
+        _check(lib().llmcad_extend_tree(self.ctx, _ptr(self.packed), _ptr(self.kv), prefix_len, _ptr(tokens), _ptr(parent),
+                                        n_old, n_tree, top_k, _ptr(out["logits"]), _ptr(out["topk_ids"]),
+                                        _ptr(out["topk_probs"]), _ptr(out["status"]), _stream()), "llmcad_extend_tree")
         return out
 
     def verify_tree_host(self, prefix_len: int, tokens: torch.Tensor, parent: torch.Tensor, out):

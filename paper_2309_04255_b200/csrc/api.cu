@@ -277,7 +277,7 @@ int run_gemm(llmcad_ctx *ctx, const void *packed, int l, int which, int act, int
 // comp: q carries a lo plane kLoRows rows after the hi plane, and o gets one too (the pass);
 // the single-step entry points work on plain bf16 buffers.
 int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, int kv_stride, int P, int n, void *o,
-                  bool comp, int32_t *status, cudaStream_t st)
+                  bool comp, int32_t *status, cudaStream_t st, int n_tree = 0, int q_first = 0)
 {
     const llmcad_config &c = ctx->cfg;
     TimedLaunch tl(ctx, 1, st);
@@ -285,31 +285,37 @@ int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, 
         int launched = 0;
         CUDA_TRY(launch_attention_tc(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->attn_ws,
                                      ctx->attn_counters, ctx->n_sms, status, st, &launched, ctx->next_trace(), comp ? 1 : 0,
-                                     ctx->kv_lo));
+                                     ctx->kv_lo, n_tree, q_first));
         ctx->launches += launched;
         return LLMCAD_OK;
     }
-    if (sizeof(float) * (size_t)(c.head_dim + P + n) > 200 * 1024) return LLMCAD_ERR_UNSUPPORTED;
+    if (sizeof(float) * (size_t)(c.head_dim + P + (n_tree > 0 ? n_tree : n)) > 200 * 1024) return LLMCAD_ERR_UNSUPPORTED;
     ctx->launches++;
-    CUDA_TRY(launch_attention_simt(q, k, v, c.dtype, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, status, st));
+    CUDA_TRY(launch_attention_simt(q, k, v, c.dtype, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, status, st, n_tree,
+                                   q_first));
     return LLMCAD_OK;
 }
 
-// Decoder forward over n nodes: tree prep, embedding, all layers; K/V of node i go to cache slot
-// P+i. When logits != nullptr the final norm and lm_head run too.
+// Decoder forward over the nodes n_old .. n_tree-1 of a tree of n_tree nodes (all of them when
+// n_old = 0): tree prep of the whole tree, embedding, all layers; K/V of node i go to cache slot
+// P+i, where the nodes below n_old already have theirs. When logits != nullptr the final norm and
+// lm_head run too (one row per processed node).
 int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, const int32_t *tokens,
-                const int32_t *parent, int n, float *logits, int32_t *status, cudaStream_t st)
+                const int32_t *parent, int n_tree, float *logits, int32_t *status, cudaStream_t st, int n_old = 0)
 {
     const llmcad_config &c = ctx->cfg;
     const int d = c.d_model, f = c.d_ffn, hd = c.head_dim, H = c.n_heads, S = c.max_seq;
+    const int n = n_tree - n_old;                    // nodes this call computes
     const int n_pad = (n + 15) / 16 * 16;
+    const int32_t *new_tokens = tokens + n_old;
     const char *base = static_cast<const char *>(packed);
     int rc;
     if ((rc = ensure_weight_maps(ctx, packed)) != LLMCAD_OK) return rc;
     if ((rc = ensure_act_maps(ctx, n_pad)) != LLMCAD_OK) return rc;
 
-    CUDA_TRY(launch_tree_prep(parent, tokens, n, P, c.vocab, hd, c.rope_base, ctx->tb, status, st));
+    CUDA_TRY(launch_tree_prep(parent, tokens, n_tree, P, c.vocab, hd, c.rope_base, ctx->tb, status, st));
     ctx->launches += 2;
+    const float2 *rope_new = ctx->tb.rope_cs + (size_t)n_old * (hd / 2);
     const size_t kv_layer = (size_t)2 * H * S * hd * ctx->elem;
 
     if (ctx->tc_gemm) {
@@ -318,14 +324,14 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
         // partial sums of squares; the consuming GEMM scales its accumulators by the per-node
         // rsqrt(mean(x^2) + eps). Activations travel as bf16 hi + lo planes (ctx->comp).
         const int tiles4 = 4 * ((d + 127) / 128);
-        CUDA_TRY(launch_embed_norm(base + ctx->lay.tok_embed, tokens, n, d,
+        CUDA_TRY(launch_embed_norm(base + ctx->lay.tok_embed, new_tokens, n, d,
                                    c.n_layers > 0 ? base + ctx->lay.attn_norm : base + ctx->lay.final_norm, ctx->x, ctx->xn,
                                    ctx->ssq[0], ctx->comp ? 1 : 0, status, st));
         auto qkv_ep = [&](int l, int parts) {
             char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)l;
             EpiParams ep{};
             ep.n = n; ep.mode = EPI_QKV; ep.n_out = 3 * d; ep.q_out = ctx->q; ep.k_cache = kl; ep.v_cache = kl + kv_layer / 2;
-            ep.rope_cs = ctx->tb.rope_cs; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P;
+            ep.rope_cs = rope_new; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P + n_old;
             ep.ssq_in = ctx->ssq[0]; ep.ssq_in_parts = parts; ep.norm_d = d; ep.eps = c.rms_eps;
             ep.comp = ctx->comp ? 1 : 0; ep.kv_lo = ctx->kv_lo;
             return ep;
@@ -372,7 +378,8 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
             if (specs[i].attention_first) {
                 char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)specs[i].l;
                 // without the tensor-core attention kernel the lo plane of att stays zero, as allocated
-                if ((rc = run_attention(ctx, ctx->q, kl, kl + kv_layer / 2, S, P, n, ctx->att, ctx->comp && ctx->tc_attn, status, st)) != LLMCAD_OK) return rc;
+                if ((rc = run_attention(ctx, ctx->q, kl, kl + kv_layer / 2, S, P, n, ctx->att, ctx->comp && ctx->tc_attn, status, st,
+                                        n_tree, n_old)) != LLMCAD_OK) return rc;
             }
             Chain ch;
             size_t j = i;
@@ -387,7 +394,7 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
         return LLMCAD_OK;
     }
 
-    CUDA_TRY(launch_embed(base + ctx->lay.tok_embed, c.dtype, tokens, n, d, ctx->x, status, st));
+    CUDA_TRY(launch_embed(base + ctx->lay.tok_embed, c.dtype, new_tokens, n, d, ctx->x, status, st));
     for (int l = 0; l < c.n_layers; ++l) {
         const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
         char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)l;
@@ -398,10 +405,10 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
         CUDA_TRY(launch_rmsnorm(ctx->x, lb + ctx->lay.attn_norm, c.dtype, n, d, c.rms_eps, ctx->xn, status, st));
         ctx->launches++;
         ep.mode = EPI_QKV; ep.n_out = 3 * d; ep.q_out = ctx->q; ep.k_cache = kl; ep.v_cache = vl;
-        ep.rope_cs = ctx->tb.rope_cs; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P;
+        ep.rope_cs = rope_new; ep.d = d; ep.hd = hd; ep.S = S; ep.P = P + n_old;
         if ((rc = run_gemm(ctx, packed, l, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
 
-        if ((rc = run_attention(ctx, ctx->q, kl, vl, S, P, n, ctx->att, false, status, st)) != LLMCAD_OK) return rc;
+        if ((rc = run_attention(ctx, ctx->q, kl, vl, S, P, n, ctx->att, false, status, st, n_tree, n_old)) != LLMCAD_OK) return rc;
 
         ep = EpiParams{}; ep.n = n; ep.mode = EPI_RESID; ep.n_out = d; ep.x = ctx->x;
         if ((rc = run_gemm(ctx, packed, l, 1, 1, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
@@ -693,6 +700,28 @@ int llmcad_prefill(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t 
         if (last && last_logits != nullptr)
             CUDA_TRY(cudaMemcpyAsync(last_logits, ctx->logits + (size_t)(m - 1) * ctx->cfg.vocab,
                                      (size_t)ctx->cfg.vocab * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    }
+    return LLMCAD_OK;
+}
+
+int llmcad_extend_tree(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t prefix_len, const int32_t *tree_tokens,
+                       const int32_t *parent_idx, int32_t n_old, int32_t n_tree, int32_t top_k, float *logits,
+                       int32_t *topk_ids, float *topk_probs, int32_t *status, void *stream)
+{
+    int rc = check_pass_args(ctx, packed, kv_cache, prefix_len, tree_tokens, parent_idx, n_tree);
+    if (rc != LLMCAD_OK) return rc;
+    if (status == nullptr || n_old < 0 || n_old >= n_tree || top_k < 0 || top_k > LLMCAD_MAX_TOPK) return LLMCAD_ERR_INVALID_ARG;
+    if (top_k > 0 && (topk_ids == nullptr || topk_probs == nullptr)) return LLMCAD_ERR_INVALID_ARG;
+    if (top_k > ctx->cfg.vocab) return LLMCAD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float *lg = logits != nullptr ? logits : ctx->logits;
+    CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    if ((rc = reset_chain_sync(ctx, st)) != LLMCAD_OK) return rc;
+    if ((rc = run_forward(ctx, packed, kv_cache, prefix_len, tree_tokens, parent_idx, n_tree, lg, status, st, n_old)) != LLMCAD_OK)
+        return rc;
+    if (top_k > 0) {
+        CUDA_TRY(launch_topk_softmax(lg, n_tree - n_old, ctx->cfg.vocab, top_k, topk_ids, topk_probs, status, st));
+        ctx->launches++;
     }
     return LLMCAD_OK;
 }

@@ -2,7 +2,8 @@
 // as a debugging stand-in for the tensor-core kernel. Keys are the prefix slots 0..P-1 (all
 // visible) followed by the tree nodes at slots P..P+n-1, of which node i sees only those whose
 // bit is set in its ancestor-or-self row (Sec. 3.2 "Tree decoder": ones only at the earlier
-// positions of the same branch). Masked keys get weight exactly zero.
+// positions of the same branch). Masked keys get weight exactly zero. When a tree is extended the
+// queries are only its new nodes q_first .. q_first + n - 1, the keys all n_tree nodes.
 #include "common.cuh"
 
 namespace llmcad {
@@ -12,7 +13,8 @@ constexpr int kAttnThreads = 128;
 template <typename T>
 __global__ void __launch_bounds__(kAttnThreads)
 attention_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, int n_heads, int hd,
-                      int kv_stride, int P, int n, const uint32_t *__restrict__ anc, T *o, const int32_t *status)
+                      int kv_stride, int P, int n, int n_tree, int q_first, const uint32_t *__restrict__ anc, T *o,
+                      const int32_t *status)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -25,14 +27,14 @@ attention_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T 
 
     const int i = blockIdx.x, h = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int n_keys = P + n;
+    const int n_keys = P + n_tree;
     const float scale = rsqrtf((float)hd);
     const T *kh = k + (size_t)h * kv_stride * hd;
     const T *vh = v + (size_t)h * kv_stride * hd;
 
     for (int e = tid; e < hd; e += kAttnThreads) s_q[e] = to_f32<T>(q[((size_t)i * n_heads + h) * hd + e]);
     uint32_t my_anc[4];
-    for (int w = 0; w < 4; ++w) my_anc[w] = anc[i * 4 + w];
+    for (int w = 0; w < 4; ++w) my_anc[w] = anc[(q_first + i) * 4 + w];
     __syncthreads();
 
     // scores: one warp per key, lanes split the head dimension
@@ -85,23 +87,24 @@ attention_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T 
 
 cudaError_t launch_attention_simt(const void *q, const void *k, const void *v, int dtype, int n_heads, int hd,
                                   int kv_stride, int P, int n, const uint32_t *anc, void *o, const int32_t *status,
-                                  cudaStream_t st)
+                                  cudaStream_t st, int n_tree, int q_first)
 {
-    const size_t smem = sizeof(float) * (size_t)(hd + P + n);
+    if (n_tree <= 0) n_tree = n;
+    const size_t smem = sizeof(float) * (size_t)(hd + P + n_tree);
     dim3 grid(n, n_heads);
     if (dtype == LLMCAD_F32) {
         if (smem > 48 * 1024)
             cudaFuncSetAttribute(attention_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         LaunchCfg lc(grid, kAttnThreads, smem, st);
         return cudaLaunchKernelEx(&lc.cfg, attention_simt_kernel<float>, (const float *)q, (const float *)k,
-                                  (const float *)v, n_heads, hd, kv_stride, P, n, anc, (float *)o, status);
+                                  (const float *)v, n_heads, hd, kv_stride, P, n, n_tree, q_first, anc, (float *)o, status);
     } else {
         if (smem > 48 * 1024)
             cudaFuncSetAttribute(attention_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         LaunchCfg lc(grid, kAttnThreads, smem, st);
         return cudaLaunchKernelEx(&lc.cfg, attention_simt_kernel<__nv_bfloat16>, (const __nv_bfloat16 *)q,
-                                  (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, n_heads, hd, kv_stride, P, n, anc,
-                                  (__nv_bfloat16 *)o, status);
+                                  (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, n_heads, hd, kv_stride, P, n, n_tree, q_first,
+                                  anc, (__nv_bfloat16 *)o, status);
     }
 }
 

@@ -97,8 +97,11 @@ __global__ void __launch_bounds__(kAtThreads)
 attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
                     const __nv_bfloat16 *__restrict__ v, int n_heads, int kv_stride, int P, int n, int n_pad,
                     const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
-                    const int32_t *status, unsigned long long *trace, const __nv_bfloat16 *__restrict__ kv_lo)
+                    const int32_t *status, unsigned long long *trace, const __nv_bfloat16 *__restrict__ kv_lo,
+                    int n_tree, int q_first)
 {
+    // n query rows = the tree nodes q_first .. q_first + n - 1 (all of them in a verification pass,
+    // the new ones when a tree is extended); the keys are the prefix and all n_tree tree nodes
     // ring depth: with 128 nodes and the lo planes three stages are what fits in shared memory
     constexpr int kStages = (COMP && GROUPS == 1) ? 3 : kMaxStages;
     constexpr int KW = kKeyTile / GROUPS;     // keys per warp per tile: 64, 32 or 16
@@ -117,7 +120,7 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     const size_t lo_off = (size_t)kLoRows * n_heads * kHd;  // elements from a hi plane of q / o to its lo plane
     const int split = blockIdx.x, head = blockIdx.y;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n_keys = P + n;
+    const int n_keys = P + n_tree;
     const int n_tiles = (n_keys + kKeyTile - 1) / kKeyTile;
     const int t_begin = split * tiles_per_split;
     const int t_end = min(n_tiles, t_begin + tiles_per_split);
@@ -185,8 +188,8 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     uint32_t anc0[4] = {0, 0, 0, 0}, anc1[4] = {0, 0, 0, 0};
     if (active) {
         for (int w = 0; w < 4; ++w) {
-            if (row0 < n) anc0[w] = anc[row0 * 4 + w];
-            if (row1 < n) anc1[w] = anc[row1 * 4 + w];
+            if (row0 < n) anc0[w] = anc[(q_first + row0) * 4 + w];
+            if (row1 < n) anc1[w] = anc[(q_first + row1) * 4 + w];
         }
     }
 
@@ -238,7 +241,7 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         const int key_base = t * kKeyTile + key_off;
         const bool needs_mask = key_base + KW > P;          // this warp's keys reach into the tree nodes
         // row of the lo buffers that holds the remainder of key `key` (the zero row for prefix keys)
-        auto lo_row = [&](int key) { const int node = key - P; return (node >= 0 && node < n) ? node : n_pad; };
+        auto lo_row = [&](int key) { const int node = key - P - q_first; return (node >= 0 && node < n) ? node : n_pad; };
         if (COMP && needs_mask) {
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
@@ -264,7 +267,7 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
                     if (key >= P) {
                         const int node = key - P;
                         const uint32_t *a = (e < 2) ? anc0 : anc1;
-                        const bool vis = node < n && ((a[node >> 5] >> (node & 31)) & 1u);
+                        const bool vis = node < n_tree && ((a[node >> 5] >> (node & 31)) & 1u);
                         if (!vis) val = -INFINITY;
                     }
                 }
@@ -454,12 +457,13 @@ size_t attention_tc_workspace_bytes(int n_heads, int n_sms)
 cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, float *ws, uint32_t *counters, int n_sms,
                                 int32_t *status, cudaStream_t st, int *launched, unsigned long long *trace, int comp,
-                                const void *kv_lo)
+                                const void *kv_lo, int n_tree, int q_first)
 {
+    if (n_tree <= 0) n_tree = n;
     (void)ws; (void)counters;
     if (hd != kHd) return cudaErrorInvalidValue;
     const int n_pad = (n + 15) / 16 * 16;
-    const int n_tiles = (P + n + kKeyTile - 1) / kKeyTile;
+    const int n_tiles = (P + n_tree + kKeyTile - 1) / kKeyTile;
     // one CTA per SM is resident (register file): aim for a single wave of heads x splits CTAs
     int splits = n_sms / n_heads;
     if (splits > kMaxSplits) splits = kMaxSplits;
@@ -477,7 +481,7 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     const size_t smem = ring > part ? ring : part;
     typedef void (*Kern)(const __nv_bfloat16 *, const __nv_bfloat16 *, const __nv_bfloat16 *, int, int, int, int, int,
                          const uint32_t *, __nv_bfloat16 *, int, int, const int32_t *, unsigned long long *,
-                         const __nv_bfloat16 *);
+                         const __nv_bfloat16 *, int, int);
     static const Kern kerns[2][3] = {{attention_tc_kernel<1, false>, attention_tc_kernel<2, false>, attention_tc_kernel<4, false>},
                                      {attention_tc_kernel<1, true>, attention_tc_kernel<2, true>, attention_tc_kernel<4, true>}};
     static bool attr_set = false;
@@ -495,7 +499,7 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     Kern kern = kerns[comp ? 1 : 0][groups == 4 ? 2 : (groups == 2 ? 1 : 0)];
     return cudaLaunchKernelEx(&lc.cfg, kern, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                               (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc, (__nv_bfloat16 *)o, splits,
-                              tiles_per_split, (const int32_t *)status, trace, (const __nv_bfloat16 *)kv_lo);
+                              tiles_per_split, (const int32_t *)status, trace, (const __nv_bfloat16 *)kv_lo, n_tree, q_first);
 }
 
 }  // namespace llmcad

@@ -10,10 +10,12 @@ size_t attention_tc_workspace_bytes(int n_heads, int n_sms);
 // q, o: [n][H][128] bf16; k, v: [H][kv_stride][128] bf16; anc: [n][4] ancestor-or-self bit rows.
 // comp != 0: q and o each consist of a hi and a lo plane, the lo plane kLoRows rows ([H][128] each)
 // after the hi plane, and kv_lo holds the bf16 remainders of the tree nodes' keys and values,
-// [2][H][kLoRows][128] (K then V, row = node).
+// [2][H][kLoRows][128] (K then V, row = query index).
+// n_tree > 0: the queries are only the tree nodes q_first .. q_first + n - 1 (anc holds the rows of
+// all n_tree nodes), the keys the prefix and all n_tree tree nodes; 0 means n_tree = n, q_first = 0.
 cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, float *ws, uint32_t *counters, int n_sms,
                                 int32_t *status, cudaStream_t st, int *launched, unsigned long long *trace = nullptr, int comp = 0,
-                                const void *kv_lo = nullptr);
+                                const void *kv_lo = nullptr, int n_tree = 0, int q_first = 0);
 
 }  // namespace llmcad

@@ -198,6 +198,9 @@ cudaError_t launch_gemm_simt(const void *W, const void *x, int dtype, int n_in, 
                              const int32_t *status, cudaStream_t st);
 cudaError_t launch_attention_simt(const void *q, const void *k, const void *v, int dtype, int n_heads, int hd,
                                   int kv_stride, int P, int n, const uint32_t *anc, void *o, const int32_t *status,
-                                  cudaStream_t st);
+                                  cudaStream_t st, int n_tree = 0, int q_first = 0);
+// softmax probabilities and ids of the k largest logits of every node (ties: lowest id; NaN -> status)
+cudaError_t launch_topk_softmax(const float *logits, int n, int vocab, int k, int32_t *ids, float *probs, int32_t *status,
+                                cudaStream_t st);
 
 }  // namespace llmcad

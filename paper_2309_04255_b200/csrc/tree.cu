@@ -261,6 +261,96 @@ cudaError_t launch_argmax(const float *logits, int n, int vocab, int32_t *argmax
 }
 
 // ------------------------------------------------------------------------------------------
+// Confidences of the generating side (Sec. 3.2: a candidate above a confidence threshold opens a
+// branch): per node the k most probable next tokens and their softmax probabilities. One block
+// per node: the row maximum and the sum of exponentials first, then k rounds of "largest logit
+// not yet taken" (ties to the lower id). The row (vocab x 4 bytes) stays in L2 between the rounds.
+constexpr int kTopkThreads = 1024;
+
+__global__ void __launch_bounds__(kTopkThreads)
+topk_softmax_kernel(const float *__restrict__ logits, int vocab, int k, int32_t *ids, float *probs, int32_t *status)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    if (*status) return;
+    __shared__ float s_v[32];
+    __shared__ int s_i[32];
+    __shared__ float s_max, s_sum;
+    __shared__ int s_taken[LLMCAD_MAX_TOPK];
+    const int node = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float *row = logits + (size_t)node * vocab;
+
+    auto block_max = [&](float v, int i, float &out_v, int &out_i) {     // argmax over the block, ties to the lower id
+        for (int o = 16; o; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+            if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+        }
+        if (lane == 0) { s_v[warp] = v; s_i[warp] = i; }
+        __syncthreads();
+        if (warp == 0) {
+            v = s_v[lane]; i = s_i[lane];
+            for (int o = 16; o; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+                if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+            }
+            if (lane == 0) { s_v[0] = v; s_i[0] = i; }
+        }
+        __syncthreads();
+        out_v = s_v[0]; out_i = s_i[0];
+        __syncthreads();
+    };
+
+    // maximum (and NaN check), then the sum of exp(x - max)
+    float best = -INFINITY;
+    int bi = 0x7fffffff;
+    bool nan = false;
+    for (int t = tid; t < vocab; t += kTopkThreads) argmax_take(__ldcg(row + t), t, best, bi, nan);
+    if (nan) atomicCAS(status, 0, LLMCAD_ERR_NAN);
+    float mx; int mi;
+    block_max(best, bi, mx, mi);
+    float sum = 0.f;
+    for (int t = tid; t < vocab; t += kTopkThreads) sum += expf(__ldcg(row + t) - mx);
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) s_v[warp] = sum;
+    __syncthreads();
+    if (tid == 0) {
+        float t = 0.f;
+        for (int w = 0; w < kTopkThreads / 32; ++w) t += s_v[w];
+        s_sum = t; s_max = mx;
+    }
+    __syncthreads();
+    const float inv = 1.0f / s_sum;
+
+    for (int r = 0; r < k; ++r) {
+        float v = -INFINITY;
+        int vi = 0x7fffffff;
+        for (int t = tid; t < vocab; t += kTopkThreads) {
+            bool taken = false;
+            for (int q = 0; q < r; ++q) taken |= (s_taken[q] == t);
+            const float x = __ldcg(row + t);
+            if (!taken && (x > v || (x == v && t < vi))) { v = x; vi = t; }
+        }
+        float bv; int bidx;
+        block_max(v, vi, bv, bidx);
+        if (tid == 0) {
+            s_taken[r] = bidx;
+            ids[(size_t)node * k + r] = bidx == 0x7fffffff ? 0 : bidx;
+            probs[(size_t)node * k + r] = expf(bv - s_max) * inv;
+        }
+        __syncthreads();
+    }
+}
+
+cudaError_t launch_topk_softmax(const float *logits, int n, int vocab, int k, int32_t *ids, float *probs, int32_t *status,
+                                cudaStream_t st)
+{
+    LaunchCfg lc(n, kTopkThreads, 0, st);
+    return cudaLaunchKernelEx(&lc.cfg, topk_softmax_kernel, logits, vocab, k, ids, probs, status);
+}
+
+// ------------------------------------------------------------------------------------------
 // Verified-sequence search (Sec. 3.2 "Depth-first verified sequence searching"), data-parallel
 // form: node c is verified iff every link on its root path is correct (the child's draft token
 // equals the target's output at the parent). The verified sequence ends at the deepest verified

@@ -4,6 +4,7 @@ reads its operands from HBM, not from L2).
     python -m paper_2309_04255_b200.kernel_bench attention            # prefix x tree-size sweep (config 4)
     python -m paper_2309_04255_b200.kernel_bench gemm [--n 32] [--model 7b] [--only qkv,o]
     python -m paper_2309_04255_b200.kernel_bench avnav [--model 7b] [--prefix 512] [--nodes 2,4,...]
+    python -m paper_2309_04255_b200.kernel_bench extend [--model 7b] [--prefix 512] [--nodes 32] [--steps 1,2,4,8]
 
 Each line of output is one JSON object. `--reps` launches are timed per case after `--warmup`.
 """
@@ -185,6 +186,53 @@ def bench_avnav(args):
             "chain_vs_steps_max_rel_diff": diff}), flush=True)
 
 
+def build_model(cfg, dev, max_seq, P):
+    v = B.Verifier(cfg, max_seq, device=dev)
+    v.pack_globals({k: gen.gen_tensor_device(cfg, k, -1, dev) for k in ("tok_embed", "final_norm", "lm_head")})
+    for l in range(cfg.n_layers):
+        v.pack_layer(l, {k: gen.gen_tensor_device(cfg, k, l, dev) for k in gen.LAYER_TENSORS})
+    kvv = v.kv_view()
+    g = torch.Generator(device=dev)
+    g.manual_seed(gen.MASTER_SEED)
+    for l in range(cfg.n_layers):
+        kvv[l, :, :, :P] = torch.randn((2, cfg.n_heads, P, cfg.head_dim), generator=g, device=dev, dtype=torch.float32).to(kvv.dtype)
+    return v
+
+
+def bench_extend(args):
+    """Tree extension (the generating side's tree decoder): a tree of --nodes nodes grown m nodes at
+    a time; every call streams all weights once, like a decoding step."""
+    cfg = gen.MODELS[args.model]
+    dev = torch.device("cuda:0")
+    P, n = args.prefix, args.nodes
+    v = build_model(cfg, dev, P + n + 8, P)
+    peak, kind = _peak()
+    wbytes = cfg.weight_bytes()
+    tokens = torch.as_tensor(gen.gen_tokens(cfg, n), device=dev)
+    parent = torch.as_tensor(gen.tree_random(n, 16, "uniform4", 1), device=dev)
+    for m in [int(x) for x in args.steps.split(",")]:
+        cuts = list(range(m, n, m)) + [n]
+
+        def grow():
+            old = 0
+            for c in cuts:
+                v.extend_tree(P, tokens[:c], parent[:c], old, top_k=4, want_logits=False)
+                old = c
+
+        grow()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.reps):
+            grow()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.reps / len(cuts)
+        print(json.dumps({"bench": "extend_tree", "model": cfg.name, "prefix": P, "tree_nodes": n, "new_nodes_per_call": m,
+                          "calls": len(cuts), "ms_per_call": ms, "weight_gbs": wbytes / ms / 1e6,
+                          "frac": wbytes / ms / 1e6 / peak, "peak": kind}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -205,10 +253,16 @@ def main():
     n.add_argument("--prefix", type=int, default=512)
     n.add_argument("--nodes", default="2,4,8,16,32,64,128")
     n.add_argument("--reps", type=int, default=3)
+    x = sub.add_parser("extend")
+    x.add_argument("--model", default="7b")
+    x.add_argument("--prefix", type=int, default=512)
+    x.add_argument("--nodes", type=int, default=32)
+    x.add_argument("--steps", default="1,2,4,8,32")
+    x.add_argument("--reps", type=int, default=3)
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("kernel_bench needs a CUDA device")
-    {"attention": bench_attention, "gemm": bench_gemm, "avnav": bench_avnav}[args.cmd](args)
+    {"attention": bench_attention, "gemm": bench_gemm, "avnav": bench_avnav, "extend": bench_extend}[args.cmd](args)
 
 
 if __name__ == "__main__":

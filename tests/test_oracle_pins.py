@@ -469,3 +469,28 @@ def test_tree_confidence_is_the_maximum():
     c = rng.uniform(0.01, 1.0, 17)
     assert orc.tree_confidence(c) == c.max()
     assert orc.tree_confidence([0.3]) == 0.3
+
+
+# ------------------------------------------------------------------ confidences of the generating side
+
+def test_topk_softmax_against_library_and_closed_forms():
+    rng = np.random.default_rng(3)
+    lg = rng.normal(0, 2, (5, 97))
+    ids, probs = orc.topk_softmax(lg, 6)
+    ref = torch.softmax(torch.from_numpy(lg), dim=-1).numpy()
+    order = np.argsort(-lg, axis=1, kind="stable")[:, :6]
+    assert np.array_equal(ids, order)
+    np.testing.assert_allclose(probs, np.take_along_axis(ref, order, 1), rtol=1e-12)
+    # equal logits: uniform probabilities, the lowest ids first
+    ids, probs = orc.topk_softmax(np.zeros((1, 10)), 3)
+    assert ids.tolist() == [[0, 1, 2]] and np.allclose(probs, 0.1)
+    # two-token vocabulary: the logistic function
+    ids, probs = orc.topk_softmax(np.array([[0.0, np.log(3.0)]]), 2)
+    assert ids.tolist() == [[1, 0]] and np.allclose(probs, [[0.75, 0.25]])
+    # all of the vocabulary: the probabilities add up to one and come in descending order
+    ids, probs = orc.topk_softmax(lg[:1], 97)
+    assert abs(probs.sum() - 1.0) < 1e-12 and np.all(np.diff(probs[0]) <= 0) and sorted(ids[0]) == list(range(97))
+    # shift invariance, and no overflow on large logits
+    a = orc.topk_softmax(lg, 4)[1]
+    b = orc.topk_softmax(lg + 1000.0, 4)[1]
+    np.testing.assert_allclose(a, b, rtol=1e-9)
