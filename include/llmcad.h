@@ -136,7 +136,8 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out);
 void llmcad_destroy(llmcad_ctx *ctx);
 
 /* Bytes of the KV cache / of the packed weight buffer for this configuration.
- * The caller allocates both as DEVICE memory (256-byte aligned). */
+ * The caller allocates both as DEVICE memory, 256-byte aligned (the pass refuses other pointers
+ * with LLMCAD_ERR_INVALID_ARG: weight tiles travel as bulk copies, K/V rows as vector stores). */
 size_t llmcad_kv_cache_bytes(const llmcad_config *cfg);
 size_t llmcad_packed_weight_bytes(const llmcad_config *cfg);
 

@@ -447,6 +447,8 @@ int reset_chain_sync(llmcad_ctx *ctx, cudaStream_t st)
 int check_pass_args(const llmcad_ctx *ctx, const void *packed, const void *kv, int P, const void *tok, const void *par, int n)
 {
     if (ctx == nullptr || packed == nullptr || kv == nullptr || tok == nullptr || par == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    // bulk copies of weight tiles and 8/16-byte vector stores into the cache: the header asks for 256-byte alignment
+    if ((reinterpret_cast<uintptr_t>(packed) & 255) != 0 || (reinterpret_cast<uintptr_t>(kv) & 255) != 0) return LLMCAD_ERR_INVALID_ARG;
     if (n < 1 || P < 0) return LLMCAD_ERR_INVALID_ARG;
     if (n > ctx->cfg.max_tree) return LLMCAD_ERR_UNSUPPORTED;
     if ((long long)P + n > ctx->cfg.max_seq) return LLMCAD_ERR_CAPACITY;
