@@ -241,3 +241,32 @@ def test_host_entry_equals_device_entry():
     assert np.array_equal(host["scalars"].numpy(), a["scalars"])
     L = a["scalars"][B.S_ACCEPTED_LEN]
     assert np.array_equal(host["accepted_path"].numpy()[:L], a["accepted_path"][:L])
+
+
+# ----------------------------------------------------------------------------- tuning paths
+
+_TUNING_SCRIPT = r"""
+import sys, os
+sys.path.insert(0, os.path.join(sys.argv[1], "tests")); sys.path.insert(0, sys.argv[1])
+import numpy as np
+import test_gpu_pass as T
+twin, parent, tokens = T.bf16_case(T.SMALL_BF16, 100, 40, 10, "uniform4", seed=7, scale=3.0)
+T.run_bf16_parity(twin, 100, parent, tokens)
+twin, parent, tokens = T.bf16_case(T.SMALL_BF16, 64, 128, 12, "uniform4", seed=8, scale=3.0)
+T.run_bf16_parity(twin, 64, parent, tokens, plant=False)
+print("ok")
+"""
+
+
+@pytest.mark.parametrize("env", [{"LLMCAD_CHAIN_MAX": "4"}, {"LLMCAD_CHAIN_MAX": "2", "LLMCAD_PDL": "0"}, {"LLMCAD_COMP": "0"},
+                                 {"LLMCAD_GEMM_PAIR_K": "1"}, {"LLMCAD_GEMM_STAGES": "2", "LLMCAD_GEMM_L2_AHEAD": "0"}])
+def test_tuning_paths_stay_correct(env):
+    """The environment knobs select other code paths of the same kernels (several dependent GEMMs per
+    launch with grid barriers, no programmatic dependent launch, plain bf16 activations, ring items
+    of one k-block, a two-stage ring): each must still match the oracle. The knobs are read once per
+    process, hence the child process."""
+    import os, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    e = dict(os.environ, **env)
+    r = subprocess.run([sys.executable, "-c", _TUNING_SCRIPT, root], env=e, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and r.stdout.strip().endswith("ok"), r.stdout[-2000:] + r.stderr[-4000:]
