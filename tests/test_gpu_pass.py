@@ -270,3 +270,37 @@ def test_tuning_paths_stay_correct(env):
     e = dict(os.environ, **env)
     r = subprocess.run([sys.executable, "-c", _TUNING_SCRIPT, root], env=e, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and r.stdout.strip().endswith("ok"), r.stdout[-2000:] + r.stderr[-4000:]
+
+
+def test_queued_passes_of_changing_size_are_reproducible():
+    """Passes over trees of different sizes queued back to back on one stream (no host
+    synchronisation in between) must each give, bit for bit, what the same pass gives alone: the
+    arrival counters, the alternating counter sets and the helpers' flags of the GEMM tail leave no
+    state behind that depends on timing or on the previous launch's shape."""
+    cfg = gen.shrink(gen.MODELS["7b"], 2)
+    P = 200
+    twin = Twin(cfg, P + 136, keep_host=False)
+    twin.fill_prefix_synthetic(P)
+    v = twin.v
+    cases = []
+    for n in (1, 16, 32, 64, 128):
+        tokens = torch.as_tensor(gen.gen_tokens(cfg, n, seed=n), device=DEV)
+        parent = torch.as_tensor(gen.tree_random(n, 12, "uniform4", n) if n > 1 else np.array([-1], np.int32), device=DEV)
+        out = v.verify_tree(P, tokens, parent)
+        torch.cuda.synchronize()
+        assert out["scalars"][B.S_STATUS].item() == 0
+        cases.append((n, tokens, parent, {k: t.clone() for k, t in out.items()}))
+    rng = np.random.default_rng(1)
+    for _ in range(4):
+        outs = []
+        for _ in range(40):
+            ci = int(rng.integers(len(cases)))
+            n, tokens, parent, _ref = cases[ci]
+            o = v.new_outputs(n)
+            v.verify_tree(P, tokens, parent, out=o)
+            outs.append((ci, o))
+        torch.cuda.synchronize()
+        for ci, o in outs:
+            ref = cases[ci][3]
+            assert torch.equal(o["logits"], ref["logits"]) and torch.equal(o["argmax"], ref["argmax"])
+            assert torch.equal(o["scalars"], ref["scalars"]) and torch.equal(o["accepted_path"], ref["accepted_path"])
