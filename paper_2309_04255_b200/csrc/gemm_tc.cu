@@ -525,6 +525,34 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
 #define LLMCAD_TRACE(slot) do { if (p.trace) p.trace[(size_t)blockIdx.x * 16 + (slot)] = global_timer_ns(); } while (0)
     if (threadIdx.x == 0) LLMCAD_TRACE(0);
 
+    // State of the weight producer (thread 0). It lives across the start-up barrier: the first
+    // ring-full of copies goes out right after the barriers are initialised, before TMEM allocation
+    // and before the other warps are even needed.
+    Cursor<PK> pc;
+    int ps = 0;
+    uint32_t ppar = 1, pissued = 0;    // a fresh barrier passes a wait on parity 1: no special first lap
+    uint64_t pol_stream = 0;
+    auto issue_item = [&]() {          // the next item of the stream into ring stage ps (which must be free)
+        const GemmDesc &d = p.g[pc.g];
+        const int nk = pc.nk();
+        const uint32_t full = smem_u32(&ctl.full[ps]);
+        const uint32_t dst = smem_base + ps * stage_bytes;
+        mbar_expect_tx(full, (uint32_t)nk * (kATileBytes + b_tile_bytes));
+        if (d.w_tiled != nullptr) {
+            // consecutive k-blocks of a tile are contiguous in the tiled layout: one copy
+            const size_t t = (size_t)(pc.tile + (pc.half ? d.up_tile_offset : 0)) * d.kb_per_tile + pc.kb0();
+            bulk_load_1d(dst, d.w_tiled + t * kATileBytes, (uint32_t)nk * kATileBytes, full, pol_stream);
+        } else {
+            for (int k = 0; k < nk; ++k)
+                tma_load_2d(dst + k * kATileBytes, &maps.w[pc.g], (pc.kb0() + k) * kBlockK,
+                            (pc.half ? d.up_row_offset : 0) + pc.tile * kTileM, full, pol_stream);
+        }
+        __threadfence_block();
+        if (pissued == 0) LLMCAD_TRACE(2);
+        ctl.a_issued = ++pissued;      // the activation loader may now add its bytes to this stage
+        pc.advance(p);
+        if (++ps == p.stages) { ps = 0; ppar ^= 1u; }
+    };
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&ctl.full[s]), 1);
@@ -540,6 +568,9 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         for (int w = 0; w < 4; ++w) ctl.dumped[w] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+        pc.init(p);
+        while (!pc.done(p) && pissued < (uint32_t)p.stages && pissued < (uint32_t)p.pre_items) issue_item();
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
@@ -562,56 +593,34 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         // Streams this CTA's weight tiles of the whole chain, in order, as fast as ring slots
         // free up; it never looks at activations or barriers between GEMMs.
         if (lane == 0) {
-            uint64_t pol_stream;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            Cursor<PK> c, cpf;                   // next item to copy into the ring / to prefetch into L2
-            c.init(p);
+            Cursor<PK> cpf;                      // next item to prefetch into L2 (pc: next item to copy into the ring)
             cpf.init(p);
-            int s = 0;
-            uint32_t par = 1, issued = 0, prefetched = 0;   // a fresh barrier passes a wait on parity 1: no special first lap
+            uint32_t prefetched = 0;
             uint64_t t_idle = 0;
-            while (!c.done(p)) {
+            while (!pc.done(p)) {
                 // While the previous kernel is still in its tail, a full-speed fill of every ring of the
                 // grid would sit in the memory system in front of that tail's few, latency-bound accesses
                 // and stretch it by more than the head start is worth: hold back after pre_items.
-                if (issued >= (uint32_t)p.pre_items && !ctl.dep_ok) {
+                if (pissued >= (uint32_t)p.pre_items && !ctl.dep_ok) {
                     __nanosleep(64);
                     if (t_idle == 0) t_idle = global_timer_ns();
                     else if (*abort_flag || global_timer_ns() - t_idle > kWaitLimitNs) { timed_out = true; break; }
                     continue;
                 }
-                if (mbar_try(smem_u32(&ctl.empty[s]), par)) {
-                    const GemmDesc &d = p.g[c.g];
-                    const int nk = c.nk();
-                    const uint32_t full = smem_u32(&ctl.full[s]);
-                    const uint32_t dst = smem_base + s * stage_bytes;
-                    mbar_expect_tx(full, (uint32_t)nk * (kATileBytes + b_tile_bytes));
-                    if (d.w_tiled != nullptr) {
-                        // consecutive k-blocks of a tile are contiguous in the tiled layout: one copy
-                        const size_t t = (size_t)(c.tile + (c.half ? d.up_tile_offset : 0)) * d.kb_per_tile + c.kb0();
-                        bulk_load_1d(dst, d.w_tiled + t * kATileBytes, (uint32_t)nk * kATileBytes, full, pol_stream);
-                    } else {
-                        for (int k = 0; k < nk; ++k)
-                            tma_load_2d(dst + k * kATileBytes, &maps.w[c.g], (c.kb0() + k) * kBlockK,
-                                        (c.half ? d.up_row_offset : 0) + c.tile * kTileM, full, pol_stream);
-                    }
-                    __threadfence_block();
-                    if (issued == 0) LLMCAD_TRACE(2);
-                    ctl.a_issued = ++issued;     // the activation loader may now add its bytes to this stage
-                    c.advance(p);
-                    if (++s == p.stages) { s = 0; par ^= 1u; }
+                if (mbar_try(smem_u32(&ctl.empty[ps]), ppar)) {
+                    issue_item();
                     t_idle = 0;
                     continue;
                 }
                 // The ring is full: the consumers are busy with a tail or a barrier between two GEMMs.
                 // Weights do not depend on any of that, so pull the next ones from HBM into L2 now;
                 // when the ring moves again it refills at L2 speed.
-                if (prefetched < issued) {       // the ring overtook the prefetch cursor: catch up
-                    while (prefetched < issued && !cpf.done(p)) { cpf.advance(p); ++prefetched; }
+                if (prefetched < pissued) {       // the ring overtook the prefetch cursor: catch up
+                    while (prefetched < pissued && !cpf.done(p)) { cpf.advance(p); ++prefetched; }
                 }
-                if (!cpf.done(p) && prefetched < issued + (uint32_t)p.stages + (uint32_t)p.l2_ahead) {
+                if (!cpf.done(p) && prefetched < pissued + (uint32_t)p.stages + (uint32_t)p.l2_ahead) {
                     const GemmDesc &d = p.g[cpf.g];
-                    if (prefetched >= issued + (uint32_t)p.stages && d.w_tiled != nullptr) {
+                    if (prefetched >= pissued + (uint32_t)p.stages && d.w_tiled != nullptr) {
                         const size_t t = (size_t)(cpf.tile + (cpf.half ? d.up_tile_offset : 0)) * d.kb_per_tile + cpf.kb0();
                         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(d.w_tiled + t * kATileBytes),
                                      "r"((uint32_t)cpf.nk() * kATileBytes) : "memory");
