@@ -105,14 +105,14 @@ struct llmcad_ctx {
     TreeBuffers tb{};
     int32_t *ibuf = nullptr;  // tokens[128], parent[128], argmax[128], path[128], scalars[8], chain[128]
     float *partials = nullptr;
-    uint32_t *flags = nullptr;
+    uint32_t *arrivals = nullptr;        // arrival counters of the GEMM tails (two sets)
     float *ssq[2] = {nullptr, nullptr};   // partial sums of squares for the folded attention / FFN norms
     float *attn_ws = nullptr;
     uint32_t *attn_counters = nullptr;
     uint32_t *grid_counter = nullptr;   // grid barrier of the GEMM chains
     uint32_t barrier_base = 0;          // its value once everything enqueued so far has run
-    int ticket_set = 0;                 // arrival-counter set of the next GEMM launch (launches alternate)
-    int prev_gemms = 0, prev_ticket_words = 0;   // what the last GEMM launch touched in its set
+    int arrival_set = 0;                 // arrival-counter set of the next GEMM launch (launches alternate)
+    int prev_gemms = 0, prev_arrival_words = 0;   // what the last GEMM launch touched in its set
     int64_t launches = 0;
     unsigned long long *trace = nullptr;   // optional timeline buffer (llmcad_set_gemm_trace): [launch][256][16]
     int trace_launch = 0, trace_capacity = 0;
@@ -233,15 +233,15 @@ struct Chain {
     {
         if (p.n_gemms == 0) return LLMCAD_OK;
         p.partials = ctx->partials;
-        p.tickets = ctx->flags;
-        p.ticket_set = ctx->ticket_set;
+        p.arrivals = ctx->arrivals;
+        p.arrival_set = ctx->arrival_set;
         p.prev_gemms = ctx->prev_gemms;
-        p.prev_ticket_words = ctx->prev_ticket_words;
-        ctx->ticket_set ^= 1;
+        p.prev_arrival_words = ctx->prev_arrival_words;
+        ctx->arrival_set ^= 1;
         ctx->prev_gemms = p.n_gemms;
-        ctx->prev_ticket_words = 0;
+        ctx->prev_arrival_words = 0;
         for (int g = 0; g < p.n_gemms; ++g)
-            if (p.g[g].n_tiles * 4 > ctx->prev_ticket_words) ctx->prev_ticket_words = p.g[g].n_tiles * 4;
+            if (p.g[g].n_tiles * 4 > ctx->prev_arrival_words) ctx->prev_arrival_words = p.g[g].n_tiles * 4;
         p.grid_counter = ctx->grid_counter;
         p.barrier_base = ctx->barrier_base;
         p.status = status;
@@ -431,16 +431,16 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
     return LLMCAD_OK;
 }
 
-// The chain kernels synchronise through a grid counter and per-tile tickets. Both return to a
+// The chain kernels synchronise through a grid counter and per-tile arrival counters. Both return to a
 // known state by themselves, but not when a wait ran out: start every call from zero.
 int reset_chain_sync(llmcad_ctx *ctx, cudaStream_t st)
 {
     if (!ctx->tc_gemm) return LLMCAD_OK;
     CUDA_TRY(cudaMemsetAsync(ctx->grid_counter, 0, sizeof(uint32_t), st));
-    CUDA_TRY(cudaMemsetAsync(ctx->flags, 0, kTicketWords * sizeof(uint32_t), st));
+    CUDA_TRY(cudaMemsetAsync(ctx->arrivals, 0, kArrivalWords * sizeof(uint32_t), st));
     ctx->barrier_base = 0;
-    ctx->ticket_set = 0;
-    ctx->prev_gemms = ctx->prev_ticket_words = 0;
+    ctx->arrival_set = 0;
+    ctx->prev_gemms = ctx->prev_arrival_words = 0;
     return LLMCAD_OK;
 }
 
@@ -541,7 +541,7 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ok = ok && alloc((void **)&ctx->tb.rope_cs, 128 * (hd / 2) * sizeof(float2));
     ok = ok && alloc((void **)&ctx->ibuf, (520 + 128) * 4);
     ok = ok && alloc((void **)&ctx->partials, gemm_tc_partial_floats(2 * ctx->n_sms, 128) * 4);
-    ok = ok && alloc((void **)&ctx->flags, kTicketWords * 4);   // arrival counters
+    ok = ok && alloc((void **)&ctx->arrivals, kArrivalWords * 4);   // arrival counters
     ok = ok && alloc((void **)&ctx->grid_counter, 256);
     const size_t ssq_floats = (size_t)4 * ((d + 127) / 128) * LLMCAD_MAX_TREE;
     ok = ok && alloc((void **)&ctx->ssq[0], ssq_floats * 4);
@@ -565,7 +565,7 @@ void llmcad_destroy(llmcad_ctx *ctx)
 {
     if (ctx == nullptr) return;
     void *ptrs[] = {ctx->x, ctx->xn, ctx->q, ctx->att, ctx->h, ctx->kv_lo, ctx->logits, ctx->tb.depth, ctx->tb.pos, ctx->tb.anc,
-                    ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->flags, ctx->attn_ws, ctx->attn_counters, ctx->ssq[0],
+                    ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->arrivals, ctx->attn_ws, ctx->attn_counters, ctx->ssq[0],
                     ctx->ssq[1], ctx->grid_counter};
     for (void *p : ptrs)
         if (p != nullptr) cudaFree(p);

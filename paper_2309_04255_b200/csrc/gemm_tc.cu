@@ -291,7 +291,7 @@ struct Cursor {
 // ------------------------------------------------------------------------------------------------
 // Finishing a 32-row group of an output tile. Every CTA that holds a share of a tile leaves its
 // accumulators in the workspace as [row group][gate|up][node][32 rows] fp32; the warp that arrives
-// last at the group's ticket (or the only holder) adds the shares in CTA order and applies the fused
+// last at the group's arrival counter (or the only holder) adds the shares in CTA order and applies the fused
 // epilogue. It works on four output rows at a time: lane = (node sub-index ns = lane / 8, row quad
 // r4 = lane % 8) and iteration `it` handles node 4 * it + ns, so that the shares, the residual stream
 // and every output move as 16- or 8-byte vectors, a rotary pair sits in one thread, and the loads of
@@ -751,8 +751,8 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         // The previous launch (complete now) counted arrivals in the other counter set; the launch
         // after this one will use that set again: put the words it touched back to zero.
         for (int g = 0; g < p.prev_gemms; ++g) {
-            uint32_t *old = p.tickets + ((size_t)(p.ticket_set ^ 1) * kMaxChain + g) * kTicketsPerGemm;
-            for (int i = (int)blockIdx.x * 128 + (int)threadIdx.x - 64; i < p.prev_ticket_words; i += (int)gridDim.x * 128) old[i] = 0;
+            uint32_t *old = p.arrivals + ((size_t)(p.arrival_set ^ 1) * kMaxChain + g) * kArrivalsPerGemm;
+            for (int i = (int)blockIdx.x * 128 + (int)threadIdx.x - 64; i < p.prev_arrival_words; i += (int)gridDim.x * 128) old[i] = 0;
         }
         uint32_t seg = 0;
         for (int g = 0; g < p.n_gemms && !timed_out; ++g) {
@@ -815,7 +815,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
             const bool dual = d.halves == 2;
             const size_t part_stride = (size_t)2 * p.n_pad * kTileM;   // floats per workspace slot (gate | up)
-            uint32_t *tickets = p.tickets + ((size_t)p.ticket_set * kMaxChain + g) * kTicketsPerGemm;
+            uint32_t *arrivals = p.arrivals + ((size_t)p.arrival_set * kMaxChain + g) * kArrivalsPerGemm;
             for (int seg_begin = r.begin; seg_begin < r.end && !timed_out; ++seg) {
                 const int tile = seg_begin / ipt;
                 const int tile_i0 = tile * ipt;
@@ -883,7 +883,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     fa.it_first = 0; fa.it_step = helped ? 2 : 1;
                     finish_rows(fa, lane);
                 } else {
-                    uint32_t *ctr = tickets + (size_t)tile * 4 + lane_grp;
+                    uint32_t *ctr = arrivals + (size_t)tile * 4 + lane_grp;
                     __syncwarp();
                     // release: the share written by all lanes of this warp is visible to whoever sees the count
                     if (lane == 0) {
@@ -945,7 +945,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             const int first_cta = tile_i0 / d.items_per_cta, last_cta = (tile_i0 + ipt - 1) / d.items_per_cta;
             const int n_parts = last_cta - first_cta + 1;
             const int n_fin = n_parts == 1 ? 1 : n_parts - ((min((last_cta + 1) * d.items_per_cta, d.n_tiles * ipt) > tile_i0 + ipt) ? 1 : 0);
-            const uint32_t *ctr = p.tickets + ((size_t)p.ticket_set * kMaxChain + g) * kTicketsPerGemm + (size_t)tile * 4 + lane_grp;
+            const uint32_t *ctr = p.arrivals + ((size_t)p.arrival_set * kMaxChain + g) * kArrivalsPerGemm + (size_t)tile * 4 + lane_grp;
             int bad = 0;
             if (lane == 0) {
                 // this CTA's own share first (a flag in shared memory), then everybody's (the arrival counter)
@@ -1068,7 +1068,7 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
     for (int g = 0; g < p.n_gemms; ++g) p.g[g].pair_k = pair_k;
     auto items_of = [](const GemmDesc &d) { return (long long)d.n_tiles * pairs_per_tile(d) * d.halves; };
     for (int g = 0; g < p.n_gemms; ++g) {
-        if (p.g[g].n_tiles > 4096) return cudaErrorInvalidValue;   // size of the ticket array
+        if (p.g[g].n_tiles > 4096) return cudaErrorInvalidValue;   // size of the arrival-counter array
         const long long total = items_of(p.g[g]);
         if (total > max_items) max_items = total;
     }

@@ -36,9 +36,9 @@ struct ChainParams {
     int stages;         // depth of the shared-memory ring
     int tmem_cols;      // allocated TMEM columns (power of two)
     float *partials;    // [grid][2 slots][2 halves][n_pad][128] fp32 partial tiles
-    uint32_t *tickets;  // [2 sets][kMaxChain][4096][4] arrivals per (GEMM, tile, 32-row group)
-    int ticket_set;     // the set this launch counts in (launches alternate); it finds it all zero
-    int prev_gemms, prev_ticket_words;   // what the previous launch touched in the other set: this launch zeroes it
+    uint32_t *arrivals;  // [2 sets][kMaxChain][4096][4] arrivals per (GEMM, tile, 32-row group)
+    int arrival_set;     // the set this launch counts in (launches alternate); it finds it all zero
+    int prev_gemms, prev_arrival_words;   // what the previous launch touched in the other set: this launch zeroes it
     uint32_t *grid_counter;   // grid barrier between the GEMMs of a chain (monotonic)
     uint32_t barrier_base;    // value of the counter when this launch starts
     int32_t *status;
@@ -61,8 +61,8 @@ bool make_act_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64
                        uint64_t plane_rows);
 
 size_t gemm_tc_partial_floats(int n_sms, int max_n_pad);
-constexpr size_t kTicketsPerGemm = 4096 * 4;
-constexpr size_t kTicketWords = 2 * kMaxChain * kTicketsPerGemm;   // both sets
+constexpr size_t kArrivalsPerGemm = 4096 * 4;
+constexpr size_t kArrivalWords = 2 * kMaxChain * kArrivalsPerGemm;   // both sets
 
 // Describes one GEMM for a chain (fills everything but items_per_cta, which the launcher sets).
 GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled = nullptr);
