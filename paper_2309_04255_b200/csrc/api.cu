@@ -205,20 +205,12 @@ struct Chain {
     Chain() { p = ChainParams{}; }
     // W is `which` (0 qkv, 1 o, 2 gate/up, 3 down) of layer l, or the lm_head when l < 0;
     // act selects the activation buffer it multiplies (0 normalised stream, 1 attention output, 2 SwiGLU output)
-    bool has_next = false;
-    GemmDesc next{};
     static const char *weight_ptr(llmcad_ctx *ctx, int l, int which)
     {
         const char *base = static_cast<const char *>(ctx->maps_for);
         if (l < 0) return base + ctx->lay.lm_head;
         const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
         return lb + (which == 0 ? ctx->lay.wqkv : which == 1 ? ctx->lay.wo : which == 2 ? ctx->lay.wgu : ctx->lay.wdown);
-    }
-    // the GEMM that the launch after this one will run: its first tiles get prefetched into L2
-    void set_next(llmcad_ctx *ctx, int l, int which, int n_in, const EpiParams &ep)
-    {
-        next = make_gemm_desc(n_in, ep, weight_ptr(ctx, l, which));
-        has_next = true;
     }
     void add(llmcad_ctx *ctx, int l, int which, int act, int n_in, const EpiParams &ep, int n_pad)
     {
@@ -249,7 +241,7 @@ struct Chain {
         uint32_t arrivals = 0;
         ctx->launches++;
         TimedLaunch tl(ctx, 0, st);
-        CUDA_TRY(launch_gemm_chain(maps, p, ctx->n_sms, st, &arrivals, has_next ? &next : nullptr));
+        CUDA_TRY(launch_gemm_chain(maps, p, ctx->n_sms, st, &arrivals));
         ctx->barrier_base += arrivals;
         return LLMCAD_OK;
     }
@@ -387,7 +379,6 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
                 ch.add(ctx, specs[j].l, specs[j].which, specs[j].act, specs[j].n_in, specs[j].ep, n_pad);
                 ++j;
             } while (j < specs.size() && ch.p.n_gemms < chain_max && !specs[j].attention_first);
-            if (j < specs.size()) ch.set_next(ctx, specs[j].l, specs[j].which, specs[j].n_in, specs[j].ep);
             if ((rc = ch.launch(ctx, status, st)) != LLMCAD_OK) return rc;
             i = j;
         }

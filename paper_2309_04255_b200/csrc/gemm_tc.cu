@@ -210,7 +210,6 @@ struct SharedCtl {
     uint32_t tmem_base;
     volatile int abort_flag;
     volatile uint32_t a_issued;     // ring items whose weight copy (and expect_tx) has been issued
-    volatile uint32_t dep_ok;       // the grid dependency is resolved: the previous kernel of the stream is complete
     volatile uint32_t dumped[4];    // per row group: this CTA's share of its last tile is in the workspace
     float rs[4][LLMCAD_MAX_TREE];   // per epilogue warp: rsqrt(mean(x^2) + eps) of the folded input RMSNorm
 };
@@ -564,13 +563,12 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         }
         ctl.abort_flag = 0;
         ctl.a_issued = 0;
-        ctl.dep_ok = 0;
         for (int w = 0; w < 4; ++w) ctl.dumped[w] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
         pc.init(p);
-        while (!pc.done(p) && pissued < (uint32_t)p.stages && pissued < (uint32_t)p.pre_items) issue_item();
+        while (!pc.done(p) && pissued < (uint32_t)p.stages) issue_item();
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
@@ -598,15 +596,6 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             uint32_t prefetched = 0;
             uint64_t t_idle = 0;
             while (!pc.done(p)) {
-                // While the previous kernel is still in its tail, a full-speed fill of every ring of the
-                // grid would sit in the memory system in front of that tail's few, latency-bound accesses
-                // and stretch it by more than the head start is worth: hold back after pre_items.
-                if (pissued >= (uint32_t)p.pre_items && !ctl.dep_ok) {
-                    __nanosleep(64);
-                    if (t_idle == 0) t_idle = global_timer_ns();
-                    else if (*abort_flag || global_timer_ns() - t_idle > kWaitLimitNs) { timed_out = true; break; }
-                    continue;
-                }
                 if (mbar_try(smem_u32(&ctl.empty[ps]), ppar)) {
                     issue_item();
                     t_idle = 0;
@@ -634,22 +623,6 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 else if (*abort_flag || global_timer_ns() - t_idle > kWaitLimitNs) { timed_out = true; break; }
             }
             if (p.n_gemms == 1) LLMCAD_TRACE(6);
-            // This CTA's weight stream has ended; its tail (partial-tile reduction, epilogue) and the
-            // hand-over to the next kernel leave HBM idle. Pull the first tiles that the CTA with this
-            // index will want in the next launch into L2 meanwhile.
-            if (p.next_items > 0 && p.next.w_tiled != nullptr && !timed_out) {
-                const GemmDesc &d = p.next;
-                const int ppt = pairs_per_tile_c<PK>(d), ipt = ppt * d.halves;
-                const Range r = cta_range<PK>(d);
-                const int end = min(r.end, r.begin + p.next_items);
-                for (int it = r.begin; it < end; ++it) {
-                    const int tile = it / ipt, q = it - tile * ipt, kp = q / d.halves, half = q - kp * d.halves;
-                    const int kb0 = kp * PK, nk = min(PK, d.kb_per_tile - kb0);
-                    const size_t t = (size_t)(tile + (half ? d.up_tile_offset : 0)) * d.kb_per_tile + kb0;
-                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(d.w_tiled + t * kATileBytes),
-                                 "r"((uint32_t)nk * kATileBytes) : "memory");
-                }
-            }
         }
     } else if (warp == 6) {
         // ================================================= activation loader
@@ -664,7 +637,6 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             int s = 0, ready = 0, traced_g = 0;
             uint32_t i = 0;
             pdl_wait();
-            ctl.dep_ok = 1;
             while (!c.done(p) && !timed_out) {
                 uint64_t t0 = 0;
                 // (1) the stage is ours: the producer has passed its "empty" wait and armed the barrier
@@ -1052,8 +1024,7 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)
     return d;
 }
 
-cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, cudaStream_t st, uint32_t *barrier_arrivals,
-                              const GemmDesc *next)
+cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, cudaStream_t st, uint32_t *barrier_arrivals)
 {
     if (p.n_gemms < 1 || p.n_gemms > kMaxChain) return cudaErrorInvalidValue;
     // a chain needs every CTA at every barrier: the grid is the SM count; a single GEMM may use fewer
@@ -1112,23 +1083,9 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    p.pre_items = 1 << 30;   // no holding back: measured best on B200 (the knob stays as a tuning aid)
-    if (const char *e = getenv("LLMCAD_GEMM_PRE_ITEMS")) p.pre_items = atoi(e);   // tuning aid
     // weight tiles pulled into L2 beyond the ring while the ring is blocked
     p.l2_ahead = 8;
     if (const char *e = getenv("LLMCAD_GEMM_L2_AHEAD")) p.l2_ahead = atoi(e);
-    // what the following launch will stream first (it uses the same grid and the same split)
-    p.next_items = 0;
-    if (next != nullptr && next->w_tiled != nullptr && grid == n_sms) {
-        p.next = *next;
-        p.next.pair_k = pair_k;
-        const long long total = items_of(p.next);
-        long long ipc = (total + grid - 1) / grid;
-        if (p.next.halves == 2) ipc += ipc & 1;
-        p.next.items_per_cta = (int)ipc;
-        p.next_items = 24 / pair_k;             // 12 x 32 KB x 148 CTAs = 57 MB, under half of L2
-        if (const char *e = getenv("LLMCAD_GEMM_NEXT_ITEMS")) p.next_items = atoi(e);
-    }
     if (barrier_arrivals) *barrier_arrivals = 4u * (uint32_t)grid * (uint32_t)(p.n_gemms - 1);
     LaunchCfg lc(grid, kThreads, smem, st);
     if (pair_k == 1) return cudaLaunchKernelEx(&lc.cfg, gemm_chain_kernel<__nv_bfloat16, 1>, maps, p);

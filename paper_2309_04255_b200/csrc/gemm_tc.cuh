@@ -43,10 +43,7 @@ struct ChainParams {
     uint32_t barrier_base;    // value of the counter when this launch starts
     int32_t *status;
     unsigned long long *trace;  // optional [grid][16] timeline in ns (nullptr: off)
-    int pre_items;      // ring items a CTA may request before the previous kernel of the stream is complete
     int l2_ahead;       // ring items the producer may prefetch into L2 beyond the ring
-    int next_items;     // leading items of `next` (the GEMM of the following launch) each CTA pulls into L2 when its own stream ends
-    GemmDesc next;
     GemmDesc g[kMaxChain];
 };
 
@@ -69,7 +66,6 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled = nul
 
 // Launches a chain of 1..kMaxChain dependent GEMMs as one persistent kernel. Returns in
 // *barrier_arrivals how far the grid counter advances (the caller adds it to its running base).
-cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, cudaStream_t st, uint32_t *barrier_arrivals,
-                              const GemmDesc *next = nullptr);
+cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, cudaStream_t st, uint32_t *barrier_arrivals);
 
 }  // namespace llmcad
