@@ -337,14 +337,17 @@ struct FinishArgs {
 // G node groups travel together (one round trip per G iterations), kB shares per node group at a
 // time: tiles held by many CTAs have many shares and few iterations per finisher (G = 2, kB = 4),
 // tiles held by one or two have few shares and many iterations (G = 4, kB = 2).
-template <int G, int kB>
+// One instantiation per epilogue mode as well: the routine is cold whenever it runs, and what it
+// costs in instruction-cache misses is the code it walks through, not the code that exists.
+template <int G, int kB, int MODE>
 __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
 {
     typedef __nv_bfloat16 T;
     const ChainParams &p = *fa.p;
     const GemmDesc &d = *fa.d;
     const EpiParams &ep = d.ep;
-    const int mode = ep.mode, n_nodes = ep.n, n_out = ep.n_out, n_pad = p.n_pad;
+    constexpr int mode = MODE;
+    const int n_nodes = ep.n, n_out = ep.n_out, n_pad = p.n_pad;
     const bool dual = d.halves == 2, comp = ep.comp != 0, has_rs = ep.ssq_in != nullptr, has_xg = ep.xg_out != nullptr;
     const bool resid = mode == EPI_RESID;
     const int tile = fa.tile, lane_grp = fa.lane_grp;
@@ -481,10 +484,21 @@ __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
     }
 }
 
+template <int G, int kB>
+__device__ __forceinline__ void finish_rows_m(const FinishArgs &fa, int lane)
+{
+    switch (fa.d->ep.mode) {
+    case EPI_QKV: finish_rows_t<G, kB, EPI_QKV>(fa, lane); break;
+    case EPI_RESID: finish_rows_t<G, kB, EPI_RESID>(fa, lane); break;
+    case EPI_SWIGLU: finish_rows_t<G, kB, EPI_SWIGLU>(fa, lane); break;
+    default: finish_rows_t<G, kB, EPI_PLAIN>(fa, lane); break;
+    }
+}
+
 __device__ __forceinline__ void finish_rows(const FinishArgs &fa, int lane)
 {
-    if (fa.last_cta - fa.first_cta + 1 > 3) finish_rows_t<2, 4>(fa, lane);
-    else finish_rows_t<4, 2>(fa, lane);
+    if (fa.last_cta - fa.first_cta + 1 > 3) finish_rows_m<2, 4>(fa, lane);
+    else finish_rows_m<4, 2>(fa, lane);
 }
 
 }  // namespace
