@@ -348,8 +348,9 @@ __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
     const EpiParams &ep = d.ep;
     constexpr int mode = MODE;
     const int n_nodes = ep.n, n_out = ep.n_out, n_pad = p.n_pad;
-    const bool dual = d.halves == 2, comp = ep.comp != 0, has_rs = ep.ssq_in != nullptr, has_xg = ep.xg_out != nullptr;
-    const bool resid = mode == EPI_RESID;
+    constexpr bool dual = MODE == EPI_SWIGLU;      // the one mode with two accumulators per tile (gate, up)
+    const bool comp = ep.comp != 0, has_rs = ep.ssq_in != nullptr, has_xg = ep.xg_out != nullptr;
+    constexpr bool resid = mode == EPI_RESID;
     const int tile = fa.tile, lane_grp = fa.lane_grp;
     const int ns = lane >> 3, r4 = lane & 7;
     const int row0 = tile * kTileM + lane_grp * 32 + 4 * r4;   // first of this lane's four output rows
