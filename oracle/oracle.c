@@ -329,3 +329,47 @@ void orc_topk_softmax(const double *logits, int n, int vocab, int k, int *ids, d
     }
     free(p);
 }
+
+/* Branches of a token tree (Sec. 3.2): one per leaf, the path from the root to that leaf. For the
+ * leaves in ascending node order: the leaf, the cumulative confidence of the branch (the product
+ * of the confidences of its tokens) and the number of draft tokens on it. The root is the last
+ * committed token, not a draft token: it counts in neither. Returns the number of branches. */
+int orc_tree_branches(const int *parent, const double *node_conf, int n, int *leaf, double *cum_conf, int *branch_len)
+{
+    int nb = 0;
+    for (int i = 0; i < n; ++i) {
+        int has_child = 0;
+        for (int j = i + 1; j < n; ++j)
+            if (parent[j] == i) has_child = 1;
+        if (has_child) continue;
+        double c = 1.0;
+        int len = 0;
+        for (int a = i; parent[a] >= 0; a = parent[a]) {
+            c *= node_conf[a];
+            ++len;
+        }
+        leaf[nb] = i;
+        cum_conf[nb] = c;
+        branch_len[nb] = len;
+        ++nb;
+    }
+    return nb;
+}
+
+/* Confidence-based branch pacer, Eq. 1-2. With N branches, M tokens to share out, branch x
+ * holding T_x tokens at cumulative confidence C_x:  f(x) = M * C_x / sum_i C_i - T_x, the share
+ * of the M tokens that the branch's confidence entitles it to minus what it has. Max-min fairness
+ * keeps the smallest f as large as possible, so the next token goes to the branch whose f is
+ * largest (every other choice lowers an f that is already smaller); ties go to the lower index.
+ * Fills f[0..N) and returns that branch. */
+int orc_branch_pacer(const double *cum_conf, const int *branch_len, int n_branches, double m_tokens, double *f)
+{
+    double total = 0.0;
+    for (int i = 0; i < n_branches; ++i) total += cum_conf[i];
+    int next = 0;
+    for (int x = 0; x < n_branches; ++x) {
+        f[x] = m_tokens * (cum_conf[x] / total) - (double)branch_len[x];
+        if (f[x] > f[next]) next = x;
+    }
+    return next;
+}

@@ -292,3 +292,28 @@ def topk_softmax(logits: np.ndarray, k: int):
     probs = np.zeros((n, k), np.float64)
     lib().orc_topk_softmax(_p(lg), C.c_int(n), C.c_int(vocab), C.c_int(k), _p(ids), _p(probs))
     return ids, probs
+
+
+def tree_branches(parent, node_conf):
+    """Sec. 3.2: the root-to-leaf branches of a tree: (leaf ids, cumulative confidences, draft tokens per branch)."""
+    par = np.ascontiguousarray(parent, dtype=np.int32)
+    conf = np.ascontiguousarray(node_conf, dtype=np.float64)
+    n = len(par)
+    leaf = np.zeros(n, np.int32)
+    cum = np.zeros(n, np.float64)
+    length = np.zeros(n, np.int32)
+    f = lib().orc_tree_branches
+    f.restype = C.c_int
+    nb = int(f(_p(par), _p(conf), C.c_int(n), _p(leaf), _p(cum), _p(length)))
+    return leaf[:nb].copy(), cum[:nb].copy(), length[:nb].copy()
+
+
+def branch_pacer(cum_conf, branch_len, m_tokens: float):
+    """Eq. 1-2: (f(x) for every branch, the branch that gets the next token)."""
+    c = np.ascontiguousarray(cum_conf, dtype=np.float64)
+    t = np.ascontiguousarray(branch_len, dtype=np.int32)
+    out = np.zeros(len(c), np.float64)
+    f = lib().orc_branch_pacer
+    f.restype = C.c_int
+    nxt = int(f(_p(c), _p(t), C.c_int(len(c)), C.c_double(float(m_tokens)), _p(out)))
+    return out, nxt

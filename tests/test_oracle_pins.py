@@ -494,3 +494,85 @@ def test_topk_softmax_against_library_and_closed_forms():
     a = orc.topk_softmax(lg, 4)[1]
     b = orc.topk_softmax(lg + 1000.0, 4)[1]
     np.testing.assert_allclose(a, b, rtol=1e-9)
+
+
+def test_tree_branches_on_trees_with_known_branches():
+    """Sec. 3.2: a branch per leaf, cumulative confidence = product over its draft tokens."""
+    conf = np.array([0.123, 0.9, 0.8, 0.5, 0.25])          # the root's entry must not matter
+    # chain root-1-2-3-4: one branch through everything
+    leaf, cum, length = orc.tree_branches([-1, 0, 1, 2, 3], conf)
+    assert leaf.tolist() == [4] and length.tolist() == [4]
+    assert cum[0] == pytest.approx(0.9 * 0.8 * 0.5 * 0.25, rel=1e-15)
+    # star: every child of the root is a branch of one token
+    leaf, cum, length = orc.tree_branches([-1, 0, 0, 0, 0], conf)
+    assert leaf.tolist() == [1, 2, 3, 4] and length.tolist() == [1, 1, 1, 1] and cum.tolist() == conf[1:].tolist()
+    # root alone: one branch without draft tokens, confidence of the empty product
+    leaf, cum, length = orc.tree_branches([-1], conf[:1])
+    assert leaf.tolist() == [0] and length.tolist() == [0] and cum.tolist() == [1.0]
+    # the tree of the verification figure's shape: 0 -> (1 -> (3, 4), 2 -> 5)
+    leaf, cum, length = orc.tree_branches([-1, 0, 0, 1, 1, 2], np.array([1.0, 0.5, 0.4, 0.3, 0.2, 0.1]))
+    assert leaf.tolist() == [3, 4, 5] and length.tolist() == [2, 2, 2]
+    np.testing.assert_allclose(cum, [0.15, 0.10, 0.04], rtol=1e-15)
+
+
+def test_tree_branches_against_path_walking():
+    rng = np.random.default_rng(11)
+    for n in (2, 7, 33, 128):
+        parent = np.array(gen.tree_random(n, 10, "uniform4", n), dtype=np.int64)
+        conf = rng.uniform(0.05, 1.0, n)
+        leaf, cum, length = orc.tree_branches(parent, conf)
+        children = {i: [j for j in range(n) if parent[j] == i] for i in range(n)}
+        want = [i for i in range(n) if not children[i]]
+        assert leaf.tolist() == want
+        for b, i in enumerate(want):
+            path = []
+            while parent[i] >= 0:
+                path.append(i)
+                i = int(parent[i])
+            assert length[b] == len(path)
+            assert cum[b] == pytest.approx(float(np.prod(conf[path])) if path else 1.0, rel=1e-12)
+
+
+def test_branch_pacer_closed_forms():
+    """Eq. 1: f(x) = M C_x / sum C - T_x on values that can be checked by hand."""
+    f, nxt = orc.branch_pacer([0.75, 0.25], [4, 4], 8)
+    assert f.tolist() == [2.0, -2.0] and nxt == 0           # shares 6 and 2 of 8 tokens, each holds 4
+    f, nxt = orc.branch_pacer([0.75, 0.25], [7, 1], 8)
+    assert f.tolist() == [-1.0, 1.0] and nxt == 1           # the confident branch ran ahead of its share
+    # equal confidences: everybody is entitled to M / N, the shortest branch goes next
+    f, nxt = orc.branch_pacer([0.3] * 4, [3, 1, 2, 1], 10)
+    np.testing.assert_allclose(f, [-0.5, 1.5, 0.5, 1.5], rtol=1e-15)
+    assert nxt == 1                                         # tie between 1 and 3: the lower index
+    # one branch: it owns every token
+    f, nxt = orc.branch_pacer([0.01], [5], 9)
+    assert f.tolist() == [4.0] and nxt == 0
+
+
+def test_branch_pacer_invariants_and_max_min_choice():
+    """sum_x f(x) = M - sum_x T_x; f only depends on confidence ratios; and the branch it picks is
+    the one that leaves the smallest f largest after receiving a token (max-min fairness, Eq. 2),
+    found here by trying every branch."""
+    rng = np.random.default_rng(12)
+    for n in (2, 3, 8, 31):
+        c = rng.uniform(1e-4, 1.0, n) ** 3
+        t = rng.integers(0, 12, n)
+        m = float(t.sum() + rng.integers(0, 5))
+        f, nxt = orc.branch_pacer(c, t, m)
+        assert f.sum() == pytest.approx(m - t.sum(), abs=1e-9)
+        f2, nxt2 = orc.branch_pacer(c * 0.37, t, m)
+        np.testing.assert_allclose(f2, f, rtol=1e-12, atol=1e-12)
+        assert nxt2 == nxt
+        share = m * c / c.sum()
+        np.testing.assert_allclose(f, share - t, rtol=1e-12, atol=1e-12)
+        best = None
+        for y in range(n):
+            t_after = t.copy()
+            t_after[y] += 1
+            worst = (share - t_after).min()
+            if best is None or worst > best[0] + 1e-12:
+                best = (worst, y)
+        # several branches can leave the same minimum; the chosen one must be among the best
+        t_after = t.copy()
+        t_after[nxt] += 1
+        assert (share - t_after).min() == pytest.approx(best[0], abs=1e-9)
+        assert f[nxt] == f.max()
