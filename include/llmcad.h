@@ -299,6 +299,27 @@ int llmcad_extend_tree(llmcad_ctx *ctx, const void *packed_weights, void *kv_cac
 int llmcad_tree_confidence(const double *branch_conf, int32_t n_branches, double *t_c);
 int llmcad_update_threshold(double alpha, int32_t n_correct, int32_t n_all, double tree_confidence, double *alpha_next);
 
+/* Host-side scalars of the confidence-based branch pacer (Sec. 3.2, Eq. 1-2); plain arithmetic, no
+ * device work, all pointers host pointers.
+ * llmcad_tree_branches: the branches of a token tree, one per leaf (root-to-leaf paths), leaves in
+ * ascending node order. parent_idx[n] as for llmcad_verify_tree (parent_idx[0] = -1,
+ * parent_idx[i] < i); node_conf[n] = the confidence with which the generating model proposed each
+ * node's token, in (0, 1] (entry 0, the root, is the last committed token and is ignored). Outputs,
+ * each with room for n entries: leaf[b] = node index of the branch's leaf, cum_conf[b] = product
+ * of the confidences of the branch's draft tokens (1 for a tree of the root alone), branch_len[b] =
+ * number of draft tokens on it (the leaf's depth); *n_branches = number of entries written.
+ * llmcad_branch_pacer: f[x] = m_tokens * cum_conf[x] / sum_i cum_conf[i] - branch_len[x] for each
+ * of the n_branches branches (Eq. 1): the share of m_tokens tokens that the branch's confidence
+ * entitles it to, minus the tokens it holds. *next_branch = the branch with the largest f, the
+ * lower index on ties: giving the next token to any other branch would lower an f that is already
+ * smaller, so this choice keeps min_x f(x) (Eq. 2) as large as possible (max-min fairness).
+ * LLMCAD_ERR_INVALID_ARG for null pointers, n < 1 or n > LLMCAD_MAX_TREE, an invalid parent_idx,
+ * n_branches < 1, a negative length or m_tokens, or a confidence outside (0, 1]. */
+int llmcad_tree_branches(const int32_t *parent_idx, const double *node_conf, int32_t n, int32_t *leaf,
+                         double *cum_conf, int32_t *branch_len, int32_t *n_branches);
+int llmcad_branch_pacer(const double *cum_conf, const int32_t *branch_len, int32_t n_branches, double m_tokens,
+                        double *f, int32_t *next_branch);
+
 /* Number of kernels this library has launched through this context so far. */
 int64_t llmcad_launch_count(const llmcad_ctx *ctx);
 

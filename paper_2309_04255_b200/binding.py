@@ -30,7 +30,7 @@ EXPORTS = [
     "llmcad_verify_tree", "llmcad_verify_tree_host", "llmcad_prefill", "llmcad_tree_prep",
     "llmcad_accept_compact", "llmcad_tree_attention", "llmcad_skinny_gemm", "llmcad_launch_count",
     "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace", "llmcad_tiled_weight_bytes", "llmcad_tile_weight", "llmcad_skinny_gemm_tiled", "llmcad_tree_attention_noalloc", "llmcad_noalloc_last_error",
-    "llmcad_tree_confidence", "llmcad_update_threshold", "llmcad_extend_tree",
+    "llmcad_tree_confidence", "llmcad_update_threshold", "llmcad_extend_tree", "llmcad_tree_branches", "llmcad_branch_pacer",
 ]
 
 
@@ -321,6 +321,37 @@ def update_threshold(alpha: float, n_correct: int, n_all: int, t_c: float) -> fl
     f.argtypes = [C.c_double, C.c_int32, C.c_int32, C.c_double, C.POINTER(C.c_double)]
     _check(f(alpha, n_correct, n_all, t_c, C.byref(out)), "llmcad_update_threshold")
     return out.value
+
+
+def tree_branches(parent_idx, node_conf):
+    """Branches (root-to-leaf paths) of a token tree: (leaf ids, cumulative confidences, draft tokens per
+    branch), Sec. 3.2 (host arithmetic)."""
+    n = len(parent_idx)
+    par = (C.c_int32 * n)(*[int(x) for x in parent_idx])
+    conf = (C.c_double * n)(*[float(x) for x in node_conf])
+    leaf = (C.c_int32 * n)()
+    cum = (C.c_double * n)()
+    length = (C.c_int32 * n)()
+    nb = C.c_int32(0)
+    f = lib().llmcad_tree_branches
+    f.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_double), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_double),
+                  C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    _check(f(par, conf, n, leaf, cum, length, C.byref(nb)), "llmcad_tree_branches")
+    return list(leaf[:nb.value]), list(cum[:nb.value]), list(length[:nb.value])
+
+
+def branch_pacer(cum_conf, branch_len, m_tokens: float):
+    """Eq. 1-2: (f(x) per branch, index of the branch that gets the next token) (host arithmetic)."""
+    n = len(cum_conf)
+    c = (C.c_double * n)(*[float(x) for x in cum_conf])
+    t = (C.c_int32 * n)(*[int(x) for x in branch_len])
+    out = (C.c_double * n)()
+    nxt = C.c_int32(-1)
+    f = lib().llmcad_branch_pacer
+    f.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int32), C.c_int32, C.c_double, C.POINTER(C.c_double),
+                  C.POINTER(C.c_int32)]
+    _check(f(c, t, n, float(m_tokens), out, C.byref(nxt)), "llmcad_branch_pacer")
+    return list(out), nxt.value
 
 
 def tree_prep(parent: torch.Tensor, prefix_len: int):

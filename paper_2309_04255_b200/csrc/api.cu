@@ -916,6 +916,57 @@ int llmcad_update_threshold(double alpha, int32_t n_correct, int32_t n_all, doub
     return LLMCAD_OK;
 }
 
+int llmcad_tree_branches(const int32_t *parent_idx, const double *node_conf, int32_t n, int32_t *leaf,
+                         double *cum_conf, int32_t *branch_len, int32_t *n_branches)
+{
+    if (parent_idx == nullptr || node_conf == nullptr || leaf == nullptr || cum_conf == nullptr ||
+        branch_len == nullptr || n_branches == nullptr || n < 1 || n > LLMCAD_MAX_TREE)
+        return LLMCAD_ERR_INVALID_ARG;
+    if (parent_idx[0] != -1) return LLMCAD_ERR_INVALID_ARG;
+    bool inner[LLMCAD_MAX_TREE] = {};
+    double cum[LLMCAD_MAX_TREE];
+    int32_t depth[LLMCAD_MAX_TREE];
+    cum[0] = 1.0;
+    depth[0] = 0;
+    for (int32_t i = 1; i < n; ++i) {                         // parents come first: one sweep
+        const int32_t par = parent_idx[i];
+        if (par < 0 || par >= i || !(node_conf[i] > 0.0 && node_conf[i] <= 1.0)) return LLMCAD_ERR_INVALID_ARG;
+        inner[par] = true;
+        cum[i] = cum[par] * node_conf[i];
+        depth[i] = depth[par] + 1;
+    }
+    int32_t nb = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        if (inner[i]) continue;
+        leaf[nb] = i;
+        cum_conf[nb] = cum[i];
+        branch_len[nb] = depth[i];
+        ++nb;
+    }
+    *n_branches = nb;
+    return LLMCAD_OK;
+}
+
+int llmcad_branch_pacer(const double *cum_conf, const int32_t *branch_len, int32_t n_branches, double m_tokens,
+                        double *f, int32_t *next_branch)
+{
+    if (cum_conf == nullptr || branch_len == nullptr || f == nullptr || next_branch == nullptr || n_branches < 1 ||
+        !(m_tokens >= 0.0))
+        return LLMCAD_ERR_INVALID_ARG;
+    double total = 0.0;
+    for (int32_t i = 0; i < n_branches; ++i) {
+        if (!(cum_conf[i] > 0.0 && cum_conf[i] <= 1.0) || branch_len[i] < 0) return LLMCAD_ERR_INVALID_ARG;
+        total += cum_conf[i];
+    }
+    int32_t best = 0;
+    for (int32_t x = 0; x < n_branches; ++x) {
+        f[x] = m_tokens * (cum_conf[x] / total) - (double)branch_len[x];
+        if (f[x] > f[best]) best = x;
+    }
+    *next_branch = best;
+    return LLMCAD_OK;
+}
+
 int64_t llmcad_launch_count(const llmcad_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
 }  // extern "C"

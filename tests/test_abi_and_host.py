@@ -165,3 +165,34 @@ def test_fallback_scalars_match_the_oracle():
             B.update_threshold(*bad)
     with pytest.raises(B.LlmcadError):
         B.tree_confidence([0.5, 0.0])
+
+
+def test_branch_pacer_matches_the_oracle():
+    """llmcad_tree_branches / llmcad_branch_pacer (host arithmetic of Eq. 1-2) against the oracle on
+    random trees, and their argument checks."""
+    from oracle import oracle as orc
+    from paper_2309_04255_b200 import binding as B
+    from paper_2309_04255_b200 import inputs as gen
+    rng = np.random.default_rng(21)
+    for n in (1, 2, 5, 32, 77, 128):
+        for shape in ("uniform4", "geometric4", "chain"):
+            parent = np.arange(-1, n - 1) if shape == "chain" else gen.tree_random(n, 10, shape, n)
+            conf = rng.uniform(0.02, 1.0, n)
+            leaf, cum, length = B.tree_branches(parent, conf)
+            o_leaf, o_cum, o_len = orc.tree_branches(parent, conf)
+            assert leaf == o_leaf.tolist() and length == o_len.tolist()
+            np.testing.assert_allclose(cum, o_cum, rtol=1e-12)
+            m = float(sum(length)) + float(rng.integers(0, 4))
+            f, nxt = B.branch_pacer(cum, length, m)
+            o_f, o_nxt = orc.branch_pacer(o_cum, o_len, m)
+            np.testing.assert_allclose(f, o_f, rtol=1e-12, atol=1e-12)
+            if np.sort(o_f)[-1] - (np.sort(o_f)[-2] if len(o_f) > 1 else -np.inf) > 1e-9:
+                assert nxt == o_nxt                       # a unique maximum must be found by both
+            else:
+                assert abs(f[nxt] - o_f.max()) <= 1e-9
+    for bad in [([0, 0], [1.0, 0.5]), ([-1, 1], [1.0, 0.5]), ([-1, 0], [1.0, 0.0]), ([-1, 0], [1.0, 1.5]), ([-1] * 129, [0.5] * 129)]:
+        with pytest.raises(B.LlmcadError):
+            B.tree_branches(*bad)
+    for bad in [([0.5, 0.0], [1, 1], 2), ([0.5, 0.5], [1, -1], 2), ([0.5, 0.5], [1, 1], -1.0)]:
+        with pytest.raises(B.LlmcadError):
+            B.branch_pacer(*bad)
