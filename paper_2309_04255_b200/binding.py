@@ -21,7 +21,7 @@ MAX_TREE = 128
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CUDA = 0, -1, -2, -3, -4
 ERR_BAD_TREE, ERR_BAD_TOKEN, ERR_TIMEOUT, ERR_NAN = 1, 2, 3, 4
 F32, BF16 = 0, 1
-FLAG_SIMT_GEMM, FLAG_SIMT_ATTN = 1, 2
+FLAG_SIMT_GEMM, FLAG_SIMT_ATTN, FLAG_T5_ATTN, FLAG_MMA_ATTN = 1, 2, 4, 8
 S_ACCEPTED_LEN, S_NEXT_TOKEN, S_NEW_PREFIX_LEN, S_N_CORRECT, S_N_ALL, S_RECTIFIED, S_STATUS = range(7)
 
 EXPORTS = [

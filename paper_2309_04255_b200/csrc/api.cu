@@ -275,6 +275,14 @@ int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, 
     TimedLaunch tl(ctx, 1, st);
     if (ctx->tc_attn) {
         int launched = 0;
+        const bool t5 = (c.flags & LLMCAD_FLAG_T5_ATTN) ? true
+                        : (c.flags & LLMCAD_FLAG_MMA_ATTN) ? false : attention_prefers_t5(n);
+        if (t5) {
+            CUDA_TRY(launch_attention_t5(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->n_sms, status, st,
+                                         &launched, ctx->next_trace(), comp ? 1 : 0, ctx->kv_lo, n_tree, q_first));
+            ctx->launches += launched;
+            return LLMCAD_OK;
+        }
         CUDA_TRY(launch_attention_tc(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->attn_ws,
                                      ctx->attn_counters, ctx->n_sms, status, st, &launched, ctx->next_trace(), comp ? 1 : 0,
                                      ctx->kv_lo, n_tree, q_first));

@@ -18,4 +18,15 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
                                 int32_t *status, cudaStream_t st, int *launched, unsigned long long *trace = nullptr, int comp = 0,
                                 const void *kv_lo = nullptr, int n_tree = 0, int q_first = 0);
 
+// The same operation on the tcgen05 tensor cores (attention_t5.cu), for larger trees; arguments as above.
+cudaError_t launch_attention_t5(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
+                                int n, const uint32_t *anc, void *o, int n_sms, int32_t *status, cudaStream_t st,
+                                int *launched, unsigned long long *trace = nullptr, int comp = 0, const void *kv_lo = nullptr,
+                                int n_tree = 0, int q_first = 0);
+
+// Which of the two serves a tree of n query rows by default: the tcgen05 kernel above 64 rows (measured on
+// B200 in whole passes: 3-8 % of the pass faster at 96 and 128 nodes, level at 48-64, clearly slower at 32
+// and below). LLMCAD_ATTN_T5_MIN_N moves the switch (tuning aid, read once; 0 = never).
+bool attention_prefers_t5(int n);
+
 }  // namespace llmcad

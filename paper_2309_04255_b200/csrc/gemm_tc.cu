@@ -1022,6 +1022,21 @@ bool make_act_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64
     return r == CUDA_SUCCESS;
 }
 
+bool make_tensor_map_bf16_3d(CUtensorMap *map, const void *base, const uint64_t dims[3], const uint64_t strides_bytes[2],
+                             const uint32_t box[3])
+{
+    auto fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t d[3] = {dims[0], dims[1], dims[2]};
+    cuuint64_t s[2] = {strides_bytes[0], strides_bytes[1]};
+    cuuint32_t b[3] = {box[0], box[1], box[2]};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), d, s, b, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 size_t gemm_tc_partial_floats(int n_sms, int max_n_pad) { return (size_t)n_sms * 2 /*slots*/ * 2 /*gate|up*/ * max_n_pad * kTileM; }
 
 GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)

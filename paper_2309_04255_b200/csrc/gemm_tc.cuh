@@ -56,6 +56,10 @@ bool make_tensor_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uin
 // of an activation k-block, one after the other, into shared memory. Rows beyond `rows` read as zero.
 bool make_act_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t planes,
                        uint64_t plane_rows);
+// Any three-dimensional bf16 tensor with 128-byte swizzle and zero fill outside its bounds: dims and box
+// innermost first, strides (bytes) of dimensions 1 and 2.
+bool make_tensor_map_bf16_3d(CUtensorMap *map, const void *base, const uint64_t dims[3], const uint64_t strides_bytes[2],
+                             const uint32_t box[3]);
 
 size_t gemm_tc_partial_floats(int n_sms, int max_n_pad);
 constexpr size_t kArrivalsPerGemm = 4096 * 4;

@@ -77,8 +77,13 @@ extern "C" int llmcad_tree_attention_noalloc(const void *q, const void *k, const
     if (e == cudaSuccess) {
         int sms = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess)
-            e = launch_attention_tc(q, k, v, n_heads, 128, kv_stride, prefix_len, n, tb.anc, o, nullptr, nullptr, sms, status, st, nullptr);
+        if (e == cudaSuccess) {
+            // neither kernel needs global scratch; same choice as the regular entry point
+            if (attention_prefers_t5(n))
+                e = launch_attention_t5(q, k, v, n_heads, 128, kv_stride, prefix_len, n, tb.anc, o, sms, status, st, nullptr);
+            else
+                e = launch_attention_tc(q, k, v, n_heads, 128, kv_stride, prefix_len, n, tb.anc, o, nullptr, nullptr, sms, status, st, nullptr);
+        }
     }
     if (e == cudaSuccess && status_out != nullptr)
         e = cudaMemcpyAsync(status_out, status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st);

@@ -259,11 +259,13 @@ print("ok")
 
 
 @pytest.mark.parametrize("env", [{"LLMCAD_CHAIN_MAX": "4"}, {"LLMCAD_CHAIN_MAX": "2", "LLMCAD_PDL": "0"}, {"LLMCAD_COMP": "0"},
-                                 {"LLMCAD_GEMM_PAIR_K": "1"}, {"LLMCAD_GEMM_STAGES": "2", "LLMCAD_GEMM_L2_AHEAD": "0"}])
+                                 {"LLMCAD_GEMM_PAIR_K": "1"}, {"LLMCAD_GEMM_STAGES": "2", "LLMCAD_GEMM_L2_AHEAD": "0"},
+                                 {"LLMCAD_ATTN_T5_MIN_N": "1"}, {"LLMCAD_ATTN_T5_MIN_N": "0"}])
 def test_tuning_paths_stay_correct(env):
     """The environment knobs select other code paths of the same kernels (several dependent GEMMs per
     launch with grid barriers, no programmatic dependent launch, plain bf16 activations, ring items
-    of one k-block, a two-stage ring): each must still match the oracle. The knobs are read once per
+    of one k-block, a two-stage ring, the tcgen05 attention kernel for every tree size, the mma.sync
+    attention kernel for every tree size): each must still match the oracle. The knobs are read once per
     process, hence the child process."""
     import os, subprocess, sys
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))

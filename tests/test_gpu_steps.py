@@ -160,17 +160,19 @@ def test_skinny_gemm(shape, mode):
 
 # ----------------------------------------------------------------------------- tree attention
 
-ATTN_CASES = [(0, 1), (0, 15), (5, 8), (64, 33), (300, 32), (1024, 64), (257, 128), (2048, 17)]
+ATTN_CASES = [(0, 1), (0, 15), (5, 8), (64, 33), (300, 32), (1024, 64), (257, 128), (2048, 17), (1000, 97), (4095, 128)]
 
 
 @pytest.mark.parametrize("case", ATTN_CASES)
-@pytest.mark.parametrize("mode", ["f32", "bf16_simt", "bf16_tc"])
+@pytest.mark.parametrize("mode", ["f32", "bf16_simt", "bf16_mma", "bf16_t5"])
 def test_tree_attention(case, mode):
+    """Every attention kernel family on every shape: plain ALU (fp32, bf16), mma.sync and tcgen05."""
     P, n = case
     H, hd = 4, 128
     dtype = "f32" if mode == "f32" else "bf16"
     cfg = gen.ModelConfig("a", 0, H * hd, H, hd, 256, 512, dtype)
-    v = B.Verifier(cfg, 16, flags=B.FLAG_SIMT_ATTN if mode == "bf16_simt" else 0)
+    flags = {"f32": 0, "bf16_simt": B.FLAG_SIMT_ATTN, "bf16_mma": B.FLAG_MMA_ATTN, "bf16_t5": B.FLAG_T5_ATTN}[mode]
+    v = B.Verifier(cfg, 16, flags=flags)
     if n == 1:
         parent = np.array([-1], np.int32)
     elif n == 15:
