@@ -36,7 +36,7 @@ namespace {
 constexpr int kHd = 128;
 constexpr int kKeyTile = 64;
 constexpr int kT5Threads = 192;
-constexpr int kStages = 6;                       // >= 4: two tiles in flight, each with a remainder stage
+constexpr int kStages = 6;                       // three tiles in flight, each possibly with a remainder stage
 constexpr int kSubTile = 64 * 64 * 2;            // [64 rows][64 columns] bf16, 128-byte rows
 constexpr int kStageBytes = 4 * kSubTile;        // K dims 0-63, K dims 64-127, V dims 0-63, V dims 64-127
 constexpr int kWsRow = kHd + 4;                  // partial row: 128 outputs, reference, sum, padding to 16 bytes
@@ -56,7 +56,6 @@ struct Ctl {
     uint64_t empty[kStages];
     uint64_t q_full;
     uint64_t s_full[2];
-    uint64_t s_empty[2];
     uint64_t p_full[2];
     uint64_t o_full[2];
     uint32_t tmem_base;
@@ -271,7 +270,6 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
         mbar_init(smem_u32(&ctl.q_full), 4);
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.s_full[b]), 1);
-            mbar_init(smem_u32(&ctl.s_empty[b]), 4);
             mbar_init(smem_u32(&ctl.p_full[b]), 4);
             mbar_init(smem_u32(&ctl.o_full[b]), 1);
         }
@@ -343,26 +341,26 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
             constexpr uint32_t idesc_o = make_idesc(128, kHd, true);
             int s = 0;
             uint32_t ph = 0;
-            int st_kv[2] = {0, 0}, st_lo[2] = {-1, -1};   // ring stages of the tiles in flight (by tile parity)
+            int st_kv[4] = {0, 0, 0, 0}, st_lo[4] = {-1, -1, -1, -1};   // ring stages of the (up to three) tiles in flight, by tile & 3
             auto issue_s = [&](int i) -> bool {             // S of tile t_begin + i into score buffer i & 1
                 const int t = t_begin + i, b = i & 1;
                 const bool lo = comp && reaches_tree(t);
-                st_kv[b] = s;
+                st_kv[i & 3] = s;
                 if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) return false;
                 if (++s == kStages) { s = 0; ph ^= 1u; }
-                st_lo[b] = -1;
+                st_lo[i & 3] = -1;
                 if (lo) {
-                    st_lo[b] = s;
+                    st_lo[i & 3] = s;
                     if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) return false;
                     if (++s == kStages) { s = 0; ph ^= 1u; }
                 }
-                // the softmax warps must have read tile i - 2 out of this buffer
-                if (i >= 2 && !mbar_wait(smem_u32(&ctl.s_empty[b]), (uint32_t)((i >> 1) - 1) & 1u, abort_flag)) return false;
+                // (the softmax warps have read tile i - 2 out of this score buffer: their P of that tile, which
+                // the caller has waited for, came after it)
                 tc_fence_after();
                 // One thread issues every MMA, so the code between two of them is what limits the rate:
                 // descriptors are a base plus compile-time offsets (address field in units of 16 bytes).
                 const uint32_t d = tmem_base + (uint32_t)b * kKeyTile;
-                const uint64_t dk = desc_k_major(s_ring + st_kv[b] * kStageBytes);
+                const uint64_t dk = desc_k_major(s_ring + st_kv[i & 3] * kStageBytes);
                 // k-step ks = 16 head dims: 8 columns of the queries in tensor memory, 32 bytes in a row of
                 // the K sub-tile that holds dims 64 * (ks / 4) ..
 #pragma unroll
@@ -374,7 +372,7 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
                         tc_mma_ts(d, tmem_base + kColQ + 64 + 8 * ks, dk + (uint64_t)(((ks >> 2) * kSubTile >> 4) + 2 * (ks & 3)), idesc_s, 1u);
                 }
                 if (lo) {
-                    const uint64_t dl = desc_k_major(s_ring + st_lo[b] * kStageBytes);
+                    const uint64_t dl = desc_k_major(s_ring + st_lo[i & 3] * kStageBytes);
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
                         tc_mma_ts(d, tmem_base + kColQ + 8 * ks, dl + (uint64_t)(((ks >> 2) * kSubTile >> 4) + 2 * (ks & 3)), idesc_s, 1u);
@@ -383,18 +381,20 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
                 return true;
             };
             if (!mbar_wait(smem_u32(&ctl.q_full), 0, abort_flag)) failed = true;
+            // An idle tensor pipe takes a few hundred cycles to get going again, so the MMAs go out in long
+            // runs: after a two-tile prologue, the scores of tile i + 2 and the P V of tile i back to back
+            // once the weights of tile i have arrived, while the softmax warps work on tile i + 1.
             if (!failed && !issue_s(0)) failed = true;
+            if (!failed && T > 1 && !issue_s(1)) failed = true;
             for (int i = 0; i < T && !failed; ++i) {
-                // The scores of the next tile go out before this tile's P V so that the softmax warps never wait
-                // for them (two tiles hold at most four of the six ring stages).
-                if (i + 1 < T && !issue_s(i + 1)) { failed = true; break; }
                 if (!mbar_wait(smem_u32(&ctl.p_full[i & 1]), (uint32_t)(i >> 1) & 1u, abort_flag)) { failed = true; break; }
+                if (i + 2 < T && !issue_s(i + 2)) { failed = true; break; }
                 tc_fence_after();
                 const int b = i & 1;
                 const uint32_t d = tmem_base + kColO;
                 // 16 keys further: 8 columns of P in tensor memory, 16 rows (2048 bytes) in V
                 const uint32_t tp = tmem_base + kColP + 64 * (uint32_t)b;
-                const uint64_t dv = desc_mn_major(s_ring + st_kv[b] * kStageBytes + 2 * kSubTile, kSubTile);
+                const uint64_t dv = desc_mn_major(s_ring + st_kv[i & 3] * kStageBytes + 2 * kSubTile, kSubTile);
                 if (i > 0) {                              // the outputs accumulate in TMEM over the tiles
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) tc_mma_ts(d, tp + 8 * ks, dv + (uint64_t)(ks * 2048 >> 4), idesc_o, 1u);
@@ -406,14 +406,14 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) tc_mma_ts(d, tp + 32 + 8 * ks, dv + (uint64_t)(ks * 2048 >> 4), idesc_o, 1u);
                 }
-                if (st_lo[b] >= 0) {
-                    const uint64_t dvl = desc_mn_major(s_ring + st_lo[b] * kStageBytes + 2 * kSubTile, kSubTile);
+                if (st_lo[i & 3] >= 0) {
+                    const uint64_t dvl = desc_mn_major(s_ring + st_lo[i & 3] * kStageBytes + 2 * kSubTile, kSubTile);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) tc_mma_ts(d, tp + 8 * ks, dvl + (uint64_t)(ks * 2048 >> 4), idesc_o, 1u);
                 }
                 tc_commit(smem_u32(&ctl.o_full[b]));
-                tc_commit(smem_u32(&ctl.empty[st_kv[b]]));
-                if (st_lo[b] >= 0) tc_commit(smem_u32(&ctl.empty[st_lo[b]]));
+                tc_commit(smem_u32(&ctl.empty[st_kv[i & 3]]));
+                if (st_lo[i & 3] >= 0) tc_commit(smem_u32(&ctl.empty[st_lo[i & 3]]));
             }
         }
     } else {
@@ -467,9 +467,6 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
             if (trace && tid == 64 && cta < 256 && i == 0) trace[(size_t)cta * 16 + 2] = global_timer_ns();
             float sc[kKeyTile];
             if (warp_active) tc_ld64(tlane + (uint32_t)b * kKeyTile, sc);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl.s_empty[b]));
             // Visibility of the tile's 64 keys for this row, one bit each: prefix keys always, tree keys by
             // the row's ancestor-or-self bits (bits of nodes that do not exist are never set).
             float tmax = -INFINITY;
