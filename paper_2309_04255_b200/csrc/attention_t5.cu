@@ -227,6 +227,65 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
+// Merge of the splits of a head for the rows split, split + splits, ... of this CTA: out = sum_s O_s
+// 2^(m_s - M) / sum_s l_s 2^(m_s - M), from the partials ([128 outputs][reference][sum] per row) in the
+// shared memory of the NS (or fewer) CTAs of the cluster. Remote shared memory answers slowly and the
+// compiler will not move loads across the stores of an earlier item, so every thread first collects
+// the operands of B items (four outputs of one row each) and only then computes and stores.
+template <int NS, int B>
+__device__ __forceinline__ void merge_splits(const float *part, cg::cluster_group &cluster, int splits, int split, int n,
+                                             int n_heads, int head, __nv_bfloat16 *o, size_t lo_off, int comp, int tid)
+{
+    const float *peer[NS];
+#pragma unroll
+    for (int sp = 0; sp < NS; ++sp) peer[sp] = sp < splits ? cluster.map_shared_rank(part, sp) : part;
+    const int my_rows = (n - split + splits - 1) / splits;
+    const int items = my_rows * (kHd / 4);
+    for (int base = tid; base < items; base += B * kT5Threads) {
+        float2 ml[B][NS];
+        float4 ov[B][NS];
+#pragma unroll
+        for (int b = 0; b < B; ++b) {
+            const int idx = min(base + b * kT5Threads, items - 1);      // a clamped item is loaded twice and stored once
+            const int row = split + (idx / (kHd / 4)) * splits, dim = (idx % (kHd / 4)) * 4;
+#pragma unroll
+            for (int sp = 0; sp < NS; ++sp) {
+                if (sp < splits) {
+                    ml[b][sp] = *reinterpret_cast<const float2 *>(peer[sp] + (size_t)row * kWsRow + kHd);
+                    ov[b][sp] = *reinterpret_cast<const float4 *>(peer[sp] + (size_t)row * kWsRow + dim);
+                } else {
+                    ml[b][sp] = make_float2(-INFINITY, 0.f);
+                    ov[b][sp] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < B; ++b) {
+            const int idx = base + b * kT5Threads;
+            if (idx >= items) break;
+            const int row = split + (idx / (kHd / 4)) * splits, dim = (idx % (kHd / 4)) * 4;
+            float M = -INFINITY;
+#pragma unroll
+            for (int sp = 0; sp < NS; ++sp) M = fmaxf(M, ml[b][sp].x);
+            float L = 0.f;
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int sp = 0; sp < NS; ++sp) {
+                const float wgt = (ml[b][sp].x == -INFINITY) ? 0.f : ex2(ml[b][sp].x - M);
+                L += ml[b][sp].y * wgt;
+                a.x += ov[b][sp].x * wgt; a.y += ov[b][sp].y * wgt; a.z += ov[b][sp].z * wgt; a.w += ov[b][sp].w * wgt;
+            }
+            const float inv = L > 0.f ? 1.f / L : 0.f;
+            uint32_t h0, l0, h1, l1;
+            pack_split(a.x * inv, a.y * inv, h0, l0);
+            pack_split(a.z * inv, a.w * inv, h1, l1);
+            __nv_bfloat16 *dst = o + ((size_t)row * n_heads + head) * kHd + dim;
+            *reinterpret_cast<uint2 *>(dst) = make_uint2(h0, h1);
+            if (comp) *reinterpret_cast<uint2 *>(dst + lo_off) = make_uint2(l0, l1);
+        }
+    }
+}
+
 }  // namespace
 
 // q: [planes][rows][H*128] (the lo plane kLoRows rows after the hi plane);
@@ -598,41 +657,10 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
     cg::cluster_group cluster = cg::this_cluster();
     cluster.sync();                                          // all partials of this head are written
     if (trace && tid == 0 && cta < 256) trace[(size_t)cta * 16 + 5] = global_timer_ns();
-    // merge rows split, split + splits, ...: out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M)
     if (!bad) {
-        const float *peer[kMaxSplits];
-#pragma unroll
-        for (int sp = 0; sp < kMaxSplits; ++sp) peer[sp] = sp < splits ? cluster.map_shared_rank(part, sp) : part;
-        const int my_rows = (n - split + splits - 1) / splits;   // rows split, split+splits, ... below n
-        // remote shared memory answers slowly: several independent items per thread in flight
-#pragma unroll 4
-        for (int idx = tid; idx < my_rows * (kHd / 4); idx += kT5Threads) {
-            const int row = split + (idx / (kHd / 4)) * splits, dim = (idx % (kHd / 4)) * 4;
-            float2 ml[kMaxSplits];
-            float4 ov[kMaxSplits];
-#pragma unroll
-            for (int sp = 0; sp < kMaxSplits; ++sp) {
-                if (sp < splits) {
-                    ml[sp] = *reinterpret_cast<const float2 *>(peer[sp] + (size_t)row * kWsRow + kHd);
-                    ov[sp] = *reinterpret_cast<const float4 *>(peer[sp] + (size_t)row * kWsRow + dim);
-                } else {
-                    ml[sp] = make_float2(-INFINITY, 0.f);
-                    ov[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            }
-            float M = -INFINITY;
-#pragma unroll
-            for (int sp = 0; sp < kMaxSplits; ++sp) M = fmaxf(M, ml[sp].x);
-            float L = 0.f;
-            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int sp = 0; sp < kMaxSplits; ++sp) {
-                const float wgt = (ml[sp].x == -INFINITY) ? 0.f : ex2(ml[sp].x - M);
-                L += ml[sp].y * wgt;
-                a.x += ov[sp].x * wgt; a.y += ov[sp].y * wgt; a.z += ov[sp].z * wgt; a.w += ov[sp].w * wgt;
-            }
-            store4(row, dim, a, L > 0.f ? 1.f / L : 0.f);
-        }
+        if (splits <= 2) merge_splits<2, 4>(part, cluster, splits, split, n, n_heads, head, o, lo_off, comp, tid);
+        else if (splits <= 4) merge_splits<4, 2>(part, cluster, splits, split, n, n_heads, head, o, lo_off, comp, tid);
+        else merge_splits<kMaxSplits, 1>(part, cluster, splits, split, n, n_heads, head, o, lo_off, comp, tid);
     }
     if (trace && tid == 0 && cta < 256) trace[(size_t)cta * 16 + 6] = global_timer_ns();
     cluster.sync();                                          // peers may still be reading this CTA's partial
