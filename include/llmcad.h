@@ -68,7 +68,7 @@ enum { LLMCAD_F32 = 0, LLMCAD_BF16 = 1 };
 enum {
     LLMCAD_FLAG_SIMT_GEMM = 1, /* use the plain-ALU GEMM even for bf16 (debugging aid) */
     LLMCAD_FLAG_SIMT_ATTN = 2, /* use the plain-ALU attention even for bf16 (debugging aid) */
-    LLMCAD_FLAG_T5_ATTN = 4,   /* bf16, head_dim 128: tcgen05 attention kernel for every tree size (default: above 64 nodes) */
+    LLMCAD_FLAG_T5_ATTN = 4,   /* bf16, head_dim 128: tcgen05 attention kernel for every tree size (default: above 32 nodes) */
     LLMCAD_FLAG_MMA_ATTN = 8   /* bf16, head_dim 128: mma.sync attention kernel for every tree size */
 };
 

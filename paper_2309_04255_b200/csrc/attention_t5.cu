@@ -669,7 +669,7 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
 
 bool attention_prefers_t5(int n)
 {
-    static const int min_n = [] { const char *e = getenv("LLMCAD_ATTN_T5_MIN_N"); return e ? atoi(e) : 65; }();
+    static const int min_n = [] { const char *e = getenv("LLMCAD_ATTN_T5_MIN_N"); return e ? atoi(e) : 33; }();
     return min_n > 0 && n >= min_n;
 }
 

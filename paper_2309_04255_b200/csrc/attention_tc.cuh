@@ -24,9 +24,10 @@ cudaError_t launch_attention_t5(const void *q, const void *k, const void *v, int
                                 int *launched, unsigned long long *trace = nullptr, int comp = 0, const void *kv_lo = nullptr,
                                 int n_tree = 0, int q_first = 0);
 
-// Which of the two serves a tree of n query rows by default: the tcgen05 kernel above 64 rows (measured on
-// B200 in whole passes: 3-8 % of the pass faster at 96 and 128 nodes, level at 48-64, clearly slower at 32
-// and below). LLMCAD_ATTN_T5_MIN_N moves the switch (tuning aid, read once; 0 = never).
+// Which of the two serves a tree of n query rows by default: the tcgen05 kernel above 32 rows (measured on
+// B200 in whole passes of the 7B shape: 1-3 % of the pass faster at 33-64 nodes, 4-8 % at 96-128; at 32 nodes
+// and below, where only one of its four softmax warps has rows to work on, 1-2 % slower).
+// LLMCAD_ATTN_T5_MIN_N moves the switch (tuning aid, read once; 0 = never).
 bool attention_prefers_t5(int n);
 
 }  // namespace llmcad
