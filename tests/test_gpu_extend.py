@@ -80,6 +80,24 @@ def test_extension_bf16_full_width(cuts):
     check_topk(ids, pr, ref.logits, BF16_TOL * np.abs(ref.logits).max())
 
 
+@pytest.mark.parametrize("flags,n,cuts", [(B.FLAG_T5_ATTN, 32, [3, 4, 20, 31, 32]), (B.FLAG_MMA_ATTN, 32, [3, 4, 20, 31, 32]),
+                                          (0, 96, [40, 41, 96])])
+def test_extension_through_both_attention_kernels(flags, n, cuts):
+    """The same at 7B widths with each tensor-core attention kernel pinned (a query block that starts
+    inside the tree, remainders only for the new nodes), and a 96-node tree grown by 40, 1 and 55 nodes,
+    which the default choice sends to the tcgen05, the mma.sync and again the tcgen05 kernel."""
+    cfg = gen.shrink(gen.MODELS["7b"], 2)
+    P = 300
+    tw = Twin(cfg, P + n + 8, flags=flags)
+    tw.fill_prefix_synthetic(P)
+    parent = gen.tree_random(n, 12, "uniform4", n)
+    tokens = gen.gen_tokens(cfg, n)
+    ref = tw.oracle_pass(P, tokens, parent)
+    lg, ids, pr = grow(tw, P, tokens, parent, cuts, 4)
+    logits_close(lg, ref.logits, BF16_TOL)
+    check_topk(ids, pr, ref.logits, BF16_TOL * np.abs(ref.logits).max())
+
+
 def test_extension_argument_checks():
     cfg = gen.MODELS["tiny"]
     v = B.Verifier(cfg, 64)
