@@ -62,7 +62,8 @@ struct Ctl {
     volatile int abort_flag;
 };
 
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(Ctl);
+constexpr int kQStage = 32 * 256;                   // per softmax warp: 32 query rows of one plane on their way to TMEM
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 4 * kQStage + sizeof(Ctl);
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -306,7 +307,8 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
     const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled tiles want 1024-byte alignment
     uint8_t *smp = sm_raw + (base - raw);
     const uint32_t s_ring = base;
-    Ctl &ctl = *reinterpret_cast<Ctl *>(smp + (size_t)kStages * kStageBytes);
+    uint8_t *q_stage = smp + (size_t)kStages * kStageBytes;
+    Ctl &ctl = *reinterpret_cast<Ctl *>(q_stage + 4 * kQStage);
     float *part = reinterpret_cast<float *>(smp);   // the ring's space, once the loop is over
 
     const int split = blockIdx.x, head = blockIdx.y;
@@ -488,22 +490,47 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
 #pragma unroll
             for (int w = 0; w < 4; ++w) a4[w] = anc[(q_first + row) * 4 + w];
         }
-        // This row of the queries goes from global memory straight into tensor memory as the A operand of
-        // Q K^T: 64 packed columns per plane. Rows beyond n stay as they are: a row of A only ever
-        // influences the same row of the product, and nobody reads those rows of the result.
+        // The queries become the A operand of Q K^T in tensor memory: 64 packed columns per plane, thread =
+        // row. A warp fetches its 32 rows with coalesced loads (two rows of 256 bytes per instruction, both
+        // planes in flight together), turns them through a small shared-memory buffer (16-byte chunks
+        // XOR-swizzled by row) and every thread stores its own row. Rows beyond n repeat row n - 1: a row
+        // of A only ever influences the same row of the product, and nobody reads those rows of the result.
         if (warp_active) {
+            const int planes = comp ? 2 : 1;
+            uint4 g[2][16];
 #pragma unroll
             for (int pl = 0; pl < 2; ++pl) {
-                if (pl == 1 && !comp) break;
-                uint32_t qr[64];
-                const uint4 *src = reinterpret_cast<const uint4 *>(q + (size_t)pl * lo_off + ((size_t)min(row, n - 1) * n_heads + head) * kHd);
+                if (pl < planes) {
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const uint4 v4 = __ldg(src + c);
-                    qr[4 * c] = v4.x; qr[4 * c + 1] = v4.y; qr[4 * c + 2] = v4.z; qr[4 * c + 3] = v4.w;
+                    for (int it = 0; it < 16; ++it) {
+                        const int rr = it * 2 + (lane >> 4);
+                        const int qrow = min(lg * 32 + rr, n - 1);
+                        g[pl][it] = __ldg(reinterpret_cast<const uint4 *>(q + (size_t)pl * lo_off + ((size_t)qrow * n_heads + head) * kHd) + (lane & 15));
+                    }
                 }
-                tc_st32(tlane + kColQ + 64 * pl, qr);
-                tc_st32(tlane + kColQ + 64 * pl + 32, qr + 32);
+            }
+            const uint32_t stg = smem_u32(q_stage + (size_t)lg * kQStage);
+#pragma unroll
+            for (int pl = 0; pl < 2; ++pl) {
+                if (pl < planes) {
+#pragma unroll
+                    for (int it = 0; it < 16; ++it) {
+                        const int rr = it * 2 + (lane >> 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + rr * 256 + (((lane & 15) ^ (rr & 15)) << 4)),
+                                     "r"(g[pl][it].x), "r"(g[pl][it].y), "r"(g[pl][it].z), "r"(g[pl][it].w) : "memory");
+                    }
+                    __syncwarp();
+                    uint32_t qr[64];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(qr[4 * c]), "=r"(qr[4 * c + 1]), "=r"(qr[4 * c + 2]), "=r"(qr[4 * c + 3])
+                                     : "r"(stg + lane * 256 + ((c ^ (lane & 15)) << 4)) : "memory");
+                    }
+                    __syncwarp();                         // the buffer is reused for the lo plane
+                    tc_st32(tlane + kColQ + 64 * pl, qr);
+                    tc_st32(tlane + kColQ + 64 * pl + 32, qr + 32);
+                }
             }
             tc_wait_st();
         }
