@@ -179,6 +179,23 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float *v)
     for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
 }
 
+// 32 consecutive fp32 columns of this thread's TMEM lane at each of two addresses, summed. A load plus
+// its wait costs ~0.15 us whatever the width, so the two loads share one wait; everything sits in one
+// statement so that no register of the result can be touched before the wait.
+__device__ __forceinline__ void tc_ld32_sum2(uint32_t taddr_a, uint32_t taddr_b, float *v)
+{
+    uint32_t a[32], b[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%64];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%65];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]), "=r"(a[4]), "=r"(a[5]), "=r"(a[6]), "=r"(a[7]), "=r"(a[8]), "=r"(a[9]), "=r"(a[10]), "=r"(a[11]), "=r"(a[12]), "=r"(a[13]), "=r"(a[14]), "=r"(a[15]), "=r"(a[16]), "=r"(a[17]), "=r"(a[18]), "=r"(a[19]), "=r"(a[20]), "=r"(a[21]), "=r"(a[22]), "=r"(a[23]), "=r"(a[24]), "=r"(a[25]), "=r"(a[26]), "=r"(a[27]), "=r"(a[28]), "=r"(a[29]), "=r"(a[30]), "=r"(a[31]), "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]), "=r"(b[4]), "=r"(b[5]), "=r"(b[6]), "=r"(b[7]), "=r"(b[8]), "=r"(b[9]), "=r"(b[10]), "=r"(b[11]), "=r"(b[12]), "=r"(b[13]), "=r"(b[14]), "=r"(b[15]), "=r"(b[16]), "=r"(b[17]), "=r"(b[18]), "=r"(b[19]), "=r"(b[20]), "=r"(b[21]), "=r"(b[22]), "=r"(b[23]), "=r"(b[24]), "=r"(b[25]), "=r"(b[26]), "=r"(b[27]), "=r"(b[28]), "=r"(b[29]), "=r"(b[30]), "=r"(b[31])
+        : "r"(taddr_a), "r"(taddr_b)
+        : "memory");
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(a[j]) + __uint_as_float(b[j]);
+}
+
 // Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
 // 1024 bytes apart (the layout a TMA box of 64 bf16 x rows with CU_TENSOR_MAP_SWIZZLE_128B
 // produces). Fields: start address >> 4 [0,14), leading byte offset >> 4 [16,30) (unused for
@@ -827,7 +844,17 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 float *dst = p.partials + ((size_t)blockIdx.x * 2 + (seg_begin == r.begin ? 0 : 1)) * part_stride +
                              (size_t)lane_grp * 2 * p.n_pad * 32 + lane;
                 for (int hf = 0; hf < (dual ? 2 : 1); ++hf) {
-                    for (int c0 = 0; c0 < p.n_pad; c0 += 16) {
+                    int c0 = 0;
+                    if (p.comp) {
+                        // 32 nodes at a time, hi and lo columns in one round trip
+                        for (; c0 + 32 <= p.n_pad; c0 += 32) {
+                            float v[32];
+                            tc_ld32_sum2(t_lane + hf * nb + c0, t_lane + hf * nb + p.n_pad + c0, v);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) dst[(size_t)(hf * p.n_pad + c0 + j) * 32] = v[j];
+                        }
+                    }
+                    for (; c0 < p.n_pad; c0 += 16) {
                         float v[16];
                         tc_ld16(t_lane + hf * nb + c0, v);
                         if (p.comp) {
