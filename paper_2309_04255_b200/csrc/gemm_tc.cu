@@ -778,8 +778,12 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             }
             // ---- RMSNorm of the GEMM input folded into the epilogue: the producer of the residual
             // stream left partial sums of squares per node; every warp keeps its own copy of the
-            // per-node factors (no block-level barrier among the epilogue warps)
-            if (ep.ssq_in != nullptr) {
+            // per-node factors (no block-level barrier among the epilogue warps). The factors are
+            // needed for finishing only, and adding up the partial rows takes tens of microseconds
+            // with many nodes: where the MMA warp has one accumulator buffer only, it happens after
+            // this warp's first share has left TMEM, so that the MMA warp is not kept waiting for it.
+            bool rs_ready = ep.ssq_in == nullptr;
+            auto compute_rs = [&]() {
                 // rows of ssq_in hold 128 floats (one per node); read them as float4 "quads". A lane
                 // owns one quad and every (32 / quads)-th partial row, eight loads in flight at a time;
                 // the lane groups are then added in a fixed order, so the sum does not depend on timing.
@@ -814,7 +818,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     my_rs[4 * quad + 3] = rsqrtf(acc.w * inv_d + ep.eps);
                 }
                 __syncwarp();
-            }
+            };
             const Range r = cta_range<PK>(d);
             const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
             const bool dual = d.halves == 2;
@@ -830,6 +834,12 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 const int last_cta = (tile_i0 + ipt - 1) / d.items_per_cta;
                 const int n_parts = last_cta - first_cta + 1;           // CTAs that hold a share of this tile
                 const bool tail = p.n_gemms == 1 && seg_end == r.end;   // (tracing) the segment that ends this CTA's work
+                // the norm factors: at once, unless the MMA warp has a single accumulator buffer and this first
+                // segment only leaves a share (then after that share has left TMEM, i.e. before the second segment)
+                if (!rs_ready && (two_bufs || n_parts == 1 || seg_end == r.end || seg_begin != r.begin)) {
+                    compute_rs();
+                    rs_ready = true;
+                }
 
                 if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), use & 1u, abort_flag, lane)) { timed_out = true; break; }
                 tc_fence_after();
