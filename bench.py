@@ -7,15 +7,27 @@ forward over all tree nodes, argmax, verified-path search, cache rollback).
 Prints ONE JSON line. The path does not shard (one GPU per model replica, no collective): with
 --gpus N > 1, launched under torchrun, every rank runs an independent replica of the same
 workload and the value is the replicas' total.
+
+What the line holds (GPU arm):
+  value / ms_per_step     median of the K per-step times (CUDA events between the steps, no host
+                          synchronisation inside the timed region), max over ranks; min, max and mean beside it
+  roofline                the dominant kernel (the weight-streaming GEMM) INSIDE an undisturbed pass: a second
+                          region of K passes records %globaltimer stamps per launch (llmcad_set_gemm_trace);
+                          a launch is charged the time from the end of its predecessor to its own end, so the
+                          kernels' times add up to the pass; `isolated` is the same kernel bracketed by events
+                          (which switches off the overlap of consecutive launches)
+  e2e                     the same pass through the host-buffer entry point, logits included
+  workloads               the 13B configuration (C3) timed in the same process, and a digest of the
+                          attention-only sweep (C4); only with the default workload on one GPU
+  cpu_baseline            the CPU oracle, as it stands, on this machine's host cores
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
-import subprocess
 import sys
-import tempfile
+import threading
 import time
 
 import numpy as np
@@ -28,9 +40,10 @@ from paper_2309_04255_b200 import inputs as gen  # noqa: E402
 
 METRIC = "tree_verification_passes_per_sec"
 UNIT = "passes/s"
-# ncu capture of gemm_chain_kernel (profiles/gemm_chain_kernel__7b_qkv_n32.md): DRAM bytes per launch relative to the launch's
-# algorithmic bytes; None until a capture exists for the workload.
-GEMM_TRAFFIC_RATIO = 1.02
+# DRAM traffic of one gemm_chain_kernel launch from the ncu capture named here (dram__bytes_read.sum +
+# dram__bytes_write.sum) next to the launch's algorithmic bytes; the kernel's traffic is the weight stream,
+# which grows in proportion to the bytes, so other launches are scaled by the ratio.
+NCU_GEMM_CAPTURE = {"summary": "profiles/gemm_chain_kernel__7b_qkv_n32.md", "dram_bytes": 104.80e6, "algorithmic_bytes": 102.5e6}
 
 
 def algorithmic_bytes(cfg, P, n):
@@ -64,43 +77,60 @@ def flops(cfg, P, n):
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples during the timed region."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """SM clock, power and throttle reasons read through NVML every few milliseconds by a thread of this
+    process (reading only; nothing is set). `mark()` opens and closes named windows, so that the samples
+    taken during the timed region can be told from the rest."""
+    REASONS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
 
-    def __init__(self, index: int):
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.samples, self.windows, self.period = [], {}, period_s
+        self.h = None
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
-                                      stderr=subprocess.DEVNULL)
-        except OSError:
-            self.p = None
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_sm = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:   # no NVML: the line says so
+            self.err = repr(e)
+        self._stop = threading.Event()
+        self.t = threading.Thread(target=self._run, daemon=True)
+        if self.h is not None:
+            self.t.start()
 
-    def stop(self):
-        if self.p is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except Exception:
-            self.p.kill()
-        self.f.flush()
-        rows = [r.split(", ") for r in open(self.f.name).read().strip().splitlines() if r.strip()]
-        os.unlink(self.f.name)
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in rows:
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
             try:
-                sm.append(float(r[1])); smax.append(float(r[2]))
-            except (ValueError, IndexError):
-                continue
-            for nm, val in zip(names, r[5:9]):
-                if val.strip().lower().startswith("active"):
-                    reasons.add(nm)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                self.samples.append((time.perf_counter(), float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)),
+                                     nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0,
+                                     int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def mark(self, name, t0, t1):
+        self.windows[name] = (t0, t1)
+
+    def stop(self, window):
+        if self.h is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["NVML unavailable: " + getattr(self, "err", "")]}
+        self._stop.set()
+        self.t.join(timeout=2)
+        t0, t1 = self.windows.get(window, (0.0, float("inf")))
+        sel = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples
+        bits = 0
+        for s in sel:
+            bits |= s[3]
+        allb = 0
+        for s in self.samples:
+            allb |= s[3]
+        return {"sm_mhz": float(np.median([s[1] for s in sel])), "sm_max_mhz": self.max_sm, "samples": len(sel),
+                "window": window, "power_w_max": max(s[2] for s in sel),
+                "reasons": sorted(k for k, b in self.REASONS.items() if bits & b),
+                "whole_run": {"samples": len(self.samples), "sm_mhz": float(np.median([s[1] for s in self.samples])),
+                              "power_w_max": max(s[2] for s in self.samples),
+                              "reasons": sorted(k for k, b in self.REASONS.items() if allb & b)}}
 
 
 def measured_peaks():
@@ -114,26 +144,36 @@ def measured_peaks():
 # ------------------------------------------------------------------------------------------ oracle legs
 
 class OracleSample:
-    """The CPU oracle, as it stands, on a bounded sample of the workload: `n_layers` decoder layers
-    at full width plus the lm_head, on this machine's host cores; the per-layer time is extrapolated
-    to the model's depth (every layer costs the same arithmetic)."""
+    """The CPU oracle, as it stands, on this machine's host cores. It runs `n_layers` decoder layers of the
+    workload at full width plus the lm_head; with n_layers = the model's depth that is one whole pass.
+    One synthetic layer's weights serve every layer (the arithmetic, and so the time, is the same;
+    generating 13-65 GB on the host would take longer than the pass)."""
 
     def __init__(self, cfg, P, parent, tokens):
         from oracle import oracle as orc
         self.orc, self.cfg, self.P, self.parent, self.tokens = orc, cfg, P, parent, tokens
         self.glob = gen.gen_globals(cfg)
-        self.layer = gen.gen_layer(cfg, 0)              # one synthetic layer, reused for every sample layer
+        self.layer = gen.gen_layer(cfg, 0)
         self.pk, self.pv = gen.gen_prefix_kv(cfg, 0, P)
 
     def run(self, n_layers):
         small = gen.shrink(self.cfg, n_layers)
         lt = []
+        t0 = time.perf_counter()
         self.orc.verify_tree(small, self.glob, lambda l: self.layer, lambda l: (self.pk, self.pv), self.P,
                              self.tokens, self.parent, keep_kv=False, layer_times=lt)
-        sec = float(np.mean(lt[:-1])) * self.cfg.n_layers + lt[-1]
-        desc = (f"{n_layers} full-width decoder layer(s) + lm_head of the workload run by the oracle "
-                f"(N={len(self.tokens)}, P={self.P}); per-layer time x {self.cfg.n_layers} layers + head")
-        return sec, desc, self.orc.n_threads()
+        wall = time.perf_counter() - t0
+        full = n_layers == self.cfg.n_layers
+        if full:
+            sec = wall
+            desc = (f"one whole pass of the workload by the oracle: all {n_layers} layers at full width + lm_head "
+                    f"(N={len(self.tokens)}, P={self.P}), wall time including its fp32 widening of the weights; "
+                    "one synthetic layer's weights reused for every layer")
+        else:
+            sec = float(np.mean(lt[:-1])) * self.cfg.n_layers + lt[-1]
+            desc = (f"{n_layers} full-width decoder layer(s) + lm_head of the workload run by the oracle "
+                    f"(N={len(self.tokens)}, P={self.P}); per-layer time x {self.cfg.n_layers} layers + head")
+        return sec, desc, self.orc.n_threads(), not full
 
 
 def run_reference(args, w, cfg):
@@ -143,21 +183,23 @@ def run_reference(args, w, cfg):
     parent = gen.gen_tree(w)
     tokens = gen.gen_tokens(cfg, w.n_nodes)
     smp = OracleSample(cfg, w.prefix_len, parent, tokens)
+    layers = cfg.n_layers if args.oracle_layers <= 0 else min(args.oracle_layers, cfg.n_layers)
     times = []
-    desc, cores = "", 0
+    desc, cores, extrap = "", 0, False
     for i in range(args.warmup + args.steps):
-        t, desc, cores = smp.run(1)
+        t, desc, cores, extrap = smp.run(layers)
         if i >= args.warmup:
             times.append(t)
-    sec = float(np.mean(times))
+    sec = float(np.median(times))
     val = 1.0 / sec
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "ms_per_step_min": min(times) * 1e3, "ms_per_step_max": max(times) * 1e3,
+        "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "extrapolated": extrap,
         "config": {"workload": workload_name(w, cfg)},
         "tree_tokens_per_sec": val * w.n_nodes,
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "extrapolated": extrap},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -189,6 +231,192 @@ def build_verifier(cfg, w, device):
     return v
 
 
+def time_steps(step, steps, barrier):
+    """K steps with an event between consecutive steps and no host synchronisation inside: returns the
+    per-step milliseconds and the host times of the region's start and end."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    barrier()
+    t0 = time.perf_counter()
+    ev[0].record()
+    for i in range(steps):
+        step()
+        ev[i + 1].record()
+    barrier()
+    t1 = time.perf_counter()
+    return [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)], ev[0].elapsed_time(ev[steps]), (t0, t1)
+
+
+def analyze_trace(t, n_layers, passes):
+    """t: [launches][256][16] %globaltimer stamps (ns) of `passes` undisturbed passes; per pass the traced
+    launches are QKV, then per layer attention, O, gate/up, down, next QKV (lm_head at the end). A launch
+    is charged the time from the latest exit seen so far (its predecessor's end) to its own last exit;
+    the first launch of a pass from its first entry. The intervals of a pass are disjoint, so their sum is
+    at most the pass."""
+    per_pass = 1 + 5 * n_layers
+    names = ["qkv"] + ["attention", "o", "gate_up", "down", "qkv"] * n_layers
+    names[-1] = "lm_head"
+    tot = {}
+    cnt = {}
+    span = 0.0
+    for p in range(passes):
+        prev = None
+        first = None
+        for j in range(per_pass):
+            sl = t[p * per_pass + j]
+            ent = sl[:, 0]
+            ext = sl[:, 12]
+            ok = ent > 0
+            if not ok.any():
+                raise RuntimeError(f"launch {j} of pass {p} left no trace")
+            e0 = float(ent[ok].min())
+            e1 = float(ext[ext > 0].max())
+            if prev is None:
+                prev, first = e0, e0
+            dur = max(0.0, e1 - prev)
+            prev = max(prev, e1)
+            tot[names[j]] = tot.get(names[j], 0.0) + dur
+            cnt[names[j]] = cnt.get(names[j], 0) + 1
+        span += prev - first
+    out = {k: {"ms_per_step": tot[k] / passes / 1e6, "launches_per_step": cnt[k] // passes,
+               "avg_launch_us": tot[k] / cnt[k] / 1e3} for k in tot}
+    return out, span / passes / 1e6
+
+
+def bench_workload(B, v, cfg, w, args, device, barrier, clocks=None, tag="main"):
+    """Times one workload on an already built verifier: per-step events, traced passes, isolated launches."""
+    P, n = w.prefix_len, w.n_nodes
+    rank = int(os.environ.get("RANK", "0"))
+    parent_np = gen.gen_tree(w, seed=rank)
+    tokens_np = gen.gen_tokens(cfg, n, seed=rank)
+    tokens = torch.as_tensor(tokens_np, device=device)
+    parent = torch.as_tensor(parent_np, device=device)
+    out = v.new_outputs(n, want_logits=True)
+
+    def step():
+        v.verify_tree(P, tokens, parent, out=out)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sc = out["scalars"].cpu().numpy()
+    if int(sc[B.S_STATUS]) != 0:
+        raise SystemExit(f"verification pass reported device status {int(sc[B.S_STATUS])}")
+    accepted_random = int(sc[B.S_ACCEPTED_LEN])
+
+    # ---- region A: K passes, inputs resident in HBM, an event between consecutive passes
+    l0 = v.launch_count()
+    per_step, total_ms, win = time_steps(step, args.steps, barrier)
+    launches = v.launch_count() - l0
+    if clocks is not None:
+        clocks.mark(tag, *win)
+
+    res = {"per_step_ms": per_step, "total_ms": total_ms, "launches": int(launches), "accepted_len_random": accepted_random,
+           "tokens_np": tokens_np, "parent_np": parent_np}
+
+    # ---- region T: the same passes with the kernels' own time stamps (no events between launches)
+    if cfg.dtype == "bf16":
+        passes = min(args.steps, 8)
+        per_pass = 1 + 5 * cfg.n_layers
+        buf = torch.zeros((per_pass * passes, 256, 16), dtype=torch.int64, device=device)
+        v.set_gemm_trace(buf)
+        tr_steps, _, _ = time_steps(step, passes, barrier)
+        v.set_gemm_trace(None)
+        kinds, span_ms = analyze_trace(buf.cpu().numpy().astype(np.float64), cfg.n_layers, passes)
+        del buf
+        res["trace"] = {"kinds": kinds, "span_ms_per_step": span_ms, "ms_per_step_traced": float(np.median(tr_steps)), "passes": passes}
+
+    # ---- region B: every GEMM / attention launch bracketed by events (the kernels in isolation)
+    v.set_kernel_timing(True)
+    iso_steps, _, _ = time_steps(step, min(args.steps, 8), barrier)
+    gemm_ms, gemm_cnt = v.get_kernel_timing(0)
+    attn_ms, attn_cnt = v.get_kernel_timing(1)
+    v.set_kernel_timing(False)
+    res["isolated"] = {"gemm_ms": gemm_ms, "gemm_cnt": gemm_cnt, "attn_ms": attn_ms, "attn_cnt": attn_cnt,
+                       "steps": len(iso_steps), "ms_per_step": float(np.median(iso_steps))}
+
+    # ---- the planted variant (draft tokens the target really produces along some branches): accepted length
+    tok = tokens_np
+    o2 = out
+    for it in range(6):
+        tok = gen.plant_tokens(parent_np, tok, o2["argmax"].cpu().numpy(), seed=it, prob=0.7)
+        o2 = v.verify_tree(P, torch.as_tensor(tok, device=device), parent)
+    torch.cuda.synchronize()
+    res["accepted_len_planted"] = int(o2["scalars"][B.S_ACCEPTED_LEN].item())
+    return res
+
+
+def summarize(cfg, w, res, world, peaks, ms=None):
+    """ms: the median step time to report (the slowest replica's when there are several)."""
+    hbm_peak, tf_peak, peak_kind = peaks
+    P, n = w.prefix_len, w.n_nodes
+    ab = algorithmic_bytes(cfg, P, n)
+    fl = flops(cfg, P, n)
+    ms = float(np.median(res["per_step_ms"])) if ms is None else ms
+    s = {"ms_per_step": ms, "ms_per_step_min": float(min(res["per_step_ms"])), "ms_per_step_max": float(max(res["per_step_ms"])),
+         "ms_per_step_mean": res["total_ms"] / len(res["per_step_ms"]),
+         "passes_per_s": world / (ms * 1e-3), "tree_tokens_per_sec": world * n / (ms * 1e-3),
+         "pass_hbm_gbs": ab["total"] / (ms * 1e-3) / 1e9,
+         "pass_roofline": {"algorithmic_bytes": ab["total"], "flops": fl,
+                           "frac_of_measured_hbm": ab["total"] / (ms * 1e-3) / 1e9 / hbm_peak,
+                           "frac_of_8TBs": ab["total"] / (ms * 1e-3) / 8e12,
+                           "tensor_frac": fl / (ms * 1e-3) / 1e12 / tf_peak, "peaks": peak_kind},
+         "accepted_len": {"random_tokens": res["accepted_len_random"], "planted_tokens": res["accepted_len_planted"]}}
+    return s
+
+
+def roofline_block(cfg, w, res, peaks):
+    hbm_peak, _, peak_kind = peaks
+    n = w.n_nodes
+    gb, gcount = gemm_algorithmic_bytes(cfg, n)
+    iso = res["isolated"]
+    iso_avg_ms = iso["gemm_ms"] / max(iso["gemm_cnt"], 1)
+    iso_bytes = gb * iso["steps"] / max(iso["gemm_cnt"], 1)
+    iso_gbs = iso_bytes / (iso_avg_ms * 1e-3) / 1e9
+    ratio = NCU_GEMM_CAPTURE["dram_bytes"] / NCU_GEMM_CAPTURE["algorithmic_bytes"]
+    block = {"kernel": "gemm_chain_kernel", "bound": "hbm", "peak": hbm_peak, "unit": "GB/s", "of": peak_kind,
+             "algorithmic_bytes_per_launch": gb / gcount, "traffic": ratio * gb / gcount,
+             "traffic_source": f"ncu capture {NCU_GEMM_CAPTURE['summary']}: DRAM bytes / algorithmic bytes = {ratio:.3f}, scaled by bytes",
+             "isolated": {"achieved": iso_gbs, "frac": iso_gbs / hbm_peak, "avg_launch_ms": iso_avg_ms,
+                          "launches_timed": iso["gemm_cnt"], "gemm_ms_per_step": iso["gemm_ms"] / iso["steps"],
+                          "attention_ms_per_step": iso["attn_ms"] / iso["steps"], "ms_per_step_with_kernel_events": iso["ms_per_step"],
+                          "how": "CUDA events around every launch: no overlap between consecutive kernels"}}
+    tr = res.get("trace")
+    if tr:
+        k = tr["kinds"]
+        gemm_ms = sum(v["ms_per_step"] for name, v in k.items() if name != "attention")
+        attn_ms = k.get("attention", {"ms_per_step": 0.0})["ms_per_step"]
+        avg_ms = gemm_ms / gcount
+        ach = gb / (gemm_ms * 1e-3) / 1e9
+        block.update({"achieved": ach, "frac": ach / hbm_peak, "avg_launch_ms": avg_ms, "launches_per_step": gcount,
+                      "gemm_ms_per_step": gemm_ms, "attention_ms_per_step": attn_ms,
+                      "kernels_ms_per_step": gemm_ms + attn_ms, "ms_per_step_traced": tr["ms_per_step_traced"],
+                      "per_gemm": {name: {"ms_per_step": v["ms_per_step"], "avg_launch_us": v["avg_launch_us"]} for name, v in k.items()},
+                      "how": "inside undisturbed passes: %globaltimer stamps per launch; a launch is charged the time from "
+                             "its predecessor's last exit to its own last exit, so kernels_ms_per_step <= ms_per_step_traced"})
+    else:
+        block.update({"achieved": iso_gbs, "frac": iso_gbs / hbm_peak, "avg_launch_ms": iso_avg_ms})
+    return block
+
+
+def attention_digest(B, device, peaks, reps=30, warmup=5):
+    """Config 4 in short: 32 heads x 128, prefix 256..8192 x trees of 8..128 nodes (one random topology
+    each), K/V buffers rotated over more than twice the L2 so that every launch reads HBM."""
+    from paper_2309_04255_b200 import kernel_bench as KB
+    H, hd = 32, 128
+    cfg = gen.ModelConfig("attn", 0, H * hd, H, hd, 256, 512, "bf16")
+    v = B.Verifier(cfg, 16, device=device)
+    cells = []
+    for P in (256, 1024, 4096, 8192):
+        for n in (8, 32, 64, 128):
+            parent = gen.tree_random(n, 16, "uniform4", 0)
+            c = KB.attention_cell(v, P, n, parent, reps, warmup, l2_resident=False)
+            cells.append({"prefix": P, "nodes": n, "us": round(c["us_attention_kernel"], 2), "gbs": round(c["hbm_gbs"], 1),
+                          "frac": round(c["hbm_gbs"] / peaks[0], 4)})
+    v.close()
+    return {"workload": "C4: tree-masked attention alone, bf16, 32 heads x 128, K/V/Q ~ N(0,1), random trees (branching uniform 1-4)",
+            "timing": "CUDA events around each attention launch, K/V rotated over > 2 x L2", "peak_gbs": peaks[0], "cells": cells}
+
+
 def run_gpu(args, w, cfg):
     from paper_2309_04255_b200 import binding as B
     rank = int(os.environ.get("RANK", "0"))
@@ -206,117 +434,100 @@ def run_gpu(args, w, cfg):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
 
-    v = build_verifier(cfg, w, device)
-    P, n = w.prefix_len, w.n_nodes
-    parent_np = gen.gen_tree(w, seed=rank)
-    tokens_np = gen.gen_tokens(cfg, n, seed=rank)
-    tokens = torch.as_tensor(tokens_np, device=device)
-    parent = torch.as_tensor(parent_np, device=device)
-    out = v.new_outputs(n, want_logits=True)
-
     def barrier():
         torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
             torch.cuda.synchronize()
 
-    def step():
-        v.verify_tree(P, tokens, parent, out=out)
-
-    for _ in range(args.warmup):
-        step()
-    barrier()
-    st = int(out["scalars"][B.S_STATUS].item())
-    if st != 0:
-        raise SystemExit(f"verification pass reported device status {st}")
-
-    # ---- timed region A: K passes, inputs resident in HBM, CUDA events on the launching stream
+    peaks = measured_peaks()
     clocks = ClockSampler(local)
-    l0 = v.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    barrier()
-    ms = e0.elapsed_time(e1)
-    launches = v.launch_count() - l0
+    v = build_verifier(cfg, w, device)
+    P, n = w.prefix_len, w.n_nodes
+    res = bench_workload(B, v, cfg, w, args, device, barrier, clocks, "timed_region")
+    tokens_np, parent_np = res["tokens_np"], res["parent_np"]
 
-    # ---- timed region B: the same K passes with every GEMM / attention launch bracketed by events
-    v.set_kernel_timing(True)
-    barrier()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record()
-    for _ in range(args.steps):
-        step()
-    f1.record()
-    barrier()
-    gemm_ms, gemm_cnt = v.get_kernel_timing(0)
-    attn_ms, attn_cnt = v.get_kernel_timing(1)
-    v.set_kernel_timing(False)
-    ms_events = f0.elapsed_time(f1)
-
-    # ---- end to end through the host-buffer entry point (pinned host memory both ways)
+    # ---- end to end through the host-buffer entry point (pinned host memory both ways, logits included)
     th = torch.as_tensor(tokens_np).pin_memory()
     ph = torch.as_tensor(parent_np).pin_memory()
-    host = {"logits": None, "argmax": torch.empty(n, dtype=torch.int32).pin_memory(),
-            "accepted_path": torch.empty(128, dtype=torch.int32).pin_memory(),
-            "scalars": torch.empty(8, dtype=torch.int32).pin_memory()}
-    for _ in range(min(3, args.warmup)):
-        v.verify_tree_host(P, th, ph, host)
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        v.verify_tree_host(P, th, ph, host)     # synchronises the stream itself
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    clk = clocks.stop()
 
-    times = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=device)
+    def host_buffers(with_logits):
+        return {"logits": torch.empty((n, cfg.vocab), dtype=torch.float32).pin_memory() if with_logits else None,
+                "argmax": torch.empty(n, dtype=torch.int32).pin_memory(),
+                "accepted_path": torch.empty(128, dtype=torch.int32).pin_memory(),
+                "scalars": torch.empty(8, dtype=torch.int32).pin_memory()}
+
+    e2e = {}
+    for with_logits in (True, False):
+        host = host_buffers(with_logits)
+        for _ in range(min(3, args.warmup)):
+            v.verify_tree_host(P, th, ph, host)
+        barrier()
+        ts = []
+        for _ in range(args.steps):
+            t0 = time.perf_counter()
+            v.verify_tree_host(P, th, ph, host)     # synchronises the stream itself
+            ts.append(time.perf_counter() - t0)
+        e2e[with_logits] = float(np.median(ts)) * 1e3
+    clk = clocks.stop("timed_region")
+
+    ms_med = float(np.median(res["per_step_ms"]))
+    times = torch.tensor([ms_med, e2e[True], e2e[False]], dtype=torch.float64, device=device)
     if dist is not None:
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = float(times[0]), float(times[1])
+    ms_med, e2e_ms, e2e_nl_ms = float(times[0]), float(times[1]), float(times[2])
 
     if rank == 0:
-        hbm_peak, tf_peak, peak_kind = measured_peaks()
-        ab = algorithmic_bytes(cfg, P, n)
-        gb, gcount = gemm_algorithmic_bytes(cfg, n)
-        ms_per = ms / args.steps
-        value = world * args.steps / (ms * 1e-3)
-        gemm_avg_ms = gemm_ms / max(gemm_cnt, 1)
-        gb_launch = gb * args.steps / max(gemm_cnt, 1)          # a launch may chain several GEMMs
-        gemm_gbs = gb_launch / (gemm_avg_ms * 1e-3) / 1e9
-        fl = flops(cfg, P, n)
+        s = summarize(cfg, w, res, world, peaks, ms=ms_med)
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_per, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "metric": METRIC, "value": s["passes_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": s["ms_per_step"], "ms_per_step_min": s["ms_per_step_min"], "ms_per_step_max": s["ms_per_step_max"],
+            "ms_per_step_mean": s["ms_per_step_mean"], "value_is": "median over the steps",
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": cfg.dtype, "data": "synthetic",
             "config": {"workload": workload_name(w, cfg), "l2": "inputs larger than L2 (weights stream once per pass)",
                        "replicas": world},
-            "tree_tokens_per_sec": value * n,
-            "pass_hbm_gbs": ab["total"] / (ms_per * 1e-3) / 1e9,
-            "pass_roofline": {"algorithmic_bytes": ab["total"], "flops": fl,
-                              "frac_of_measured_hbm": ab["total"] / (ms_per * 1e-3) / 1e9 / hbm_peak,
-                              "frac_of_8TBs": ab["total"] / (ms_per * 1e-3) / 8e12,
-                              "tensor_frac": fl / (ms_per * 1e-3) / 1e12 / tf_peak, "peaks": peak_kind},
-            "roofline": {"kernel": "gemm_chain_kernel", "bound": "hbm", "achieved": gemm_gbs, "peak": hbm_peak,
-                         "unit": "GB/s", "frac": gemm_gbs / hbm_peak,
-                         "traffic": (GEMM_TRAFFIC_RATIO * gb_launch) if GEMM_TRAFFIC_RATIO else None,
-                         "launches_timed": gemm_cnt, "avg_launch_ms": gemm_avg_ms,
-                         "algorithmic_bytes_per_launch": gb_launch, "of": peak_kind,
-                         "ms_per_step_with_kernel_events": ms_events / args.steps,
-                         "attention_ms_per_step": attn_ms / args.steps, "gemm_ms_per_step": gemm_ms / args.steps},
-            "e2e": {"value": world * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
-                    "h2d_bytes_per_step": 2 * n * 4, "d2h_bytes_per_step": (n + n + 8) * 4},
-            "gpu_launches": int(launches),
+            "tree_tokens_per_sec": s["tree_tokens_per_sec"], "pass_hbm_gbs": s["pass_hbm_gbs"],
+            "pass_roofline": s["pass_roofline"], "accepted_len": s["accepted_len"],
+            "roofline": roofline_block(cfg, w, res, peaks),
+            "e2e": {"value": world / (e2e_ms * 1e-3), "unit": UNIT, "logits": True,
+                    "h2d_bytes_per_step": 2 * n * 4, "d2h_bytes_per_step": (n + n + 8) * 4 + n * cfg.vocab * 4,
+                    "without_logits": {"value": world / (e2e_nl_ms * 1e-3), "d2h_bytes_per_step": (n + n + 8) * 4}},
+            "gpu_launches": res["launches"],
             "clocks": clk,
         }
+        v.close()
+        del v
+        torch.cuda.empty_cache()
+        if world == 1 and args.extras and w.name == "C2":
+            extra = {}
+            w3 = gen.WORKLOADS["C3"]
+            c3 = gen.MODELS[w3.model]
+            v3 = build_verifier(c3, w3, device)
+            r3 = bench_workload(B, v3, c3, w3, args, device, barrier)
+            s3 = summarize(c3, w3, r3, 1, peaks)
+            rb3 = roofline_block(c3, w3, r3, peaks)
+            extra["C3"] = {"workload": workload_name(w3, c3), "ms_per_step": s3["ms_per_step"], "ms_per_step_min": s3["ms_per_step_min"],
+                           "ms_per_step_max": s3["ms_per_step_max"], "passes_per_s": s3["passes_per_s"],
+                           "tree_tokens_per_sec": s3["tree_tokens_per_sec"],
+                           "frac_of_measured_hbm": s3["pass_roofline"]["frac_of_measured_hbm"],
+                           "frac_of_8TBs": s3["pass_roofline"]["frac_of_8TBs"], "accepted_len": s3["accepted_len"],
+                           "gemm_frac_in_pass": rb3.get("frac"), "gemm_ms_per_step": rb3.get("gemm_ms_per_step"),
+                           "attention_ms_per_step": rb3.get("attention_ms_per_step"), "steps": args.steps}
+            v3.close()
+            del v3
+            torch.cuda.empty_cache()
+            extra["C4"] = attention_digest(B, device, peaks)
+            line["workloads"] = extra
         if world == 1 and not args.no_cpu_baseline:
-            sec, desc, cores = OracleSample(cfg, P, parent_np, tokens_np).run(args.oracle_layers)
-            line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+            smp = OracleSample(cfg, P, parent_np, tokens_np)
+            layers = cfg.n_layers if args.oracle_layers <= 0 else min(args.oracle_layers, cfg.n_layers)
+            sec, desc, cores, extrap = smp.run(layers)
+            line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                                    "extrapolated": extrap}
         print(json.dumps(line), flush=True)
-    v.close()
+    else:
+        v.close()
     if dist is not None:
         dist.destroy_process_group()
 
@@ -329,11 +540,16 @@ def main():
     ap.add_argument("--workload", default="C2", choices=sorted(gen.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--oracle-layers", type=int, default=8)
+    ap.add_argument("--no-extras", dest="extras", action="store_false", help="skip the C3 and C4 figures")
+    ap.add_argument("--oracle-layers", type=int, default=None,
+                    help="decoder layers the oracle runs per step (0 = the whole depth); default: the whole depth for "
+                         "C1/C2, 8 layers (extrapolated, and marked so) for the deeper workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = gen.WORKLOADS[args.workload]
     cfg = gen.MODELS[w.model]
+    if args.oracle_layers is None:
+        args.oracle_layers = 0 if args.workload in ("C1", "C2") else 8
     if args.impl == "reference":
         run_reference(args, w, cfg)
     else:

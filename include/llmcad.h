@@ -29,8 +29,13 @@
  * = n_heads, rotary position embedding on interleaved pairs (x[2t], x[2t+1]) with
  * angle pos * rope_base^(-2t/head_dim), softmax scale 1/sqrt(head_dim), SwiGLU
  * FFN, separate embedding and lm_head. Weights are row-major [out][in].
- * dtype bf16: weights, cached K/V and GEMM input activations are bf16; residual
- * stream, accumulators, softmax, norms and logits are fp32. dtype fp32: all fp32.
+ * dtype bf16: weights and cached K/V are bf16; residual stream, accumulators,
+ * softmax, norms and logits are fp32. Every activation that enters a tensor-core
+ * product (GEMM inputs, queries, softmax weights, attention outputs, and within a
+ * pass the tree nodes' own K/V) travels as two bf16 planes, hi = bf16(v) and
+ * lo = bf16(v - hi), i.e. with 16 significant bits: plain bf16 activations do not
+ * stay inside 2e-2 of the largest logit over tens of layers. The cache receives the
+ * hi plane of K/V only. dtype fp32: all fp32.
  *
  * KV cache layout: [n_layers][2 (K,V)][n_heads][max_seq][head_dim] in the model
  * dtype. Slots 0..prefix_len-1 hold the prefix; during a pass the tree nodes'
@@ -200,9 +205,14 @@ int llmcad_accept_compact(llmcad_ctx *ctx, void *kv_cache, int32_t prefix_len, c
                           const int32_t *parent_idx, const int32_t *argmax, int32_t n,
                           int32_t *accepted_path, int32_t *scalars, void *stream);
 
-/* Tree-masked attention alone (one layer): q [n][H][hd]; k, v [H][kv_stride][hd] with
- * the prefix at slots 0..prefix_len-1 and the tree nodes at prefix_len..prefix_len+n-1;
- * o [n][H][hd]. dtype as in llmcad_config. All DEVICE. */
+/* Tree-masked attention alone (one layer), the masked self-attention of Sec. 3.2 "Tree
+ * decoder": node i attends to every prefix slot and to the tree nodes whose bit is set in
+ * row i of the mask table (itself and its ancestors), softmax scale 1/sqrt(hd).
+ * q [n][H][hd]; k, v [H][kv_stride][hd] with the prefix at slots 0..prefix_len-1 and the
+ * tree nodes at prefix_len..prefix_len+n-1; o [n][H][hd]. dtype as in llmcad_config. All
+ * DEVICE; in bf16 contexts q, k, v and o must be 16-byte aligned (LLMCAD_ERR_INVALID_ARG
+ * otherwise). A malformed parent_idx lands in the context's status word
+ * (llmcad_last_status) and leaves o untouched. */
 int llmcad_tree_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, int32_t kv_stride,
                           int32_t prefix_len, const int32_t *parent_idx, int32_t n, void *o, void *stream);
 
@@ -216,20 +226,6 @@ int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, 
  * synchronises `stream` and returns the context's own device status word of the last such
  * call: 0, a device-detected LLMCAD_ERR_* (> 0), or LLMCAD_ERR_CUDA. */
 int llmcad_last_status(llmcad_ctx *ctx, void *stream);
-
-/* Per-launch timing for roofline reports. While enabled, every skinny-GEMM launch (kind 0) and
- * every tree-attention launch (kind 1) of this context is bracketed by CUDA events on the
- * launching stream. llmcad_get_kernel_timing waits for the recorded launches of `kind`, returns
- * their summed duration and count since the last query, and forgets them. */
-int llmcad_set_kernel_timing(llmcad_ctx *ctx, int32_t enable);
-int llmcad_get_kernel_timing(llmcad_ctx *ctx, int32_t kind, double *total_ms /*HOST*/, int64_t *n_launches /*HOST*/);
-
-/* Tracing aid: while `trace` (DEVICE, [capacity][256][16] uint64, or NULL to stop) is set, the
- * next `capacity` tensor-core GEMM and attention launches of this context each fill one
- * [256][16] slice: per CTA, nanosecond timestamps (%globaltimer) of entry (0), set-up done (1),
- * grid dependency resolved (3), per chained GEMM g first accumulator ready (4+2g) and epilogue
- * done (5+2g), exit (12). */
-int llmcad_set_gemm_trace(llmcad_ctx *ctx, uint64_t *trace, int32_t capacity);
 
 /* The tensor-core path streams each weight matrix as a sequence of 16 KB tiles (128 rows x 64
  * columns, tile-row major then k-block, 128-byte rows with the 16-byte chunk c of row r stored
@@ -256,7 +252,8 @@ int llmcad_skinny_gemm_tiled(llmcad_ctx *ctx, const void *w_tiled, const void *x
  *
  * Same computation and layouts as llmcad_tree_attention, bf16, head_dim 128 only:
  * q, o [n][n_heads][128]; k, v [n_heads][kv_stride][128]; parent_idx int32[n]; all DEVICE,
- * caller-owned. status_out (DEVICE int32, may be NULL) receives 0 or LLMCAD_ERR_BAD_TREE.
+ * caller-owned, q, k, v and o 16-byte aligned (LLMCAD_ERR_INVALID_ARG otherwise). status_out
+ * (DEVICE int32, may be NULL) receives 0 or LLMCAD_ERR_BAD_TREE; a malformed tree leaves o untouched.
  * Limits: n <= 128 (what the static scratch holds) -- larger n is refused with
  * LLMCAD_ERR_UNSUPPORTED and a message in llmcad_noalloc_last_error(); n_heads <= 65535.
  *
@@ -321,9 +318,6 @@ int llmcad_tree_branches(const int32_t *parent_idx, const double *node_conf, int
                          double *cum_conf, int32_t *branch_len, int32_t *n_branches);
 int llmcad_branch_pacer(const double *cum_conf, const int32_t *branch_len, int32_t n_branches, double m_tokens,
                         double *f, int32_t *next_branch);
-
-/* Number of kernels this library has launched through this context so far. */
-int64_t llmcad_launch_count(const llmcad_ctx *ctx);
 
 #ifdef __cplusplus
 }

@@ -31,6 +31,7 @@ EXPORTS = [
     "llmcad_accept_compact", "llmcad_tree_attention", "llmcad_skinny_gemm", "llmcad_launch_count",
     "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace", "llmcad_tiled_weight_bytes", "llmcad_tile_weight", "llmcad_skinny_gemm_tiled", "llmcad_tree_attention_noalloc", "llmcad_noalloc_last_error",
     "llmcad_tree_confidence", "llmcad_update_threshold", "llmcad_extend_tree", "llmcad_tree_branches", "llmcad_branch_pacer",
+    "llmcad_set_wait_limit_ns", "llmcad_selftest_wait_timeout",
 ]
 
 
@@ -107,6 +108,8 @@ def lib():
         L.llmcad_extend_tree.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
         L.llmcad_set_kernel_timing.argtypes = [vp, i32]
         L.llmcad_get_kernel_timing.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+        L.llmcad_set_wait_limit_ns.argtypes = [vp, C.c_uint64]
+        L.llmcad_selftest_wait_timeout.argtypes = [vp, vp]
         _lib = L
     return _lib
 
@@ -244,10 +247,10 @@ class Verifier:
                "llmcad_accept_compact")
         return path, scalars
 
-    def tree_attention(self, q, k, v, prefix_len: int, parent):
-        """q [n][H][hd]; k, v [H][kv_stride][hd]."""
+    def tree_attention(self, q, k, v, prefix_len: int, parent, o=None):
+        """q [n][H][hd]; k, v [H][kv_stride][hd]; o (optional) receives the result."""
         n = q.shape[0]
-        o = torch.empty_like(q)
+        o = torch.empty_like(q) if o is None else o
         _check(lib().llmcad_tree_attention(self.ctx, _ptr(q), _ptr(k), _ptr(v), k.shape[1], prefix_len, _ptr(parent), n,
                                            _ptr(o), _stream()), "llmcad_tree_attention")
         return o
@@ -292,11 +295,30 @@ class Verifier:
     def launch_count(self) -> int:
         return lib().llmcad_launch_count(self.ctx)
 
+    def set_wait_limit_ns(self, ns: int):
+        """Bound of every device-side wait of this context's kernels (0 = the default of 2 s)."""
+        _check(lib().llmcad_set_wait_limit_ns(self.ctx, int(ns)), "llmcad_set_wait_limit_ns")
+
+    def selftest_wait_timeout(self) -> int:
+        """Runs a small GEMM chain whose grid barrier cannot complete; returns the device status word."""
+        code = lib().llmcad_selftest_wait_timeout(self.ctx, _stream())
+        if code < 0:
+            raise LlmcadError(code, "llmcad_selftest_wait_timeout")
+        return code
+
 
 def tree_attention_noalloc(q, k, v, prefix_len: int, parent, o, status=None):
     """Context-free tree attention on caller-provided buffers (the library allocates nothing):
     q, o [n][H][128] bf16; k, v [H][kv_stride][128] bf16; parent int32[n]; status int32[1] or None."""
     n, H = q.shape[0], q.shape[1]
+    # the entry point takes raw pointers: what it cannot see (dtype, shapes) is checked here
+    for name, t in (("q", q), ("k", k), ("v", v), ("o", o)):
+        if t.dtype != torch.bfloat16 or t.dim() != 3 or t.shape[2] != 128:
+            raise ValueError(f"{name} must be a bf16 tensor [..][..][128], got {t.dtype} {tuple(t.shape)}")
+    if k.shape != v.shape or k.shape[0] != H or o.shape != q.shape:
+        raise ValueError("shapes: q, o [n][H][128]; k, v [H][kv_stride][128]")
+    if parent.dtype != torch.int32 or parent.numel() != n or (status is not None and status.dtype != torch.int32):
+        raise ValueError("parent must be int32[n] and status int32[1]")
     code = lib().llmcad_tree_attention_noalloc(_ptr(q), _ptr(k), _ptr(v), H, k.shape[1], prefix_len, _ptr(parent), n, _ptr(o),
                                                _ptr(status), _stream())
     if code != OK:

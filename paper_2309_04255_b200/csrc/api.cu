@@ -10,6 +10,7 @@
 #include <new>
 #include <vector>
 
+#include "../../include/llmcad_profile.h"
 #include "attention_tc.cuh"
 #include "common.cuh"
 #include "gemm_tc.cuh"
@@ -114,6 +115,7 @@ struct llmcad_ctx {
     int arrival_set = 0;                 // arrival-counter set of the next GEMM launch (launches alternate)
     int prev_gemms = 0, prev_arrival_words = 0;   // what the last GEMM launch touched in its set
     int64_t launches = 0;
+    uint64_t wait_limit_ns = kDefaultWaitLimitNs;   // bound of every device-side wait (llmcad_set_wait_limit_ns)
     unsigned long long *trace = nullptr;   // optional timeline buffer (llmcad_set_gemm_trace): [launch][256][16]
     int trace_launch = 0, trace_capacity = 0;
     unsigned long long *next_trace()
@@ -237,6 +239,7 @@ struct Chain {
         p.grid_counter = ctx->grid_counter;
         p.barrier_base = ctx->barrier_base;
         p.status = status;
+        p.wait_limit_ns = ctx->wait_limit_ns;
         p.trace = ctx->next_trace();
         uint32_t arrivals = 0;
         ctx->launches++;
@@ -279,7 +282,7 @@ int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, 
                         : (c.flags & LLMCAD_FLAG_MMA_ATTN) ? false : attention_prefers_t5(n);
         if (t5) {
             CUDA_TRY(launch_attention_t5(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->n_sms, status, st,
-                                         &launched, ctx->next_trace(), comp ? 1 : 0, ctx->kv_lo, n_tree, q_first));
+                                         &launched, ctx->next_trace(), comp ? 1 : 0, ctx->kv_lo, n_tree, q_first, ctx->wait_limit_ns));
             ctx->launches += launched;
             return LLMCAD_OK;
         }
@@ -770,6 +773,10 @@ int llmcad_tree_attention(llmcad_ctx *ctx, const void *q, const void *k, const v
     if (!ctx || !q || !k || !v || !parent_idx || !o) return LLMCAD_ERR_INVALID_ARG;
     if (n < 1 || prefix_len < 0 || kv_stride < prefix_len + n) return LLMCAD_ERR_INVALID_ARG;
     if (n > ctx->cfg.max_tree) return LLMCAD_ERR_UNSUPPORTED;
+    // the tensor-core kernels move rows as 16-byte vectors and bulk copies
+    if (ctx->tc_attn && ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(v) |
+                          reinterpret_cast<uintptr_t>(o)) & 15) != 0)
+        return LLMCAD_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
     CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
@@ -976,5 +983,50 @@ int llmcad_branch_pacer(const double *cum_conf, const int32_t *branch_len, int32
 }
 
 int64_t llmcad_launch_count(const llmcad_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int llmcad_set_wait_limit_ns(llmcad_ctx *ctx, uint64_t ns)
+{
+    if (ctx == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    ctx->wait_limit_ns = ns ? ns : kDefaultWaitLimitNs;
+    return LLMCAD_OK;
+}
+
+int llmcad_selftest_wait_timeout(llmcad_ctx *ctx, void *stream)
+{
+    if (ctx == nullptr) return LLMCAD_ERR_INVALID_ARG;
+    if (!ctx->tc_gemm || ctx->cfg.vocab < 160) return LLMCAD_ERR_UNSUPPORTED;
+    if (ctx->wait_limit_ns > 100000000ull) return LLMCAD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
+    CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    int rc = reset_chain_sync(ctx, st);
+    if (rc != LLMCAD_OK) return rc;
+    const int n_pad = 16;
+    if ((rc = ensure_act_maps(ctx, n_pad)) != LLMCAD_OK) return rc;
+    // Two dependent 256 x 128 GEMMs on 16 nodes. Weights: the first 64 KB of the context's logits
+    // buffer read as four pre-swizzled tiles (any bit pattern will do); input: the normalised
+    // activations; output: plain fp32 rows further up in the same buffer.
+    EpiParams ep{};
+    ep.mode = EPI_PLAIN; ep.n = n_pad; ep.n_out = 256; ep.ldy = 256;
+    ep.y = ctx->logits + (64 * 1024) / sizeof(float);
+    Chain ch;
+    for (int g = 0; g < 2; ++g) {
+        ch.maps.x[g] = ctx->act_maps[n_pad / 16][0];
+        ch.p.g[g] = make_gemm_desc(128, ep, ctx->logits);
+    }
+    ch.p.n_pad = n_pad;
+    ch.p.comp = ctx->comp ? 1 : 0;
+    ch.p.n_gemms = 2;
+    // the launch believes the barrier counter starts one higher than it does: the arrivals after the
+    // first GEMM never reach the target, and every wait at the barrier runs into the limit
+    ctx->barrier_base += 1;
+    rc = ch.launch(ctx, status, st);
+    if (rc != LLMCAD_OK) return rc;
+    int32_t v = 0;
+    CUDA_TRY(cudaMemcpyAsync(&v, status, sizeof(v), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    if ((rc = reset_chain_sync(ctx, st)) != LLMCAD_OK) return rc;
+    return v;
+}
 
 }  // extern "C"

@@ -92,8 +92,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait of one thread: gives up after kWaitLimitNs or when another role has raised `abort`.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+// Bounded wait of one thread: gives up after wait_limit ns or when another role has raised `abort`.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint64_t wait_limit)
 {
     if (mbar_try(bar, parity)) return true;
     uint64_t t0 = 0;
@@ -103,15 +103,15 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
         if ((it & 255u) == 0) {
             if (*abort_flag) return false;
             if (t0 == 0) t0 = global_timer_ns();
-            else if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+            else if (global_timer_ns() - t0 > wait_limit) return false;
         }
     }
 }
 // The same for a whole warp: lane 0 polls, the warp follows.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane)
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane, uint64_t wait_limit)
 {
     int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, wait_limit) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
@@ -298,7 +298,7 @@ __global__ void __launch_bounds__(kT5Threads, 1)
 attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_lo, int n_heads, int P,
                     int n, const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
-                    int32_t *status, unsigned long long *trace, int comp, int n_tree, int q_first)
+                    int32_t *status, unsigned long long *trace, int comp, int n_tree, int q_first, uint64_t wait_limit)
 {
     const int cta = blockIdx.y * gridDim.x + blockIdx.x;
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 0] = global_timer_ns();
@@ -351,6 +351,9 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
     const uint32_t tmem_base = ctl.tmem_base;
     volatile int *abort_flag = &ctl.abort_flag;
     bool failed = false;
+    // A pass whose tree or tokens an earlier phase refused (status word set) does no work here: every
+    // role looks at the word once the grid dependency has resolved, and all see the same value.
+    auto refused = [&]() { pdl_wait(); return *reinterpret_cast<const volatile int32_t *>(status) != 0; };
 
     if (warp == 0) {
         // ================================================= producer
@@ -384,13 +387,17 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
                 issue_kv(t++);
                 ++issued;
             }
-            pdl_wait();
+            if (refused()) {
+                // nothing will consume the tiles already requested: let them land before the ring goes away
+                for (int i = 0; i < issued; ++i) mbar_wait(smem_u32(&ctl.full[i]), 0, abort_flag, wait_limit);
+                t = t_end;
+            }
             for (; t < t_end && !failed; ++t) {
-                if (issued >= kStages && !mbar_wait(smem_u32(&ctl.empty[s]), par, abort_flag)) { failed = true; break; }
+                if (issued >= kStages && !mbar_wait(smem_u32(&ctl.empty[s]), par, abort_flag, wait_limit)) { failed = true; break; }
                 issue_kv(t);
                 ++issued;
                 if (comp && reaches_tree(t)) {
-                    if (issued >= kStages && !mbar_wait(smem_u32(&ctl.empty[s]), par, abort_flag)) { failed = true; break; }
+                    if (issued >= kStages && !mbar_wait(smem_u32(&ctl.empty[s]), par, abort_flag, wait_limit)) { failed = true; break; }
                     issue_lo(t);
                     ++issued;
                 }
@@ -398,7 +405,7 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
         }
     } else if (warp == 1) {
         // ================================================= MMA issuer of S = Q K^T
-        if (lane == 0 && T > 0) {
+        if (lane == 0 && T > 0 && !refused()) {
             constexpr uint32_t idesc_s = make_idesc(128, kKeyTile, false);
             int s = 0;
             uint32_t ph = 0;
@@ -407,12 +414,12 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
                 const int t = t_begin + i, b = i & 1;
                 const bool lo = comp && reaches_tree(t);
                 st_kv[i & 3] = s;
-                if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) return false;
+                if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag, wait_limit)) return false;
                 if (++s == kStages) { s = 0; ph ^= 1u; }
                 st_lo[i & 3] = -1;
                 if (lo) {
                     st_lo[i & 3] = s;
-                    if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) return false;
+                    if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag, wait_limit)) return false;
                     if (++s == kStages) { s = 0; ph ^= 1u; }
                 }
                 // (the softmax warps have read tile i - 2 out of this score buffer: their P of that tile, which
@@ -441,11 +448,11 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
                 tc_commit(smem_u32(&ctl.s_full[b]));
                 return true;
             };
-            if (!mbar_wait(smem_u32(&ctl.q_full), 0, abort_flag)) failed = true;
+            if (!mbar_wait(smem_u32(&ctl.q_full), 0, abort_flag, wait_limit)) failed = true;
             // Scores run two tiles ahead of the softmax: tile i goes into the buffer that the weights of
             // tile i - 2 have been computed from.
             for (int i = 0; i < T && !failed; ++i) {
-                if (i >= 2 && !mbar_wait(smem_u32(&ctl.p_full[i & 1]), (uint32_t)((i - 2) >> 1) & 1u, abort_flag)) { failed = true; break; }
+                if (i >= 2 && !mbar_wait(smem_u32(&ctl.p_full[i & 1]), (uint32_t)((i - 2) >> 1) & 1u, abort_flag, wait_limit)) { failed = true; break; }
                 if (!issue_s(i)) failed = true;
             }
         }
@@ -454,7 +461,7 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
         // A second issuing thread: a run of MMAs into one accumulator holds its thread for the ~420 cycles
         // of pipeline latency on top of the MMAs themselves, and two threads keep two runs (scores of a
         // later tile, P V of this one) in flight at once (measured: 1460 cycles for both against 1870 in turn).
-        if (lane == 0 && T > 0) {
+        if (lane == 0 && T > 0 && !refused()) {
             constexpr uint32_t idesc_o = make_idesc(128, kHd, true);
             int s = 0;                                    // walks the ring like the score issuer (it has waited for the copies)
             for (int i = 0; i < T && !failed; ++i) {
@@ -466,7 +473,7 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
                     s_lo = s;
                     if (++s == kStages) s = 0;
                 }
-                if (!mbar_wait(smem_u32(&ctl.p_full[i & 1]), (uint32_t)(i >> 1) & 1u, abort_flag)) { failed = true; break; }
+                if (!mbar_wait(smem_u32(&ctl.p_full[i & 1]), (uint32_t)(i >> 1) & 1u, abort_flag, wait_limit)) { failed = true; break; }
                 tc_fence_after();
                 const int b = i & 1;
                 const uint32_t d = tmem_base + kColO;
@@ -500,8 +507,9 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
         const int row = lg * 32 + lane;
         const bool warp_active = lg * 32 < n;             // a warp whose rows are all padding only keeps the barriers going
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
-        pdl_wait();
+        const bool skip = refused();
         if (trace && tid == 64 && cta < 256) trace[(size_t)cta * 16 + 1] = global_timer_ns();
+        if (!skip) {
         uint32_t a4[4] = {0, 0, 0, 0};
         if (row < n) {
 #pragma unroll
@@ -565,7 +573,7 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
         for (int i = 0; i < T; ++i) {
             const int t = t_begin + i, b = i & 1;
             const int key0 = t * kKeyTile;
-            if (!mbar_wait_warp(smem_u32(&ctl.s_full[b]), (uint32_t)(i >> 1) & 1u, abort_flag, lane)) { failed = true; break; }
+            if (!mbar_wait_warp(smem_u32(&ctl.s_full[b]), (uint32_t)(i >> 1) & 1u, abort_flag, lane, wait_limit)) { failed = true; break; }
             tc_fence_after();
             if (trace && tid == 64 && cta < 256 && i == 0) trace[(size_t)cta * 16 + 2] = global_timer_ns();
             float sc[kKeyTile];
@@ -595,13 +603,13 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
             }
             // P buffer b was last read by the P V of tile i - 2
             if (i > 1) {
-                if (!mbar_wait_warp(smem_u32(&ctl.o_full[b]), (uint32_t)((i - 2) >> 1) & 1u, abort_flag, lane)) { failed = true; break; }
+                if (!mbar_wait_warp(smem_u32(&ctl.o_full[b]), (uint32_t)((i - 2) >> 1) & 1u, abort_flag, lane, wait_limit)) { failed = true; break; }
             }
             if (warp_active) {
                 const bool move = tmax > ref + kSlack || (ref == -INFINITY && tmax > -INFINITY);
                 if (__any_sync(0xffffffffu, move)) {
                     // the outputs in TMEM are about to be rescaled: the P V of tile i - 1 must have retired
-                    if (i > 0 && !mbar_wait_warp(smem_u32(&ctl.o_full[b ^ 1]), (uint32_t)((i - 1) >> 1) & 1u, abort_flag, lane)) { failed = true; break; }
+                    if (i > 0 && !mbar_wait_warp(smem_u32(&ctl.o_full[b ^ 1]), (uint32_t)((i - 1) >> 1) & 1u, abort_flag, lane, wait_limit)) { failed = true; break; }
                     tc_fence_after();
                     const float factor = !move ? 1.f : (ref == -INFINITY ? 0.f : ex2(ref - tmax));
                     if (move) ref = tmax;
@@ -638,7 +646,7 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
         }
         // the last two tiles' P V
         for (int i = max(0, T - 2); i < T && !failed; ++i)
-            if (!mbar_wait_warp(smem_u32(&ctl.o_full[i & 1]), (uint32_t)(i >> 1) & 1u, abort_flag, lane)) failed = true;
+            if (!mbar_wait_warp(smem_u32(&ctl.o_full[i & 1]), (uint32_t)(i >> 1) & 1u, abort_flag, lane, wait_limit)) failed = true;
         tc_fence_after();
         if (trace && tid == 64 && cta < 256) trace[(size_t)cta * 16 + 3] = global_timer_ns();
         // every copy has landed and every MMA has retired (the last o_full): the ring is free for the
@@ -662,6 +670,7 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
             }
             if (row < n) *reinterpret_cast<float2 *>(pr + kHd) = make_float2(ref, l);
         }
+        }
         tc_fence_before();
     }
     if (failed) {
@@ -674,7 +683,8 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
-    const bool bad = ctl.abort_flag != 0;
+    // (the softmax warps have passed the grid dependency, so the status word is final for every thread)
+    const bool bad = ctl.abort_flag != 0 || *reinterpret_cast<const volatile int32_t *>(status) != 0;
 
     // four outputs of one row, normalised, as bf16 hi (and lo) to global memory
     auto store4 = [&](int row, int dim, float4 a, float inv) {
@@ -719,7 +729,7 @@ bool attention_prefers_t5(int n)
 
 cudaError_t launch_attention_t5(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, int n_sms, int32_t *status, cudaStream_t st,
-                                int *launched, unsigned long long *trace, int comp, const void *kv_lo, int n_tree, int q_first)
+                                int *launched, unsigned long long *trace, int comp, const void *kv_lo, int n_tree, int q_first, uint64_t wait_limit_ns)
 {
     if (n_tree <= 0) n_tree = n;
     if (hd != kHd || n < 1 || n > 128 || P + n_tree > kv_stride) return cudaErrorInvalidValue;
@@ -749,16 +759,16 @@ cudaError_t launch_attention_t5(const void *q, const void *k, const void *v, int
     } else {
         ml = mk;      // never dereferenced without compensation
     }
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    if (attr_set.needed()) {
         cudaError_t e = cudaFuncSetAttribute(attention_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set.mark();
     }
     LaunchCfg lc(dim3(splits, n_heads), dim3(kT5Threads), kSmemBytes, st, splits);
     if (launched) *launched = 1;
     return cudaLaunchKernelEx(&lc.cfg, attention_t5_kernel, (const __nv_bfloat16 *)q, mk, mv, ml, n_heads, P, n, anc, (__nv_bfloat16 *)o, splits,
-                              tiles_per_split, status, trace, comp, n_tree, q_first);
+                              tiles_per_split, status, trace, comp, n_tree, q_first, wait_limit_ns);
 }
 
 }  // namespace llmcad

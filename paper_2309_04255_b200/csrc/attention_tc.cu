@@ -484,15 +484,15 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
                          const __nv_bfloat16 *, int, int);
     static const Kern kerns[2][3] = {{attention_tc_kernel<1, false>, attention_tc_kernel<2, false>, attention_tc_kernel<4, false>},
                                      {attention_tc_kernel<1, true>, attention_tc_kernel<2, true>, attention_tc_kernel<4, true>}};
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    if (attr_set.needed()) {
         const int max_smem = 2 * 128 * kRowBytes + 2 * 3 * kKeyTile * kRowBytes + 2 * 129 * kRowBytes;   // 128 nodes, hi + lo
         for (int c = 0; c < 2; ++c)
             for (int g = 0; g < 3; ++g) {
                 cudaError_t e = cudaFuncSetAttribute(kerns[c][g], cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
                 if (e != cudaSuccess) return e;
             }
-        attr_set = true;
+        attr_set.mark();
     }
     LaunchCfg lc(dim3(splits, n_heads), dim3(kAtThreads), smem, st, splits);
     if (launched) *launched = 1;

@@ -22,7 +22,7 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
 cudaError_t launch_attention_t5(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, int n_sms, int32_t *status, cudaStream_t st,
                                 int *launched, unsigned long long *trace = nullptr, int comp = 0, const void *kv_lo = nullptr,
-                                int n_tree = 0, int q_first = 0);
+                                int n_tree = 0, int q_first = 0, uint64_t wait_limit_ns = kDefaultWaitLimitNs);
 
 // Which of the two serves a tree of n query rows by default: the tcgen05 kernel above 32 rows (measured on
 // B200 in whole passes of the 7B shape: 1-3 % of the pass faster at 33-64 nodes, 4-8 % at 96-128; at 32 nodes

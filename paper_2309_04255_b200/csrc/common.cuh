@@ -138,7 +138,7 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t) :: "memory");   // the clobber keeps the read where it is written
     return t;
 }
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every device-side wait gives up after 2 s
+constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;  // every device-side wait gives up after 2 s unless the context says otherwise
 
 // ---------------------------------------------------------------- programmatic dependent launch
 // Every kernel of the pass is launched with programmatic stream serialization: it lets its
@@ -170,6 +170,19 @@ struct LaunchCfg {
         }
         cfg.attrs = attrs;
     }
+};
+
+// A function attribute (cudaFuncSetAttribute) belongs to the device it was set on: remember per device
+// whether a launcher has done its one-time set-up there.
+struct PerDeviceOnce {
+    bool done[64] = {};
+    int dev = -1;
+    bool needed()
+    {
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { dev = -1; return true; }
+        return !done[dev];
+    }
+    void mark() { if (dev >= 0) done[dev] = true; }
 };
 
 // ---------------------------------------------------------------- launchers (host)

@@ -78,8 +78,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kWaitLimitNs or as soon as another role has raised `abort`.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+// Bounded wait: gives up after wait_limit ns or as soon as another role has raised `abort`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint64_t wait_limit)
 {
     if (mbar_try(bar, parity)) return true;
     uint64_t t0 = 0;
@@ -90,7 +90,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if ((it & 255u) == 0) {
             if (*abort_flag) return false;
             if (t0 == 0) t0 = global_timer_ns();
-            else if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+            else if (global_timer_ns() - t0 > wait_limit) return false;
         }
     }
 }
@@ -99,7 +99,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // polls, with a short sleep between polls, and the warp follows. A warp of 32 hot pollers per
 // barrier would saturate the shared-memory pipeline that the producer's copies and barrier
 // operations also go through.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane)
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int lane, uint64_t wait_limit)
 {
     int ok = 1;
     if (lane == 0 && !mbar_try(bar, parity)) {
@@ -107,7 +107,7 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
         for (uint32_t it = 1;; ++it) {
             __nanosleep(40);
             if (mbar_try(bar, parity)) break;
-            if ((it & 63u) == 0 && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) { ok = 0; break; }
+            if ((it & 63u) == 0 && (*abort_flag || global_timer_ns() - t0 > wait_limit)) { ok = 0; break; }
         }
     }
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
@@ -548,6 +548,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t acc_cols = 2u * nb;                    // TMEM columns of one accumulator buffer (gate | up)
     const bool two_bufs = p.acc_bufs == 2;
+    const uint64_t wait_limit = p.wait_limit_ns;          // every wait below gives up after this many ns
 
     // Let the next kernel of the stream start early. This kernel in turn must not read activations,
     // the status word or the workspace, nor write anything, before pdl_wait(): until then it only
@@ -652,7 +653,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 }
                 __nanosleep(32);
                 if (t_idle == 0) t_idle = global_timer_ns();
-                else if (*abort_flag || global_timer_ns() - t_idle > kWaitLimitNs) { timed_out = true; break; }
+                else if (*abort_flag || global_timer_ns() - t_idle > wait_limit) { timed_out = true; break; }
             }
             if (p.n_gemms == 1) LLMCAD_TRACE(6);
         }
@@ -676,7 +677,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     __nanosleep(32);
                     if ((spin & 255u) == 255u) {
                         if (t0 == 0) t0 = global_timer_ns();
-                        if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) { timed_out = true; break; }
+                        if (*abort_flag || global_timer_ns() - t0 > wait_limit) { timed_out = true; break; }
                     }
                 }
                 // (2) the GEMM's input is final on every CTA
@@ -686,7 +687,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     if (c.g > ready) {
                         __nanosleep(100);
                         if (t0 == 0) t0 = global_timer_ns();
-                        if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) timed_out = true;
+                        if (*abort_flag || global_timer_ns() - t0 > wait_limit) timed_out = true;
                     }
                 }
                 if (timed_out) break;
@@ -716,11 +717,11 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 const int cg = c.g, tile = c.tile, halves = c.halves;
                 const int buf = two_bufs ? (seg & 1) : 0;
                 const uint32_t use = two_bufs ? (seg >> 1) : seg;     // how often this buffer has been used before
-                if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, abort_flag)) { timed_out = true; break; }
+                if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, abort_flag, wait_limit)) { timed_out = true; break; }
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + buf * acc_cols;
                 for (int q = 0; c.g == cg && c.tile == tile; ++q) {
-                    if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag)) { timed_out = true; break; }
+                    if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag, wait_limit)) { timed_out = true; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * stage_bytes;
                     // segments of a two-half GEMM start on a gate item, so the first `halves` items
@@ -770,7 +771,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     const uint64_t t0 = global_timer_ns();
                     for (uint32_t spin = 0; (int32_t)(ld_acquire_u32(p.grid_counter) - p.barrier_base - target) < 0; ++spin) {
                         __nanosleep(100);
-                        if ((spin & 15u) == 15u && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) { bad = 1; break; }
+                        if ((spin & 15u) == 15u && (*abort_flag || global_timer_ns() - t0 > wait_limit)) { bad = 1; break; }
                     }
                     __threadfence();
                 }
@@ -845,7 +846,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     rs_ready = true;
                 }
 
-                if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), use & 1u, abort_flag, lane)) { timed_out = true; break; }
+                if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), use & 1u, abort_flag, lane, wait_limit)) { timed_out = true; break; }
                 tc_fence_after();
                 if (threadIdx.x == 64 && g < 4 && seg_begin == r.begin) LLMCAD_TRACE(4 + 2 * g);
                 if (threadIdx.x == 64 && tail) LLMCAD_TRACE(14);
@@ -929,7 +930,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                                 __nanosleep(64);
                                 if ((spin & 15u) == 15u) {
                                     if (t0 == 0) t0 = global_timer_ns();
-                                    else if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) { bad = 1; break; }
+                                    else if (*abort_flag || global_timer_ns() - t0 > wait_limit) { bad = 1; break; }
                                 }
                             }
                         }
@@ -982,7 +983,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     __nanosleep(ctl.dumped[lane_grp] == 0 ? 200 : 64);
                     if ((spin & 15u) == 15u) {
                         if (t0 == 0) t0 = global_timer_ns();
-                        else if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) { bad = 1; break; }
+                        else if (*abort_flag || global_timer_ns() - t0 > wait_limit) { bad = 1; break; }
                     }
                 }
                 __threadfence_block();
@@ -1105,8 +1106,19 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
     // single k-blocks cost 10-17 % up to 64 nodes and gain 6 % at 128.
     const int nb = p.n_pad * (p.comp ? 2 : 1);       // MMA N
     if (nb > 256) return cudaErrorInvalidValue;
+    // tuning aids from the environment, read once per process
+    struct Tuning {
+        int pair_k = 0, stages_cap = 0, l2_ahead = 8;
+        Tuning()
+        {
+            if (const char *e = getenv("LLMCAD_GEMM_PAIR_K")) { const int v = atoi(e); if (v == 1 || v == 2) pair_k = v; }
+            if (const char *e = getenv("LLMCAD_GEMM_STAGES")) { const int v = atoi(e); if (v >= 2) stages_cap = v; }
+            if (const char *e = getenv("LLMCAD_GEMM_L2_AHEAD")) l2_ahead = atoi(e);
+        }
+    };
+    static const Tuning tune;
     int pair_k = nb > 128 ? 1 : kMaxPairK;
-    if (const char *e = getenv("LLMCAD_GEMM_PAIR_K")) { const int v = atoi(e); if (v == 1 || v == 2) pair_k = v; }   // tuning aid
+    if (tune.pair_k) pair_k = tune.pair_k;
     for (int g = 0; g < p.n_gemms; ++g) p.g[g].pair_k = pair_k;
     auto items_of = [](const GemmDesc &d) { return (long long)d.n_tiles * pairs_per_tile(d) * d.halves; };
     for (int g = 0; g < p.n_gemms; ++g) {
@@ -1137,26 +1149,23 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
     const size_t full_limit = 227 * 1024 - 1024 /*alignment slack*/ - 4096 /*static*/;
     int stages = (int)(full_limit / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
-    if (const char *e = getenv("LLMCAD_GEMM_STAGES")) {   // tuning aid: cap the ring depth
-        const int cap = atoi(e);
-        if (cap >= 2 && cap < stages) stages = cap;
-    }
+    if (tune.stages_cap && tune.stages_cap < stages) stages = tune.stages_cap;   // tuning aid: cap the ring depth
     if (stages < 2) return cudaErrorInvalidConfiguration;
     p.stages = stages;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    if (attr_set.needed()) {
         cudaError_t e = cudaFuncSetAttribute(gemm_chain_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              227 * 1024 - 4096);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(gemm_chain_kernel<__nv_bfloat16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      227 * 1024 - 4096);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set.mark();
     }
     // weight tiles pulled into L2 beyond the ring while the ring is blocked
-    p.l2_ahead = 8;
-    if (const char *e = getenv("LLMCAD_GEMM_L2_AHEAD")) p.l2_ahead = atoi(e);
+    p.l2_ahead = tune.l2_ahead;
+    if (p.wait_limit_ns == 0) p.wait_limit_ns = kDefaultWaitLimitNs;
     if (barrier_arrivals) *barrier_arrivals = 4u * (uint32_t)grid * (uint32_t)(p.n_gemms - 1);
     LaunchCfg lc(grid, kThreads, smem, st);
     if (pair_k == 1) return cudaLaunchKernelEx(&lc.cfg, gemm_chain_kernel<__nv_bfloat16, 1>, maps, p);

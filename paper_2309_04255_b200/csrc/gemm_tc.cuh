@@ -44,6 +44,7 @@ struct ChainParams {
     int32_t *status;
     unsigned long long *trace;  // optional [grid][16] timeline in ns (nullptr: off)
     int l2_ahead;       // ring items the producer may prefetch into L2 beyond the ring
+    uint64_t wait_limit_ns;   // bound of every device-side wait of the launch
     GemmDesc g[kMaxChain];
 };
 

@@ -45,6 +45,12 @@ extern "C" int llmcad_tree_attention_noalloc(const void *q, const void *k, const
         return LLMCAD_ERR_UNSUPPORTED;
     }
     if (n_heads > 65535) { snprintf(g_err, sizeof(g_err), "n_heads=%d exceeds 65535", n_heads); return LLMCAD_ERR_UNSUPPORTED; }
+    // the kernels move rows as 16-byte vectors and bulk copies: a misaligned buffer would fault on the device
+    if (((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(v) |
+          reinterpret_cast<uintptr_t>(o)) & 15) != 0) {
+        snprintf(g_err, sizeof(g_err), "q, k, v and o must be 16-byte aligned");
+        return LLMCAD_ERR_INVALID_ARG;
+    }
 
     // Set-up, once per device, with that device current: in host code the array's name is only a
     // stand-in, the address the kernels need comes from the runtime.

@@ -8,8 +8,8 @@ here.
 The paper evaluates on public text datasets with trained checkpoints; none of
 that is available offline, so every input is synthetic:
 
-* weights ~ N(0, 0.02), one independent stream per (layer, tensor), rounded to
-  bf16 for the bf16 configurations; RMSNorm gains are 1.0;
+* weights ~ N(0, 0.02), one independent stream per (layer, tensor, block of 1024
+  rows), rounded to bf16 for the bf16 configurations; RMSNorm gains are 1.0;
 * prefix K/V ~ N(0, 1) (the natural scale of q = x_hat W with std 0.02 sqrt(d));
 * draft trees follow the paper's draft rule (a successor opens a branch when its
   confidence exceeds ~30 %, hence at most 3-4 children per node; branches are
@@ -115,15 +115,37 @@ def tensor_shape(cfg: ModelConfig, name: str):
     }[name]
 
 
+_GEN_BLOCK_ROWS = 1024      # rows per independent random stream of a weight matrix
+_gen_pool = None
+
+
+def _gen_block(shape, key, r0, r1, out):
+    g = _rng(*key, r0 // _GEN_BLOCK_ROWS)
+    a = g.standard_normal((r1 - r0, *shape[1:]), dtype=np.float32)
+    a *= np.float32(0.02)
+    out[r0:r1] = a
+
+
 def gen_tensor(cfg: ModelConfig, name: str, layer: int = -1, seed: int = 0) -> torch.Tensor:
-    """One weight tensor, row-major [out][in], in the config's storage dtype (CPU)."""
+    """One weight tensor, row-major [out][in], in the config's storage dtype (CPU). A matrix is drawn
+    in blocks of 1024 rows, each from its own stream keyed by (seed, layer, tensor, block), so that
+    the blocks of a large matrix can be drawn on all host cores at once."""
+    global _gen_pool
     shape = tensor_shape(cfg, name)
     if name.endswith("norm"):
         return _to_dtype(np.ones(shape, dtype=np.float32), cfg.dtype)
-    g = _rng(seed, layer + 1, _TID[name])
-    a = g.standard_normal(shape, dtype=np.float32)
-    a *= np.float32(0.02)
-    return _to_dtype(a, cfg.dtype)
+    key = (seed, layer + 1, _TID[name])
+    out = np.empty(shape, dtype=np.float32)
+    blocks = [(r0, min(shape[0], r0 + _GEN_BLOCK_ROWS)) for r0 in range(0, shape[0], _GEN_BLOCK_ROWS)]
+    if len(blocks) == 1:
+        _gen_block(shape, key, 0, shape[0], out)
+    else:
+        if _gen_pool is None:
+            import os
+            from concurrent.futures import ThreadPoolExecutor
+            _gen_pool = ThreadPoolExecutor(len(os.sched_getaffinity(0)))
+        list(_gen_pool.map(lambda b: _gen_block(shape, key, b[0], b[1], out), blocks))
+    return _to_dtype(out, cfg.dtype)
 
 
 def gen_layer(cfg: ModelConfig, layer: int, seed: int = 0) -> Dict[str, torch.Tensor]:

@@ -45,11 +45,38 @@ def time_launches(fn, n_variants, reps, warmup):
     return e0.elapsed_time(e1) * 1e3 / reps      # microseconds per launch
 
 
+def attention_cell(v, P, n, parent, reps, warmup, l2_resident=True):
+    """One (prefix, tree size) case of the attention-only sweep on verifier `v` (32 heads x 128)."""
+    H, hd = v.cfg.n_heads, v.cfg.head_dim
+    dev = v.device
+    kv_bytes = 2 * H * (P + n) * hd * 2
+    io_bytes = kv_bytes + 2 * n * H * hd * 2
+    nbuf = max(2, int(2 * L2_BYTES // kv_bytes) + 1)      # rotate over > 2 x L2 of K/V
+    g = torch.Generator(device=dev)
+    g.manual_seed(gen.MASTER_SEED + P + n)
+    ks = [torch.randn((H, P + n, hd), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16) for _ in range(nbuf)]
+    vs = [torch.randn((H, P + n, hd), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16) for _ in range(nbuf)]
+    q = torch.randn((n, H, hd), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    par = torch.as_tensor(parent, device=dev)
+    us = time_launches(lambda i: v.tree_attention(q, ks[i], vs[i], P, par), nbuf, reps, warmup)
+    us_l2 = time_launches(lambda i: v.tree_attention(q, ks[0], vs[0], P, par), 1, reps, warmup) if l2_resident else None
+    assert v.last_status() == 0
+    # each call is tree-prep + attention; the attention kernel's share is timed by its own events
+    v.set_kernel_timing(True)
+    for i in range(reps):
+        v.tree_attention(q, ks[i % nbuf], vs[i % nbuf], P, par)
+    ms, cnt = v.get_kernel_timing(1)
+    v.set_kernel_timing(False)
+    k_us = ms * 1e3 / max(cnt, 1)
+    return {"algorithmic_bytes": io_bytes, "us_per_call_hbm": us, "us_per_call_l2_resident": us_l2,
+            "us_attention_kernel": k_us, "hbm_gbs": io_bytes / k_us / 1e3,
+            "flops": 4 * n * (P + n) * H * hd, "tflops": 4 * n * (P + n) * H * hd / k_us / 1e6}
+
+
 def bench_attention(args):
     H, hd = 32, 128
     cfg = gen.ModelConfig("attn", 0, H * hd, H, hd, 256, 512, "bf16")
     v = B.Verifier(cfg, 16)
-    dev = v.device
     peak, kind = _peak()
     prefixes = [int(x) for x in args.prefix.split(",")]
     sizes = [int(x) for x in args.nodes.split(",")]
@@ -62,32 +89,9 @@ def bench_attention(args):
                     parent = gen.tree_star(n)
                 else:
                     parent = gen.tree_random(n, 16, "uniform4", int(topo)) if n > 1 else np.array([-1], np.int32)
-                kv_bytes = 2 * H * (P + n) * hd * 2
-                io_bytes = kv_bytes + 2 * n * H * hd * 2
-                nbuf = max(2, int(2 * L2_BYTES // kv_bytes) + 1)      # rotate over > 2 x L2 of K/V
-                g = torch.Generator(device=dev)
-                g.manual_seed(gen.MASTER_SEED + P + n)
-                ks = [torch.randn((H, P + n, hd), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16) for _ in range(nbuf)]
-                vs = [torch.randn((H, P + n, hd), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16) for _ in range(nbuf)]
-                q = torch.randn((n, H, hd), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
-                par = torch.as_tensor(parent, device=dev)
-                us = time_launches(lambda i: v.tree_attention(q, ks[i], vs[i], P, par), nbuf, args.reps, args.warmup)
-                us_l2 = time_launches(lambda i: v.tree_attention(q, ks[0], vs[0], P, par), 1, args.reps, args.warmup)
-                assert v.last_status() == 0
-                # each call is tree-prep + attention; the attention kernel's share is timed by its own events
-                v.set_kernel_timing(True)
-                for i in range(args.reps):
-                    v.tree_attention(q, ks[i % nbuf], vs[i % nbuf], P, par)
-                ms, cnt = v.get_kernel_timing(1)
-                v.set_kernel_timing(False)
-                k_us = ms * 1e3 / max(cnt, 1)
-                print(json.dumps({
-                    "kernel": "tree_attention", "prefix": P, "nodes": n, "topology": topo, "heads": H, "head_dim": hd,
-                    "algorithmic_bytes": io_bytes, "us_per_call_hbm": us, "us_per_call_l2_resident": us_l2,
-                    "us_attention_kernel": k_us, "hbm_gbs": io_bytes / k_us / 1e3, "peak_gbs": peak, "peak": kind,
-                    "frac": io_bytes / k_us / 1e3 / peak,
-                    "flops": 4 * n * (P + n) * H * hd, "tflops": 4 * n * (P + n) * H * hd / k_us / 1e6}), flush=True)
-                del ks, vs
+                c = attention_cell(v, P, n, parent, args.reps, args.warmup)
+                print(json.dumps({"kernel": "tree_attention", "prefix": P, "nodes": n, "topology": topo, "heads": H, "head_dim": hd,
+                                  **c, "peak_gbs": peak, "peak": kind, "frac": c["hbm_gbs"] / peak}), flush=True)
 
 
 def bench_gemm(args):

@@ -223,6 +223,30 @@ def test_error_paths():
     assert out["scalars"][B.S_STATUS] == 0 and out["scalars"][B.S_ACCEPTED_LEN] >= 1
 
 
+def test_bounded_wait_runs_out_and_the_context_survives():
+    """The failure path of the device-side waits: with the limit lowered to 1 ms, a GEMM chain whose
+    grid barrier cannot complete (a host-side set-up, nothing faults) gives up, reports TIMEOUT in the
+    status word, frees its tensor memory and returns; the same context then runs a pass that is bit
+    for bit what it produced before."""
+    twin, parent, tokens = bf16_case(SMALL_BF16, 40, 20, 6, "uniform4", seed=8, scale=3.0)
+    before = twin.gpu_pass(40, tokens, parent)
+    assert before["scalars"][B.S_STATUS] == 0
+    with pytest.raises(B.LlmcadError) as e:          # refuses to run with the default limit of 2 s
+        twin.v.selftest_wait_timeout()
+    assert e.value.code == B.ERR_INVALID_ARG
+    twin.v.set_wait_limit_ns(1_000_000)
+    import time
+    t0 = time.perf_counter()
+    assert twin.v.selftest_wait_timeout() == B.ERR_TIMEOUT
+    assert time.perf_counter() - t0 < 1.0            # the kernel came back after ~1 ms + its 2 ms drain
+    assert twin.v.selftest_wait_timeout() == B.ERR_TIMEOUT     # and again: the counters start from zero every time
+    twin.v.set_wait_limit_ns(0)
+    after = twin.gpu_pass(40, tokens, parent)
+    assert after["scalars"][B.S_STATUS] == 0
+    assert np.array_equal(after["logits"], before["logits"]) and np.array_equal(after["argmax"], before["argmax"])
+    assert np.array_equal(after["scalars"], before["scalars"])
+
+
 def test_host_entry_equals_device_entry():
     twin, parent, tokens = bf16_case(SMALL_BF16, 40, 20, 6, "uniform4", seed=8, scale=3.0)
     a = twin.gpu_pass(40, tokens, parent)

@@ -197,6 +197,58 @@ def test_tree_attention(case, mode):
     assert np.abs(got - ref).max() <= tol * np.abs(ref).max()
 
 
+# Config 4 at its own head count and its extreme prefix lengths: with 32 heads there are fewer key
+# splits per head than in the 4-head cases above, so the cluster and merge shapes differ.
+C4_CASES = [(P, n, "random") for P in (256, 8192) for n in (8, 32, 64, 128)] + [(8192, 128, "chain"), (8192, 128, "star")]
+
+
+@pytest.mark.parametrize("case", C4_CASES)
+@pytest.mark.parametrize("mode", ["bf16_mma", "bf16_t5"])
+def test_tree_attention_config4(case, mode):
+    """32 heads x 128, prefix 256 and 8192, trees of 8..128 nodes (random, chain, star), each tensor
+    kernel pinned, element by element against the oracle."""
+    P, n, shape = case
+    H, hd = 32, 128
+    cfg = gen.ModelConfig("a", 0, H * hd, H, hd, 256, 512, "bf16")
+    v = B.Verifier(cfg, 16, flags={"bf16_mma": B.FLAG_MMA_ATTN, "bf16_t5": B.FLAG_T5_ATTN}[mode])
+    parent = {"random": lambda: gen.tree_random(n, 12, "uniform4", P + n), "chain": lambda: gen.tree_chain(n),
+              "star": lambda: gen.tree_star(n)}[shape]()
+    q, k, vv = gen.gen_attention_inputs(H, hd, P, n, seed=2, dtype="bf16")
+    o = v.tree_attention(q.to(DEV), k.to(DEV), vv.to(DEV), P, dev_i32(parent))
+    assert v.last_status() == 0
+    _, _, _, anc = orc.tree_prep(parent, P)
+    tk = k[:, P:].permute(1, 0, 2).reshape(n, H * hd)
+    tv = vv[:, P:].permute(1, 0, 2).reshape(n, H * hd)
+    ref = orc.tree_attention(q.reshape(n, H * hd), k[:, :P], vv[:, :P], tk, tv, anc, H, hd)
+    got = o.double().cpu().numpy().reshape(n, H * hd)
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref).max() <= 2e-2 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("mode", ["bf16_mma", "bf16_t5"])
+def test_tree_attention_refuses_a_malformed_tree_of_40_nodes(mode):
+    """Above 32 nodes the default kernel is the tcgen05 one: it too must leave o alone and report the tree."""
+    P, n, H, hd = 70, 40, 4, 128
+    cfg = gen.ModelConfig("a", 0, H * hd, H, hd, 256, 512, "bf16")
+    v = B.Verifier(cfg, 16, flags={"bf16_mma": B.FLAG_MMA_ATTN, "bf16_t5": B.FLAG_T5_ATTN}[mode])
+    parent = gen.tree_random(n, 12, "uniform4", 5)
+    parent[35] = 37                                    # a parent that comes after its child
+    q, k, vv = gen.gen_attention_inputs(H, hd, P, n, seed=4, dtype="bf16")
+    o = torch.full((n, H, hd), 7.0, dtype=torch.bfloat16, device=DEV)
+    v.tree_attention(q.to(DEV), k.to(DEV), vv.to(DEV), P, dev_i32(parent), o=o)
+    assert v.last_status() == B.ERR_BAD_TREE
+    assert (o == 7.0).all()                            # nothing was written
+    # a well-formed call afterwards works and differs from what the refused call left behind
+    parent[35] = 3
+    o2 = v.tree_attention(q.to(DEV), k.to(DEV), vv.to(DEV), P, dev_i32(parent))
+    assert v.last_status() == 0 and torch.isfinite(o2.float()).all()
+    # misaligned buffers are refused on the host
+    qd = torch.zeros(n * H * hd + 8, dtype=torch.bfloat16, device=DEV)[4:4 + n * H * hd].view(n, H, hd)
+    with pytest.raises(B.LlmcadError) as e:
+        v.tree_attention(qd, k.to(DEV), vv.to(DEV), P, dev_i32(parent))
+    assert e.value.code == B.ERR_INVALID_ARG
+
+
 def test_attention_head_dim_64_f32():
     P, n, H, hd = 40, 15, 4, 64
     cfg = gen.ModelConfig("a", 0, H * hd, H, hd, 256, 512, "f32")

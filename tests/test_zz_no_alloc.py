@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as orc
 from paper_2309_04255_b200 import binding as B
 from paper_2309_04255_b200 import inputs as gen
 
@@ -30,15 +31,31 @@ def test_noalloc_matches_regular_entry_point_twice():
         want = ref.tree_attention(q, k, v, P, parent)
         got = torch.full_like(q, float("nan"))
         status = torch.full((1,), -7, dtype=torch.int32, device=dev)
-        before = torch.cuda.memory_allocated(dev)
+        if seed == 1:
+            # the very first call loads the kernels' module and looks up the scratch address; what
+            # must not allocate is every call, so the free-memory reading brackets a call after it
+            B.tree_attention_noalloc(q, k, v, P, parent, got, status)
+            torch.cuda.synchronize()
+            got.fill_(float("nan"))
+        # free device memory as the driver reports it (cudaMemGetInfo): an allocation by the
+        # library itself, which torch's own counters cannot see, would lower it
+        free_before, _ = torch.cuda.mem_get_info(dev)
         B.tree_attention_noalloc(q, k, v, P, parent, got, status)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated(dev) == before
+        free_after, _ = torch.cuda.mem_get_info(dev)
+        assert free_after == free_before
         assert int(status.item()) == 0
         g, w = got.float().cpu().numpy(), want.float().cpu().numpy()
         assert np.isfinite(g).all()
         assert np.abs(g - w).max() <= 2e-2 * np.abs(w).max()
         assert np.array_equal(g, w)              # same kernels on the same inputs
+        # and directly against the CPU oracle's tree attention
+        par = parent.cpu().numpy()
+        _, _, _, anc = orc.tree_prep(par, P)
+        kc, vc = k.cpu(), v.cpu()
+        ref_o = orc.tree_attention(q.cpu().reshape(n, H * hd), kc[:, :P], vc[:, :P], kc[:, P:].permute(1, 0, 2).reshape(n, H * hd),
+                                   vc[:, P:].permute(1, 0, 2).reshape(n, H * hd), anc, H, hd)
+        assert np.abs(got.double().cpu().numpy().reshape(n, H * hd) - ref_o).max() <= 2e-2 * np.abs(ref_o).max()
     # a malformed tree is reported through the status word, which the previous calls left at 0
     bad = torch.as_tensor(np.array([-1, 2, 0], np.int32), device=dev)
     q, k, v = (t.to(dev) for t in gen.gen_attention_inputs(H, hd, 5, 3, seed=3))
@@ -51,6 +68,20 @@ def test_noalloc_matches_regular_entry_point_twice():
     B.tree_attention_noalloc(q, k, v, 5, good, torch.empty_like(q), status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    # the same with a tree large enough for the tcgen05 kernel: refused, and o left as it was
+    n = 40
+    par = gen.tree_random(n, 12, "uniform4", 9)
+    par[30] = 33
+    q, k, v = (t.to(dev) for t in gen.gen_attention_inputs(H, hd, 20, n, seed=5))
+    o = torch.full_like(q, 7.0)
+    B.tree_attention_noalloc(q, k, v, 20, torch.as_tensor(par, device=dev), o, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.ERR_BAD_TREE and bool((o == 7.0).all())
+    # buffers the kernels could not read as 16-byte vectors are refused before anything is launched
+    flat = torch.zeros(q.numel() + 8, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(B.LlmcadError) as e:
+        B.tree_attention_noalloc(flat[4:4 + q.numel()].view(q.shape), k, v, 20, torch.as_tensor(par, device=dev), o, status)
+    assert e.value.code == B.ERR_INVALID_ARG
 
 
 def test_noalloc_rejects_sizes_beyond_the_static_scratch():
