@@ -23,27 +23,29 @@ int llmcad_set_kernel_timing(llmcad_ctx *ctx, int32_t enable);
 int llmcad_get_kernel_timing(llmcad_ctx *ctx, int32_t kind, double *total_ms /*HOST*/, int64_t *n_launches /*HOST*/);
 
 /* Timeline of the kernels inside an undisturbed pass. While `trace` (DEVICE, [capacity][256][16]
- * uint64, or NULL to stop) is set, the next `capacity` tensor-core GEMM and attention launches of
- * this context each fill one [256][16] slice: per CTA, nanosecond timestamps (%globaltimer) of
- * entry (0), set-up done (1), grid dependency resolved (3), per chained GEMM g first accumulator
- * ready (4+2g) and epilogue done (5+2g), exit (12). Launch order of a pass: QKV GEMM, then per
- * layer attention, O, gate/up, down, next QKV (lm_head after the last layer). The stamps cost a
- * predicated store each and do not change how consecutive kernels overlap. */
+ * uint64, or NULL to stop) is set, the next `capacity` tensor-core GEMMs and attention launches of
+ * this context each fill one [256][16] slice: per CTA, nanosecond timestamps (%globaltimer). A GEMM
+ * (streaming kernel + finishing kernel) shares one slice: streaming CTA entry (0), set-up done (1),
+ * first weight copy issued (2), grid dependency resolved (3), first accumulator ready (4), last
+ * weight copy issued (6), last MMA issued (7), accumulators in the workspace (8), streaming CTA
+ * exit (13); finishing CTA entry (9), its grid dependency resolved (10), exit (12). Attention:
+ * entry (0), exit (12). Launch order of a pass: QKV GEMM, then per layer attention, O, gate/up,
+ * down, next QKV (lm_head after the last layer). The stamps cost a predicated store each and do not
+ * change how consecutive kernels overlap. */
 int llmcad_set_gemm_trace(llmcad_ctx *ctx, uint64_t *trace, int32_t capacity);
 
 /* Number of kernels this library has launched through this context so far. */
 int64_t llmcad_launch_count(const llmcad_ctx *ctx);
 
-/* Every device-side wait of this context's kernels (shared-memory barriers, arrival counters of
- * the GEMM tails, the grid barrier of chained GEMMs) gives up after `ns` nanoseconds; the kernel
+/* Every device-side wait of this context's kernels (the shared-memory barriers between the roles of
+ * a CTA; no kernel waits for another CTA) gives up after `ns` nanoseconds; the kernel
  * then sets LLMCAD_ERR_TIMEOUT in the status word, lets all its roles fall out of their loops,
  * frees its tensor memory and returns. Default 2 s; 0 restores the default. */
 int llmcad_set_wait_limit_ns(llmcad_ctx *ctx, uint64_t ns);
 
-/* Self-test of that path (bf16 tensor-core contexts only, vocab >= 160): runs a small chain of two
- * dependent GEMMs on the context's own work buffers whose grid barrier is set up so that it can
- * never complete (the launch is told that the barrier counter starts one higher than it does), so
- * the waits at the barrier run out. Nothing faults or traps: the kernel returns after the wait
+/* Self-test of that path (bf16 tensor-core contexts only, vocab >= 160): runs a small GEMM on the
+ * context's own work buffers whose activation copies are withheld (a launch flag), so that its ring
+ * stages never fill and every role's wait runs out. Nothing faults or traps: the kernel returns after the wait
  * limit (set a short one first: the call refuses limits above 100 ms with LLMCAD_ERR_INVALID_ARG).
  * Synchronises `stream` and returns the device status word, LLMCAD_ERR_TIMEOUT when the path
  * works, or a negative host-detected error. The context is usable afterwards. */

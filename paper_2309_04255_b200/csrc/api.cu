@@ -105,15 +105,11 @@ struct llmcad_ctx {
     float *logits = nullptr;  // [128][V], used when the caller does not want logits
     TreeBuffers tb{};
     int32_t *ibuf = nullptr;  // tokens[128], parent[128], argmax[128], path[128], scalars[8], chain[128]
-    float *partials = nullptr;
-    uint32_t *arrivals = nullptr;        // arrival counters of the GEMM tails (two sets)
+    float *partials = nullptr;            // segment workspace of the tensor-core GEMMs
+    size_t partial_floats = 0;
     float *ssq[2] = {nullptr, nullptr};   // partial sums of squares for the folded attention / FFN norms
     float *attn_ws = nullptr;
     uint32_t *attn_counters = nullptr;
-    uint32_t *grid_counter = nullptr;   // grid barrier of the GEMM chains
-    uint32_t barrier_base = 0;          // its value once everything enqueued so far has run
-    int arrival_set = 0;                 // arrival-counter set of the next GEMM launch (launches alternate)
-    int prev_gemms = 0, prev_arrival_words = 0;   // what the last GEMM launch touched in its set
     int64_t launches = 0;
     uint64_t wait_limit_ns = kDefaultWaitLimitNs;   // bound of every device-side wait (llmcad_set_wait_limit_ns)
     unsigned long long *trace = nullptr;   // optional timeline buffer (llmcad_set_gemm_trace): [launch][256][16]
@@ -200,11 +196,11 @@ int ensure_act_maps(llmcad_ctx *ctx, int n_pad)
     return LLMCAD_OK;
 }
 
-// A chain of dependent tensor-core GEMMs that goes out as one persistent kernel.
-struct Chain {
-    ChainMaps maps;
-    ChainParams p;
-    Chain() { p = ChainParams{}; }
+// One tensor-core GEMM of the pass: the streaming kernel and its finishing kernel.
+struct TcGemm {
+    GemmMaps maps;
+    GemmParams p;
+    TcGemm() { p = GemmParams{}; }
     // W is `which` (0 qkv, 1 o, 2 gate/up, 3 down) of layer l, or the lm_head when l < 0;
     // act selects the activation buffer it multiplies (0 normalised stream, 1 attention output, 2 SwiGLU output)
     static const char *weight_ptr(llmcad_ctx *ctx, int l, int which)
@@ -214,38 +210,25 @@ struct Chain {
         const char *lb = base + ctx->lay.layer_bytes * (size_t)l;
         return lb + (which == 0 ? ctx->lay.wqkv : which == 1 ? ctx->lay.wo : which == 2 ? ctx->lay.wgu : ctx->lay.wdown);
     }
-    void add(llmcad_ctx *ctx, int l, int which, int act, int n_in, const EpiParams &ep, int n_pad)
+    void set(llmcad_ctx *ctx, int l, int which, int act, int n_in, const EpiParams &ep, int n_pad)
     {
-        const char *w = weight_ptr(ctx, l, which);
-        maps.x[p.n_gemms] = ctx->act_maps[n_pad / 16][act];
-        p.g[p.n_gemms] = make_gemm_desc(n_in, ep, w);
+        maps.x = ctx->act_maps[n_pad / 16][act];
+        p.g = make_gemm_desc(n_in, ep, weight_ptr(ctx, l, which));
         p.n_pad = n_pad;
         p.comp = ctx->comp ? 1 : 0;
-        ++p.n_gemms;
     }
     int launch(llmcad_ctx *ctx, int32_t *status, cudaStream_t st)
     {
-        if (p.n_gemms == 0) return LLMCAD_OK;
         p.partials = ctx->partials;
-        p.arrivals = ctx->arrivals;
-        p.arrival_set = ctx->arrival_set;
-        p.prev_gemms = ctx->prev_gemms;
-        p.prev_arrival_words = ctx->prev_arrival_words;
-        ctx->arrival_set ^= 1;
-        ctx->prev_gemms = p.n_gemms;
-        ctx->prev_arrival_words = 0;
-        for (int g = 0; g < p.n_gemms; ++g)
-            if (p.g[g].n_tiles * 4 > ctx->prev_arrival_words) ctx->prev_arrival_words = p.g[g].n_tiles * 4;
-        p.grid_counter = ctx->grid_counter;
-        p.barrier_base = ctx->barrier_base;
         p.status = status;
         p.wait_limit_ns = ctx->wait_limit_ns;
         p.trace = ctx->next_trace();
-        uint32_t arrivals = 0;
-        ctx->launches++;
+        int launched = 0;
         TimedLaunch tl(ctx, 0, st);
-        CUDA_TRY(launch_gemm_chain(maps, p, ctx->n_sms, st, &arrivals));
-        ctx->barrier_base += arrivals;
+        const cudaError_t e = launch_gemm_tc(maps, p, ctx->n_sms, ctx->partial_floats, st, &launched);
+        ctx->launches += launched;
+        if (e == cudaErrorInvalidValue && launched == 0) return LLMCAD_ERR_UNSUPPORTED;   // more tiles than the workspace holds
+        CUDA_TRY(e);
         return LLMCAD_OK;
     }
 };
@@ -373,25 +356,16 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
             if (!last) specs.push_back({l + 1, 0, 0, d, qkv_ep(l + 1, tiles4), false});
             else if (logits != nullptr) specs.push_back({-1, 0, 0, d, head_ep(tiles4), false});
         }
-        // Dependent GEMMs may share a launch (grid barriers between them, see gemm_tc.cu); measured
-        // on B200 one GEMM per launch, chained by programmatic dependent launch, is faster, so that
-        // is the default. LLMCAD_CHAIN_MAX is a tuning aid.
-        static const int chain_max = [] { const char *e = getenv("LLMCAD_CHAIN_MAX"); int v = e ? atoi(e) : 1; return v < 1 ? 1 : (v > kMaxChain ? kMaxChain : v); }();
-        for (size_t i = 0; i < specs.size();) {
+        for (size_t i = 0; i < specs.size(); ++i) {
             if (specs[i].attention_first) {
                 char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)specs[i].l;
                 // without the tensor-core attention kernel the lo plane of att stays zero, as allocated
                 if ((rc = run_attention(ctx, ctx->q, kl, kl + kv_layer / 2, S, P, n, ctx->att, ctx->comp && ctx->tc_attn, status, st,
                                         n_tree, n_old)) != LLMCAD_OK) return rc;
             }
-            Chain ch;
-            size_t j = i;
-            do {
-                ch.add(ctx, specs[j].l, specs[j].which, specs[j].act, specs[j].n_in, specs[j].ep, n_pad);
-                ++j;
-            } while (j < specs.size() && ch.p.n_gemms < chain_max && !specs[j].attention_first);
-            if ((rc = ch.launch(ctx, status, st)) != LLMCAD_OK) return rc;
-            i = j;
+            TcGemm g;
+            g.set(ctx, specs[i].l, specs[i].which, specs[i].act, specs[i].n_in, specs[i].ep, n_pad);
+            if ((rc = g.launch(ctx, status, st)) != LLMCAD_OK) return rc;
         }
         return LLMCAD_OK;
     }
@@ -430,19 +404,6 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
         ep.n = n; ep.mode = EPI_PLAIN; ep.n_out = c.vocab; ep.y = logits; ep.ldy = c.vocab;
         if ((rc = run_gemm(ctx, packed, -1, 0, 0, d, ep, n_pad, status, st)) != LLMCAD_OK) return rc;
     }
-    return LLMCAD_OK;
-}
-
-// The chain kernels synchronise through a grid counter and per-tile arrival counters. Both return to a
-// known state by themselves, but not when a wait ran out: start every call from zero.
-int reset_chain_sync(llmcad_ctx *ctx, cudaStream_t st)
-{
-    if (!ctx->tc_gemm) return LLMCAD_OK;
-    CUDA_TRY(cudaMemsetAsync(ctx->grid_counter, 0, sizeof(uint32_t), st));
-    CUDA_TRY(cudaMemsetAsync(ctx->arrivals, 0, kArrivalWords * sizeof(uint32_t), st));
-    ctx->barrier_base = 0;
-    ctx->arrival_set = 0;
-    ctx->prev_gemms = ctx->prev_arrival_words = 0;
     return LLMCAD_OK;
 }
 
@@ -542,9 +503,15 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ok = ok && alloc((void **)&ctx->tb.anc, 128 * 16);
     ok = ok && alloc((void **)&ctx->tb.rope_cs, 128 * (hd / 2) * sizeof(float2));
     ok = ok && alloc((void **)&ctx->ibuf, (520 + 128) * 4);
-    ok = ok && alloc((void **)&ctx->partials, gemm_tc_partial_floats(2 * ctx->n_sms, 128) * 4);
-    ok = ok && alloc((void **)&ctx->arrivals, kArrivalWords * 4);   // arrival counters
-    ok = ok && alloc((void **)&ctx->grid_counter, 256);
+    {
+        // segment workspace: the GEMM with the most tiles of this model (or 256 tiles, for the single-GEMM entry points)
+        int max_tiles = 256;
+        for (size_t rows : {3 * d, f, (size_t)cfg->vocab})
+            if ((int)((rows + 127) / 128) > max_tiles) max_tiles = (int)((rows + 127) / 128);
+        const int max_pad = (cfg->max_tree + 15) / 16 * 16;
+        ctx->partial_floats = ctx->tc_gemm ? gemm_tc_partial_floats(ctx->n_sms, max_tiles, max_pad) : 64;
+        ok = ok && alloc((void **)&ctx->partials, ctx->partial_floats * 4);
+    }
     const size_t ssq_floats = (size_t)4 * ((d + 127) / 128) * LLMCAD_MAX_TREE;
     ok = ok && alloc((void **)&ctx->ssq[0], ssq_floats * 4);
     ok = ok && alloc((void **)&ctx->ssq[1], ssq_floats * 4);
@@ -567,8 +534,8 @@ void llmcad_destroy(llmcad_ctx *ctx)
 {
     if (ctx == nullptr) return;
     void *ptrs[] = {ctx->x, ctx->xn, ctx->q, ctx->att, ctx->h, ctx->kv_lo, ctx->logits, ctx->tb.depth, ctx->tb.pos, ctx->tb.anc,
-                    ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->arrivals, ctx->attn_ws, ctx->attn_counters, ctx->ssq[0],
-                    ctx->ssq[1], ctx->grid_counter};
+                    ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->attn_ws, ctx->attn_counters, ctx->ssq[0],
+                    ctx->ssq[1]};
     for (void *p : ptrs)
         if (p != nullptr) cudaFree(p);
     for (auto &t : ctx->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
@@ -641,7 +608,6 @@ int llmcad_verify_tree(llmcad_ctx *ctx, const void *packed, void *kv_cache, int3
     int32_t *status = out->scalars + LLMCAD_S_STATUS;
     float *logits = out->logits != nullptr ? out->logits : ctx->logits;
     CUDA_TRY(cudaMemsetAsync(out->scalars, 0, 8 * sizeof(int32_t), st));
-    if ((rc = reset_chain_sync(ctx, st)) != LLMCAD_OK) return rc;
     if ((rc = run_forward(ctx, packed, kv_cache, prefix_len, tree_tokens, parent_idx, n, logits, status, st)) != LLMCAD_OK)
         return rc;
     CUDA_TRY(launch_argmax(logits, n, c.vocab, out->argmax, status, st));
@@ -689,10 +655,6 @@ int llmcad_prefill(llmcad_ctx *ctx, const void *packed, void *kv_cache, int32_t 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
     CUDA_TRY(cudaMemsetAsync(ctx->scalars_dev(), 0, 8 * sizeof(int32_t), st));
-    {
-        int rc0 = reset_chain_sync(ctx, st);
-        if (rc0 != LLMCAD_OK) return rc0;
-    }
     const int chunk = ctx->cfg.max_tree;
     for (int done = 0; done < n; done += chunk) {
         const int m = n - done < chunk ? n - done : chunk;
@@ -720,7 +682,6 @@ int llmcad_extend_tree(llmcad_ctx *ctx, const void *packed, void *kv_cache, int3
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float *lg = logits != nullptr ? logits : ctx->logits;
     CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
-    if ((rc = reset_chain_sync(ctx, st)) != LLMCAD_OK) return rc;
     if ((rc = run_forward(ctx, packed, kv_cache, prefix_len, tree_tokens, parent_idx, n_tree, lg, status, st, n_old)) != LLMCAD_OK)
         return rc;
     if (top_k > 0) {
@@ -798,22 +759,17 @@ int llmcad_skinny_gemm(llmcad_ctx *ctx, const void *w, const void *x, float *y, 
     CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
     EpiParams ep{};
     ep.mode = EPI_PLAIN; ep.n = n; ep.n_out = n_out; ep.y = y; ep.ldy = n_out;
-    {
-        int rc0 = reset_chain_sync(ctx, st);
-        if (rc0 != LLMCAD_OK) return rc0;
-    }
     if (ctx->tc_gemm) {
         const int n_pad = (n + 15) / 16 * 16;
-        Chain ch;
+        TcGemm g;
         // rows of x beyond n are outside the tensor: the copy engine fills them with zeros
-        if (!make_tensor_map_bf16(&ch.maps.w[0], w, n_out, n_in, 128) || !make_act_map_bf16(&ch.maps.x[0], x, n, n_in, n_pad, 1, n)) {
+        if (!make_tensor_map_bf16(&g.maps.w, w, n_out, n_in, 128) || !make_act_map_bf16(&g.maps.x, x, n, n_in, n_pad, 1, n)) {
             snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
             return LLMCAD_ERR_CUDA;
         }
-        ch.p.g[0] = make_gemm_desc(n_in, ep);
-        ch.p.n_pad = n_pad;
-        ch.p.n_gemms = 1;
-        return ch.launch(ctx, status, st);
+        g.p.g = make_gemm_desc(n_in, ep);
+        g.p.n_pad = n_pad;
+        return g.launch(ctx, status, st);
     }
     ctx->launches++;
     TimedLaunch tl(ctx, 0, st);
@@ -845,20 +801,17 @@ int llmcad_skinny_gemm_tiled(llmcad_ctx *ctx, const void *w_tiled, const void *x
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
     CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
-    int rc = reset_chain_sync(ctx, st);
-    if (rc != LLMCAD_OK) return rc;
     EpiParams ep{};
     ep.mode = EPI_PLAIN; ep.n = n; ep.n_out = n_out; ep.y = y; ep.ldy = n_out;
     const int n_pad = (n + 15) / 16 * 16;
-    Chain ch;
-    if (!make_act_map_bf16(&ch.maps.x[0], x, n, n_in, n_pad, 1, n)) {
+    TcGemm g;
+    if (!make_act_map_bf16(&g.maps.x, x, n, n_in, n_pad, 1, n)) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
         return LLMCAD_ERR_CUDA;
     }
-    ch.p.g[0] = make_gemm_desc(n_in, ep, w_tiled);
-    ch.p.n_pad = n_pad;
-    ch.p.n_gemms = 1;
-    return ch.launch(ctx, status, st);
+    g.p.g = make_gemm_desc(n_in, ep, w_tiled);
+    g.p.n_pad = n_pad;
+    return g.launch(ctx, status, st);
 }
 
 int llmcad_set_kernel_timing(llmcad_ctx *ctx, int32_t enable)
@@ -999,33 +952,28 @@ int llmcad_selftest_wait_timeout(llmcad_ctx *ctx, void *stream)
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
     CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
-    int rc = reset_chain_sync(ctx, st);
-    if (rc != LLMCAD_OK) return rc;
     const int n_pad = 16;
-    if ((rc = ensure_act_maps(ctx, n_pad)) != LLMCAD_OK) return rc;
-    // Two dependent 256 x 128 GEMMs on 16 nodes. Weights: the first 64 KB of the context's logits
-    // buffer read as four pre-swizzled tiles (any bit pattern will do); input: the normalised
-    // activations; output: plain fp32 rows further up in the same buffer.
+    int rc = ensure_act_maps(ctx, n_pad);
+    if (rc != LLMCAD_OK) return rc;
+    // A 256 x 128 GEMM on 16 nodes. Weights: the first 64 KB of the context's logits buffer read as
+    // four pre-swizzled tiles (any bit pattern will do); input: the normalised activations; output:
+    // plain fp32 rows further up in the same buffer.
     EpiParams ep{};
     ep.mode = EPI_PLAIN; ep.n = n_pad; ep.n_out = 256; ep.ldy = 256;
     ep.y = ctx->logits + (64 * 1024) / sizeof(float);
-    Chain ch;
-    for (int g = 0; g < 2; ++g) {
-        ch.maps.x[g] = ctx->act_maps[n_pad / 16][0];
-        ch.p.g[g] = make_gemm_desc(128, ep, ctx->logits);
-    }
-    ch.p.n_pad = n_pad;
-    ch.p.comp = ctx->comp ? 1 : 0;
-    ch.p.n_gemms = 2;
-    // the launch believes the barrier counter starts one higher than it does: the arrivals after the
-    // first GEMM never reach the target, and every wait at the barrier runs into the limit
-    ctx->barrier_base += 1;
-    rc = ch.launch(ctx, status, st);
+    TcGemm g;
+    g.maps.x = ctx->act_maps[n_pad / 16][0];
+    g.p.g = make_gemm_desc(128, ep, ctx->logits);
+    g.p.n_pad = n_pad;
+    g.p.comp = ctx->comp ? 1 : 0;
+    // the activation copies are withheld: the ring stages never fill, and every role of the streaming
+    // kernel runs into the wait limit
+    g.p.withhold_act = 1;
+    rc = g.launch(ctx, status, st);
     if (rc != LLMCAD_OK) return rc;
     int32_t v = 0;
     CUDA_TRY(cudaMemcpyAsync(&v, status, sizeof(v), cudaMemcpyDeviceToHost, st));
     CUDA_TRY(cudaStreamSynchronize(st));
-    if ((rc = reset_chain_sync(ctx, st)) != LLMCAD_OK) return rc;
     return v;
 }
 

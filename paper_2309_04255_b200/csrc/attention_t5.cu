@@ -762,6 +762,7 @@ cudaError_t launch_attention_t5(const void *q, const void *k, const void *v, int
     static PerDeviceOnce attr_set;
     if (attr_set.needed()) {
         cudaError_t e = cudaFuncSetAttribute(attention_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_t5_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set.mark();
     }

@@ -490,6 +490,8 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
         for (int c = 0; c < 2; ++c)
             for (int g = 0; g < 3; ++g) {
                 cudaError_t e = cudaFuncSetAttribute(kerns[c][g], cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+                // the largest shared-memory split of the SM, so that the next GEMM's streaming CTA can settle beside this kernel's
+                if (e == cudaSuccess) e = cudaFuncSetAttribute(kerns[c][g], cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
                 if (e != cudaSuccess) return e;
             }
         attr_set.mark();

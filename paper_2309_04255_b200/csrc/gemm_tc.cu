@@ -2,35 +2,43 @@
 //
 // The one-shot verification of Sec. 3.2 visits every parameter once for all N <= 128 tree nodes,
 // so each GEMM is D[n_out][N] = W[n_out][K] * X[N][K]^T with a tiny N: it is bound by the bytes
-// of W coming from HBM. The kernel therefore puts W on the M side of tcgen05.mma (128 weight
-// rows per tile = the 128 TMEM lanes) and the tree nodes on the N side (padded to a multiple of
-// 16; with hi + lo activation planes the MMA sees every node twice), and streams W exactly once
+// of W coming from HBM. The streaming kernel therefore puts W on the M side of tcgen05.mma (128
+// weight rows per tile = the 128 TMEM lanes) and the tree nodes on the N side (padded to a multiple
+// of 16; with hi + lo activation planes the MMA sees every node twice), and streams W exactly once
 // through a ring in shared memory: the weights are stored as pre-swizzled 16 KB tiles (pack.cu), so
 // a ring item (one tile, two k-blocks) is one contiguous 32 KB bulk copy.
 //
-// The grid is persistent, one CTA per SM. The (tile, k-block pair, half) items of a GEMM are split
-// evenly over the CTAs (stream-K): a CTA's range may start and end inside a tile; every holder of a
-// tile leaves its accumulators in an fp32 workspace, and the CTAs whose range ends in that tile add
-// all shares in a fixed (CTA) order and run the fused epilogue together (see finish_rows), so the
-// result does not depend on timing. A launch may run up to four *dependent* GEMMs with grid
-// barriers between them (the producer keeps streaming the next GEMM's weights meanwhile); one GEMM
-// per launch, chained by programmatic dependent launch, measured faster and is what the pass uses.
+// A GEMM is two kernels, chained by programmatic dependent launch.
 //
-// Warp roles (256 threads): warp 0 = weight producer, warp 1 = TMEM allocator + MMA issuer,
-// warps 2..5 = epilogue (tcgen05.ld of their 32 lanes each), warp 6 = activation loader (TMA),
-// warp 7 = spare; when the launch's last tile is finished, warps 0, 1, 6 and 7 each take half of one
-// epilogue warp's work. Accumulators are double-buffered in TMEM when two buffers fit, so that the
-// epilogue of one tile overlaps the MMAs of the next.
+// gemm_stream_kernel: persistent grid, one CTA per SM. The (tile, k-block pair, half) items of the
+// GEMM are split evenly over the CTAs (stream-K): a CTA's range may start and end inside a tile.
+// For every tile that a CTA holds items of (a "segment") it leaves its accumulators, hi and lo
+// columns added, in a workspace slot (slot = tile + CTA, unique because the CTAs' ranges are
+// ordered), and exits. Nothing in it waits for another CTA.
+//
+// gemm_finish_kernel: all warps of the GPU add the segments of every tile in CTA order (so the
+// result does not depend on timing) and apply the fused epilogue (rotary + K/V cache write,
+// residual + the next norm's gain * x and sums of squares, SwiGLU, or plain fp32 rows). It needs
+// next to no shared memory, so the NEXT GEMM's streaming CTAs become resident as soon as this
+// GEMM's streaming CTAs leave, and fill their weight rings while the finishing runs: the HBM
+// stream pauses only for as long as a ring lasts, not for the whole tail of a GEMM.
+//
+// Warp roles of the streaming kernel (224 threads): warp 0 = weight producer, warp 1 = TMEM
+// allocator + MMA issuer, warps 2..5 = accumulator dump (tcgen05.ld of their 32 lanes each),
+// warp 6 = activation loader (TMA). Accumulators are double-buffered in TMEM when two buffers fit,
+// so that the dump of one segment overlaps the MMAs of the next.
 //
 // Programmatic stream serialization: the ring is filled with weight tiles while the previous
-// kernel of the pass is still running; activations, workspace and outputs wait for the grid
-// dependency. A status word left by an earlier phase is not looked at here: the GEMMs then work on
-// stale but finite activations and write only scratch, and the search/rollback kernels at the end
-// of the pass report the error.
+// kernels of the pass are still running; activations and the workspace wait for the grid
+// dependency. The streaming kernel lets its dependents go only after its own dependency has
+// resolved, so the finishing kernel may read what earlier GEMMs produced (norm sums, gains) before
+// its own dependency, the streaming kernel, completes. A status word left by an earlier phase is
+// not looked at here: the GEMMs then work on stale but finite activations and write only scratch
+// and tree slots, and the search/rollback kernels at the end of the pass report the error.
 //
-// Every wait (mbarrier, arrival counter, grid barrier) is bounded by a deadline; on expiry the
+// Every wait of the streaming kernel (mbarriers only) is bounded by a deadline; on expiry the
 // kernel sets the status word to LLMCAD_ERR_TIMEOUT, lets every role fall out of its loop, frees
-// TMEM and returns. All CTAs of a launch are resident at once (grid <= SM count, one CTA per SM).
+// TMEM and returns.
 #include <cuda.h>
 
 #include <cstdlib>
@@ -44,8 +52,14 @@ namespace {
 
 constexpr int kTileM = 128;     // weight rows per tile
 constexpr int kBlockK = 64;     // bf16 elements per k-block = one 128-byte swizzle row
-constexpr int kThreads = 256;   // producer, MMA, 4 epilogue warps, activation loader, one spare: the four
-                                // non-epilogue warps each help one epilogue warp with the launch's last tile
+constexpr int kThreads = 224;   // producer, MMA issuer, 4 epilogue warps, activation loader
+constexpr int kFinThreads = 384;  // finishing kernel: 12 warps, up to 112 registers each beside a resident streaming CTA
+// An SM's registers come in four banks of 16K, one per warp scheduler: beside the streaming CTA's two warps per
+// scheduler (96 registers a thread) three finishing warps fit with up to 106 each.
+constexpr int kFinMaxRegs = 96;
+constexpr size_t kFinSmem = 24 * 1024;   // dynamic shared memory the finishing kernel asks for (and does not use):
+                                         // it keeps two of its CTAs from settling on one SM, which would leave no room
+                                         // there for the next GEMM's streaming CTA
 constexpr int kATileBytes = kTileM * kBlockK * 2;  // 16 KB
 constexpr int kMaxStages = 16;
 constexpr int kMaxPairK = 2;     // k-blocks per ring item (GemmDesc::pair_k): 2 = one 32 KB weight copy feeds 8 MMAs;
@@ -227,16 +241,7 @@ struct SharedCtl {
     uint32_t tmem_base;
     volatile int abort_flag;
     volatile uint32_t a_issued;     // ring items whose weight copy (and expect_tx) has been issued
-    volatile uint32_t dumped[4];    // per row group: this CTA's share of its last tile is in the workspace
-    float rs[4][LLMCAD_MAX_TREE];   // per epilogue warp: rsqrt(mean(x^2) + eps) of the folded input RMSNorm
 };
-
-__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
-{
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
 
 // A ring item is (tile, k-block pair, half): up to two consecutive 64-wide k-blocks of one
 // 128-row weight tile (32 KB, contiguous in the tiled layout) and the matching activation tiles.
@@ -244,65 +249,55 @@ __host__ __device__ __forceinline__ int pairs_per_tile(const GemmDesc &g) { retu
 // the same with the k-blocks per item as a compile-time constant (the kernel is instantiated for 1 and 2)
 template <int PK> __device__ __forceinline__ int pairs_per_tile_c(const GemmDesc &g) { return (g.kb_per_tile + PK - 1) / PK; }
 
-// This CTA's share of GEMM g: items [begin, end) of its item list.
+// CTA cta's share of the GEMM: items [begin, end) of its item list.
 struct Range {
     int begin, end;
 };
 template <int PK>
-__device__ __forceinline__ Range cta_range(const GemmDesc &g)
+__device__ __forceinline__ Range cta_range(const GemmDesc &g, int cta)
 {
     const int total = g.n_tiles * pairs_per_tile_c<PK>(g) * g.halves;
     Range r;
-    r.begin = min(total, (int)blockIdx.x * g.items_per_cta);
+    r.begin = min(total, cta * g.items_per_cta);
     r.end = min(total, r.begin + g.items_per_cta);
     return r;
 }
 
-// Cursor over the concatenated item stream of the chain (all GEMMs, this CTA's ranges, in order).
-// Coordinates are kept incrementally: the single-thread roles have well under a microsecond per item.
+// Cursor over this CTA's items, in order. Coordinates are kept incrementally: the single-thread
+// roles have well under a microsecond per item.
 template <int PK>
 struct Cursor {
-    int g;                 // current GEMM, == n_gemms when exhausted
     int tile, kp, half;    // coordinates of the current item (kp: k-block pair)
-    int left;              // items left in this CTA's range of GEMM g, the current one included
+    int left;              // items left in this CTA's range, the current one included
     int ppt, halves, kbpt;
-    __device__ void init(const ChainParams &p)
+    __device__ void init(const GemmDesc &d)
     {
-        g = -1;
-        left = 0;
-        next_gemm(p);
+        const Range r = cta_range<PK>(d, (int)blockIdx.x);
+        left = r.end - r.begin;
+        kbpt = d.kb_per_tile;
+        ppt = pairs_per_tile_c<PK>(d);
+        halves = d.halves;
+        const int ipt = ppt * halves;
+        tile = r.begin / ipt;
+        const int q = r.begin - tile * ipt;
+        kp = q / halves;
+        half = q - kp * halves;
     }
-    __device__ void next_gemm(const ChainParams &p)
-    {
-        while (true) {
-            if (++g >= p.n_gemms) { g = p.n_gemms; left = 0; return; }
-            const GemmDesc &d = p.g[g];
-            const Range r = cta_range<PK>(d);
-            left = r.end - r.begin;
-            if (left <= 0) continue;
-            kbpt = d.kb_per_tile;
-            ppt = pairs_per_tile_c<PK>(d);
-            halves = d.halves;
-            const int ipt = ppt * halves;
-            tile = r.begin / ipt;
-            const int q = r.begin - tile * ipt;
-            kp = q / halves;
-            half = q - kp * halves;
-            return;
-        }
-    }
-    __device__ bool done(const ChainParams &p) const { return g >= p.n_gemms; }
+    __device__ bool done() const { return left <= 0; }
     __device__ int kb0() const { return kp * PK; }
     __device__ int nk() const { return min(PK, kbpt - kp * PK); }   // k-blocks in this item
-    __device__ void advance(const ChainParams &p)
+    __device__ void advance()
     {
-        if (--left <= 0) { next_gemm(p); return; }
+        --left;
         if (++half == halves) {
             half = 0;
             if (++kp == ppt) { kp = 0; ++tile; }
         }
     }
 };
+
+// Floats of one segment slot of the workspace: [4 row groups][halves][n_pad nodes][32 rows].
+__host__ __device__ __forceinline__ size_t slot_floats(int halves, int n_pad) { return (size_t)halves * n_pad * kTileM; }
 
 // ------------------------------------------------------------------------------------------------
 // Finishing a 32-row group of an output tile. Every CTA that holds a share of a tile leaves its
@@ -321,23 +316,20 @@ __device__ __forceinline__ uint2 pack4_bf16(const __nv_bfloat16 (&h)[4])
     return r;
 }
 
-// Which workspace slot of CTA cc holds its share of the tile whose first item is tile_i0: slot 0
-// holds the tile in which the CTA's range starts, slot 1 any later one.
-__device__ __forceinline__ const float *share_ptr(const ChainParams &p, const GemmDesc &d, int cc, int tile_i0, int lane_grp)
+// Where CTA cc left its segment of tile `tile`, rows of row group lane_grp: slot tile + cc.
+__device__ __forceinline__ const float *share_ptr(const GemmParams &p, const GemmDesc &d, int cc, int tile, int lane_grp)
 {
-    const int slot = (cc * d.items_per_cta >= tile_i0) ? 0 : 1;
-    return p.partials + ((size_t)cc * 2 + slot) * ((size_t)2 * p.n_pad * kTileM) + (size_t)lane_grp * 2 * p.n_pad * 32;
+    return p.partials + (size_t)(tile + cc) * slot_floats(d.halves, p.n_pad) + (size_t)lane_grp * d.halves * p.n_pad * 32;
 }
 
 // Everything the finishing code needs, gathered in one place so that the function below can be a
 // real call (one copy of its code in the kernel).
 struct FinishArgs {
-    const ChainParams *p;
+    const GemmParams *p;
     const GemmDesc *d;              // in shared memory
     const float *rs;                // per-node factors of the folded input norm (shared memory)
-    int tile, tile_i0, first_cta, last_cta, lane_grp;
+    int tile, first_cta, last_cta, lane_grp;
     int it_first, it_step;          // this warp finishes node groups it_first, it_first + it_step, ...
-    unsigned long long *trace;      // optional timeline slots of this CTA (tracing)
 };
 
 // Finishing a 32-row group of an output tile: add the shares of all CTAs that hold part of the
@@ -357,10 +349,10 @@ struct FinishArgs {
 // One instantiation per epilogue mode as well: the routine is cold whenever it runs, and what it
 // costs in instruction-cache misses is the code it walks through, not the code that exists.
 template <int G, int kB, int MODE>
-__device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
+__device__ __forceinline__ void finish_rows_t(const FinishArgs &fa, int lane, const bool dry)
 {
     typedef __nv_bfloat16 T;
-    const ChainParams &p = *fa.p;
+    const GemmParams &p = *fa.p;
     const GemmDesc &d = *fa.d;
     const EpiParams &ep = d.ep;
     constexpr int mode = MODE;
@@ -409,7 +401,7 @@ __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
             float4 t[G][kB], u[G][kB];
 #pragma unroll
             for (int k = 0; k < kB; ++k) {
-                const float *sk = share_ptr(p, d, fa.first_cta + min(k0 + k, n_parts - 1), fa.tile_i0, lane_grp) + 4 * r4;
+                const float *sk = share_ptr(p, d, fa.first_cta + min(k0 + k, n_parts - 1), tile, lane_grp) + 4 * r4;
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
                     const int node = min(itg + g * fa.it_step, iters - 1) * 4 + ns;
@@ -428,11 +420,10 @@ __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
                 }
             }
         }
-        if (fa.trace && itg == fa.it_first) fa.trace[11] = (unsigned long long)(as[0].x + as[G - 1].w != 12345.f) * global_timer_ns();
         // two at a time, unrolled: the warp is alone on its scheduler and the two chains overlap
         for (int g2 = 0; g2 < G; g2 += 2) {
 #pragma unroll
-        for (int gq = 0; gq < 2; ++gq) {
+        for (int gq = 0; gq < (G < 2 ? G : 2); ++gq) {
         const int g = g2 + gq;
         const int it = itg + g * fa.it_step;
         if (it >= iters) continue;
@@ -447,7 +438,7 @@ __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
         T *dst = nullptr, *dst_lo = nullptr;
         if (resid) {
             const float xo[4] = {ok ? ax.x + v[0] : 0.f, ok ? ax.y + v[1] : 0.f, ok ? ax.z + v[2] : 0.f, ok ? ax.w + v[3] : 0.f};
-            if (ok) *reinterpret_cast<float4 *>(ep.x + (size_t)node * n_out + row0) = make_float4(xo[0], xo[1], xo[2], xo[3]);
+            if (ok && !dry) *reinterpret_cast<float4 *>(ep.x + (size_t)node * n_out + row0) = make_float4(xo[0], xo[1], xo[2], xo[3]);
 #pragma unroll
             for (int k = 0; k < 4; ++k) out[k] = xo[k] * gain[k];
             if (has_xg) {
@@ -459,7 +450,7 @@ __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
                 ss += __shfl_xor_sync(0xffffffffu, ss, 1);
                 ss += __shfl_xor_sync(0xffffffffu, ss, 2);
                 ss += __shfl_xor_sync(0xffffffffu, ss, 4);
-                if (r4 == 0) ep.ssq_out[(size_t)(tile * 4 + lane_grp) * LLMCAD_MAX_TREE + node] = ss;
+                if (r4 == 0 && !dry) ep.ssq_out[(size_t)(tile * 4 + lane_grp) * LLMCAD_MAX_TREE + node] = ss;
             }
         } else if (mode == EPI_SWIGLU) {
 #pragma unroll
@@ -479,7 +470,7 @@ __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
                 dst = reinterpret_cast<T *>(sec == 1 ? ep.k_cache : ep.v_cache) + ((size_t)head * ep.S + ep.P + node) * ep.hd + e;
                 dst_lo = reinterpret_cast<T *>(ep.kv_lo) + ((size_t)((sec - 1) * (ep.d / ep.hd) + head) * kLoRows + node) * ep.hd + e;
             }
-        } else if (node < n_nodes) {
+        } else if (node < n_nodes && !dry) {
             float *yr = ep.y + (size_t)node * ep.ldy + row0;
             if (rows_ok && (ep.ldy & 3) == 0 && (reinterpret_cast<uintptr_t>(ep.y) & 15) == 0)
                 *reinterpret_cast<float4 *>(yr) = make_float4(v[0], v[1], v[2], v[3]);
@@ -489,7 +480,7 @@ __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
                     if (k < n_valid) yr[k] = v[k];
             }
         }
-        if (dst != nullptr && ok) {
+        if (dst != nullptr && ok && !dry) {
             T hi[4], lo[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) split_bf16(out[k], hi[k], lo[k]);
@@ -498,46 +489,20 @@ __device__ __noinline__ void finish_rows_t(const FinishArgs &fa, int lane)
         }
         }
         }
-        if (fa.trace && itg == fa.it_first) fa.trace[15] = global_timer_ns();
     }
-}
-
-template <int G, int kB>
-__device__ __forceinline__ void finish_rows_m(const FinishArgs &fa, int lane)
-{
-    switch (fa.d->ep.mode) {
-    case EPI_QKV: finish_rows_t<G, kB, EPI_QKV>(fa, lane); break;
-    case EPI_RESID: finish_rows_t<G, kB, EPI_RESID>(fa, lane); break;
-    case EPI_SWIGLU: finish_rows_t<G, kB, EPI_SWIGLU>(fa, lane); break;
-    default: finish_rows_t<G, kB, EPI_PLAIN>(fa, lane); break;
-    }
-}
-
-__device__ __forceinline__ void finish_rows(const FinishArgs &fa, int lane)
-{
-    if (fa.last_cta - fa.first_cta + 1 > 3) finish_rows_m<2, 4>(fa, lane);
-    else finish_rows_m<4, 2>(fa, lane);
 }
 
 }  // namespace
 
-template <typename T, int PK>
+#define LLMCAD_TRACE(slot) do { if (p.trace && blockIdx.x < 256) p.trace[(size_t)blockIdx.x * 16 + (slot)] = global_timer_ns(); } while (0)
+
+template <int PK>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams p)
+gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ GemmParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ SharedCtl ctl;
-    // The epilogue reads its GEMM's description (pointers, sizes, mode) all over the finishing code.
-    // From the kernel parameters, indexed by the GEMM's number, every first touch of a constant-cache
-    // line is a miss that stalls the lone finishing warp for most of a microsecond; a copy in shared
-    // memory, made while the first weights are still on their way, costs nothing to read.
-    __shared__ __align__(16) GemmDesc s_desc[kMaxChain];
-    {
-        static_assert(sizeof(GemmDesc) % 4 == 0, "GemmDesc is copied word by word");
-        const uint32_t *src = reinterpret_cast<const uint32_t *>(&p.g[0]);
-        uint32_t *dst = reinterpret_cast<uint32_t *>(&s_desc[0]);
-        for (int i = threadIdx.x; i < (int)(sizeof(GemmDesc) / 4) * p.n_gemms; i += kThreads) dst[i] = src[i];
-    }
+    const GemmDesc &d = p.g;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t nb = (uint32_t)p.n_pad * (p.comp ? 2u : 1u);   // activation rows per k-block = the MMA N: nodes (hi | lo)
@@ -550,22 +515,17 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
     const bool two_bufs = p.acc_bufs == 2;
     const uint64_t wait_limit = p.wait_limit_ns;          // every wait below gives up after this many ns
 
-    // Let the next kernel of the stream start early. This kernel in turn must not read activations,
-    // the status word or the workspace, nor write anything, before pdl_wait(): until then it only
-    // prefetches weights, which no kernel writes.
-    pdl_launch_dependents();
-#define LLMCAD_TRACE(slot) do { if (p.trace) p.trace[(size_t)blockIdx.x * 16 + (slot)] = global_timer_ns(); } while (0)
     if (threadIdx.x == 0) LLMCAD_TRACE(0);
 
     // State of the weight producer (thread 0). It lives across the start-up barrier: the first
     // ring-full of copies goes out right after the barriers are initialised, before TMEM allocation
-    // and before the other warps are even needed.
+    // and before the other warps are even needed. Until pdl_wait() this kernel only prefetches
+    // weights, which no kernel writes.
     Cursor<PK> pc;
     int ps = 0;
     uint32_t ppar = 1, pissued = 0;    // a fresh barrier passes a wait on parity 1: no special first lap
     uint64_t pol_stream = 0;
     auto issue_item = [&]() {          // the next item of the stream into ring stage ps (which must be free)
-        const GemmDesc &d = p.g[pc.g];
         const int nk = pc.nk();
         const uint32_t full = smem_u32(&ctl.full[ps]);
         const uint32_t dst = smem_base + ps * stage_bytes;
@@ -576,13 +536,13 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             bulk_load_1d(dst, d.w_tiled + t * kATileBytes, (uint32_t)nk * kATileBytes, full, pol_stream);
         } else {
             for (int k = 0; k < nk; ++k)
-                tma_load_2d(dst + k * kATileBytes, &maps.w[pc.g], (pc.kb0() + k) * kBlockK,
+                tma_load_2d(dst + k * kATileBytes, &maps.w, (pc.kb0() + k) * kBlockK,
                             (pc.half ? d.up_row_offset : 0) + pc.tile * kTileM, full, pol_stream);
         }
         __threadfence_block();
         if (pissued == 0) LLMCAD_TRACE(2);
         ctl.a_issued = ++pissued;      // the activation loader may now add its bytes to this stage
-        pc.advance(p);
+        pc.advance();
         if (++ps == p.stages) { ps = 0; ppar ^= 1u; }
     };
     if (threadIdx.x == 0) {
@@ -596,12 +556,11 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         }
         ctl.abort_flag = 0;
         ctl.a_issued = 0;
-        for (int w = 0; w < 4; ++w) ctl.dumped[w] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-        pc.init(p);
-        while (!pc.done(p) && pissued < (uint32_t)p.stages) issue_item();
+        pc.init(d);
+        while (!pc.done() && pissued < (uint32_t)p.stages) issue_item();
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
@@ -616,38 +575,34 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
     volatile int *abort_flag = &ctl.abort_flag;
     bool timed_out = false;
     if (threadIdx.x == 0) LLMCAD_TRACE(1);
-    // "GEMM g of this launch is complete on every CTA": 4 epilogue warps x gridDim arrivals each.
-    const uint32_t arrivals_per_gemm = 4u * gridDim.x;
 
     if (warp == 0) {
         // ================================================= weight producer
-        // Streams this CTA's weight tiles of the whole chain, in order, as fast as ring slots
-        // free up; it never looks at activations or barriers between GEMMs.
+        // Streams this CTA's weight tiles, in order, as fast as ring slots free up.
         if (lane == 0) {
             Cursor<PK> cpf;                      // next item to prefetch into L2 (pc: next item to copy into the ring)
-            cpf.init(p);
+            cpf.init(d);
             uint32_t prefetched = 0;
             uint64_t t_idle = 0;
-            while (!pc.done(p)) {
+            while (!pc.done()) {
                 if (mbar_try(smem_u32(&ctl.empty[ps]), ppar)) {
                     issue_item();
                     t_idle = 0;
                     continue;
                 }
-                // The ring is full: the consumers are busy with a tail or a barrier between two GEMMs.
-                // Weights do not depend on any of that, so pull the next ones from HBM into L2 now;
-                // when the ring moves again it refills at L2 speed.
+                // The ring is full: the consumers wait for their input. Weights do not depend on that,
+                // so pull the next ones from HBM into L2 now; when the ring moves again it refills at
+                // L2 speed.
                 if (prefetched < pissued) {       // the ring overtook the prefetch cursor: catch up
-                    while (prefetched < pissued && !cpf.done(p)) { cpf.advance(p); ++prefetched; }
+                    while (prefetched < pissued && !cpf.done()) { cpf.advance(); ++prefetched; }
                 }
-                if (!cpf.done(p) && prefetched < pissued + (uint32_t)p.stages + (uint32_t)p.l2_ahead) {
-                    const GemmDesc &d = p.g[cpf.g];
+                if (!cpf.done() && prefetched < pissued + (uint32_t)p.stages + (uint32_t)p.l2_ahead) {
                     if (prefetched >= pissued + (uint32_t)p.stages && d.w_tiled != nullptr) {
                         const size_t t = (size_t)(cpf.tile + (cpf.half ? d.up_tile_offset : 0)) * d.kb_per_tile + cpf.kb0();
                         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(d.w_tiled + t * kATileBytes),
                                      "r"((uint32_t)cpf.nk() * kATileBytes) : "memory");
                     }
-                    cpf.advance(p);
+                    cpf.advance();
                     ++prefetched;
                     continue;
                 }
@@ -655,24 +610,24 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 if (t_idle == 0) t_idle = global_timer_ns();
                 else if (*abort_flag || global_timer_ns() - t_idle > wait_limit) { timed_out = true; break; }
             }
-            if (p.n_gemms == 1) LLMCAD_TRACE(6);
+            LLMCAD_TRACE(6);
         }
     } else if (warp == 6) {
         // ================================================= activation loader
         // Follows the weight producer item by item and adds the (small, L2-resident) activation
-        // tiles of each item, but only once the GEMM that the item belongs to may read its input:
-        // after the grid dependency for the first GEMM, after the grid barrier for the others.
+        // tiles of each item, once the grid dependency says that the GEMM's input is final.
         if (lane == 0) {
             uint64_t pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
             Cursor<PK> c;
-            c.init(p);
-            int s = 0, ready = 0, traced_g = 0;
+            c.init(d);
+            int s = 0;
             uint32_t i = 0;
             pdl_wait();
-            while (!c.done(p) && !timed_out) {
+            pdl_launch_dependents();
+            while (!c.done() && !timed_out && !p.withhold_act) {
                 uint64_t t0 = 0;
-                // (1) the stage is ours: the producer has passed its "empty" wait and armed the barrier
+                // the stage is ours: the producer has passed its "empty" wait and armed the barrier
                 for (uint32_t spin = 0; (int32_t)(ctl.a_issued - (i + 1)) < 0; ++spin) {
                     __nanosleep(32);
                     if ((spin & 255u) == 255u) {
@@ -680,47 +635,37 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                         if (*abort_flag || global_timer_ns() - t0 > wait_limit) { timed_out = true; break; }
                     }
                 }
-                // (2) the GEMM's input is final on every CTA
-                while (!timed_out && c.g > ready) {
-                    const uint32_t have = ld_acquire_u32(p.grid_counter) - p.barrier_base;
-                    ready = (int)(have / arrivals_per_gemm);       // GEMMs 0..ready-1 are complete everywhere
-                    if (c.g > ready) {
-                        __nanosleep(100);
-                        if (t0 == 0) t0 = global_timer_ns();
-                        if (*abort_flag || global_timer_ns() - t0 > wait_limit) timed_out = true;
-                    }
-                }
                 if (timed_out) break;
-                if (c.g != traced_g) { traced_g = c.g; if (c.g >= 1 && c.g <= 3) LLMCAD_TRACE(12 + c.g); }
                 const uint32_t full = smem_u32(&ctl.full[s]);
                 const uint32_t dst = smem_base + s * stage_bytes + b_off;
                 const int nk = c.nk();
                 for (int k = 0; k < nk; ++k)
-                    tma_load_3d(dst + k * b_tile_bytes, &maps.x[c.g], (c.kb0() + k) * kBlockK, full, pol_keep);
-                c.advance(p);
+                    tma_load_3d(dst + k * b_tile_bytes, &maps.x, (c.kb0() + k) * kBlockK, full, pol_keep);
+                c.advance();
                 ++i;
                 if (++s == p.stages) s = 0;
             }
         } else {
             pdl_wait();
+            pdl_launch_dependents();
         }
     } else if (warp == 1) {
         // ================================================= MMA issuer
         if (lane == 0) {
             const uint32_t idesc = make_idesc(kTileM, (int)nb);
             Cursor<PK> c;
-            c.init(p);
+            c.init(d);
             uint32_t seg = 0, ph = 0;   // ph: parity the MMA warp waits for on its stage's "full" barrier
             int s = 0;
-            while (!c.done(p) && !timed_out) {
+            while (!c.done() && !timed_out) {
                 // one segment: the items of one tile that belong to this CTA
-                const int cg = c.g, tile = c.tile, halves = c.halves;
+                const int tile = c.tile, halves = c.halves;
                 const int buf = two_bufs ? (seg & 1) : 0;
                 const uint32_t use = two_bufs ? (seg >> 1) : seg;     // how often this buffer has been used before
                 if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, abort_flag, wait_limit)) { timed_out = true; break; }
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + buf * acc_cols;
-                for (int q = 0; c.g == cg && c.tile == tile; ++q) {
+                for (int q = 0; !c.done() && c.tile == tile; ++q) {
                     if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag, wait_limit)) { timed_out = true; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * stage_bytes;
@@ -738,267 +683,72 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                         }
                     }
                     tc_commit(smem_u32(&ctl.empty[s]));  // frees the stage when these MMAs have read it
-                    c.advance(p);
+                    c.advance();
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
                 if (timed_out) break;
                 tc_commit(smem_u32(&ctl.tmem_full[buf]));
                 ++seg;
             }
-            if (p.n_gemms == 1) LLMCAD_TRACE(7);
+            LLMCAD_TRACE(7);
         }
-    } else if (warp < 6) {
-        // ================================================= epilogue (warps 2..5)
+    } else {
+        // ================================================= accumulator dump (warps 2..5)
         const int lane_grp = warp & 3;                 // TMEM lanes 32*lane_grp .. +31 belong to this warp
-        float *my_rs = ctl.rs[warp - 2];
+        // the workspace may still be read by the finishing kernel of the previous GEMM
         pdl_wait();
+        pdl_launch_dependents();
         if (threadIdx.x == 64) LLMCAD_TRACE(3);
-        // The previous launch (complete now) counted arrivals in the other counter set; the launch
-        // after this one will use that set again: put the words it touched back to zero.
-        for (int g = 0; g < p.prev_gemms; ++g) {
-            uint32_t *old = p.arrivals + ((size_t)(p.arrival_set ^ 1) * kMaxChain + g) * kArrivalsPerGemm;
-            for (int i = (int)blockIdx.x * 128 + (int)threadIdx.x - 64; i < p.prev_arrival_words; i += (int)gridDim.x * 128) old[i] = 0;
-        }
+        const Range r = cta_range<PK>(d, (int)blockIdx.x);
+        const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
+        const size_t slot_stride = slot_floats(d.halves, p.n_pad);
         uint32_t seg = 0;
-        for (int g = 0; g < p.n_gemms && !timed_out; ++g) {
-            const GemmDesc &d = s_desc[g];
-            const EpiParams &ep = d.ep;
-            // ---- grid barrier: everything GEMM g-1 wrote (activations, residual, norm sums) is final
-            if (g > 0) {
-                int bad = 0;
-                if (lane == 0) {
-                    const uint32_t target = arrivals_per_gemm * (uint32_t)g;
-                    const uint64_t t0 = global_timer_ns();
-                    for (uint32_t spin = 0; (int32_t)(ld_acquire_u32(p.grid_counter) - p.barrier_base - target) < 0; ++spin) {
-                        __nanosleep(100);
-                        if ((spin & 15u) == 15u && (*abort_flag || global_timer_ns() - t0 > wait_limit)) { bad = 1; break; }
+        for (int seg_begin = r.begin; seg_begin < r.end; ++seg) {
+            const int tile = seg_begin / ipt;
+            const int seg_end = min(r.end, (tile + 1) * ipt);
+            const int buf = two_bufs ? (seg & 1) : 0;
+            const uint32_t use = two_bufs ? (seg >> 1) : seg;
+            if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), use & 1u, abort_flag, lane, wait_limit)) { timed_out = true; break; }
+            tc_fence_after();
+            if (threadIdx.x == 64 && seg == 0) LLMCAD_TRACE(4);
+            // this CTA's segment of the tile goes to slot tile + CTA, lane = row of the 32-row group;
+            // with hi + lo activations a node's two accumulator columns are added first
+            const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * acc_cols;
+            float *dst = p.partials + (size_t)(tile + (int)blockIdx.x) * slot_stride + (size_t)lane_grp * d.halves * p.n_pad * 32 + lane;
+            for (int hf = 0; hf < d.halves; ++hf) {
+                int c0 = 0;
+                if (p.comp) {
+                    // 32 nodes at a time, hi and lo columns in one round trip
+                    for (; c0 + 32 <= p.n_pad; c0 += 32) {
+                        float v[32];
+                        tc_ld32_sum2(t_lane + hf * nb + c0, t_lane + hf * nb + p.n_pad + c0, v);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) dst[(size_t)(hf * p.n_pad + c0 + j) * 32] = v[j];
                     }
-                    __threadfence();
                 }
-                if (__shfl_sync(0xffffffffu, bad, 0)) { timed_out = true; break; }
-            }
-            // ---- RMSNorm of the GEMM input folded into the epilogue: the producer of the residual
-            // stream left partial sums of squares per node; every warp keeps its own copy of the
-            // per-node factors (no block-level barrier among the epilogue warps). The factors are
-            // needed for finishing only, and adding up the partial rows takes tens of microseconds
-            // with many nodes: where the MMA warp has one accumulator buffer only, it happens after
-            // this warp's first share has left TMEM, so that the MMA warp is not kept waiting for it.
-            bool rs_ready = ep.ssq_in == nullptr;
-            // items the MMA warp works through while the factors are being summed: a lane reads every
-            // (32 / quads)-th partial row, eight at a time, ~0.8 us per round against ~0.35 us per item
-            const int rs_items = ((ep.ssq_in_parts * (p.n_pad > 64 ? 4 : (p.n_pad > 32 ? 2 : 1)) / 4 + 7) / 8) * 2;
-            auto compute_rs = [&]() {
-                // rows of ssq_in hold 128 floats (one per node); read them as float4 "quads". A lane
-                // owns one quad and every (32 / quads)-th partial row, eight loads in flight at a time;
-                // the lane groups are then added in a fixed order, so the sum does not depend on timing.
-                int qp = 4;
-                while (qp * 4 < p.n_pad) qp <<= 1;                 // quads, rounded up to 4, 8, 16 or 32
-                const int groups = 32 / qp, quad = lane & (qp - 1), slice = lane / qp;
-                const float4 *rows = reinterpret_cast<const float4 *>(ep.ssq_in) + quad;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                int t = slice;
-                for (; t + 7 * groups < ep.ssq_in_parts; t += 8 * groups) {
-                    float4 v[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) v[u] = __ldcg(rows + (size_t)(t + u * groups) * (LLMCAD_MAX_TREE / 4));
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
-                }
-                for (; t < ep.ssq_in_parts; t += groups) {
-                    const float4 v = __ldcg(rows + (size_t)t * (LLMCAD_MAX_TREE / 4));
-                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-                }
-                for (int off = qp; off < 32; off <<= 1) {
-                    acc.x += __shfl_xor_sync(0xffffffffu, acc.x, off);
-                    acc.y += __shfl_xor_sync(0xffffffffu, acc.y, off);
-                    acc.z += __shfl_xor_sync(0xffffffffu, acc.z, off);
-                    acc.w += __shfl_xor_sync(0xffffffffu, acc.w, off);
-                }
-                if (lane < qp) {
-                    const float inv_d = 1.0f / (float)ep.norm_d;
-                    my_rs[4 * quad + 0] = rsqrtf(acc.x * inv_d + ep.eps);
-                    my_rs[4 * quad + 1] = rsqrtf(acc.y * inv_d + ep.eps);
-                    my_rs[4 * quad + 2] = rsqrtf(acc.z * inv_d + ep.eps);
-                    my_rs[4 * quad + 3] = rsqrtf(acc.w * inv_d + ep.eps);
-                }
-                __syncwarp();
-            };
-            const Range r = cta_range<PK>(d);
-            const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
-            const bool dual = d.halves == 2;
-            const size_t part_stride = (size_t)2 * p.n_pad * kTileM;   // floats per workspace slot (gate | up)
-            uint32_t *arrivals = p.arrivals + ((size_t)p.arrival_set * kMaxChain + g) * kArrivalsPerGemm;
-            for (int seg_begin = r.begin; seg_begin < r.end && !timed_out; ++seg) {
-                const int tile = seg_begin / ipt;
-                const int tile_i0 = tile * ipt;
-                const int seg_end = min(r.end, tile_i0 + ipt);
-                const int buf = two_bufs ? (seg & 1) : 0;
-                const uint32_t use = two_bufs ? (seg >> 1) : seg;
-                const int first_cta = tile_i0 / d.items_per_cta;
-                const int last_cta = (tile_i0 + ipt - 1) / d.items_per_cta;
-                const int n_parts = last_cta - first_cta + 1;           // CTAs that hold a share of this tile
-                const bool tail = p.n_gemms == 1 && seg_end == r.end;   // (tracing) the segment that ends this CTA's work
-                // the norm factors: at once, unless the MMA warp has a single accumulator buffer and this first
-                // segment only leaves a share and is shorter than the summing takes (then after that share has
-                // left TMEM, i.e. before the second segment)
-                if (!rs_ready && (two_bufs || n_parts == 1 || seg_end == r.end || seg_begin != r.begin || seg_end - seg_begin >= rs_items)) {
-                    compute_rs();
-                    rs_ready = true;
-                }
-
-                if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), use & 1u, abort_flag, lane, wait_limit)) { timed_out = true; break; }
-                tc_fence_after();
-                if (threadIdx.x == 64 && g < 4 && seg_begin == r.begin) LLMCAD_TRACE(4 + 2 * g);
-                if (threadIdx.x == 64 && tail) LLMCAD_TRACE(14);
-
-                // ---- this CTA's share of the tile goes to the workspace, lane = row of the 32-row group.
-                // With hi + lo activations a node's two accumulator columns are added first. Slot 0 of a
-                // CTA holds the tile in which its range starts, slot 1 any later one (a later tile is
-                // finished, by this same warp, before the next one is written).
-                const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * acc_cols;
-                float *dst = p.partials + ((size_t)blockIdx.x * 2 + (seg_begin == r.begin ? 0 : 1)) * part_stride +
-                             (size_t)lane_grp * 2 * p.n_pad * 32 + lane;
-                for (int hf = 0; hf < (dual ? 2 : 1); ++hf) {
-                    int c0 = 0;
+                for (; c0 < p.n_pad; c0 += 16) {
+                    float v[16];
+                    tc_ld16(t_lane + hf * nb + c0, v);
                     if (p.comp) {
-                        // 32 nodes at a time, hi and lo columns in one round trip
-                        for (; c0 + 32 <= p.n_pad; c0 += 32) {
-                            float v[32];
-                            tc_ld32_sum2(t_lane + hf * nb + c0, t_lane + hf * nb + p.n_pad + c0, v);
+                        float t[16];
+                        tc_ld16(t_lane + hf * nb + p.n_pad + c0, t);
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) dst[(size_t)(hf * p.n_pad + c0 + j) * 32] = v[j];
-                        }
+                        for (int j = 0; j < 16; ++j) v[j] += t[j];
                     }
-                    for (; c0 < p.n_pad; c0 += 16) {
-                        float v[16];
-                        tc_ld16(t_lane + hf * nb + c0, v);
-                        if (p.comp) {
-                            float t[16];
-                            tc_ld16(t_lane + hf * nb + p.n_pad + c0, t);
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) v[j] += t[j];
-                        }
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) dst[(size_t)(hf * p.n_pad + c0 + j) * 32] = v[j];
-                    }
-                }
-                if (threadIdx.x == 64 && tail) LLMCAD_TRACE(8);
-                // the accumulator has left TMEM: hand the buffer back to the MMA warp
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
-
-                // ---- finishing. The rows of a tile are independent per warp (32 rows each), so each
-                // warp works with the same-numbered warps of the other CTAs that hold a share of the
-                // tile, through one arrival counter per (tile, row group). The CTAs whose range ends in
-                // this tile (all holders, except the last one when its range goes on into the next tile)
-                // have nothing left to do: each waits until every share has arrived and finishes its
-                // part of the nodes. A CTA that goes on only announces its share; it held the tile's
-                // last k-blocks first thing in the kernel, so nobody waits for it in practice, and it
-                // waits for nobody. The counters are put back to zero by the next launch.
-                FinishArgs fa;
-                fa.p = &p; fa.d = &d; fa.rs = my_rs;
-                fa.tile = tile; fa.tile_i0 = tile_i0; fa.first_cta = first_cta; fa.last_cta = last_cta; fa.lane_grp = lane_grp;
-                fa.trace = (threadIdx.x == 64 && tail && p.trace) ? p.trace + (size_t)blockIdx.x * 16 : nullptr;
-                // The segment that ends this CTA's work in the launch: the warp of another role with
-                // the same row group (idle by now) takes every other node group (see the helpers below).
-                const bool helped = g + 1 == p.n_gemms && seg_end == r.end;
-                if (n_parts == 1) {
-                    if (helped) {
-                        __threadfence_block();
-                        __syncwarp();
-                        if (lane == 0) ctl.dumped[lane_grp] = 1;
-                    }
-                    fa.it_first = 0; fa.it_step = helped ? 2 : 1;
-                    finish_rows(fa, lane);
-                } else {
-                    uint32_t *ctr = arrivals + (size_t)tile * 4 + lane_grp;
-                    __syncwarp();
-                    // release: the share written by all lanes of this warp is visible to whoever sees the count
-                    if (lane == 0) {
-                        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
-                        if (helped) ctl.dumped[lane_grp] = 1;
-                    }
-                    if (threadIdx.x == 64 && tail) LLMCAD_TRACE(9);
-                    if (seg_end == r.end) {
-                        // (a range never goes beyond the last tile)
-                        const int n_fin = n_parts - ((min((last_cta + 1) * d.items_per_cta, d.n_tiles * ipt) > tile_i0 + ipt) ? 1 : 0);
-                        int bad = 0;
-                        if (lane == 0) {
-                            uint64_t t0 = 0;
-                            for (uint32_t spin = 0; ld_acquire_u32(ctr) < (uint32_t)n_parts; ++spin) {
-                                __nanosleep(64);
-                                if ((spin & 15u) == 15u) {
-                                    if (t0 == 0) t0 = global_timer_ns();
-                                    else if (*abort_flag || global_timer_ns() - t0 > wait_limit) { bad = 1; break; }
-                                }
-                            }
-                        }
-                        if (__shfl_sync(0xffffffffu, bad, 0)) { timed_out = true; break; }
-                        if (threadIdx.x == 64 && tail) LLMCAD_TRACE(10);
-                        fa.it_first = ((int)blockIdx.x - first_cta) * (helped ? 2 : 1); fa.it_step = n_fin * (helped ? 2 : 1);
-                        finish_rows(fa, lane);
-                    }
-                }
-                if (threadIdx.x == 64 && tail) LLMCAD_TRACE(13);
-                seg_begin = seg_end;
-            }
-            if (timed_out) break;
-            if (threadIdx.x == 64 && g < 4) LLMCAD_TRACE(5 + 2 * g);
-            // ---- this warp is done with GEMM g: arrive at the grid barrier that gates GEMM g+1
-            if (g + 1 < p.n_gemms) {
-                __syncwarp();
-                if (lane == 0) {
-                    __threadfence();
-                    atomicAdd(p.grid_counter, 1u);
+                    for (int j = 0; j < 16; ++j) dst[(size_t)(hf * p.n_pad + c0 + j) * 32] = v[j];
                 }
             }
+            // the accumulator has left TMEM: hand the buffer back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+            seg_begin = seg_end;
         }
+        if (threadIdx.x == 64) LLMCAD_TRACE(8);
     }
     __syncwarp();   // lanes that skipped their role's single-thread section rejoin their warp here
     timed_out = __any_sync(0xffffffffu, timed_out);   // keep the warp together on the way out
-
-    // ================================================= helpers
-    // The producer, MMA, loader and spare warps have nothing left to do when the launch's last GEMM
-    // reaches its tail, which is exactly when the epilogue warps have the most: each takes the row
-    // group warp % 4 of this CTA's last tile and finishes every other node group of it, next to the
-    // epilogue warp that owns the group (which takes the others).
-    if (!timed_out && (warp < 2 || warp > 5)) {
-        const int g = p.n_gemms - 1;
-        const GemmDesc &d = s_desc[g];
-        const Range r = cta_range<PK>(d);
-        if (r.end > r.begin) {
-            const int lane_grp = warp & 3;
-            const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
-            const int tile = (r.end - 1) / ipt, tile_i0 = tile * ipt;
-            const int first_cta = tile_i0 / d.items_per_cta, last_cta = (tile_i0 + ipt - 1) / d.items_per_cta;
-            const int n_parts = last_cta - first_cta + 1;
-            const int n_fin = n_parts == 1 ? 1 : n_parts - ((min((last_cta + 1) * d.items_per_cta, d.n_tiles * ipt) > tile_i0 + ipt) ? 1 : 0);
-            const uint32_t *ctr = p.arrivals + ((size_t)p.arrival_set * kMaxChain + g) * kArrivalsPerGemm + (size_t)tile * 4 + lane_grp;
-            int bad = 0;
-            if (lane == 0) {
-                // this CTA's own share first (a flag in shared memory), then everybody's (the arrival counter)
-                uint64_t t0 = 0;
-                for (uint32_t spin = 0; ctl.dumped[lane_grp] == 0 || (n_parts > 1 && ld_acquire_u32(ctr) < (uint32_t)n_parts); ++spin) {
-                    __nanosleep(ctl.dumped[lane_grp] == 0 ? 200 : 64);
-                    if ((spin & 15u) == 15u) {
-                        if (t0 == 0) t0 = global_timer_ns();
-                        else if (*abort_flag || global_timer_ns() - t0 > wait_limit) { bad = 1; break; }
-                    }
-                }
-                __threadfence_block();
-            }
-            if (__shfl_sync(0xffffffffu, bad, 0)) timed_out = true;
-            else {
-                FinishArgs fa;
-                fa.p = &p; fa.d = &d; fa.rs = ctl.rs[lane_grp < 2 ? lane_grp + 2 : lane_grp - 2];   // of the epilogue warp of this row group
-                fa.tile = tile; fa.tile_i0 = tile_i0; fa.first_cta = first_cta; fa.last_cta = last_cta; fa.lane_grp = lane_grp;
-                fa.trace = nullptr;
-                fa.it_first = ((int)blockIdx.x - first_cta) * 2 + 1; fa.it_step = n_fin * 2;
-                finish_rows(fa, lane);
-            }
-        }
-    }
 
     if (timed_out) {
         *abort_flag = 1;
@@ -1011,8 +761,102 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
-        if (lane == 0) LLMCAD_TRACE(12);
+        if (lane == 0) LLMCAD_TRACE(13);
     }
+}
+
+// Adds the segments of every tile and applies the fused epilogue; see the head of the file. The
+// work is cut into (tile, 32-row group) pairs; k warps share a pair's node groups, k chosen so that
+// all warps of the grid have work. G node groups and KB segments of each are loaded in one go
+// (the launcher picks them so that a warp normally needs a single round trip to L2).
+//
+// Until the grid dependency (the streaming kernel) resolves, the CTA has nothing to do but sits on
+// its SM already. It uses the time (a) to read what earlier GEMMs left: the description, the norm
+// sums, the gains; (b) for a dry run of its own work with the stores switched off, on whatever the
+// workspace holds: the code of this kernel runs once per launch and would be fetched from L2 line
+// by line otherwise, which costs more than the work itself.
+template <int MODE, int G, int KB>
+__global__ void __maxnreg__(kFinMaxRegs)
+gemm_finish_kernel(const __grid_constant__ GemmParams p)
+{
+    // The finishing code reads the GEMM's description (pointers, sizes, mode) all over. From the kernel
+    // parameters every first touch of a constant-cache line is a miss; a copy in shared memory costs
+    // nothing to read.
+    __shared__ __align__(16) GemmDesc s_desc;
+    __shared__ float s_part[kFinThreads / LLMCAD_MAX_TREE][LLMCAD_MAX_TREE];
+    __shared__ float s_rs[LLMCAD_MAX_TREE];
+    {
+        static_assert(sizeof(GemmDesc) % 4 == 0, "GemmDesc is copied word by word");
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(&p.g);
+        uint32_t *dst = reinterpret_cast<uint32_t *>(&s_desc);
+        for (int i = threadIdx.x; i < (int)(sizeof(GemmDesc) / 4); i += kFinThreads) dst[i] = src[i];
+    }
+    pdl_launch_dependents();     // the next GEMM's streaming kernel may take the SMs as they free up
+    if (threadIdx.x == 0) LLMCAD_TRACE(9);
+    __syncthreads();
+    const GemmDesc &d = s_desc;
+    const EpiParams &ep = d.ep;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- RMSNorm of the GEMM input folded into the epilogue: the producer of the residual stream
+    // left partial sums of squares per node ([parts][128]); the accumulators of node i are multiplied
+    // by rsqrt(mean(x^2) + eps). Three threads per node add every third partial row, in a fixed order.
+    if (ep.ssq_in != nullptr) {
+        constexpr int kSlices = kFinThreads / LLMCAD_MAX_TREE;
+        const int node = threadIdx.x & (LLMCAD_MAX_TREE - 1), slice = threadIdx.x / LLMCAD_MAX_TREE;
+        float acc = 0.f;
+        if (node < p.n_pad) {
+            const float *col = ep.ssq_in + node;
+            int t = slice;
+            for (; t + 7 * kSlices < ep.ssq_in_parts; t += 8 * kSlices) {
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = __ldcg(col + (size_t)(t + kSlices * u) * LLMCAD_MAX_TREE);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) acc += v[u];
+            }
+            for (; t < ep.ssq_in_parts; t += kSlices) acc += __ldcg(col + (size_t)t * LLMCAD_MAX_TREE);
+        }
+        s_part[slice][node] = acc;
+        __syncthreads();
+        if (threadIdx.x < LLMCAD_MAX_TREE) {
+            float sum = 0.f;
+#pragma unroll
+            for (int q = 0; q < kSlices; ++q) sum += s_part[q][threadIdx.x];
+            s_rs[threadIdx.x] = rsqrtf(sum / (float)ep.norm_d + ep.eps);
+        }
+        __syncthreads();
+    }
+
+    const int ipt = pairs_per_tile(d) * d.halves;
+    const int pairs = d.n_tiles * 4, iters = p.n_pad >> 2;
+    const int W = (int)gridDim.x * (kFinThreads / 32);
+    int k = W / pairs;
+    k = k < 1 ? 1 : (k > iters ? iters : k);
+    const int groups = W / k;
+    const int wg = warp * (int)gridDim.x + (int)blockIdx.x;      // consecutive pairs on different SMs
+
+    for (int round = 0; round < 2; ++round) {
+        const bool dry = round == 0;
+        if (!dry) {
+            pdl_wait();                  // every segment is in the workspace
+            if (threadIdx.x == 0) LLMCAD_TRACE(10);
+        }
+        if (wg < groups * k) {
+            for (int pair = wg / k; pair < pairs; pair += groups) {
+                FinishArgs fa;
+                fa.p = &p; fa.d = &d; fa.rs = s_rs;
+                fa.tile = pair >> 2; fa.lane_grp = pair & 3;
+                const int tile_i0 = fa.tile * ipt;
+                fa.first_cta = tile_i0 / d.items_per_cta;
+                fa.last_cta = (tile_i0 + ipt - 1) / d.items_per_cta;
+                fa.it_first = wg % k; fa.it_step = k;
+                finish_rows_t<G, KB, MODE>(fa, lane, dry);
+                if (dry) break;          // one pair is enough to have walked through the code
+            }
+        }
+    }
+    if (threadIdx.x == 0) LLMCAD_TRACE(12);
 }
 
 // ------------------------------------------------------------------------------------------ host
@@ -1079,7 +923,7 @@ bool make_tensor_map_bf16_3d(CUtensorMap *map, const void *base, const uint64_t 
     return r == CUDA_SUCCESS;
 }
 
-size_t gemm_tc_partial_floats(int n_sms, int max_n_pad) { return (size_t)n_sms * 2 /*slots*/ * 2 /*gate|up*/ * max_n_pad * kTileM; }
+size_t gemm_tc_partial_floats(int n_sms, int max_tiles, int max_n_pad) { return (size_t)(max_tiles + n_sms) * slot_floats(2, max_n_pad); }
 
 GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)
 {
@@ -1090,22 +934,16 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)
     d.pair_k = kMaxPairK;
     d.up_row_offset = ep.n_out;
     d.items_per_cta = 0;
+    d.grid = 0;
     d.w_tiled = static_cast<const uint8_t *>(w_tiled);
     d.up_tile_offset = d.n_tiles;
     d.ep = ep;
     return d;
 }
 
-cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, cudaStream_t st, uint32_t *barrier_arrivals)
+cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_t partial_floats, cudaStream_t st, int *launched)
 {
-    if (p.n_gemms < 1 || p.n_gemms > kMaxChain) return cudaErrorInvalidValue;
-    // a chain needs every CTA at every barrier: the grid is the SM count; a single GEMM may use fewer
-    long long max_items = 0;
-    // Ring items of two k-blocks (one 32 KB weight copy each) unless the activation tiles are so wide
-    // (hi | lo planes of more than 64 nodes) that only two stages would fit; measured on B200:
-    // single k-blocks cost 10-17 % up to 64 nodes and gain 6 % at 128.
-    const int nb = p.n_pad * (p.comp ? 2 : 1);       // MMA N
-    if (nb > 256) return cudaErrorInvalidValue;
+    if (launched) *launched = 0;
     // tuning aids from the environment, read once per process
     struct Tuning {
         int pair_k = 0, stages_cap = 0, l2_ahead = 8;
@@ -1117,36 +955,34 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
         }
     };
     static const Tuning tune;
+    // Ring items of two k-blocks (one 32 KB weight copy each) unless the activation tiles are so wide
+    // (hi | lo planes of more than 64 nodes) that only two stages would fit; measured on B200:
+    // single k-blocks cost 10-17 % up to 64 nodes and gain 6 % at 128.
+    const int nb = p.n_pad * (p.comp ? 2 : 1);       // MMA N
+    if (nb > 256 || p.n_pad < 16 || p.n_pad % 16) return cudaErrorInvalidValue;
     int pair_k = nb > 128 ? 1 : kMaxPairK;
     if (tune.pair_k) pair_k = tune.pair_k;
-    for (int g = 0; g < p.n_gemms; ++g) p.g[g].pair_k = pair_k;
-    auto items_of = [](const GemmDesc &d) { return (long long)d.n_tiles * pairs_per_tile(d) * d.halves; };
-    for (int g = 0; g < p.n_gemms; ++g) {
-        if (p.g[g].n_tiles > 4096) return cudaErrorInvalidValue;   // size of the arrival-counter array
-        const long long total = items_of(p.g[g]);
-        if (total > max_items) max_items = total;
-    }
-    int grid = n_sms;
-    if (p.n_gemms == 1 && max_items < grid) grid = (int)max_items;
-    for (int g = 0; g < p.n_gemms; ++g) {
-        const long long total = items_of(p.g[g]);
-        long long ipc = (total + grid - 1) / grid;
-        if (p.g[g].halves == 2) ipc += ipc & 1;   // ranges of a two-half GEMM start on a gate item
-        p.g[g].items_per_cta = (int)ipc;
-    }
-    if (p.n_gemms == 1) {
-        const long long total = items_of(p.g[0]);
-        grid = (int)((total + p.g[0].items_per_cta - 1) / p.g[0].items_per_cta);
-    }
+    GemmDesc &d = p.g;
+    d.pair_k = pair_k;
+    // the items are split evenly over one CTA per SM (fewer CTAs when there are fewer items)
+    const long long total = (long long)d.n_tiles * pairs_per_tile(d) * d.halves;
+    if (total < 1) return cudaErrorInvalidValue;
+    int grid = total < n_sms ? (int)total : n_sms;
+    long long ipc = (total + grid - 1) / grid;
+    if (d.halves == 2) ipc += ipc & 1;   // ranges of a two-half GEMM start on a gate item
+    d.items_per_cta = (int)ipc;
+    grid = (int)((total + ipc - 1) / ipc);
+    d.grid = grid;
+    if ((size_t)(d.n_tiles + grid) * slot_floats(d.halves, p.n_pad) > partial_floats) return cudaErrorInvalidValue;
     const size_t stage_bytes = (size_t)pair_k * ((size_t)kATileBytes + (size_t)nb * kBlockK * 2);
-    // One CTA per SM with the whole shared memory as the ring. (Two CTAs per SM with half-size rings,
-    // so that the next kernel is resident during this one's tail, measured slower on B200.)
+    // One CTA per SM with the whole shared memory as the ring.
     // accumulators: (gate | up) x MMA N columns each, double-buffered when two of them fit
     p.acc_bufs = 4 * nb <= 512 ? 2 : 1;
     int cols = p.acc_bufs * 2 * nb, pow2 = 32;
     while (pow2 < cols) pow2 <<= 1;
     p.tmem_cols = pow2;
-    const size_t full_limit = 227 * 1024 - 1024 /*alignment slack*/ - 4096 /*static*/;
+    // the ring takes what the SM has, less the room that the finishing CTA of the previous GEMM needs beside it
+    const size_t full_limit = 227 * 1024 - 1024 /*alignment slack*/ - 2048 /*static*/ - (kFinSmem + 4096);
     int stages = (int)(full_limit / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (tune.stages_cap && tune.stages_cap < stages) stages = tune.stages_cap;   // tuning aid: cap the ring depth
@@ -1155,21 +991,65 @@ cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, 
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     static PerDeviceOnce attr_set;
     if (attr_set.needed()) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_chain_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             227 * 1024 - 4096);
+        cudaError_t e = cudaFuncSetAttribute(gemm_stream_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(gemm_chain_kernel<__nv_bfloat16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     227 * 1024 - 4096);
+            e = cudaFuncSetAttribute(gemm_stream_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
+        // An SM splits its on-chip memory between shared memory and L1 when it is empty, to fit the kernel that
+        // arrives; a streaming CTA of 195 KB would get a 196 KB split, and the finishing CTA of the same GEMM
+        // could not settle beside it. Every kernel of the GEMM asks for the largest shared-memory split.
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_stream_kernel<1>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_stream_kernel<2>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set.mark();
     }
     // weight tiles pulled into L2 beyond the ring while the ring is blocked
     p.l2_ahead = tune.l2_ahead;
     if (p.wait_limit_ns == 0) p.wait_limit_ns = kDefaultWaitLimitNs;
-    if (barrier_arrivals) *barrier_arrivals = 4u * (uint32_t)grid * (uint32_t)(p.n_gemms - 1);
-    LaunchCfg lc(grid, kThreads, smem, st);
-    if (pair_k == 1) return cudaLaunchKernelEx(&lc.cfg, gemm_chain_kernel<__nv_bfloat16, 1>, maps, p);
-    return cudaLaunchKernelEx(&lc.cfg, gemm_chain_kernel<__nv_bfloat16, 2>, maps, p);
+    {
+        LaunchCfg lc(grid, kThreads, smem, st);
+        const cudaError_t e = pair_k == 1 ? cudaLaunchKernelEx(&lc.cfg, gemm_stream_kernel<1>, maps, p)
+                                          : cudaLaunchKernelEx(&lc.cfg, gemm_stream_kernel<2>, maps, p);
+        if (e != cudaSuccess) return e;
+        if (launched) ++*launched;
+    }
+    // finishing: (tile, row group) pairs x node groups of four, one warp-iteration each; G node groups and
+    // KB segments per round trip so that the warps get through in one round where registers allow
+    const long long units = (long long)d.n_tiles * 4 * (p.n_pad / 4);
+    const int warps_per_cta = kFinThreads / 32;
+    int fgrid = (int)((units + warps_per_cta - 1) / warps_per_cta);
+    if (fgrid > n_sms) fgrid = n_sms;
+    const long long per_warp = (units + (long long)fgrid * warps_per_cta - 1) / ((long long)fgrid * warps_per_cta);
+    const int max_parts = (int)(((long long)pairs_per_tile(d) * d.halves + ipc - 1) / ipc) + 1;
+    const bool wide = max_parts > 4;           // many segments per tile (tiles split over many CTAs)
+    const bool two = per_warp >= 2;            // several node groups per warp
+    typedef void (*FinKernel)(GemmParams);
+    FinKernel fk = nullptr;
+#define LLMCAD_PICK(MODE)                                                                                            \
+    fk = wide ? (FinKernel)gemm_finish_kernel<MODE, 1, 8>                                                            \
+              : (two ? (FinKernel)gemm_finish_kernel<MODE, 2, 4> : (FinKernel)gemm_finish_kernel<MODE, 1, 4>)
+    switch (d.ep.mode) {
+    case EPI_QKV: LLMCAD_PICK(EPI_QKV); break;
+    case EPI_RESID: LLMCAD_PICK(EPI_RESID); break;
+    case EPI_SWIGLU:
+        fk = wide ? (FinKernel)gemm_finish_kernel<EPI_SWIGLU, 1, 4> : (two ? (FinKernel)gemm_finish_kernel<EPI_SWIGLU, 2, 2> : (FinKernel)gemm_finish_kernel<EPI_SWIGLU, 1, 4>);
+        break;
+    default: LLMCAD_PICK(EPI_PLAIN); break;
+    }
+#undef LLMCAD_PICK
+    {
+        // once per finishing kernel and device (see above)
+        static PerDeviceOnce fin_set[4][3];
+        PerDeviceOnce &once = fin_set[d.ep.mode & 3][wide ? 0 : (two ? 1 : 2)];
+        if (once.needed()) {
+            const cudaError_t e = cudaFuncSetAttribute(fk, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+            if (e != cudaSuccess) return e;
+            once.mark();
+        }
+    }
+    LaunchCfg lf(fgrid, kFinThreads, kFinSmem, st);
+    const cudaError_t e = cudaLaunchKernelEx(&lf.cfg, fk, p);
+    if (e == cudaSuccess && launched) ++*launched;
+    return e;
 }
 
 }  // namespace llmcad

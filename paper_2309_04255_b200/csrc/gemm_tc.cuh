@@ -1,4 +1,6 @@
-// Host-visible interface of the tensor-core skinny-GEMM chain kernel (gemm_tc.cu).
+// Host-visible interface of the tensor-core skinny GEMM (gemm_tc.cu): a weight-streaming kernel that
+// leaves the accumulators of every tile segment in a workspace, and a finishing kernel that adds the
+// segments of each tile and applies the fused epilogue.
 #pragma once
 
 #include <cuda.h>
@@ -7,45 +9,40 @@
 
 namespace llmcad {
 
-constexpr int kMaxChain = 4;
-
-// One GEMM of a chain: D[n_out][n] = W[n_out][n_in] X[n][n_in]^T followed by its fused epilogue.
+// One GEMM: D[n_out][n] = W[n_out][n_in] X[n][n_in]^T followed by its fused epilogue.
 struct GemmDesc {
     int n_tiles;        // tiles of 128 output features
     int kb_per_tile;    // 64-wide k-blocks per tile
     int pair_k;         // k-blocks per ring item (1 or 2), set by the launcher
     int halves;         // 2: every tile carries a gate and an up accumulator (SwiGLU), else 1
     int up_row_offset;  // row of the first up-projection row in the packed [2f][d] matrix
-    int items_per_cta;  // ring items ((tile, k-block, half) triples) per CTA of the persistent grid
+    int items_per_cta;  // ring items ((tile, k-block, half) triples) per CTA of the streaming grid
+    int grid;           // CTAs of the streaming grid
     const uint8_t *w_tiled;  // weights as a sequence of pre-swizzled 16 KB tiles [tile][k-block] (see pack.cu),
                              // or nullptr: row-major weights through the tensor map
     int up_tile_offset;      // first tile of the up projection in the tiled sequence
     EpiParams ep;
 };
 
-struct ChainMaps {
-    CUtensorMap w[kMaxChain];  // weight matrices, box 64 x 128 rows
-    CUtensorMap x[kMaxChain];  // the activation matrix each GEMM multiplies, box 64 x n_pad rows x planes (hi, lo)
+struct GemmMaps {
+    CUtensorMap w;  // weight matrix, box 64 x 128 rows (row-major weights only)
+    CUtensorMap x;  // the activation matrix, box 64 x n_pad rows x planes (hi, lo)
 };
 
-struct ChainParams {
-    int n_gemms;
+struct GemmParams {
     int n_pad;          // tree nodes padded to a multiple of 16
-    int comp;           // 1: activations come as hi + lo planes; the MMA N is 2 * n_pad and the epilogue adds the two
+    int comp;           // 1: activations come as hi + lo planes; the MMA N is 2 * n_pad and the two columns of a node are added
     int acc_bufs;       // accumulator buffers in TMEM: 2, or 1 when 2 x (gate | up) x MMA N exceeds the 512 columns
     int stages;         // depth of the shared-memory ring
     int tmem_cols;      // allocated TMEM columns (power of two)
-    float *partials;    // [grid][2 slots][2 halves][n_pad][128] fp32 partial tiles
-    uint32_t *arrivals;  // [2 sets][kMaxChain][4096][4] arrivals per (GEMM, tile, 32-row group)
-    int arrival_set;     // the set this launch counts in (launches alternate); it finds it all zero
-    int prev_gemms, prev_arrival_words;   // what the previous launch touched in the other set: this launch zeroes it
-    uint32_t *grid_counter;   // grid barrier between the GEMMs of a chain (monotonic)
-    uint32_t barrier_base;    // value of the counter when this launch starts
+    float *partials;    // segment slots [n_tiles + grid][4 row groups][halves][n_pad][32 rows] fp32: the segment of
+                        // tile t held by CTA c sits in slot t + c
     int32_t *status;
-    unsigned long long *trace;  // optional [grid][16] timeline in ns (nullptr: off)
+    unsigned long long *trace;  // optional [256][16] timeline in ns of this GEMM (nullptr: off)
     int l2_ahead;       // ring items the producer may prefetch into L2 beyond the ring
+    int withhold_act;   // self-test of the wait limit: the activation copies are never issued
     uint64_t wait_limit_ns;   // bound of every device-side wait of the launch
-    GemmDesc g[kMaxChain];
+    GemmDesc g;
 };
 
 // Tensor map over a row-major bf16 matrix [rows][cols] with a box of 64 columns x box_rows rows
@@ -62,15 +59,15 @@ bool make_act_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64
 bool make_tensor_map_bf16_3d(CUtensorMap *map, const void *base, const uint64_t dims[3], const uint64_t strides_bytes[2],
                              const uint32_t box[3]);
 
-size_t gemm_tc_partial_floats(int n_sms, int max_n_pad);
-constexpr size_t kArrivalsPerGemm = 4096 * 4;
-constexpr size_t kArrivalWords = 2 * kMaxChain * kArrivalsPerGemm;   // both sets
+// Floats of segment workspace that GEMMs of up to max_tiles tiles on up to max_n_pad nodes need.
+size_t gemm_tc_partial_floats(int n_sms, int max_tiles, int max_n_pad);
 
-// Describes one GEMM for a chain (fills everything but items_per_cta, which the launcher sets).
+// Describes one GEMM (fills everything but items_per_cta and grid, which the launcher sets).
 GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled = nullptr);
 
-// Launches a chain of 1..kMaxChain dependent GEMMs as one persistent kernel. Returns in
-// *barrier_arrivals how far the grid counter advances (the caller adds it to its running base).
-cudaError_t launch_gemm_chain(const ChainMaps &maps, ChainParams &p, int n_sms, cudaStream_t st, uint32_t *barrier_arrivals);
+// Enqueues one GEMM: the streaming kernel, then the finishing kernel (both with programmatic
+// stream serialization). partial_floats is the size of p.partials; cudaErrorInvalidValue if the
+// GEMM needs more. *launched (optional) receives the number of kernels enqueued.
+cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_t partial_floats, cudaStream_t st, int *launched);
 
 }  // namespace llmcad
