@@ -86,6 +86,8 @@ int check_config(const llmcad_config *c)
 
 }  // namespace
 
+constexpr int kSyncCounters = 2048;
+
 struct llmcad_ctx {
     llmcad_config cfg;
     PackedLayout lay;
@@ -110,6 +112,13 @@ struct llmcad_ctx {
     float *ssq[2] = {nullptr, nullptr};   // partial sums of squares for the folded attention / FFN norms
     float *attn_ws = nullptr;
     uint32_t *attn_counters = nullptr;
+    // completion counters through which the kernels of a tensor-core pass hand over (common.cuh): one per
+    // kernel, taken in launch order, all zeroed at the start of a forward. LLMCAD_SYNC_COUNTERS=0 (tuning
+    // aid, read at creation) falls back to grid dependencies.
+    uint32_t *sync_ctrs = nullptr;
+    int sync_next = 0;
+    bool use_counters = true;
+    uint32_t *next_ctr() { return (use_counters && sync_next < kSyncCounters) ? sync_ctrs + sync_next++ : nullptr; }
     int64_t launches = 0;
     uint64_t wait_limit_ns = kDefaultWaitLimitNs;   // bound of every device-side wait (llmcad_set_wait_limit_ns)
     unsigned long long *trace = nullptr;   // optional timeline buffer (llmcad_set_gemm_trace): [launch][256][16]
@@ -255,7 +264,7 @@ int run_gemm(llmcad_ctx *ctx, const void *packed, int l, int which, int act, int
 // comp: q carries a lo plane kLoRows rows after the hi plane, and o gets one too (the pass);
 // the single-step entry points work on plain bf16 buffers.
 int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, int kv_stride, int P, int n, void *o,
-                  bool comp, int32_t *status, cudaStream_t st, int n_tree = 0, int q_first = 0)
+                  bool comp, int32_t *status, cudaStream_t st, int n_tree = 0, int q_first = 0, const AttnSync *sync = nullptr)
 {
     const llmcad_config &c = ctx->cfg;
     TimedLaunch tl(ctx, 1, st);
@@ -265,13 +274,13 @@ int run_attention(llmcad_ctx *ctx, const void *q, const void *k, const void *v, 
                         : (c.flags & LLMCAD_FLAG_MMA_ATTN) ? false : attention_prefers_t5(n);
         if (t5) {
             CUDA_TRY(launch_attention_t5(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->n_sms, status, st,
-                                         &launched, ctx->next_trace(), comp ? 1 : 0, ctx->kv_lo, n_tree, q_first, ctx->wait_limit_ns));
+                                         &launched, ctx->next_trace(), comp ? 1 : 0, ctx->kv_lo, n_tree, q_first, ctx->wait_limit_ns, sync));
             ctx->launches += launched;
             return LLMCAD_OK;
         }
         CUDA_TRY(launch_attention_tc(q, k, v, c.n_heads, c.head_dim, kv_stride, P, n, ctx->tb.anc, o, ctx->attn_ws,
                                      ctx->attn_counters, ctx->n_sms, status, st, &launched, ctx->next_trace(), comp ? 1 : 0,
-                                     ctx->kv_lo, n_tree, q_first));
+                                     ctx->kv_lo, n_tree, q_first, sync));
         ctx->launches += launched;
         return LLMCAD_OK;
     }
@@ -356,16 +365,46 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
             if (!last) specs.push_back({l + 1, 0, 0, d, qkv_ep(l + 1, tiles4), false});
             else if (logits != nullptr) specs.push_back({-1, 0, 0, d, head_ep(tiles4), false});
         }
+        // every GEMM is planned first, so that each can tell its predecessor where its weights start
+        std::vector<TcGemm> gemms(specs.size());
+        for (size_t i = 0; i < specs.size(); ++i) {
+            gemms[i].set(ctx, specs[i].l, specs[i].which, specs[i].act, specs[i].n_in, specs[i].ep, n_pad);
+            CUDA_TRY(plan_gemm_tc(gemms[i].p, ctx->n_sms));
+        }
+        // Hand-over between the kernels: completion counters (one per kernel, zeroed here) where both sides are
+        // tensor-core kernels of this library, the grid dependency otherwise. `dep` is what the next kernel
+        // waits for: null after the embedding kernel and after a plain-ALU attention kernel.
+        ctx->sync_next = 0;
+        if (ctx->use_counters) CUDA_TRY(cudaMemsetAsync(ctx->sync_ctrs, 0, kSyncCounters * sizeof(uint32_t), st));
+        const uint32_t *dep = nullptr;
+        uint32_t dep_target = 0;
         for (size_t i = 0; i < specs.size(); ++i) {
             if (specs[i].attention_first) {
                 char *kl = static_cast<char *>(kv_cache) + kv_layer * (size_t)specs[i].l;
+                AttnSync sync{dep, dep_target, ctx->tc_attn ? ctx->next_ctr() : nullptr, ctx->wait_limit_ns, 0};
+                const bool with_sync = ctx->tc_attn && sync.done_ctr != nullptr;
                 // without the tensor-core attention kernel the lo plane of att stays zero, as allocated
                 if ((rc = run_attention(ctx, ctx->q, kl, kl + kv_layer / 2, S, P, n, ctx->att, ctx->comp && ctx->tc_attn, status, st,
-                                        n_tree, n_old)) != LLMCAD_OK) return rc;
+                                        n_tree, n_old, with_sync ? &sync : nullptr)) != LLMCAD_OK) return rc;
+                dep = with_sync ? sync.done_ctr : nullptr;
+                dep_target = sync.arrivals;
             }
-            TcGemm g;
-            g.set(ctx, specs[i].l, specs[i].which, specs[i].act, specs[i].n_in, specs[i].ep, n_pad);
-            if ((rc = g.launch(ctx, status, st)) != LLMCAD_OK) return rc;
+            // The first ring-fulls per CTA of the next GEMM's weights go to L2 during this GEMM's tail. Measured on
+            // B200 (7B shape, 32 nodes): 12 items gain 2.5 % of the pass, 24 items gain more for the QKV GEMM
+            // that follows the down projection and lose elsewhere (the burst competes with this GEMM's own
+            // tail); with more than 32 nodes the L2-to-SM path is the busy one and the prefetch only costs.
+            if (i + 1 < specs.size() && n_pad <= 32) {
+                const int mode_next = specs[i + 1].ep.mode;
+                gemms[i].p.next = next_weights(gemms[i + 1].p, (mode_next == EPI_QKV || mode_next == EPI_PLAIN) ? 24 : 12);
+            }
+            GemmParams &gp = gemms[i].p;
+            gp.dep_ctr = dep; gp.dep_target = dep_target;
+            gp.s_done = ctx->next_ctr();
+            gp.f_done = gp.s_done != nullptr ? ctx->next_ctr() : nullptr;
+            if (gp.f_done == nullptr) gp.s_done = nullptr;
+            if ((rc = gemms[i].launch(ctx, status, st)) != LLMCAD_OK) return rc;
+            dep = gp.f_done;
+            dep_target = (uint32_t)gp.f_grid;
         }
         return LLMCAD_OK;
     }
@@ -517,6 +556,11 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ok = ok && alloc((void **)&ctx->ssq[1], ssq_floats * 4);
     ok = ok && alloc((void **)&ctx->attn_ws, attention_tc_workspace_bytes(cfg->n_heads, ctx->n_sms));
     ok = ok && alloc((void **)&ctx->attn_counters, (size_t)cfg->n_heads * 8 * 4);
+    ok = ok && alloc((void **)&ctx->sync_ctrs, kSyncCounters * sizeof(uint32_t));
+    {
+        const char *e = getenv("LLMCAD_SYNC_COUNTERS");
+        ctx->use_counters = !(e != nullptr && atoi(e) == 0);
+    }
     if (ok) {
         std::vector<int32_t> chain(128);
         for (int i = 0; i < 128; ++i) chain[i] = i - 1;
@@ -534,7 +578,7 @@ void llmcad_destroy(llmcad_ctx *ctx)
 {
     if (ctx == nullptr) return;
     void *ptrs[] = {ctx->x, ctx->xn, ctx->q, ctx->att, ctx->h, ctx->kv_lo, ctx->logits, ctx->tb.depth, ctx->tb.pos, ctx->tb.anc,
-                    ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->attn_ws, ctx->attn_counters, ctx->ssq[0],
+                    ctx->tb.rope_cs, ctx->ibuf, ctx->partials, ctx->attn_ws, ctx->attn_counters, ctx->sync_ctrs, ctx->ssq[0],
                     ctx->ssq[1]};
     for (void *p : ptrs)
         if (p != nullptr) cudaFree(p);

@@ -298,7 +298,8 @@ __global__ void __launch_bounds__(kT5Threads, 1)
 attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_lo, int n_heads, int P,
                     int n, const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
-                    int32_t *status, unsigned long long *trace, int comp, int n_tree, int q_first, uint64_t wait_limit)
+                    int32_t *status, unsigned long long *trace, int comp, int n_tree, int q_first, uint64_t wait_limit,
+                    DepWait dep, uint32_t *done_ctr)
 {
     const int cta = blockIdx.y * gridDim.x + blockIdx.x;
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 0] = global_timer_ns();
@@ -353,7 +354,17 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
     bool failed = false;
     // A pass whose tree or tokens an earlier phase refused (status word set) does no work here: every
     // role looks at the word once the grid dependency has resolved, and all see the same value.
-    auto refused = [&]() { pdl_wait(); return *reinterpret_cast<const volatile int32_t *>(status) != 0; };
+    // (the dependency is the grid dependency or the producer's completion counter; the one thread that feeds the
+    // copy engine with data written by ordinary stores puts a proxy fence behind its wait)
+    auto refused = [&]() {
+        dep_wait_thread(dep);
+        fence_proxy_async();
+        return *reinterpret_cast<const volatile int32_t *>(status) != 0;
+    };
+    auto refused_warp = [&]() {
+        dep_wait_warp(dep, lane);
+        return *reinterpret_cast<const volatile int32_t *>(status) != 0;
+    };
 
     if (warp == 0) {
         // ================================================= producer
@@ -507,13 +518,13 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
         const int row = lg * 32 + lane;
         const bool warp_active = lg * 32 < n;             // a warp whose rows are all padding only keeps the barriers going
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
-        const bool skip = refused();
+        const bool skip = refused_warp();
         if (trace && tid == 64 && cta < 256) trace[(size_t)cta * 16 + 1] = global_timer_ns();
         if (!skip) {
         uint32_t a4[4] = {0, 0, 0, 0};
         if (row < n) {
 #pragma unroll
-            for (int w = 0; w < 4; ++w) a4[w] = anc[(q_first + row) * 4 + w];
+            for (int w = 0; w < 4; ++w) a4[w] = __ldcg(anc + (q_first + row) * 4 + w);   // L2: written earlier in this pass
         }
         // The queries become the A operand of Q K^T in tensor memory: 64 packed columns per plane, thread =
         // row. A warp fetches its 32 rows with coalesced loads (two rows of 256 bytes per instruction, both
@@ -530,7 +541,7 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
                     for (int it = 0; it < 16; ++it) {
                         const int rr = it * 2 + (lane >> 4);
                         const int qrow = min(lg * 32 + rr, n - 1);
-                        g[pl][it] = __ldg(reinterpret_cast<const uint4 *>(q + (size_t)pl * lo_off + ((size_t)qrow * n_heads + head) * kHd) + (lane & 15));
+                        g[pl][it] = __ldcg(reinterpret_cast<const uint4 *>(q + (size_t)pl * lo_off + ((size_t)qrow * n_heads + head) * kHd) + (lane & 15));
                     }
                 }
             }
@@ -703,6 +714,10 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
                 store4(row, dim, *reinterpret_cast<const float4 *>(part + (size_t)row * kWsRow + dim), L > 0.f ? 1.f / L : 0.f);
             }
         }
+        if (done_ctr != nullptr) {
+            __syncthreads();
+            if (tid == 0) dep_arrive(done_ctr);
+        }
         if (trace && tid == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
         return;
     }
@@ -717,6 +732,10 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
         else merge_splits<kMaxSplits, 1>(part, cluster, splits, split, n, n_heads, head, o, lo_off, comp, tid);
     }
     if (trace && tid == 0 && cta < 256) trace[(size_t)cta * 16 + 6] = global_timer_ns();
+    if (done_ctr != nullptr) {
+        __syncthreads();                                     // this CTA's rows of the output are written
+        if (tid == 0) dep_arrive(done_ctr);
+    }
     cluster.sync();                                          // peers may still be reading this CTA's partial
     if (trace && tid == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
 }
@@ -729,7 +748,8 @@ bool attention_prefers_t5(int n)
 
 cudaError_t launch_attention_t5(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, int n_sms, int32_t *status, cudaStream_t st,
-                                int *launched, unsigned long long *trace, int comp, const void *kv_lo, int n_tree, int q_first, uint64_t wait_limit_ns)
+                                int *launched, unsigned long long *trace, int comp, const void *kv_lo, int n_tree, int q_first, uint64_t wait_limit_ns,
+                                const AttnSync *sync)
 {
     if (n_tree <= 0) n_tree = n;
     if (hd != kHd || n < 1 || n > 128 || P + n_tree > kv_stride) return cudaErrorInvalidValue;
@@ -768,8 +788,15 @@ cudaError_t launch_attention_t5(const void *q, const void *k, const void *v, int
     }
     LaunchCfg lc(dim3(splits, n_heads), dim3(kT5Threads), kSmemBytes, st, splits);
     if (launched) *launched = 1;
+    DepWait dep{nullptr, 0, wait_limit_ns};
+    uint32_t *done = nullptr;
+    if (sync != nullptr) {
+        dep = DepWait{sync->dep_ctr, sync->dep_target, wait_limit_ns};
+        done = sync->done_ctr;
+        sync->arrivals = (uint32_t)(splits * n_heads);
+    }
     return cudaLaunchKernelEx(&lc.cfg, attention_t5_kernel, (const __nv_bfloat16 *)q, mk, mv, ml, n_heads, P, n, anc, (__nv_bfloat16 *)o, splits,
-                              tiles_per_split, status, trace, comp, n_tree, q_first, wait_limit_ns);
+                              tiles_per_split, status, trace, comp, n_tree, q_first, wait_limit_ns, dep, done);
 }
 
 }  // namespace llmcad

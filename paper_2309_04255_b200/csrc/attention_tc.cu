@@ -98,7 +98,7 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
                     const __nv_bfloat16 *__restrict__ v, int n_heads, int kv_stride, int P, int n, int n_pad,
                     const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
                     const int32_t *status, unsigned long long *trace, const __nv_bfloat16 *__restrict__ kv_lo,
-                    int n_tree, int q_first)
+                    int n_tree, int q_first, DepWait dep, uint32_t *done_ctr)
 {
     // n query rows = the tree nodes q_first .. q_first + n - 1 (all of them in a verification pass,
     // the new ones when a tree is extended); the keys are the prefix and all n_tree tree nodes
@@ -149,11 +149,17 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         early[st] = t_begin + st < t_end && (t_begin + st + 1) * kKeyTile <= P;
         if (early[st]) load_tile(t_begin + st, st);
     }
-    pdl_wait();
+    // the queries and the tree nodes' K/V are final: grid dependency, or the producer's completion counter
+    if (dep.ctr == nullptr) pdl_wait();
+    else {
+        if (threadIdx.x == 0) dep_wait_thread(dep);      // a wait that runs out lets the pass go on: the status word tells
+        __syncthreads();
+    }
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 1] = global_timer_ns();
-    if (*status) {             // uniform over the grid: set only by kernels that ran before this one
+    if (*reinterpret_cast<const volatile int32_t *>(status)) {   // uniform over the grid: set only by kernels that ran before this one
         cp_commit();
         cp_wait<0>();          // nothing may still be writing this CTA's shared memory when it exits
+        if (threadIdx.x == 0) dep_arrive(done_ctr);
         return;
     }
     // queries of this head (rows >= n are zero) and the remaining first key tiles
@@ -188,8 +194,8 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     uint32_t anc0[4] = {0, 0, 0, 0}, anc1[4] = {0, 0, 0, 0};
     if (active) {
         for (int w = 0; w < 4; ++w) {
-            if (row0 < n) anc0[w] = anc[(q_first + row0) * 4 + w];
-            if (row1 < n) anc1[w] = anc[(q_first + row1) * 4 + w];
+            if (row0 < n) anc0[w] = __ldcg(anc + (q_first + row0) * 4 + w);     // L2: written earlier in this pass
+            if (row1 < n) anc1[w] = __ldcg(anc + (q_first + row1) * 4 + w);
         }
     }
 
@@ -401,6 +407,10 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
             *reinterpret_cast<uint32_t *>(dst) = hi;
             if (COMP) *reinterpret_cast<uint32_t *>(dst + lo_off) = lo;
         }
+        if (done_ctr != nullptr) {
+            __syncthreads();
+            if (threadIdx.x == 0) dep_arrive(done_ctr);
+        }
         if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
         return;
     }
@@ -444,6 +454,10 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         if (COMP) *reinterpret_cast<uint32_t *>(dst + lo_off) = lo;
     }
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 6] = global_timer_ns();
+    if (done_ctr != nullptr) {
+        __syncthreads();                                     // this CTA's rows of the output are written
+        if (threadIdx.x == 0) dep_arrive(done_ctr);
+    }
     cluster.sync();                                          // peers may still be reading this CTA's partial
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
 }
@@ -457,7 +471,7 @@ size_t attention_tc_workspace_bytes(int n_heads, int n_sms)
 cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int n_heads, int hd, int kv_stride, int P,
                                 int n, const uint32_t *anc, void *o, float *ws, uint32_t *counters, int n_sms,
                                 int32_t *status, cudaStream_t st, int *launched, unsigned long long *trace, int comp,
-                                const void *kv_lo, int n_tree, int q_first)
+                                const void *kv_lo, int n_tree, int q_first, const AttnSync *sync)
 {
     if (n_tree <= 0) n_tree = n;
     (void)ws; (void)counters;
@@ -481,7 +495,7 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     const size_t smem = ring > part ? ring : part;
     typedef void (*Kern)(const __nv_bfloat16 *, const __nv_bfloat16 *, const __nv_bfloat16 *, int, int, int, int, int,
                          const uint32_t *, __nv_bfloat16 *, int, int, const int32_t *, unsigned long long *,
-                         const __nv_bfloat16 *, int, int);
+                         const __nv_bfloat16 *, int, int, DepWait, uint32_t *);
     static const Kern kerns[2][3] = {{attention_tc_kernel<1, false>, attention_tc_kernel<2, false>, attention_tc_kernel<4, false>},
                                      {attention_tc_kernel<1, true>, attention_tc_kernel<2, true>, attention_tc_kernel<4, true>}};
     static PerDeviceOnce attr_set;
@@ -499,9 +513,16 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     LaunchCfg lc(dim3(splits, n_heads), dim3(kAtThreads), smem, st, splits);
     if (launched) *launched = 1;
     Kern kern = kerns[comp ? 1 : 0][groups == 4 ? 2 : (groups == 2 ? 1 : 0)];
+    DepWait dep{nullptr, 0, kDefaultWaitLimitNs};
+    uint32_t *done = nullptr;
+    if (sync != nullptr) {
+        dep = DepWait{sync->dep_ctr, sync->dep_target, sync->wait_limit_ns ? sync->wait_limit_ns : kDefaultWaitLimitNs};
+        done = sync->done_ctr;
+        sync->arrivals = (uint32_t)(splits * n_heads);
+    }
     return cudaLaunchKernelEx(&lc.cfg, kern, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                               (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc, (__nv_bfloat16 *)o, splits,
-                              tiles_per_split, (const int32_t *)status, trace, (const __nv_bfloat16 *)kv_lo, n_tree, q_first);
+                              tiles_per_split, (const int32_t *)status, trace, (const __nv_bfloat16 *)kv_lo, n_tree, q_first, dep, done);
 }
 
 }  // namespace llmcad

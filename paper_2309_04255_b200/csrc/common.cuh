@@ -147,6 +147,66 @@ constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;  // every device-side wa
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// ---------------------------------------------------------------- completion counters
+// Programmatic dependent launch orders two kernels through griddepcontrol.wait, which returns only when
+// the earlier grid has exited and its memory is flushed: ~1.3 us after the last CTA's exit on B200. The
+// kernels of the tensor-core pass hand over through counters in global memory instead: every CTA (or
+// warp) of a kernel adds one to the kernel's counter, with release semantics, when its results are
+// written, and the consumer polls, with acquire semantics, until the counter reaches the number of
+// arrivals it was told to expect. All CTAs of the producer are resident (or done) before any CTA of the
+// consumer starts, because a kernel lets its dependents launch only from inside its CTAs, so a poll
+// cannot starve the kernel it waits for. A null counter means "use the grid dependency".
+struct DepWait {
+    const uint32_t *ctr;     // nullptr: griddepcontrol.wait
+    uint32_t target;
+    uint64_t limit_ns;       // the wait gives up after this long
+};
+
+__device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// One thread waits; false when the limit ran out.
+__device__ __forceinline__ bool dep_wait_thread(const DepWait &d)
+{
+    if (d.ctr == nullptr) { pdl_wait(); return true; }
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (ld_acquire_gpu_u32(d.ctr) >= d.target) return true;
+        __nanosleep(32);
+        if ((it & 63u) == 63u) {
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > d.limit_ns) return false;
+        }
+    }
+}
+
+// A whole warp waits: lane 0 polls, the barrier orders the other lanes' later reads after its acquire.
+__device__ __forceinline__ bool dep_wait_warp(const DepWait &d, int lane)
+{
+    int ok = 1;
+    if (d.ctr == nullptr) { pdl_wait(); return true; }
+    if (lane == 0) ok = dep_wait_thread(d) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
+}
+
+// One arrival: everything this thread wrote, and everything it has observed through a CTA or warp barrier,
+// is visible to whoever sees the count.
+__device__ __forceinline__ void dep_arrive(uint32_t *ctr)
+{
+    if (ctr == nullptr) return;
+    __threadfence();
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
+}
+
+// Data that arrived through ordinary stores of other SMs is about to be read by the copy engine (TMA).
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
 struct LaunchCfg {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attrs[2];

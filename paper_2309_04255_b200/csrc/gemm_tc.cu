@@ -514,6 +514,7 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
     const uint32_t acc_cols = 2u * nb;                    // TMEM columns of one accumulator buffer (gate | up)
     const bool two_bufs = p.acc_bufs == 2;
     const uint64_t wait_limit = p.wait_limit_ns;          // every wait below gives up after this many ns
+    const DepWait dep{p.dep_ctr, p.dep_target, wait_limit};
 
     if (threadIdx.x == 0) LLMCAD_TRACE(0);
 
@@ -611,6 +612,22 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
                 else if (*abort_flag || global_timer_ns() - t_idle > wait_limit) { timed_out = true; break; }
             }
             LLMCAD_TRACE(6);
+            // This CTA's weights are all requested. HBM would now idle through the tail of this GEMM and
+            // the start of the next: ask L2 for the first items of the next GEMM's CTA of the same number.
+            const NextWeights &nx = p.next;
+            if (nx.w_tiled != nullptr && !timed_out && (int)blockIdx.x < nx.grid) {
+                const int ppt = (nx.kb_per_tile + nx.pair_k - 1) / nx.pair_k, ipt = ppt * nx.halves;
+                const int begin = (int)blockIdx.x * nx.items_per_cta;
+                const int end = min(nx.n_tiles * ipt, begin + min(nx.items_per_cta, nx.items));
+                for (int i = begin; i < end; ++i) {
+                    const int tile = i / ipt, q = i - tile * ipt;
+                    const int kp = q / nx.halves, half = q - kp * nx.halves;
+                    const int kb0 = kp * nx.pair_k, nk = min(nx.pair_k, nx.kb_per_tile - kb0);
+                    const size_t t = (size_t)(tile + (half ? nx.up_tile_offset : 0)) * nx.kb_per_tile + kb0;
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(nx.w_tiled + t * kATileBytes),
+                                 "r"((uint32_t)nk * kATileBytes) : "memory");
+                }
+            }
         }
     } else if (warp == 6) {
         // ================================================= activation loader
@@ -623,7 +640,8 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
             c.init(d);
             int s = 0;
             uint32_t i = 0;
-            pdl_wait();
+            if (!dep_wait_thread(dep)) timed_out = true;
+            fence_proxy_async();          // the activations were written by ordinary stores; the copies below read them
             pdl_launch_dependents();
             while (!c.done() && !timed_out && !p.withhold_act) {
                 uint64_t t0 = 0;
@@ -645,9 +663,6 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
                 ++i;
                 if (++s == p.stages) s = 0;
             }
-        } else {
-            pdl_wait();
-            pdl_launch_dependents();
         }
     } else if (warp == 1) {
         // ================================================= MMA issuer
@@ -696,14 +711,14 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
         // ================================================= accumulator dump (warps 2..5)
         const int lane_grp = warp & 3;                 // TMEM lanes 32*lane_grp .. +31 belong to this warp
         // the workspace may still be read by the finishing kernel of the previous GEMM
-        pdl_wait();
+        if (!dep_wait_warp(dep, lane)) timed_out = true;
         pdl_launch_dependents();
         if (threadIdx.x == 64) LLMCAD_TRACE(3);
         const Range r = cta_range<PK>(d, (int)blockIdx.x);
         const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
         const size_t slot_stride = slot_floats(d.halves, p.n_pad);
         uint32_t seg = 0;
-        for (int seg_begin = r.begin; seg_begin < r.end; ++seg) {
+        for (int seg_begin = r.begin; seg_begin < r.end && !timed_out; ++seg) {
             const int tile = seg_begin / ipt;
             const int seg_end = min(r.end, (tile + 1) * ipt);
             const int buf = two_bufs ? (seg & 1) : 0;
@@ -749,6 +764,8 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
     }
     __syncwarp();   // lanes that skipped their role's single-thread section rejoin their warp here
     timed_out = __any_sync(0xffffffffu, timed_out);   // keep the warp together on the way out
+    // this dump warp's segments are in the workspace (also said after a wait ran out, so that nobody waits for this CTA)
+    if (warp >= 2 && warp <= 5 && lane == 0) dep_arrive(p.s_done);
 
     if (timed_out) {
         *abort_flag = 1;
@@ -793,6 +810,10 @@ gemm_finish_kernel(const __grid_constant__ GemmParams p)
     }
     pdl_launch_dependents();     // the next GEMM's streaming kernel may take the SMs as they free up
     if (threadIdx.x == 0) LLMCAD_TRACE(9);
+    // what earlier GEMMs left (norm sums, residual, gains) is final: the streaming kernel of this GEMM
+    // waited for the same counter before it let this kernel launch, so this returns at once
+    bool late = false;
+    if (threadIdx.x == 0 && p.dep_ctr != nullptr) late = !dep_wait_thread(DepWait{p.dep_ctr, p.dep_target, p.wait_limit_ns});
     __syncthreads();
     const GemmDesc &d = s_desc;
     const EpiParams &ep = d.ep;
@@ -839,7 +860,12 @@ gemm_finish_kernel(const __grid_constant__ GemmParams p)
     for (int round = 0; round < 2; ++round) {
         const bool dry = round == 0;
         if (!dry) {
-            pdl_wait();                  // every segment is in the workspace
+            // every segment is in the workspace
+            if (p.s_done == nullptr) pdl_wait();
+            else {
+                if (threadIdx.x == 0) late |= !dep_wait_thread(DepWait{p.s_done, 4u * (uint32_t)d.grid, p.wait_limit_ns});
+                __syncthreads();
+            }
             if (threadIdx.x == 0) LLMCAD_TRACE(10);
         }
         if (wg < groups * k) {
@@ -854,6 +880,13 @@ gemm_finish_kernel(const __grid_constant__ GemmParams p)
                 finish_rows_t<G, KB, MODE>(fa, lane, dry);
                 if (dry) break;          // one pair is enough to have walked through the code
             }
+        }
+    }
+    if (p.f_done != nullptr) {
+        __syncthreads();             // all of this CTA's results are written
+        if (threadIdx.x == 0) {
+            if (late) atomicCAS(p.status, 0, LLMCAD_ERR_TIMEOUT);
+            dep_arrive(p.f_done);
         }
     }
     if (threadIdx.x == 0) LLMCAD_TRACE(12);
@@ -941,20 +974,28 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)
     return d;
 }
 
-cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_t partial_floats, cudaStream_t st, int *launched)
+namespace {
+// tuning aids from the environment, read once per process
+struct Tuning {
+    int pair_k = 0, stages_cap = 0, l2_ahead = 8, next_items = -1;
+    Tuning()
+    {
+        if (const char *e = getenv("LLMCAD_GEMM_PAIR_K")) { const int v = atoi(e); if (v == 1 || v == 2) pair_k = v; }
+        if (const char *e = getenv("LLMCAD_GEMM_STAGES")) { const int v = atoi(e); if (v >= 2) stages_cap = v; }
+        if (const char *e = getenv("LLMCAD_GEMM_L2_AHEAD")) l2_ahead = atoi(e);
+        if (const char *e = getenv("LLMCAD_GEMM_NEXT_ITEMS")) next_items = atoi(e);
+    }
+};
+const Tuning &tuning()
 {
-    if (launched) *launched = 0;
-    // tuning aids from the environment, read once per process
-    struct Tuning {
-        int pair_k = 0, stages_cap = 0, l2_ahead = 8;
-        Tuning()
-        {
-            if (const char *e = getenv("LLMCAD_GEMM_PAIR_K")) { const int v = atoi(e); if (v == 1 || v == 2) pair_k = v; }
-            if (const char *e = getenv("LLMCAD_GEMM_STAGES")) { const int v = atoi(e); if (v >= 2) stages_cap = v; }
-            if (const char *e = getenv("LLMCAD_GEMM_L2_AHEAD")) l2_ahead = atoi(e);
-        }
-    };
-    static const Tuning tune;
+    static const Tuning t;
+    return t;
+}
+}  // namespace
+
+cudaError_t plan_gemm_tc(GemmParams &p, int n_sms)
+{
+    const Tuning &tune = tuning();
     // Ring items of two k-blocks (one 32 KB weight copy each) unless the activation tiles are so wide
     // (hi | lo planes of more than 64 nodes) that only two stages would fit; measured on B200:
     // single k-blocks cost 10-17 % up to 64 nodes and gain 6 % at 128.
@@ -973,6 +1014,32 @@ cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_
     d.items_per_cta = (int)ipc;
     grid = (int)((total + ipc - 1) / ipc);
     d.grid = grid;
+    return cudaSuccess;
+}
+
+NextWeights next_weights(const GemmParams &planned, int items)
+{
+    const GemmDesc &d = planned.g;
+    NextWeights nx{};
+    nx.w_tiled = d.w_tiled;
+    nx.n_tiles = d.n_tiles; nx.kb_per_tile = d.kb_per_tile; nx.pair_k = d.pair_k; nx.halves = d.halves;
+    nx.items_per_cta = d.items_per_cta; nx.up_tile_offset = d.up_tile_offset; nx.grid = d.grid;
+    nx.items = tuning().next_items >= 0 ? tuning().next_items : items;
+    return nx;
+}
+
+cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_t partial_floats, cudaStream_t st, int *launched)
+{
+    if (launched) *launched = 0;
+    const Tuning &tune = tuning();
+    {
+        const cudaError_t e = plan_gemm_tc(p, n_sms);
+        if (e != cudaSuccess) return e;
+    }
+    GemmDesc &d = p.g;
+    const int nb = p.n_pad * (p.comp ? 2 : 1);
+    const int pair_k = d.pair_k, grid = d.grid;
+    const long long ipc = d.items_per_cta;
     if ((size_t)(d.n_tiles + grid) * slot_floats(d.halves, p.n_pad) > partial_floats) return cudaErrorInvalidValue;
     const size_t stage_bytes = (size_t)pair_k * ((size_t)kATileBytes + (size_t)nb * kBlockK * 2);
     // One CTA per SM with the whole shared memory as the ring.
@@ -1046,6 +1113,7 @@ cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_
             once.mark();
         }
     }
+    p.f_grid = fgrid;
     LaunchCfg lf(fgrid, kFinThreads, kFinSmem, st);
     const cudaError_t e = cudaLaunchKernelEx(&lf.cfg, fk, p);
     if (e == cudaSuccess && launched) ++*launched;
