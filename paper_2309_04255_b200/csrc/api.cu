@@ -113,11 +113,13 @@ struct llmcad_ctx {
     float *attn_ws = nullptr;
     uint32_t *attn_counters = nullptr;
     // completion counters through which the kernels of a tensor-core pass hand over (common.cuh): one per
-    // kernel, taken in launch order, all zeroed at the start of a forward. LLMCAD_SYNC_COUNTERS=0 (tuning
-    // aid, read at creation) falls back to grid dependencies.
+    // kernel, taken in launch order, all zeroed at the start of a forward. Off by default: measured on B200
+    // (7B shape, 32 nodes) the hand-over through counters costs 4 % of the pass against grid dependencies
+    // (a release after a burst of stores takes 2-4 us under the weight stream; the grid dependency's flush
+    // takes 1.3). LLMCAD_SYNC_COUNTERS=1 (tuning aid, read at creation) switches it on.
     uint32_t *sync_ctrs = nullptr;
     int sync_next = 0;
-    bool use_counters = true;
+    bool use_counters = false;
     uint32_t *next_ctr() { return (use_counters && sync_next < kSyncCounters) ? sync_ctrs + sync_next++ : nullptr; }
     int64_t launches = 0;
     uint64_t wait_limit_ns = kDefaultWaitLimitNs;   // bound of every device-side wait (llmcad_set_wait_limit_ns)
@@ -559,7 +561,7 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ok = ok && alloc((void **)&ctx->sync_ctrs, kSyncCounters * sizeof(uint32_t));
     {
         const char *e = getenv("LLMCAD_SYNC_COUNTERS");
-        ctx->use_counters = !(e != nullptr && atoi(e) == 0);
+        ctx->use_counters = e != nullptr && atoi(e) != 0;
     }
     if (ok) {
         std::vector<int32_t> chain(128);

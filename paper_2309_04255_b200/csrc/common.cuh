@@ -149,8 +149,9 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 
 // ---------------------------------------------------------------- completion counters
 // Programmatic dependent launch orders two kernels through griddepcontrol.wait, which returns only when
-// the earlier grid has exited and its memory is flushed: ~1.3 us after the last CTA's exit on B200. The
-// kernels of the tensor-core pass hand over through counters in global memory instead: every CTA (or
+// the earlier grid has exited and its memory is flushed: ~1.3 us after the last CTA's exit on B200. As an
+// alternative (an option of the context, off by default: it measured slower) the kernels of the
+// tensor-core pass can hand over through counters in global memory: every CTA (or
 // warp) of a kernel adds one to the kernel's counter, with release semantics, when its results are
 // written, and the consumer polls, with acquire semantics, until the counter reaches the number of
 // arrivals it was told to expect. All CTAs of the producer are resident (or done) before any CTA of the
@@ -200,8 +201,7 @@ __device__ __forceinline__ bool dep_wait_warp(const DepWait &d, int lane)
 __device__ __forceinline__ void dep_arrive(uint32_t *ctr)
 {
     if (ctr == nullptr) return;
-    __threadfence();
-    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");   // release is cumulative: no separate fence
 }
 
 // Data that arrived through ordinary stores of other SMs is about to be read by the copy engine (TMA).
