@@ -373,3 +373,45 @@ int orc_branch_pacer(const double *cum_conf, const int *branch_len, int n_branch
     }
     return next;
 }
+
+/* INT4 group quantisation of the weights (Sec. 4.1: the target model's weights are held as INT4
+ * through group-wise post-training quantisation). Reading, where the paper only names the format:
+ * symmetric codes q in [-8, 7], one scale per row and group of `group` consecutive input columns,
+ * the scale a power of two 2^e, e the smallest integer with max|w| <= 7 * 2^e over the group (a
+ * group of zeros gets e = -126), q = w / 2^e rounded to the nearest integer, halves to even.
+ * Power-of-two scales make every dequantised weight q * 2^e a value bf16 holds exactly, so the
+ * quantised model is an ordinary model over those weights and the rest of the oracle applies
+ * unchanged. w: [rows][cols] fp32, cols a multiple of group; q: [rows][cols] int8;
+ * e: [rows][cols / group] int8. */
+void orc_quantize_int4(const float *w, int rows, int cols, int group, signed char *q, signed char *e)
+{
+    const int ng = cols / group;
+    for (int r = 0; r < rows; ++r)
+        for (int g = 0; g < ng; ++g) {
+            const float *x = w + (size_t)r * cols + (size_t)g * group;
+            double m = 0.0;
+            for (int c = 0; c < group; ++c)
+                if (fabs((double)x[c]) > m) m = fabs((double)x[c]);
+            int ex = -126;
+            if (m > 0.0) {
+                ex = -126;
+                while (ex < 127 && m > 7.0 * ldexp(1.0, ex)) ++ex;    /* smallest e with m <= 7 * 2^e */
+            }
+            e[(size_t)r * ng + g] = (signed char)ex;
+            for (int c = 0; c < group; ++c) {
+                double v = nearbyint(ldexp((double)x[c], -ex));   /* default rounding mode: to nearest, halves to even */
+                if (v > 7.0) v = 7.0;
+                if (v < -8.0) v = -8.0;
+                q[(size_t)r * cols + (size_t)g * group + c] = (signed char)v;
+            }
+        }
+}
+
+/* The weights a quantised model computes with: w[r][c] = q[r][c] * 2^e[r][c / group]. */
+void orc_dequantize_int4(const signed char *q, const signed char *e, int rows, int cols, int group, float *w)
+{
+    const int ng = cols / group;
+    for (int r = 0; r < rows; ++r)
+        for (int c = 0; c < cols; ++c)
+            w[(size_t)r * cols + c] = (float)ldexp((double)q[(size_t)r * cols + c], e[(size_t)r * ng + c / group]);
+}

@@ -317,3 +317,40 @@ def branch_pacer(cum_conf, branch_len, m_tokens: float):
     f.restype = C.c_int
     nxt = int(f(_p(c), _p(t), C.c_int(len(c)), C.c_double(float(m_tokens)), _p(out)))
     return out, nxt
+
+
+INT4_GROUP = 64
+
+
+def quantize_int4(w, group: int = INT4_GROUP):
+    """Sec. 4.1 (INT4 weights): symmetric group quantisation with power-of-two scales.
+    w [rows][cols] -> (q int8 [rows][cols] in [-8, 7], e int8 [rows][cols / group])."""
+    w = _f32(w)
+    rows, cols = w.shape
+    assert cols % group == 0
+    q = np.zeros((rows, cols), np.int8)
+    e = np.zeros((rows, cols // group), np.int8)
+    lib().orc_quantize_int4(_p(w), C.c_int(rows), C.c_int(cols), C.c_int(group), _p(q), _p(e))
+    return q, e
+
+
+def dequantize_int4(q, e, group: int = INT4_GROUP) -> np.ndarray:
+    """q * 2^e as fp32 (every value is exactly representable in bf16)."""
+    q = np.ascontiguousarray(q, dtype=np.int8)
+    e = np.ascontiguousarray(e, dtype=np.int8)
+    rows, cols = q.shape
+    w = np.zeros((rows, cols), np.float32)
+    lib().orc_dequantize_int4(_p(q), _p(e), C.c_int(rows), C.c_int(cols), C.c_int(group), _p(w))
+    return w
+
+
+def int4_weights(layer: Dict, group: int = INT4_GROUP) -> Dict:
+    """The layer a quantised model computes with: every matrix replaced by its dequantised INT4 form
+    (norm gains stay as they are)."""
+    out = {}
+    for k, v in layer.items():
+        if k.endswith("norm"):
+            out[k] = v
+        else:
+            out[k] = dequantize_int4(*quantize_int4(v, group), group)
+    return out

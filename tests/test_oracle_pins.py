@@ -576,3 +576,47 @@ def test_branch_pacer_invariants_and_max_min_choice():
         t_after[nxt] += 1
         assert (share - t_after).min() == pytest.approx(best[0], abs=1e-9)
         assert f[nxt] == f.max()
+
+
+# ----------------------------------------------------------------------------- INT4 weights (Sec. 4.1)
+
+def test_int4_quantisation_hand_computed_groups():
+    """Groups worked out by hand: the scale is the smallest power of two with max|w| <= 7 * 2^e, codes
+    are w / 2^e rounded to nearest (halves to even) and clamped to [-8, 7]."""
+    g = 4
+    w = np.array([[0.7, -0.35, 0.0625, 0.0,          # max 0.7: 7 * 2^-4 = 0.4375 < 0.7 <= 7 * 2^-3 = 0.875 -> e = -3
+                   7.0, -7.0, 3.5, 2.5,              # max 7 = 7 * 2^0 -> e = 0; 3.5 -> 4 (half to even), 2.5 -> 2
+                   0.0, 0.0, 0.0, 0.0,               # all zero -> e = -126, codes 0
+                   -8.0, 1.0, 0.5, -0.5]],           # max 8 > 7 -> e = 1: -8/2 = -4, 1/2 = 0.5 -> 0, 0.25 -> 0, -0.25 -> 0
+                 np.float32)
+    q, e = orc.quantize_int4(w, g)
+    assert e.tolist() == [[-3, 0, -126, 1]]
+    assert q.tolist() == [[6, -3, 0, 0, 7, -7, 4, 2, 0, 0, 0, 0, -4, 0, 0, 0]]     # 0.7/0.125 = 5.6 -> 6; -2.8 -> -3; 0.5 -> 0
+    d = orc.dequantize_int4(q, e, g)
+    assert d.tolist() == [[0.75, -0.375, 0.0, 0.0, 7.0, -7.0, 4.0, 2.0, 0.0, 0.0, 0.0, 0.0, -8.0, 0.0, 0.0, 0.0]]
+
+
+def test_int4_quantisation_invariants():
+    rng = np.random.default_rng(5)
+    w = (rng.standard_normal((37, 256)) * 0.02).astype(np.float32)
+    w[3, 64:128] = 0.0
+    w[5, 0] = 1.5                                    # an outlier sets its group's scale
+    q, e = orc.quantize_int4(w)
+    d = orc.dequantize_int4(q, e)
+    assert q.min() >= -8 and q.max() <= 7
+    scale = np.exp2(e.astype(np.float64)).repeat(64, axis=1)
+    # nearest code: the error is at most half a step (the largest magnitude is at most 7 steps, so nothing clips)
+    assert (np.abs(d.astype(np.float64) - w) <= 0.5 * scale + 1e-12).all()
+    # the scale is the smallest admissible power of two: the group's largest magnitude exceeds 7 steps of the next smaller one
+    gmax = np.abs(w).reshape(37, 4, 64).max(axis=2)
+    nz = gmax > 0
+    assert (gmax[nz] <= 7 * np.exp2(e[nz].astype(np.float64))).all() and (gmax[nz] > 7 * np.exp2(e[nz].astype(np.float64) - 1)).all()
+    assert (e[~nz] == -126).all() and (d[3, 64:128] == 0).all()
+    # dequantised weights are bf16 values, and quantising them again changes nothing
+    assert torch.equal(torch.from_numpy(d).to(torch.bfloat16).float(), torch.from_numpy(d))
+    q2, e2 = orc.quantize_int4(d)
+    d2 = orc.dequantize_int4(q2, e2)
+    assert np.array_equal(d2, d)
+    # a linear layer over the quantised weights is the plain linear layer over the dequantised ones
+    x = rng.standard_normal((3, 256))
+    assert np.allclose(orc.linear(d, x), x @ d.astype(np.float64).T, rtol=1e-12, atol=1e-12)
