@@ -46,11 +46,14 @@ UNIT = "passes/s"
 NCU_GEMM_CAPTURE = {"summary": "profiles/gemm_chain_kernel__7b_qkv_n32.md", "dram_bytes": 104.80e6, "algorithmic_bytes": 102.5e6}
 
 
-def algorithmic_bytes(cfg, P, n):
+def algorithmic_bytes(cfg, P, n, int4=False):
     """Bytes one pass must move: every weight matrix once, the prefix K/V once, the tree nodes'
-    K/V written and read once, the embedding rows of the n tokens, the fp32 logits."""
+    K/V written and read once, the embedding rows of the n tokens, the fp32 logits. With INT4 weights
+    the layer matrices take half a byte per element plus one exponent byte per group of 64."""
     e = cfg.elem_bytes
     weights = cfg.weight_bytes()
+    if int4:
+        weights = int(cfg.n_layers * cfg.layer_weight_elems() * (0.5 + 1.0 / 64)) + cfg.vocab * cfg.d_model * e
     prefix_kv = 2 * cfg.n_layers * P * cfg.d_model * e
     tree_kv = 2 * 2 * cfg.n_layers * n * cfg.d_model * e
     logits = n * cfg.vocab * 4
@@ -214,9 +217,9 @@ def workload_name(w, cfg):
 
 # ------------------------------------------------------------------------------------------ GPU arm
 
-def build_verifier(cfg, w, device):
+def build_verifier(cfg, w, device, flags=0):
     from paper_2309_04255_b200 import binding as B
-    v = B.Verifier(cfg, w.prefix_len + 128 + 8, device=device)
+    v = B.Verifier(cfg, w.prefix_len + 128 + 8, device=device, flags=flags)
     v.pack_globals({k: gen.gen_tensor_device(cfg, k, -1, device) for k in ("tok_embed", "final_norm", "lm_head")})
     for l in range(cfg.n_layers):
         v.pack_layer(l, {k: gen.gen_tensor_device(cfg, k, l, device) for k in gen.LAYER_TENSORS})
@@ -345,11 +348,11 @@ def bench_workload(B, v, cfg, w, args, device, barrier, clocks=None, tag="main")
     return res
 
 
-def summarize(cfg, w, res, world, peaks, ms=None):
+def summarize(cfg, w, res, world, peaks, ms=None, int4=False):
     """ms: the median step time to report (the slowest replica's when there are several)."""
     hbm_peak, tf_peak, peak_kind = peaks
     P, n = w.prefix_len, w.n_nodes
-    ab = algorithmic_bytes(cfg, P, n)
+    ab = algorithmic_bytes(cfg, P, n, int4)
     fl = flops(cfg, P, n)
     ms = float(np.median(res["per_step_ms"])) if ms is None else ms
     s = {"ms_per_step": ms, "ms_per_step_min": float(min(res["per_step_ms"])), "ms_per_step_max": float(max(res["per_step_ms"])),
@@ -516,6 +519,19 @@ def run_gpu(args, w, cfg):
                            "attention_ms_per_step": rb3.get("attention_ms_per_step"), "steps": args.steps}
             v3.close()
             del v3
+            torch.cuda.empty_cache()
+            # the benchmarked workload with INT4 weights (Sec. 4.1 of the paper: the target runs INT4 on its devices)
+            v4 = build_verifier(cfg, w, device, flags=B.FLAG_INT4_WEIGHTS)
+            r4 = bench_workload(B, v4, cfg, w, args, device, barrier)
+            s4 = summarize(cfg, w, r4, 1, peaks, int4=True)
+            extra["C2_int4_weights"] = {"workload": workload_name(w, cfg) + "; layer matrices as INT4 codes with power-of-two group scales (groups of 64)",
+                                        "ms_per_step": s4["ms_per_step"], "ms_per_step_min": s4["ms_per_step_min"],
+                                        "ms_per_step_max": s4["ms_per_step_max"], "passes_per_s": s4["passes_per_s"],
+                                        "algorithmic_bytes": s4["pass_roofline"]["algorithmic_bytes"],
+                                        "frac_of_measured_hbm": s4["pass_roofline"]["frac_of_measured_hbm"],
+                                        "speedup_over_bf16": s["ms_per_step"] / s4["ms_per_step"], "steps": args.steps}
+            v4.close()
+            del v4
             torch.cuda.empty_cache()
             extra["C4"] = attention_digest(B, device, peaks)
             line["workloads"] = extra

@@ -74,7 +74,8 @@ enum {
     LLMCAD_FLAG_SIMT_GEMM = 1, /* use the plain-ALU GEMM even for bf16 (debugging aid) */
     LLMCAD_FLAG_SIMT_ATTN = 2, /* use the plain-ALU attention even for bf16 (debugging aid) */
     LLMCAD_FLAG_T5_ATTN = 4,   /* bf16, head_dim 128: tcgen05 attention kernel for every tree size (default: above 32 nodes) */
-    LLMCAD_FLAG_MMA_ATTN = 8   /* bf16, head_dim 128: mma.sync attention kernel for every tree size */
+    LLMCAD_FLAG_MMA_ATTN = 8,  /* bf16, head_dim 128: mma.sync attention kernel for every tree size */
+    LLMCAD_FLAG_INT4_WEIGHTS = 16 /* bf16 contexts: the seven matrices of every layer are held as INT4 (see llmcad_quantize_int4) */
 };
 
 /* indices into the scalars[8] output */
@@ -238,6 +239,26 @@ int llmcad_tile_weight(const void *w, int32_t n_out, int32_t n_in, void *tiled /
 /* llmcad_skinny_gemm on a matrix in that layout (bf16 contexts only). */
 int llmcad_skinny_gemm_tiled(llmcad_ctx *ctx, const void *w_tiled, const void *x, float *y, int32_t n_out, int32_t n_in,
                              int32_t n, void *stream);
+
+/* INT4 weights (Sec. 4.1: the target model runs with INT4 group-quantised weights). Format of this
+ * library, where the paper only names the precision: symmetric codes q in [-8, 7], one scale per row and
+ * group of 64 consecutive input columns, the scale a power of two 2^e with e the smallest integer such
+ * that max|w| <= 7 * 2^e over the group (-126 for a group of zeros), q = w / 2^e rounded to nearest,
+ * halves to even. Every dequantised weight q * 2^e is a value bf16 holds exactly, so a pass with INT4
+ * weights is the bf16 pass over the dequantised weights, bit for bit, at a quarter of the weight bytes.
+ * A context created with LLMCAD_FLAG_INT4_WEIGHTS (bf16, d_model and d_ffn multiples of 64) quantises
+ * the layer matrices inside llmcad_pack_layer and streams them as INT4 tiles, which the GEMM kernel
+ * expands to bf16 tiles in shared memory; embedding and lm_head stay bf16.
+ * llmcad_quantize_int4: codes and exponents of a row-major bf16 matrix [n_out][n_in] (DEVICE), n_in a
+ * multiple of 64, as plain arrays q [n_out][n_in] and e [n_out][n_in / 64] (DEVICE int8).
+ * llmcad_tile_weight_int4 / llmcad_tiled_weight_int4_bytes: the same quantisation in the layout the GEMM
+ * streams (4224 bytes per tile of 128 rows and 64 columns: 128 x 8 words of eight codes, 128 exponents).
+ * llmcad_skinny_gemm_tiled_int4: llmcad_skinny_gemm on a matrix in that layout (bf16 contexts only). */
+int llmcad_quantize_int4(const void *w, int32_t n_out, int32_t n_in, int8_t *q, int8_t *e, void *stream);
+size_t llmcad_tiled_weight_int4_bytes(int32_t n_out, int32_t n_in);
+int llmcad_tile_weight_int4(const void *w, int32_t n_out, int32_t n_in, void *tiled /*DEVICE*/, void *stream);
+int llmcad_skinny_gemm_tiled_int4(llmcad_ctx *ctx, const void *w_tiled, const void *x, float *y, int32_t n_out, int32_t n_in,
+                                  int32_t n, void *stream);
 
 /* Tree attention without any allocation. (The paper has no counterpart: this entry point exists
  * for the way the library is embedded, not for the method.)

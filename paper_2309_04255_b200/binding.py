@@ -21,7 +21,7 @@ MAX_TREE = 128
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CUDA = 0, -1, -2, -3, -4
 ERR_BAD_TREE, ERR_BAD_TOKEN, ERR_TIMEOUT, ERR_NAN = 1, 2, 3, 4
 F32, BF16 = 0, 1
-FLAG_SIMT_GEMM, FLAG_SIMT_ATTN, FLAG_T5_ATTN, FLAG_MMA_ATTN = 1, 2, 4, 8
+FLAG_SIMT_GEMM, FLAG_SIMT_ATTN, FLAG_T5_ATTN, FLAG_MMA_ATTN, FLAG_INT4_WEIGHTS = 1, 2, 4, 8, 16
 S_ACCEPTED_LEN, S_NEXT_TOKEN, S_NEW_PREFIX_LEN, S_N_CORRECT, S_N_ALL, S_RECTIFIED, S_STATUS = range(7)
 
 EXPORTS = [
@@ -32,6 +32,7 @@ EXPORTS = [
     "llmcad_last_status", "llmcad_set_kernel_timing", "llmcad_get_kernel_timing", "llmcad_set_gemm_trace", "llmcad_tiled_weight_bytes", "llmcad_tile_weight", "llmcad_skinny_gemm_tiled", "llmcad_tree_attention_noalloc", "llmcad_noalloc_last_error",
     "llmcad_tree_confidence", "llmcad_update_threshold", "llmcad_extend_tree", "llmcad_tree_branches", "llmcad_branch_pacer",
     "llmcad_set_wait_limit_ns", "llmcad_selftest_wait_timeout",
+    "llmcad_quantize_int4", "llmcad_tiled_weight_int4_bytes", "llmcad_tile_weight_int4", "llmcad_skinny_gemm_tiled_int4",
 ]
 
 
@@ -108,6 +109,11 @@ def lib():
         L.llmcad_extend_tree.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
         L.llmcad_set_kernel_timing.argtypes = [vp, i32]
         L.llmcad_get_kernel_timing.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+        L.llmcad_quantize_int4.argtypes = [vp, i32, i32, vp, vp, vp]
+        L.llmcad_tiled_weight_int4_bytes.argtypes = [i32, i32]
+        L.llmcad_tiled_weight_int4_bytes.restype = sz
+        L.llmcad_tile_weight_int4.argtypes = [vp, i32, i32, vp, vp]
+        L.llmcad_skinny_gemm_tiled_int4.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
         L.llmcad_set_wait_limit_ns.argtypes = [vp, C.c_uint64]
         L.llmcad_selftest_wait_timeout.argtypes = [vp, vp]
         _lib = L
@@ -276,6 +282,20 @@ class Verifier:
                "llmcad_skinny_gemm_tiled")
         return y
 
+    def tile_weight_int4(self, w):
+        """Row-major bf16 [n_out][n_in] -> INT4 codes and group exponents in the layout the GEMM streams."""
+        n_out, n_in = w.shape
+        t = torch.empty(lib().llmcad_tiled_weight_int4_bytes(n_out, n_in), dtype=torch.uint8, device=self.device)
+        _check(lib().llmcad_tile_weight_int4(_ptr(w), n_out, n_in, _ptr(t), _stream()), "llmcad_tile_weight_int4")
+        return t
+
+    def skinny_gemm_tiled_int4(self, w_tiled, n_out, x):
+        n, n_in = x.shape
+        y = torch.empty((n, n_out), dtype=torch.float32, device=self.device)
+        _check(lib().llmcad_skinny_gemm_tiled_int4(self.ctx, _ptr(w_tiled), _ptr(x), _ptr(y), n_out, n_in, n, _stream()),
+               "llmcad_skinny_gemm_tiled_int4")
+        return y
+
     def last_status(self) -> int:
         return lib().llmcad_last_status(self.ctx, _stream())
 
@@ -324,6 +344,15 @@ def tree_attention_noalloc(q, k, v, prefix_len: int, parent, o, status=None):
     if code != OK:
         raise LlmcadError(code, "llmcad_tree_attention_noalloc: " + lib().llmcad_noalloc_last_error().decode())
     return o
+
+
+def quantize_int4(w: torch.Tensor):
+    """INT4 codes [n_out][n_in] and group exponents [n_out][n_in / 64] (both int8, on w's device) of a bf16 matrix."""
+    n_out, n_in = w.shape
+    q = torch.empty((n_out, n_in), dtype=torch.int8, device=w.device)
+    e = torch.empty((n_out, n_in // 64), dtype=torch.int8, device=w.device)
+    _check(lib().llmcad_quantize_int4(_ptr(w), n_out, n_in, _ptr(q), _ptr(e), _stream()), "llmcad_quantize_int4")
+    return q, e
 
 
 def tree_confidence(branch_conf) -> float:

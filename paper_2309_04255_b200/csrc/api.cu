@@ -52,7 +52,9 @@ PackedLayout packed_layout(const llmcad_config &c)
     const size_t e = c.dtype == LLMCAD_F32 ? 4 : 2;
     const size_t d = c.d_model, f = c.d_ffn, v = c.vocab;
     const bool tiled = want_tiled(c);
-    auto mat = [&](size_t n_out, size_t n_in) { return tiled ? tiled_weight_bytes((int)n_out, (int)n_in) : n_out * n_in * e; };
+    const bool w4 = tiled && (c.flags & LLMCAD_FLAG_INT4_WEIGHTS);     // the layer matrices only; the lm_head stays bf16
+    auto mat_head = [&](size_t n_out, size_t n_in) { return tiled ? tiled_weight_bytes((int)n_out, (int)n_in) : n_out * n_in * e; };
+    auto mat = [&](size_t n_out, size_t n_in) { return w4 ? tiled_weight_int4_bytes((int)n_out, (int)n_in) : mat_head(n_out, n_in); };
     PackedLayout L{};
     size_t o = 0;
     L.attn_norm = o; o = align_up(o + d * e, 1024);
@@ -65,7 +67,7 @@ PackedLayout packed_layout(const llmcad_config &c)
     o = L.layer_bytes * (size_t)c.n_layers;
     L.tok_embed = o;  o = align_up(o + v * d * e, 1024);
     L.final_norm = o; o = align_up(o + d * e, 1024);
-    L.lm_head = o;    o = align_up(o + mat(v, d), 1024);
+    L.lm_head = o;    o = align_up(o + mat_head(v, d), 1024);
     L.total = o;
     return L;
 }
@@ -81,6 +83,8 @@ int check_config(const llmcad_config *c)
     if (c->head_dim != 64 && c->head_dim != 128) return LLMCAD_ERR_UNSUPPORTED;
     if (c->n_heads * c->head_dim != c->d_model) return LLMCAD_ERR_UNSUPPORTED;
     if (c->d_model % 8 || c->d_ffn % 8) return LLMCAD_ERR_UNSUPPORTED;
+    // INT4 weights: the tensor-core path only, groups of 64 input columns
+    if ((c->flags & LLMCAD_FLAG_INT4_WEIGHTS) && (!want_tiled(*c) || c->d_model % 64 || c->d_ffn % 64)) return LLMCAD_ERR_UNSUPPORTED;
     return LLMCAD_OK;
 }
 
@@ -94,6 +98,7 @@ struct llmcad_ctx {
     int n_sms = 0;
     size_t elem = 2;
     bool tc_gemm = false, tc_attn = false;
+    bool w4 = false;          // the layer matrices are held as INT4 tiles (LLMCAD_FLAG_INT4_WEIGHTS)
     // Tensor-core path: activations travel as bf16 hi + lo planes (common.cuh); a tuning aid
     // (LLMCAD_COMP=0) turns the lo planes off.
     bool comp = false;
@@ -224,7 +229,7 @@ struct TcGemm {
     void set(llmcad_ctx *ctx, int l, int which, int act, int n_in, const EpiParams &ep, int n_pad)
     {
         maps.x = ctx->act_maps[n_pad / 16][act];
-        p.g = make_gemm_desc(n_in, ep, weight_ptr(ctx, l, which));
+        p.g = make_gemm_desc(n_in, ep, weight_ptr(ctx, l, which), ctx->w4 && l >= 0);
         p.n_pad = n_pad;
         p.comp = ctx->comp ? 1 : 0;
     }
@@ -515,6 +520,7 @@ int llmcad_create(const llmcad_config *cfg, llmcad_ctx **out)
     ctx->elem = cfg->dtype == LLMCAD_F32 ? 4 : 2;
     const bool sm100 = prop.major == 10;
     ctx->tc_gemm = want_tiled(*cfg);
+    ctx->w4 = ctx->tc_gemm && (cfg->flags & LLMCAD_FLAG_INT4_WEIGHTS);
     if (ctx->tc_gemm && !sm100) {   // the tensor-core kernels are sm_100a only
         delete ctx;
         snprintf(g_cuda_err, sizeof(g_cuda_err), "device is not sm_100");
@@ -602,6 +608,20 @@ int llmcad_pack_layer(llmcad_ctx *ctx, int32_t layer, const llmcad_layer_weights
     auto cp = [&](size_t off, const void *s, size_t bytes) {
         return cudaMemcpyAsync(lb + off, s, bytes, cudaMemcpyDeviceToDevice, st);
     };
+    if (ctx->w4) {
+        // quantised on the way in: INT4 codes and power-of-two group scales, tiled for the streaming kernel
+        const size_t t_dd = tiled_weight_int4_bytes((int)d, (int)d), t_fd = tiled_weight_int4_bytes((int)f, (int)d);
+        CUDA_TRY(cp(ctx->lay.attn_norm, src->attn_norm, d * e));
+        CUDA_TRY(cp(ctx->lay.ffn_norm, src->ffn_norm, d * e));
+        CUDA_TRY(launch_tile_weight_int4(src->wq, (int)d, (int)d, lb + ctx->lay.wqkv, st));
+        CUDA_TRY(launch_tile_weight_int4(src->wk, (int)d, (int)d, lb + ctx->lay.wqkv + t_dd, st));
+        CUDA_TRY(launch_tile_weight_int4(src->wv, (int)d, (int)d, lb + ctx->lay.wqkv + 2 * t_dd, st));
+        CUDA_TRY(launch_tile_weight_int4(src->wo, (int)d, (int)d, lb + ctx->lay.wo, st));
+        CUDA_TRY(launch_tile_weight_int4(src->w_gate, (int)f, (int)d, lb + ctx->lay.wgu, st));
+        CUDA_TRY(launch_tile_weight_int4(src->w_up, (int)f, (int)d, lb + ctx->lay.wgu + t_fd, st));
+        CUDA_TRY(launch_tile_weight_int4(src->w_down, (int)d, (int)f, lb + ctx->lay.wdown, st));
+        return LLMCAD_OK;
+    }
     if (ctx->tc_gemm) {
         const size_t t_dd = tiled_weight_bytes((int)d, (int)d), t_fd = tiled_weight_bytes((int)f, (int)d);
         CUDA_TRY(cp(ctx->lay.attn_norm, src->attn_norm, d * e));
@@ -856,6 +876,52 @@ int llmcad_skinny_gemm_tiled(llmcad_ctx *ctx, const void *w_tiled, const void *x
         return LLMCAD_ERR_CUDA;
     }
     g.p.g = make_gemm_desc(n_in, ep, w_tiled);
+    g.p.n_pad = n_pad;
+    return g.launch(ctx, status, st);
+}
+
+int llmcad_quantize_int4(const void *w, int32_t n_out, int32_t n_in, int8_t *q, int8_t *e, void *stream)
+{
+    if (!w || !q || !e) return LLMCAD_ERR_INVALID_ARG;
+    if (n_out < 1 || n_in < 1) return LLMCAD_ERR_INVALID_ARG;
+    if (n_in % 64) return LLMCAD_ERR_UNSUPPORTED;
+    CUDA_TRY(launch_quantize_int4_plain(w, n_out, n_in, q, e, static_cast<cudaStream_t>(stream)));
+    return LLMCAD_OK;
+}
+
+size_t llmcad_tiled_weight_int4_bytes(int32_t n_out, int32_t n_in)
+{
+    if (n_out < 1 || n_in < 1 || n_in % 64) return 0;
+    return tiled_weight_int4_bytes(n_out, n_in);
+}
+
+int llmcad_tile_weight_int4(const void *w, int32_t n_out, int32_t n_in, void *tiled, void *stream)
+{
+    if (!w || !tiled) return LLMCAD_ERR_INVALID_ARG;
+    if (n_out < 1 || n_in < 1) return LLMCAD_ERR_INVALID_ARG;
+    if (n_in % 64) return LLMCAD_ERR_UNSUPPORTED;
+    CUDA_TRY(launch_tile_weight_int4(w, n_out, n_in, tiled, static_cast<cudaStream_t>(stream)));
+    return LLMCAD_OK;
+}
+
+int llmcad_skinny_gemm_tiled_int4(llmcad_ctx *ctx, const void *w_tiled, const void *x, float *y, int32_t n_out, int32_t n_in,
+                                  int32_t n, void *stream)
+{
+    if (!ctx || !w_tiled || !x || !y) return LLMCAD_ERR_INVALID_ARG;
+    if (n_out < 1 || n_in < 1 || n < 1) return LLMCAD_ERR_INVALID_ARG;
+    if (n > ctx->cfg.max_tree || n_in % 64 || !ctx->tc_gemm) return LLMCAD_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *status = ctx->scalars_dev() + LLMCAD_S_STATUS;
+    CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    EpiParams ep{};
+    ep.mode = EPI_PLAIN; ep.n = n; ep.n_out = n_out; ep.y = y; ep.ldy = n_out;
+    const int n_pad = (n + 15) / 16 * 16;
+    TcGemm g;
+    if (!make_act_map_bf16(&g.maps.x, x, n, n_in, n_pad, 1, n)) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed");
+        return LLMCAD_ERR_CUDA;
+    }
+    g.p.g = make_gemm_desc(n_in, ep, w_tiled, true);
     g.p.n_pad = n_pad;
     return g.launch(ctx, status, st);
 }

@@ -267,6 +267,11 @@ cudaError_t launch_compact(void *kv, int dtype, int n_layers, int n_heads, int S
                            const int32_t *scalars, cudaStream_t st);
 size_t tiled_weight_bytes(int n_out, int n_in);
 cudaError_t launch_tile_weight(const void *w, int n_out, int n_in, void *dst, cudaStream_t st);
+// INT4 weights (pack.cu): bytes of one (128 rows x 64 columns) tile: 4 KB of codes + 128 exponents
+constexpr int kW4TileBytes = 4096 + 128;
+size_t tiled_weight_int4_bytes(int n_out, int n_in);       // n_in a multiple of 64
+cudaError_t launch_tile_weight_int4(const void *w, int n_out, int n_in, void *dst, cudaStream_t st);
+cudaError_t launch_quantize_int4_plain(const void *w, int n_out, int n_in, int8_t *q, int8_t *e, cudaStream_t st);
 cudaError_t launch_gemm_simt(const void *W, const void *x, int dtype, int n_in, const EpiParams &ep,
                              const int32_t *status, cudaStream_t st);
 cudaError_t launch_attention_simt(const void *q, const void *k, const void *v, int dtype, int n_heads, int hd,

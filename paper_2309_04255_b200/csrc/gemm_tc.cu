@@ -62,6 +62,7 @@ constexpr size_t kFinSmem = 24 * 1024;   // dynamic shared memory the finishing 
                                          // there for the next GEMM's streaming CTA
 constexpr int kATileBytes = kTileM * kBlockK * 2;  // 16 KB
 constexpr int kMaxStages = 16;
+constexpr int kMaxPStages = 24;   // INT4 weights: ring of packed tiles
 constexpr int kMaxPairK = 2;     // k-blocks per ring item (GemmDesc::pair_k): 2 = one 32 KB weight copy feeds 8 MMAs;
                                  // 1 for wide activation tiles, which would leave too few ring stages otherwise
 
@@ -241,6 +242,8 @@ struct SharedCtl {
     uint32_t tmem_base;
     volatile int abort_flag;
     volatile uint32_t a_issued;     // ring items whose weight copy (and expect_tx) has been issued
+    uint64_t pfull[kMaxPStages];    // INT4 weights: packed tile landed / packed stage free again
+    uint64_t pempty[kMaxPStages];
 };
 
 // A ring item is (tile, k-block pair, half): up to two consecutive 64-wide k-blocks of one
@@ -496,7 +499,7 @@ __device__ __forceinline__ void finish_rows_t(const FinishArgs &fa, int lane, co
 
 #define LLMCAD_TRACE(slot) do { if (p.trace && blockIdx.x < 256) p.trace[(size_t)blockIdx.x * 16 + (slot)] = global_timer_ns(); } while (0)
 
-template <int PK>
+template <int PK, bool W4>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ GemmParams p)
 {
@@ -511,6 +514,9 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
     const uint32_t stage_bytes = PK * (kATileBytes + b_tile_bytes);
     const uint32_t b_off = PK * kATileBytes;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    // INT4 weights: behind the ring of MMA stages lies a ring of packed items (PK tiles of 4224 bytes each)
+    constexpr uint32_t pstage_bytes = PK * kW4TileBytes;
+    const uint32_t packed_base = smem_base + (uint32_t)p.stages * stage_bytes;
     const uint32_t acc_cols = 2u * nb;                    // TMEM columns of one accumulator buffer (gate | up)
     const bool two_bufs = p.acc_bufs == 2;
     const uint64_t wait_limit = p.wait_limit_ns;          // every wait below gives up after this many ns
@@ -528,6 +534,18 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
     uint64_t pol_stream = 0;
     auto issue_item = [&]() {          // the next item of the stream into ring stage ps (which must be free)
         const int nk = pc.nk();
+        if (W4) {
+            // packed tiles go to the packed ring; the dump warps turn them into MMA stages
+            const uint32_t pf = smem_u32(&ctl.pfull[ps]);
+            mbar_expect_tx(pf, (uint32_t)nk * kW4TileBytes);
+            const size_t t = (size_t)(pc.tile + (pc.half ? d.up_tile_offset : 0)) * d.kb_per_tile + pc.kb0();
+            bulk_load_1d(packed_base + ps * pstage_bytes, d.w_tiled + t * kW4TileBytes, (uint32_t)nk * kW4TileBytes, pf, pol_stream);
+            if (pissued == 0) LLMCAD_TRACE(2);
+            ++pissued;
+            pc.advance();
+            if (++ps == p.pstages) { ps = 0; ppar ^= 1u; }
+            return;
+        }
         const uint32_t full = smem_u32(&ctl.full[ps]);
         const uint32_t dst = smem_base + ps * stage_bytes;
         mbar_expect_tx(full, (uint32_t)nk * (kATileBytes + b_tile_bytes));
@@ -548,8 +566,16 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
     };
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&ctl.full[s]), 1);
+            // INT4: a stage is full when its activation bytes have landed (armed by one arrival) and the four
+            // dump warps have written their quarters of the weight tile
+            mbar_init(smem_u32(&ctl.full[s]), W4 ? 5 : 1);
             mbar_init(smem_u32(&ctl.empty[s]), 1);
+        }
+        if (W4) {
+            for (int s = 0; s < p.pstages; ++s) {
+                mbar_init(smem_u32(&ctl.pfull[s]), 1);
+                mbar_init(smem_u32(&ctl.pempty[s]), 4);
+            }
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.tmem_full[b]), 1);
@@ -561,7 +587,7 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
         pc.init(d);
-        while (!pc.done() && pissued < (uint32_t)p.stages) issue_item();
+        while (!pc.done() && pissued < (uint32_t)(W4 ? p.pstages : p.stages)) issue_item();
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
@@ -586,9 +612,15 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
             uint32_t prefetched = 0;
             uint64_t t_idle = 0;
             while (!pc.done()) {
-                if (mbar_try(smem_u32(&ctl.empty[ps]), ppar)) {
+                if (mbar_try(smem_u32(W4 ? &ctl.pempty[ps] : &ctl.empty[ps]), ppar)) {
                     issue_item();
                     t_idle = 0;
+                    continue;
+                }
+                if (W4) {      // the packed ring is deep enough by itself
+                    __nanosleep(32);
+                    if (t_idle == 0) t_idle = global_timer_ns();
+                    else if (*abort_flag || global_timer_ns() - t_idle > wait_limit) { timed_out = true; break; }
                     continue;
                 }
                 // The ring is full: the consumers wait for their input. Weights do not depend on that,
@@ -711,18 +743,87 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
         // ================================================= accumulator dump (warps 2..5)
         const int lane_grp = warp & 3;                 // TMEM lanes 32*lane_grp .. +31 belong to this warp
         // the workspace may still be read by the finishing kernel of the previous GEMM
-        if (!dep_wait_warp(dep, lane)) timed_out = true;
-        pdl_launch_dependents();
-        if (threadIdx.x == 64) LLMCAD_TRACE(3);
+        bool dep_ok = false;
+        if (!W4) {
+            if (!dep_wait_warp(dep, lane)) timed_out = true;
+            pdl_launch_dependents();
+            dep_ok = true;
+            if (threadIdx.x == 64) LLMCAD_TRACE(3);
+        }
         const Range r = cta_range<PK>(d, (int)blockIdx.x);
         const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
         const size_t slot_stride = slot_floats(d.halves, p.n_pad);
+        // ---- INT4 weights: these warps also turn every packed item into the bf16 tiles the MMA reads, a quarter
+        // of the rows each, in the MMA stage that they claim for it. Element j of a word sits where
+        // (word >> 4k) & 0x000f000f picks elements 2k, 2k+1; OR-ing 0x4300 into each half makes the bf16 values
+        // 128 + u (u = q + 8), and one fused multiply-add per pair, (128 + u) * 2^e - 136 * 2^e, gives q * 2^e exactly.
+        Cursor<PK> dc;
+        dc.init(d);
+        int ds = 0, dps = 0;
+        uint32_t dpar = 1, dppar = 0, dcount = 0;      // a fresh "empty" barrier passes a wait on parity 1
+        uint8_t *const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+        auto dequant_item = [&]() -> bool {
+            const int nk = dc.nk();
+            if (!mbar_wait_warp(smem_u32(&ctl.empty[ds]), dpar, abort_flag, lane, wait_limit)) return false;
+            if (warp == 2 && lane == 0) {
+                mbar_expect_tx(smem_u32(&ctl.full[ds]), (uint32_t)nk * b_tile_bytes);
+                __threadfence_block();
+                ctl.a_issued = ++dcount;       // the activation loader may now add its bytes to this stage
+            }
+            if (!mbar_wait_warp(smem_u32(&ctl.pfull[dps]), dppar, abort_flag, lane, wait_limit)) return false;
+            const uint8_t *pk = smem_gen + (size_t)p.stages * stage_bytes + (size_t)dps * pstage_bytes;
+            uint8_t *wt = smem_gen + (size_t)ds * stage_bytes;
+            for (int k = 0; k < nk; ++k) {
+                const uint32_t *words = reinterpret_cast<const uint32_t *>(pk + (size_t)k * kW4TileBytes);
+                const int8_t *exps = reinterpret_cast<const int8_t *>(pk + (size_t)k * kW4TileBytes + 4096);
+#pragma unroll 4
+                for (int it = 0; it < 8; ++it) {
+                    const int row = lane_grp * 32 + it * 4 + (lane >> 3), c = lane & 7;
+                    const uint32_t x = words[row * 8 + c];
+                    const int e = exps[row];
+                    const uint32_t s16 = (uint32_t)(e + 127) << 7;                       // bf16 bits of 2^e
+                    const uint32_t b16 = 0x8000u | ((uint32_t)(e + 134) << 7) | 8u;      // bf16 bits of -136 * 2^e
+                    const uint32_t s2 = s16 | (s16 << 16), b2 = b16 | (b16 << 16);
+                    uint32_t o[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t t2 = ((x >> (4 * j)) & 0x000f000fu) | 0x43004300u;
+                        const __nv_bfloat162 rr = __hfma2(*reinterpret_cast<const __nv_bfloat162 *>(&t2),
+                                                          *reinterpret_cast<const __nv_bfloat162 *>(&s2),
+                                                          *reinterpret_cast<const __nv_bfloat162 *>(&b2));
+                        o[j] = *reinterpret_cast<const uint32_t *>(&rr);
+                    }
+                    *reinterpret_cast<uint4 *>(wt + (size_t)k * kATileBytes + row * 128 + ((c ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the tensor core reads what these threads wrote
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&ctl.full[ds]));
+                mbar_arrive(smem_u32(&ctl.pempty[dps]));
+            }
+            dc.advance();
+            if (++ds == p.stages) { ds = 0; dpar ^= 1u; }
+            if (++dps == p.pstages) { dps = 0; dppar ^= 1u; }
+            return true;
+        };
         uint32_t seg = 0;
         for (int seg_begin = r.begin; seg_begin < r.end && !timed_out; ++seg) {
             const int tile = seg_begin / ipt;
             const int seg_end = min(r.end, (tile + 1) * ipt);
             const int buf = two_bufs ? (seg & 1) : 0;
             const uint32_t use = two_bufs ? (seg >> 1) : seg;
+            if (W4) {
+                for (int i = seg_begin; i < seg_end && !timed_out; ++i)
+                    if (!dequant_item()) timed_out = true;
+                if (timed_out) break;
+                if (!dep_ok) {          // the workspace may still be read by the previous GEMM's finishing kernel
+                    if (!dep_wait_warp(dep, lane)) { timed_out = true; break; }
+                    pdl_launch_dependents();
+                    dep_ok = true;
+                    if (threadIdx.x == 64) LLMCAD_TRACE(3);
+                }
+            }
             if (!mbar_wait_warp(smem_u32(&ctl.tmem_full[buf]), use & 1u, abort_flag, lane, wait_limit)) { timed_out = true; break; }
             tc_fence_after();
             if (threadIdx.x == 64 && seg == 0) LLMCAD_TRACE(4);
@@ -958,7 +1059,7 @@ bool make_tensor_map_bf16_3d(CUtensorMap *map, const void *base, const uint64_t 
 
 size_t gemm_tc_partial_floats(int n_sms, int max_tiles, int max_n_pad) { return (size_t)(max_tiles + n_sms) * slot_floats(2, max_n_pad); }
 
-GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)
+GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled, bool w4)
 {
     GemmDesc d{};
     d.halves = ep.mode == EPI_SWIGLU ? 2 : 1;
@@ -970,6 +1071,7 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled)
     d.grid = 0;
     d.w_tiled = static_cast<const uint8_t *>(w_tiled);
     d.up_tile_offset = d.n_tiles;
+    d.w4 = w4 ? 1 : 0;
     d.ep = ep;
     return d;
 }
@@ -1054,18 +1156,35 @@ cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_
     if (stages > kMaxStages) stages = kMaxStages;
     if (tune.stages_cap && tune.stages_cap < stages) stages = tune.stages_cap;   // tuning aid: cap the ring depth
     if (stages < 2) return cudaErrorInvalidConfiguration;
+    size_t smem = (size_t)stages * stage_bytes + 1024;
+    p.pstages = 0;
+    if (d.w4) {
+        // INT4 weights: the MMA ring keeps what covers the latency of the activation copies (three stages where
+        // they fit), the rest of the shared memory holds packed items, four times as many weights per byte
+        if (d.w_tiled == nullptr) return cudaErrorInvalidValue;
+        const size_t pstage = (size_t)pair_k * kW4TileBytes;
+        if (stages > 3) stages = 3;
+        while (stages > 2 && full_limit - (size_t)stages * stage_bytes < 8 * pstage) --stages;   // room for eight packed items
+        int pst = (int)((full_limit - (size_t)stages * stage_bytes) / pstage);
+        if (pst > kMaxPStages) pst = kMaxPStages;
+        if (pst < 2) return cudaErrorInvalidConfiguration;
+        p.pstages = pst;
+        smem = (size_t)stages * stage_bytes + (size_t)pst * pstage + 1024;
+        p.next = NextWeights{};
+    }
     p.stages = stages;
-    const size_t smem = (size_t)stages * stage_bytes + 1024;
     static PerDeviceOnce attr_set;
     if (attr_set.needed()) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_stream_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(gemm_stream_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
+        cudaError_t e = cudaSuccess;
+        typedef void (*SKernel)(GemmMaps, GemmParams);
+        const SKernel all[4] = {gemm_stream_kernel<1, false>, gemm_stream_kernel<2, false>, gemm_stream_kernel<1, true>, gemm_stream_kernel<2, true>};
         // An SM splits its on-chip memory between shared memory and L1 when it is empty, to fit the kernel that
         // arrives; a streaming CTA of 195 KB would get a 196 KB split, and the finishing CTA of the same GEMM
         // could not settle beside it. Every kernel of the GEMM asks for the largest shared-memory split.
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_stream_kernel<1>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_stream_kernel<2>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+            e = cudaFuncSetAttribute(all[i], cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(all[i], cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        }
         if (e != cudaSuccess) return e;
         attr_set.mark();
     }
@@ -1074,8 +1193,11 @@ cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_
     if (p.wait_limit_ns == 0) p.wait_limit_ns = kDefaultWaitLimitNs;
     {
         LaunchCfg lc(grid, kThreads, smem, st);
-        const cudaError_t e = pair_k == 1 ? cudaLaunchKernelEx(&lc.cfg, gemm_stream_kernel<1>, maps, p)
-                                          : cudaLaunchKernelEx(&lc.cfg, gemm_stream_kernel<2>, maps, p);
+        cudaError_t e;
+        if (d.w4) e = pair_k == 1 ? cudaLaunchKernelEx(&lc.cfg, gemm_stream_kernel<1, true>, maps, p)
+                                  : cudaLaunchKernelEx(&lc.cfg, gemm_stream_kernel<2, true>, maps, p);
+        else e = pair_k == 1 ? cudaLaunchKernelEx(&lc.cfg, gemm_stream_kernel<1, false>, maps, p)
+                             : cudaLaunchKernelEx(&lc.cfg, gemm_stream_kernel<2, false>, maps, p);
         if (e != cudaSuccess) return e;
         if (launched) ++*launched;
     }

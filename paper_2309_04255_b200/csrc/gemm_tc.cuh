@@ -21,6 +21,8 @@ struct GemmDesc {
     const uint8_t *w_tiled;  // weights as a sequence of pre-swizzled 16 KB tiles [tile][k-block] (see pack.cu),
                              // or nullptr: row-major weights through the tensor map
     int up_tile_offset;      // first tile of the up projection in the tiled sequence
+    int w4;                  // 1: w_tiled holds INT4 tiles (pack.cu, 4224 bytes per tile and k-block) that the kernel
+                             // turns into bf16 tiles in shared memory on their way to the MMA
     EpiParams ep;
 };
 
@@ -43,6 +45,7 @@ struct GemmParams {
     int comp;           // 1: activations come as hi + lo planes; the MMA N is 2 * n_pad and the two columns of a node are added
     int acc_bufs;       // accumulator buffers in TMEM: 2, or 1 when 2 x (gate | up) x MMA N exceeds the 512 columns
     int stages;         // depth of the shared-memory ring
+    int pstages;        // INT4 weights: depth of the ring of packed tiles that feeds it
     int tmem_cols;      // allocated TMEM columns (power of two)
     float *partials;    // segment slots [n_tiles + grid][4 row groups][halves][n_pad][32 rows] fp32: the segment of
                         // tile t held by CTA c sits in slot t + c
@@ -80,7 +83,7 @@ bool make_tensor_map_bf16_3d(CUtensorMap *map, const void *base, const uint64_t 
 size_t gemm_tc_partial_floats(int n_sms, int max_tiles, int max_n_pad);
 
 // Describes one GEMM (fills everything but items_per_cta and grid, which the launcher sets).
-GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled = nullptr);
+GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled = nullptr, bool w4 = false);
 
 // Fixes how the GEMM is cut up (k-blocks per ring item, items per CTA, grid); launch_gemm_tc calls it
 // itself, callers that want to describe a GEMM to its predecessor (next_weights) call it first.
