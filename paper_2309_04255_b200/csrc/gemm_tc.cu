@@ -773,27 +773,37 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
             if (!mbar_wait_warp(smem_u32(&ctl.pfull[dps]), dppar, abort_flag, lane, wait_limit)) return false;
             const uint8_t *pk = smem_gen + (size_t)p.stages * stage_bytes + (size_t)dps * pstage_bytes;
             uint8_t *wt = smem_gen + (size_t)ds * stage_bytes;
+            // lane = (row within a group of four, chunk): iteration `it` handles row 32 * lane_grp + 4 * it + lane / 8,
+            // words and stores of a warp instruction are contiguous (no bank conflicts). All loads of a k-block go
+            // out before the first conversion: a warp is alone on its scheduler here, so latency is what counts.
+            const int r_in = lane >> 3, c = lane & 7;
             for (int k = 0; k < nk; ++k) {
-                const uint32_t *words = reinterpret_cast<const uint32_t *>(pk + (size_t)k * kW4TileBytes);
-                const int8_t *exps = reinterpret_cast<const int8_t *>(pk + (size_t)k * kW4TileBytes + 4096);
-#pragma unroll 4
+                const uint32_t *words = reinterpret_cast<const uint32_t *>(pk + (size_t)k * kW4TileBytes) + (lane_grp * 32 + r_in) * 8 + c;
+                const int8_t *exps = reinterpret_cast<const int8_t *>(pk + (size_t)k * kW4TileBytes + 4096) + lane_grp * 32 + r_in;
+                uint8_t *dst = wt + (size_t)k * kATileBytes + (size_t)(lane_grp * 32 + r_in) * 128;
+                uint32_t x[8];
+                int e[8];
+#pragma unroll
                 for (int it = 0; it < 8; ++it) {
-                    const int row = lane_grp * 32 + it * 4 + (lane >> 3), c = lane & 7;
-                    const uint32_t x = words[row * 8 + c];
-                    const int e = exps[row];
-                    const uint32_t s16 = (uint32_t)(e + 127) << 7;                       // bf16 bits of 2^e
-                    const uint32_t b16 = 0x8000u | ((uint32_t)(e + 134) << 7) | 8u;      // bf16 bits of -136 * 2^e
+                    x[it] = words[it * 32];
+                    e[it] = exps[it * 4];
+                }
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const uint32_t s16 = (uint32_t)(e[it] + 127) << 7;                       // bf16 bits of 2^e
+                    const uint32_t b16 = 0x8000u | ((uint32_t)(e[it] + 134) << 7) | 8u;      // bf16 bits of -136 * 2^e
                     const uint32_t s2 = s16 | (s16 << 16), b2 = b16 | (b16 << 16);
                     uint32_t o[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint32_t t2 = ((x >> (4 * j)) & 0x000f000fu) | 0x43004300u;
+                        const uint32_t t2 = ((x[it] >> (4 * j)) & 0x000f000fu) | 0x43004300u;
                         const __nv_bfloat162 rr = __hfma2(*reinterpret_cast<const __nv_bfloat162 *>(&t2),
                                                           *reinterpret_cast<const __nv_bfloat162 *>(&s2),
                                                           *reinterpret_cast<const __nv_bfloat162 *>(&b2));
                         o[j] = *reinterpret_cast<const uint32_t *>(&rr);
                     }
-                    *reinterpret_cast<uint4 *>(wt + (size_t)k * kATileBytes + row * 128 + ((c ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    // row & 7 = (4 * it + r_in) & 7: the 128-byte swizzle of the MMA tile
+                    *reinterpret_cast<uint4 *>(dst + (size_t)it * 512 + ((c ^ ((4 * it + r_in) & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the tensor core reads what these threads wrote
