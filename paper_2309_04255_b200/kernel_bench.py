@@ -5,6 +5,7 @@ reads its operands from HBM, not from L2).
     python -m paper_2309_04255_b200.kernel_bench gemm [--n 32] [--model 7b] [--only qkv,o]
     python -m paper_2309_04255_b200.kernel_bench avnav [--model 7b] [--prefix 512] [--nodes 2,4,...]
     python -m paper_2309_04255_b200.kernel_bench extend [--model 7b] [--prefix 512] [--nodes 32] [--steps 1,2,4,8]
+    python -m paper_2309_04255_b200.kernel_bench timeline [--workload C2] [--layers 4] [--int4]   # per-kernel time stamps of one pass
 
 Each line of output is one JSON object. `--reps` launches are timed per case after `--warmup`.
 """
@@ -237,6 +238,62 @@ def bench_extend(args):
                           "frac": wbytes / ms / 1e6 / peak, "peak": kind}), flush=True)
 
 
+def bench_timeline(args):
+    """One undisturbed pass of a workload (a few layers of its model) with the kernels' own %globaltimer
+    stamps (llmcad_set_gemm_trace): where every GEMM's streaming kernel (S) and finishing kernel (F) and
+    every attention kernel starts, sees its dependency, ends; a launch is charged the time from its
+    predecessor's end to its own. Microseconds since the first stamp, median over the CTAs unless a
+    range min..max is given."""
+    dev = torch.device("cuda:0")
+    w = gen.WORKLOADS[args.workload]
+    L = args.layers
+    cfg = gen.shrink(gen.MODELS[w.model], L)
+    P, n = w.prefix_len, w.n_nodes
+    v = B.Verifier(cfg, P + 136, device=dev, flags=B.FLAG_INT4_WEIGHTS if args.int4 else 0)
+    v.pack_globals({k: gen.gen_tensor_device(cfg, k, -1, dev) for k in ("tok_embed", "final_norm", "lm_head")})
+    for l in range(L):
+        v.pack_layer(l, {k: gen.gen_tensor_device(cfg, k, l, dev) for k in gen.LAYER_TENSORS})
+    kvv = v.kv_view()
+    kvv[:, :, :, :P] = torch.randn((L, 2, cfg.n_heads, P, cfg.head_dim), device=dev).to(kvv.dtype)
+    tokens = torch.as_tensor(gen.gen_tokens(cfg, n), device=dev)
+    parent = torch.as_tensor(gen.gen_tree(w), device=dev)
+    out = v.new_outputs(n)
+    for _ in range(3):
+        v.verify_tree(P, tokens, parent, out=out)
+    torch.cuda.synchronize()
+    cap = 1 + 5 * L
+    buf = torch.zeros(cap, 256, 16, dtype=torch.int64, device=dev)
+    v.set_gemm_trace(buf)
+    v.verify_tree(P, tokens, parent, out=out)
+    torch.cuda.synchronize()
+    v.set_gemm_trace(None)
+    t = buf.cpu().numpy().astype(np.float64)
+    names = ["qkv"] + ["attention", "o", "gate_up", "down", "qkv"] * L
+    names[-1] = "lm_head"
+    base = t[0][:, 0][t[0][:, 0] > 0].min()
+
+    def st(T, slot):
+        x = T[:, slot]
+        x = x[x > 0]
+        return ((x.min() - base) / 1e3, (np.median(x) - base) / 1e3, (x.max() - base) / 1e3) if len(x) else (-1.0, -1.0, -1.0)
+
+    prev = 0.0
+    for i in range(cap):
+        T = t[i]
+        end = st(T, 12)[2]
+        row = {"launch": i, "kernel": names[i], "charged_us": round(end - prev, 2)}
+        prev = end
+        if names[i] == "attention":
+            keys = {"entry": 0, "dependency": 1, "first_tile": 2, "loop_end": 3, "cta_merged": 4, "cluster_sync": 5, "stored": 6, "exit": 12}
+        else:
+            keys = {"S_entry": 0, "S_first_copy": 2, "S_dependency": 3, "S_last_copy": 6, "S_last_mma": 7, "S_dumped": 8, "S_exit": 13,
+                    "F_entry": 9, "F_dependency": 10, "F_exit": 12}
+        for k, slot in keys.items():
+            a, m, b = st(T, slot)
+            row[k] = f"{m:.2f} ({a:.2f}..{b:.2f})"
+        print(json.dumps(row), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -263,10 +320,15 @@ def main():
     x.add_argument("--nodes", type=int, default=32)
     x.add_argument("--steps", default="1,2,4,8,32")
     x.add_argument("--reps", type=int, default=3)
+    t = sub.add_parser("timeline")
+    t.add_argument("--workload", default="C2")
+    t.add_argument("--layers", type=int, default=4)
+    t.add_argument("--int4", action="store_true")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("kernel_bench needs a CUDA device")
-    {"attention": bench_attention, "gemm": bench_gemm, "avnav": bench_avnav, "extend": bench_extend}[args.cmd](args)
+    {"attention": bench_attention, "gemm": bench_gemm, "avnav": bench_avnav, "extend": bench_extend,
+     "timeline": bench_timeline}[args.cmd](args)
 
 
 if __name__ == "__main__":
