@@ -303,14 +303,8 @@ struct Cursor {
 __host__ __device__ __forceinline__ size_t slot_floats(int halves, int n_pad) { return (size_t)halves * n_pad * kTileM; }
 
 // ------------------------------------------------------------------------------------------------
-// Finishing a 32-row group of an output tile. Every CTA that holds a share of a tile leaves its
-// accumulators in the workspace as [row group][gate|up][node][32 rows] fp32; the warp that arrives
-// last at the group's arrival counter (or the only holder) adds the shares in CTA order and applies the fused
-// epilogue. It works on four output rows at a time: lane = (node sub-index ns = lane / 8, row quad
-// r4 = lane % 8) and iteration `it` handles node 4 * it + ns, so that the shares, the residual stream
-// and every output move as 16- or 8-byte vectors, a rotary pair sits in one thread, and the loads of
-// several nodes and several shares are in flight together (this warp is alone on its scheduler:
-// what it costs is the number of dependent round trips, not the bytes).
+// Finishing (the work of gemm_finish_kernel). Every streaming CTA that holds items of a tile has left
+// its accumulators in the workspace as [row group][gate|up][node][32 rows] fp32 (a "segment").
 __device__ __forceinline__ uint2 pack4_bf16(const __nv_bfloat16 (&h)[4])
 {
     uint2 r;
@@ -325,8 +319,7 @@ __device__ __forceinline__ const float *share_ptr(const GemmParams &p, const Gem
     return p.partials + (size_t)(tile + cc) * slot_floats(d.halves, p.n_pad) + (size_t)lane_grp * d.halves * p.n_pad * 32;
 }
 
-// Everything the finishing code needs, gathered in one place so that the function below can be a
-// real call (one copy of its code in the kernel).
+// What a warp of the finishing kernel works on.
 struct FinishArgs {
     const GemmParams *p;
     const GemmDesc *d;              // in shared memory
@@ -335,22 +328,17 @@ struct FinishArgs {
     int it_first, it_step;          // this warp finishes node groups it_first, it_first + it_step, ...
 };
 
-// Finishing a 32-row group of an output tile: add the shares of all CTAs that hold part of the
-// tile, in CTA order, and apply the fused epilogue. This is the one stretch of the kernel that runs
-// with nothing to hide behind: a warp alone on its scheduler, once per launch, after the weight
-// stream has ended. What it costs is the length of its dependent chain: round trips to L2 (a lone
-// warp gets a global load or store through only every 50 to 150 ns) and plain instruction latency;
-// and, the code being cold every time, instruction-cache misses, so it is kept small (one copy,
-// rolled loops, no specialisation per mode or shape). Hence: lane = (node sub-index ns = lane / 8,
-// row quad r4 = lane % 8), iteration `it` handles the four output rows 4 * r4 .. + 3 of node
-// 4 * it + ns, everything moves as 16- or 8-byte vectors, a rotary pair sits in one thread; and the
-// iterations of a group are dealt out to all the CTAs that end their work on this tile (it_first,
-// it_step), each of which would otherwise idle while one of them did everything.
-// G node groups travel together (one round trip per G iterations), kB shares per node group at a
-// time: tiles held by many CTAs have many shares and few iterations per finisher (G = 2, kB = 4),
-// tiles held by one or two have few shares and many iterations (G = 4, kB = 2).
-// One instantiation per epilogue mode as well: the routine is cold whenever it runs, and what it
-// costs in instruction-cache misses is the code it walks through, not the code that exists.
+// Finishing a 32-row group of an output tile: add the segments of all CTAs that hold part of the
+// tile, in CTA order (so the result does not depend on timing), and apply the fused epilogue. What
+// this costs is the length of its dependent chain, round trips to L2 and plain instruction latency,
+// not bytes. Hence: lane = (node sub-index ns = lane / 8, row quad r4 = lane % 8), iteration `it`
+// handles the four output rows 4 * r4 .. + 3 of node 4 * it + ns, everything moves as 16- or 8-byte
+// vectors, a rotary pair sits in one thread; the iterations of a group are dealt out to several
+// warps of the grid (it_first, it_step); G node groups travel together and kB segments of each are
+// loaded at a time, all loads issued before the first use. With `dry` nothing is stored: the
+// finishing kernel walks through its code once that way before its input exists (see there).
+// One instantiation per epilogue mode: the code is cold whenever it runs, and what that costs is
+// the code walked through, not the code that exists.
 template <int G, int kB, int MODE>
 __device__ __forceinline__ void finish_rows_t(const FinishArgs &fa, int lane, const bool dry)
 {
@@ -423,7 +411,7 @@ __device__ __forceinline__ void finish_rows_t(const FinishArgs &fa, int lane, co
                 }
             }
         }
-        // two at a time, unrolled: the warp is alone on its scheduler and the two chains overlap
+        // two at a time, unrolled, so that the two dependent chains overlap
         for (int g2 = 0; g2 < G; g2 += 2) {
 #pragma unroll
         for (int gq = 0; gq < (G < 2 ? G : 2); ++gq) {
