@@ -518,25 +518,20 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
         const int row = lg * 32 + lane;
         const bool warp_active = lg * 32 < n;             // a warp whose rows are all padding only keeps the barriers going
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
-        const bool skip = refused_warp();
+        dep_wait_warp(dep, lane);
         if (trace && tid == 64 && cta < 256) trace[(size_t)cta * 16 + 1] = global_timer_ns();
-        if (!skip) {
+        // The loads below go out before the status word is looked at (they read buffers that exist whatever an
+        // earlier phase found), so that its round trip overlaps theirs.
         uint32_t a4[4] = {0, 0, 0, 0};
         if (row < n) {
 #pragma unroll
             for (int w = 0; w < 4; ++w) a4[w] = __ldcg(anc + (q_first + row) * 4 + w);   // L2: written earlier in this pass
         }
-        // The queries become the A operand of Q K^T in tensor memory: 64 packed columns per plane, thread =
-        // row. A warp fetches its 32 rows with coalesced loads (two rows of 256 bytes per instruction, both
-        // planes in flight together), turns them through a small shared-memory buffer (16-byte chunks
-        // XOR-swizzled by row) and every thread stores its own row. Rows beyond n repeat row n - 1: a row
-        // of A only ever influences the same row of the product, and nobody reads those rows of the result.
+        uint4 g[2][16];
         if (warp_active) {
-            const int planes = comp ? 2 : 1;
-            uint4 g[2][16];
 #pragma unroll
             for (int pl = 0; pl < 2; ++pl) {
-                if (pl < planes) {
+                if (pl < (comp ? 2 : 1)) {
 #pragma unroll
                     for (int it = 0; it < 16; ++it) {
                         const int rr = it * 2 + (lane >> 4);
@@ -545,6 +540,16 @@ attention_t5_kernel(const __nv_bfloat16 *__restrict__ q, const __grid_constant__
                     }
                 }
             }
+        }
+        const bool skip = *reinterpret_cast<const volatile int32_t *>(status) != 0;
+        if (!skip) {
+        // The queries become the A operand of Q K^T in tensor memory: 64 packed columns per plane, thread =
+        // row. A warp fetches its 32 rows with coalesced loads (two rows of 256 bytes per instruction, both
+        // planes in flight together), turns them through a small shared-memory buffer (16-byte chunks
+        // XOR-swizzled by row) and every thread stores its own row. Rows beyond n repeat row n - 1: a row
+        // of A only ever influences the same row of the product, and nobody reads those rows of the result.
+        if (warp_active) {
+            const int planes = comp ? 2 : 1;
             const uint32_t stg = smem_u32(q_stage + (size_t)lg * kQStage);
 #pragma unroll
             for (int pl = 0; pl < 2; ++pl) {

@@ -156,12 +156,6 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         __syncthreads();
     }
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 1] = global_timer_ns();
-    if (*reinterpret_cast<const volatile int32_t *>(status)) {   // uniform over the grid: set only by kernels that ran before this one
-        cp_commit();
-        cp_wait<0>();          // nothing may still be writing this CTA's shared memory when it exits
-        if (threadIdx.x == 0) dep_arrive(done_ctr);
-        return;
-    }
     // queries of this head (rows >= n are zero) and the remaining first key tiles
     for (int c = tid; c < n_pad * 16; c += kAtThreads) {
         const int r = c >> 4, ch = c & 15;
@@ -185,6 +179,13 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     for (int st = 0; st < kStages - 1; ++st) {
         if (t_begin + st < t_end && !early[st]) load_tile(t_begin + st, st);
         cp_commit();                            // group 0 also carries the queries and everything requested early
+    }
+    // The status word is looked at only now, with the copies above already on their way (they read buffers that
+    // exist whatever an earlier phase found): a refused pass waits for them and leaves.
+    if (*reinterpret_cast<const volatile int32_t *>(status)) {   // uniform over the grid: set only by kernels that ran before this one
+        cp_wait<0>();          // nothing may still be writing this CTA's shared memory when it exits
+        if (threadIdx.x == 0) dep_arrive(done_ctr);
+        return;
     }
 
     const int q_tiles = n_pad >> 4;
