@@ -64,7 +64,8 @@ enum {
     LLMCAD_ERR_BAD_TREE = 1,  /* parent_idx[0] != -1, or parent_idx[i] not in [0, i) */
     LLMCAD_ERR_BAD_TOKEN = 2, /* token id outside [0, vocab) */
     LLMCAD_ERR_TIMEOUT = 3,   /* a bounded device-side wait ran out */
-    LLMCAD_ERR_NAN = 4        /* a logit was NaN */
+    LLMCAD_ERR_NAN = 4,       /* a logit was NaN */
+    LLMCAD_ERR_CHECK = 5      /* debug build (-DLLMCAD_CHECKS) only: a device-side bounds check failed; the access was skipped */
 };
 
 enum { LLMCAD_F32 = 0, LLMCAD_BF16 = 1 };

@@ -15,11 +15,12 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libllmcad.so")
+# LLMCAD_LIB selects another build of the same library (the debug build with device-side checks)
+LIB_PATH = os.environ.get("LLMCAD_LIB") or os.path.join(_HERE, "libllmcad.so")
 MAX_TREE = 128
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CUDA = 0, -1, -2, -3, -4
-ERR_BAD_TREE, ERR_BAD_TOKEN, ERR_TIMEOUT, ERR_NAN = 1, 2, 3, 4
+ERR_BAD_TREE, ERR_BAD_TOKEN, ERR_TIMEOUT, ERR_NAN, ERR_CHECK = 1, 2, 3, 4, 5
 F32, BF16 = 0, 1
 FLAG_SIMT_GEMM, FLAG_SIMT_ATTN, FLAG_T5_ATTN, FLAG_MMA_ATTN, FLAG_INT4_WEIGHTS = 1, 2, 4, 8, 16
 S_ACCEPTED_LEN, S_NEXT_TOKEN, S_NEW_PREFIX_LEN, S_N_CORRECT, S_N_ALL, S_RECTIFIED, S_STATUS = range(7)

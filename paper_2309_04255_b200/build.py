@@ -8,6 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libllmcad.so")
+LIB_CHECKS = os.path.join(HERE, "libllmcad_checks.so")     # the same sources with -DLLMCAD_CHECKS (device-side bounds checks)
 SOURCES = ["api.cu", "tree.cu", "gemm_simt.cu", "attention_simt.cu", "gemm_tc.cu", "attention_tc.cu", "attention_t5.cu", "pack.cu", "noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
@@ -20,20 +21,24 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def needs_build(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(HERE, "..", "include", "llmcad.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
-        return LIB
-    objdir = os.path.join(HERE, "build")
+def build(force: bool = False, verbose: bool = False, checks: bool = False) -> str:
+    """Builds libllmcad.so, or with checks=True libllmcad_checks.so (the debug build with device-side bounds checks)."""
+    lib = LIB_CHECKS if checks else LIB
+    if not force and not needs_build(lib):
+        return lib
+    objdir = os.path.join(HERE, "build_checks" if checks else "build")
     os.makedirs(objdir, exist_ok=True)
     flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    if checks:
+        flags += ["-DLLMCAD_CHECKS"]
     if verbose:
         flags += ["-Xptxas", "-v"]
     procs = []
@@ -53,11 +58,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
             print("FAILED:", " ".join(cmd), file=sys.stderr)
     if failed:
         raise RuntimeError("nvcc failed")
-    tmp = LIB + f".tmp{os.getpid()}"
+    tmp = lib + f".tmp{os.getpid()}"
     subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-lcudart"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checks="--checks" in sys.argv))

@@ -483,6 +483,7 @@ const char *llmcad_strerror(int code)
     case LLMCAD_ERR_BAD_TOKEN: return "token id out of range";
     case LLMCAD_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case LLMCAD_ERR_NAN: return "NaN logit";
+    case LLMCAD_ERR_CHECK: return "a device-side bounds check of the debug build failed";
     default: return "unknown error";
     }
 }

@@ -131,6 +131,18 @@ __device__ __forceinline__ void epilogue_pair(const EpiParams &ep, int r0, int i
     }
 }
 
+// ---------------------------------------------------------------- debug checks
+// compute-sanitizer is not available where this library is developed. A build with -DLLMCAD_CHECKS
+// (build.py: libllmcad_checks.so) verifies, on the device, the indices that are derived from data or
+// from the launch arithmetic (workspace slots, cache slots, node and row numbers, path entries) right
+// before they are used: a failed check writes LLMCAD_ERR_CHECK into the pass's status word and the
+// access is skipped, so that nothing faults. In the normal build the macro is the constant `true`.
+#ifdef LLMCAD_CHECKS
+#define LLMCAD_CHECK(cond, status_ptr) ((cond) ? true : (atomicCAS(reinterpret_cast<int *>(const_cast<int32_t *>(status_ptr)), 0, (int)LLMCAD_ERR_CHECK), false))
+#else
+#define LLMCAD_CHECK(cond, status_ptr) (true)
+#endif
+
 // ---------------------------------------------------------------- bounded waits
 __device__ __forceinline__ uint64_t global_timer_ns()
 {

@@ -379,7 +379,8 @@ __global__ void accept_kernel(const int32_t *__restrict__ parent, const int32_t 
         return;
     }
     if (c < n) {
-        const int p = parent[c];
+        int p = parent[c];
+        if (!LLMCAD_CHECK(c == 0 ? p == -1 : (p >= 0 && p < c), scalars + LLMCAD_S_STATUS)) p = c == 0 ? -1 : 0;
         s_par[c] = p;
         s_link[c] = (c == 0) ? 1 : (tokens[c] == argmax[p]);
     }
@@ -447,7 +448,8 @@ __global__ void compact_kernel(uint4 *kv, int n_lkh, int S, int chunks, int P, c
     pdl_launch_dependents();
     pdl_wait();
     if (scalars[LLMCAD_S_STATUS]) return;
-    const int len = scalars[LLMCAD_S_ACCEPTED_LEN];
+    int len = scalars[LLMCAD_S_ACCEPTED_LEN];
+    if (!LLMCAD_CHECK(len >= 0 && P + len <= S && len <= LLMCAD_MAX_TREE, scalars + LLMCAD_S_STATUS)) len = 0;
     const long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (w >= (long long)n_lkh * chunks) return;
     const int lkh = (int)(w / chunks), ch = (int)(w % chunks);
@@ -458,7 +460,8 @@ __global__ void compact_kernel(uint4 *kv, int n_lkh, int S, int chunks, int P, c
         uint4 tmp[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-            if (j + u < len) tmp[u] = base[(size_t)path[j + u] * chunks];
+            if (j + u < len && LLMCAD_CHECK(path[j + u] >= j + u && P + path[j + u] < S, scalars + LLMCAD_S_STATUS))
+                tmp[u] = base[(size_t)path[j + u] * chunks];
 #pragma unroll
         for (int u = 0; u < 8; ++u)
             if (j + u < len) base[(size_t)(j + u) * chunks] = tmp[u];

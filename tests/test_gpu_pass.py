@@ -298,6 +298,19 @@ def test_tuning_paths_stay_correct(env):
     assert r.returncode == 0 and r.stdout.strip().endswith("ok"), r.stdout[-2000:] + r.stderr[-4000:]
 
 
+def test_debug_build_with_device_side_checks_finds_nothing():
+    """The library built with -DLLMCAD_CHECKS verifies, on the device, the indices it derives from data
+    and from the launch arithmetic (workspace slots, cache slots, path entries) and reports a failed
+    check through the status word instead of touching memory. The same parity cases must pass under it
+    with status 0: the stand-in for a memory checker on a machine that has none."""
+    import os, subprocess, sys
+    from paper_2309_04255_b200 import build as libbuild
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    e = dict(os.environ, LLMCAD_LIB=libbuild.build(checks=True))
+    r = subprocess.run([sys.executable, "-c", _TUNING_SCRIPT, root], env=e, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and r.stdout.strip().endswith("ok"), r.stdout[-2000:] + r.stderr[-4000:]
+
+
 def test_queued_passes_of_changing_size_are_reproducible():
     """Passes over trees of different sizes queued back to back on one stream (no host
     synchronisation in between) must each give, bit for bit, what the same pass gives alone: the
