@@ -62,7 +62,6 @@ constexpr size_t kFinSmem = 24 * 1024;   // dynamic shared memory the finishing 
                                          // there for the next GEMM's streaming CTA
 constexpr int kATileBytes = kTileM * kBlockK * 2;  // 16 KB
 constexpr int kMaxStages = 16;
-constexpr int kMaxAStages = 8;    // ring of activation tiles
 constexpr int kMaxPStages = 24;   // INT4 weights: ring of packed tiles
 constexpr int kMaxPairK = 2;     // k-blocks per ring item (GemmDesc::pair_k): 2 = one 32 KB weight copy feeds 8 MMAs;
                                  // 1 for wide activation tiles, which would leave too few ring stages otherwise
@@ -236,14 +235,13 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n)
 }
 
 struct SharedCtl {
-    uint64_t full[kMaxStages];      // weight ring: the item's tiles have landed (or, INT4, have been expanded)
-    uint64_t empty[kMaxStages];     //              the MMAs that read the stage are done
-    uint64_t afull[kMaxAStages];    // activation ring, one stage per item as well
-    uint64_t aempty[kMaxAStages];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
+    volatile uint32_t a_issued;     // ring items whose weight copy (and expect_tx) has been issued
     uint64_t pfull[kMaxPStages];    // INT4 weights: packed tile landed / packed stage free again
     uint64_t pempty[kMaxPStages];
 };
@@ -502,16 +500,13 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t nb = (uint32_t)p.n_pad * (p.comp ? 2u : 1u);   // activation rows per k-block = the MMA N: nodes (hi | lo)
     const uint32_t b_tile_bytes = nb * kBlockK * 2;
-    // Two rings, one stage per item in each: the weight tiles (PK x 16 KB; they do not depend on anything, so this
-    // ring fills before the grid dependency and is what carries the stream over the gap between two GEMMs) and
-    // the activation tiles (PK x nb x 128 bytes from L2, which only need to cover the latency of their copies).
-    constexpr uint32_t stage_bytes = PK * kATileBytes;
-    const uint32_t astage_bytes = PK * b_tile_bytes;
+    // stage: [weights k-block 0 | weights k-block 1 | activations k-block 0 | activations k-block 1]
+    const uint32_t stage_bytes = PK * (kATileBytes + b_tile_bytes);
+    const uint32_t b_off = PK * kATileBytes;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t act_base = smem_base + (uint32_t)p.stages * stage_bytes;
-    // INT4 weights: behind them lies a ring of packed items (PK tiles of 4224 bytes each)
+    // INT4 weights: behind the ring of MMA stages lies a ring of packed items (PK tiles of 4224 bytes each)
     constexpr uint32_t pstage_bytes = PK * kW4TileBytes;
-    const uint32_t packed_base = act_base + (uint32_t)p.astages * astage_bytes;
+    const uint32_t packed_base = smem_base + (uint32_t)p.stages * stage_bytes;
     const uint32_t acc_cols = 2u * nb;                    // TMEM columns of one accumulator buffer (gate | up)
     const bool two_bufs = p.acc_bufs == 2;
     const uint64_t wait_limit = p.wait_limit_ns;          // every wait below gives up after this many ns
@@ -543,7 +538,7 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
         }
         const uint32_t full = smem_u32(&ctl.full[ps]);
         const uint32_t dst = smem_base + ps * stage_bytes;
-        mbar_expect_tx(full, (uint32_t)nk * kATileBytes);
+        mbar_expect_tx(full, (uint32_t)nk * (kATileBytes + b_tile_bytes));
         if (d.w_tiled != nullptr) {
             // consecutive k-blocks of a tile are contiguous in the tiled layout: one copy
             const size_t t = (size_t)(pc.tile + (pc.half ? d.up_tile_offset : 0)) * d.kb_per_tile + pc.kb0();
@@ -553,20 +548,18 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
                 tma_load_2d(dst + k * kATileBytes, &maps.w, (pc.kb0() + k) * kBlockK,
                             (pc.half ? d.up_row_offset : 0) + pc.tile * kTileM, full, pol_stream);
         }
+        __threadfence_block();
         if (pissued == 0) LLMCAD_TRACE(2);
-        ++pissued;
+        ctl.a_issued = ++pissued;      // the activation loader may now add its bytes to this stage
         pc.advance();
         if (++ps == p.stages) { ps = 0; ppar ^= 1u; }
     };
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            // INT4: a weight stage is full when the four dump warps have written their quarters of the tile
-            mbar_init(smem_u32(&ctl.full[s]), W4 ? 4 : 1);
+            // INT4: a stage is full when its activation bytes have landed (armed by one arrival) and the four
+            // dump warps have written their quarters of the weight tile
+            mbar_init(smem_u32(&ctl.full[s]), W4 ? 5 : 1);
             mbar_init(smem_u32(&ctl.empty[s]), 1);
-        }
-        for (int s = 0; s < p.astages; ++s) {
-            mbar_init(smem_u32(&ctl.afull[s]), 1);
-            mbar_init(smem_u32(&ctl.aempty[s]), 1);
         }
         if (W4) {
             for (int s = 0; s < p.pstages; ++s) {
@@ -579,6 +572,7 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
             mbar_init(smem_u32(&ctl.tmem_empty[b]), 4);
         }
         ctl.abort_flag = 0;
+        ctl.a_issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
@@ -659,28 +653,37 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
         }
     } else if (warp == 6) {
         // ================================================= activation loader
-        // Walks the items in order and brings the (small, L2-resident) activation tiles of each into the
-        // activation ring, once the grid dependency says that the GEMM's input is final.
+        // Follows the weight producer item by item and adds the (small, L2-resident) activation
+        // tiles of each item, once the grid dependency says that the GEMM's input is final.
         if (lane == 0) {
             uint64_t pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
             Cursor<PK> c;
             c.init(d);
             int s = 0;
-            uint32_t apar = 1;            // a fresh barrier passes a wait on parity 1
+            uint32_t i = 0;
             if (!dep_wait_thread(dep)) timed_out = true;
             fence_proxy_async();          // the activations were written by ordinary stores; the copies below read them
             pdl_launch_dependents();
             while (!c.done() && !timed_out && !p.withhold_act) {
-                if (!mbar_wait(smem_u32(&ctl.aempty[s]), apar, abort_flag, wait_limit)) { timed_out = true; break; }
-                const uint32_t full = smem_u32(&ctl.afull[s]);
-                const uint32_t dst = act_base + s * astage_bytes;
+                uint64_t t0 = 0;
+                // the stage is ours: the producer has passed its "empty" wait and armed the barrier
+                for (uint32_t spin = 0; (int32_t)(ctl.a_issued - (i + 1)) < 0; ++spin) {
+                    __nanosleep(32);
+                    if ((spin & 255u) == 255u) {
+                        if (t0 == 0) t0 = global_timer_ns();
+                        if (*abort_flag || global_timer_ns() - t0 > wait_limit) { timed_out = true; break; }
+                    }
+                }
+                if (timed_out) break;
+                const uint32_t full = smem_u32(&ctl.full[s]);
+                const uint32_t dst = smem_base + s * stage_bytes + b_off;
                 const int nk = c.nk();
-                mbar_expect_tx(full, (uint32_t)nk * b_tile_bytes);
                 for (int k = 0; k < nk; ++k)
                     tma_load_3d(dst + k * b_tile_bytes, &maps.x, (c.kb0() + k) * kBlockK, full, pol_keep);
                 c.advance();
-                if (++s == p.astages) { s = 0; apar ^= 1u; }
+                ++i;
+                if (++s == p.stages) s = 0;
             }
         }
     } else if (warp == 1) {
@@ -689,8 +692,8 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
             const uint32_t idesc = make_idesc(kTileM, (int)nb);
             Cursor<PK> c;
             c.init(d);
-            uint32_t seg = 0, ph = 0, aph = 0;   // parities the MMA warp waits for on its stages' "full" barriers
-            int s = 0, as = 0;
+            uint32_t seg = 0, ph = 0;   // ph: parity the MMA warp waits for on its stage's "full" barrier
+            int s = 0;
             while (!c.done() && !timed_out) {
                 // one segment: the items of one tile that belong to this CTA
                 const int tile = c.tile, halves = c.halves;
@@ -701,27 +704,24 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
                 const uint32_t d0 = tmem_base + buf * acc_cols;
                 for (int q = 0; !c.done() && c.tile == tile; ++q) {
                     if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag, wait_limit)) { timed_out = true; break; }
-                    if (!mbar_wait(smem_u32(&ctl.afull[as]), aph, abort_flag, wait_limit)) { timed_out = true; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_base + s * stage_bytes, b_addr = act_base + as * astage_bytes;
+                    const uint32_t a_addr = smem_base + s * stage_bytes;
                     // segments of a two-half GEMM start on a gate item, so the first `halves` items
                     // of a segment are the ones that must overwrite their accumulator
                     const uint32_t dcol = d0 + c.half * nb;
                     const int nk = c.nk();
                     for (int k = 0; k < nk; ++k) {
                         const uint64_t a_desc = make_smem_desc(a_addr + k * kATileBytes);
-                        const uint64_t b_desc = make_smem_desc(b_addr + k * b_tile_bytes);
+                        const uint64_t b_desc = make_smem_desc(a_addr + b_off + k * b_tile_bytes);
 #pragma unroll
                         for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
                             // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the >>4 address field
                             tc_mma_bf16(dcol, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (q >= halves || k > 0 || k4 > 0) ? 1u : 0u);
                         }
                     }
-                    tc_commit(smem_u32(&ctl.empty[s]));  // frees the stages when these MMAs have read them
-                    tc_commit(smem_u32(&ctl.aempty[as]));
+                    tc_commit(smem_u32(&ctl.empty[s]));  // frees the stage when these MMAs have read it
                     c.advance();
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
-                    if (++as == p.astages) { as = 0; aph ^= 1u; }
                 }
                 if (timed_out) break;
                 tc_commit(smem_u32(&ctl.tmem_full[buf]));
@@ -750,13 +750,18 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
         Cursor<PK> dc;
         dc.init(d);
         int ds = 0, dps = 0;
-        uint32_t dpar = 1, dppar = 0;                  // a fresh "empty" barrier passes a wait on parity 1
+        uint32_t dpar = 1, dppar = 0, dcount = 0;      // a fresh "empty" barrier passes a wait on parity 1
         uint8_t *const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
         auto dequant_item = [&]() -> bool {
             const int nk = dc.nk();
             if (!mbar_wait_warp(smem_u32(&ctl.empty[ds]), dpar, abort_flag, lane, wait_limit)) return false;
+            if (warp == 2 && lane == 0) {
+                mbar_expect_tx(smem_u32(&ctl.full[ds]), (uint32_t)nk * b_tile_bytes);
+                __threadfence_block();
+                ctl.a_issued = ++dcount;       // the activation loader may now add its bytes to this stage
+            }
             if (!mbar_wait_warp(smem_u32(&ctl.pfull[dps]), dppar, abort_flag, lane, wait_limit)) return false;
-            const uint8_t *pk = smem_gen + (size_t)p.stages * stage_bytes + (size_t)p.astages * astage_bytes + (size_t)dps * pstage_bytes;
+            const uint8_t *pk = smem_gen + (size_t)p.stages * stage_bytes + (size_t)dps * pstage_bytes;
             uint8_t *wt = smem_gen + (size_t)ds * stage_bytes;
             // lane = (row within a group of four, chunk): iteration `it` handles row 32 * lane_grp + 4 * it + lane / 8,
             // words and stores of a warp instruction are contiguous (no bank conflicts). All loads of a k-block go
@@ -1075,12 +1080,11 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled, bool
 namespace {
 // tuning aids from the environment, read once per process
 struct Tuning {
-    int pair_k = 0, stages_cap = 0, astages = 0, l2_ahead = 8, next_items = -1;
+    int pair_k = 0, stages_cap = 0, l2_ahead = 8, next_items = -1;
     Tuning()
     {
         if (const char *e = getenv("LLMCAD_GEMM_PAIR_K")) { const int v = atoi(e); if (v == 1 || v == 2) pair_k = v; }
         if (const char *e = getenv("LLMCAD_GEMM_STAGES")) { const int v = atoi(e); if (v >= 2) stages_cap = v; }
-        if (const char *e = getenv("LLMCAD_GEMM_ASTAGES")) { const int v = atoi(e); if (v >= 1 && v <= 8) astages = v; }
         if (const char *e = getenv("LLMCAD_GEMM_L2_AHEAD")) l2_ahead = atoi(e);
         if (const char *e = getenv("LLMCAD_GEMM_NEXT_ITEMS")) next_items = atoi(e);
     }
@@ -1140,48 +1144,35 @@ cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_
     const int pair_k = d.pair_k, grid = d.grid;
     const long long ipc = d.items_per_cta;
     if ((size_t)(d.n_tiles + grid) * slot_floats(d.halves, p.n_pad) > partial_floats) return cudaErrorInvalidValue;
-    // Shared memory: a ring of activation stages deep enough to cover the latency of their copies from L2 (32 KB
-    // in flight, at least two stages), and the rest, less the room the finishing CTA of the previous GEMM needs
-    // beside this CTA, for the ring of weight stages.
-    const size_t stage_bytes = (size_t)pair_k * kATileBytes;
-    const size_t astage_bytes = (size_t)pair_k * (size_t)nb * kBlockK * 2;
+    const size_t stage_bytes = (size_t)pair_k * ((size_t)kATileBytes + (size_t)nb * kBlockK * 2);
+    // One CTA per SM with the whole shared memory as the ring.
     // accumulators: (gate | up) x MMA N columns each, double-buffered when two of them fit
     p.acc_bufs = 4 * nb <= 512 ? 2 : 1;
     int cols = p.acc_bufs * 2 * nb, pow2 = 32;
     while (pow2 < cols) pow2 <<= 1;
     p.tmem_cols = pow2;
+    // the ring takes what the SM has, less the room that the finishing CTA of the previous GEMM needs beside it
     const size_t full_limit = 227 * 1024 - 1024 /*alignment slack*/ - 2048 /*static*/ - (kFinSmem + 4096);
-    int astages = (int)(32768 / astage_bytes);
-    if (astages < 2) astages = 2;
-    if (astages > 4) astages = 4;
-    if (tune.astages) astages = tune.astages;
-    if (astages > kMaxAStages) astages = kMaxAStages;
-    if ((size_t)astages * astage_bytes + 2 * stage_bytes > full_limit) return cudaErrorInvalidConfiguration;
-    int stages = (int)((full_limit - (size_t)astages * astage_bytes) / stage_bytes);
+    int stages = (int)(full_limit / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (tune.stages_cap && tune.stages_cap < stages) stages = tune.stages_cap;   // tuning aid: cap the ring depth
     if (stages < 2) return cudaErrorInvalidConfiguration;
-    size_t smem = (size_t)stages * stage_bytes + (size_t)astages * astage_bytes + 1024;
+    size_t smem = (size_t)stages * stage_bytes + 1024;
     p.pstages = 0;
     if (d.w4) {
-        // INT4 weights: two weight stages (the tile being expanded and the tile being multiplied), more activation
-        // stages (an item's activation tile is now larger than its packed weights, so it is the activation copies
-        // whose latency has to be covered), and the rest of the shared memory for packed items
+        // INT4 weights: the MMA ring keeps what covers the latency of the activation copies (three stages where
+        // they fit), the rest of the shared memory holds packed items, four times as many weights per byte
         if (d.w_tiled == nullptr) return cudaErrorInvalidValue;
         const size_t pstage = (size_t)pair_k * kW4TileBytes;
-        stages = 2;
-        astages = (int)(65536 / astage_bytes);
-        if (astages < 2) astages = 2;
-        if (astages > 6) astages = 6;
-        while (astages > 2 && (size_t)stages * stage_bytes + (size_t)astages * astage_bytes + 6 * pstage > full_limit) --astages;
-        if (full_limit < (size_t)stages * stage_bytes + (size_t)astages * astage_bytes + 2 * pstage) return cudaErrorInvalidConfiguration;
-        int pst = (int)((full_limit - (size_t)stages * stage_bytes - (size_t)astages * astage_bytes) / pstage);
+        if (stages > 3) stages = 3;
+        while (stages > 2 && full_limit - (size_t)stages * stage_bytes < 8 * pstage) --stages;   // room for eight packed items
+        int pst = (int)((full_limit - (size_t)stages * stage_bytes) / pstage);
         if (pst > kMaxPStages) pst = kMaxPStages;
+        if (pst < 2) return cudaErrorInvalidConfiguration;
         p.pstages = pst;
-        smem = (size_t)stages * stage_bytes + (size_t)astages * astage_bytes + (size_t)pst * pstage + 1024;
+        smem = (size_t)stages * stage_bytes + (size_t)pst * pstage + 1024;
         p.next = NextWeights{};
     }
-    p.astages = astages;
     p.stages = stages;
     static PerDeviceOnce attr_set;
     if (attr_set.needed()) {
