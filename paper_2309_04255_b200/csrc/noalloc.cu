@@ -59,16 +59,17 @@ extern "C" int llmcad_tree_attention_noalloc(const void *q, const void *k, const
         snprintf(g_err, sizeof(g_err), "no usable current device");
         return LLMCAD_ERR_CUDA;
     }
-    if (g_scratch_ptr[dev] == nullptr) {
+    // (two host threads making their first call at once both look the address up and store the same value)
+    if (__atomic_load_n(&g_scratch_ptr[dev], __ATOMIC_ACQUIRE) == nullptr) {
         void *ptr = nullptr;
         const cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
         if (e != cudaSuccess || ptr == nullptr) {
             snprintf(g_err, sizeof(g_err), "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
             return LLMCAD_ERR_CUDA;
         }
-        g_scratch_ptr[dev] = ptr;
+        __atomic_store_n(&g_scratch_ptr[dev], ptr, __ATOMIC_RELEASE);
     }
-    unsigned char *base = static_cast<unsigned char *>(g_scratch_ptr[dev]);
+    unsigned char *base = static_cast<unsigned char *>(__atomic_load_n(&g_scratch_ptr[dev], __ATOMIC_ACQUIRE));
     TreeBuffers tb;
     tb.depth = reinterpret_cast<int32_t *>(base);
     tb.pos = reinterpret_cast<int32_t *>(base + 512);
