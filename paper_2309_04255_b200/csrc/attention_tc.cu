@@ -6,10 +6,14 @@
 // few heads, so the key range of each head is split over the CTAs of one thread-block cluster
 // (grid = splits x heads, cluster = the splits of a head, about one CTA per SM in total): each
 // CTA streams its key range once through a four-stage cp.async ring in shared memory, keeps an
-// online softmax per query row and leaves an unnormalised partial (max, sum, output) in its own
-// shared memory; after a cluster barrier every CTA merges a share of the query rows by reading
-// the partials of its peers through distributed shared memory and writes the bf16 output. No
-// global workspace, no atomics.
+// online softmax per query row and ends with an unnormalised partial (max, sum, output) per row.
+// The splits of a head are merged through distributed shared memory: query row r belongs to CTA
+// r % splits of the cluster. With few nodes (<= 32, the common tree) every CTA pushes its partial
+// rows into a receive buffer in the owner's shared memory (remote stores are posted, remote loads
+// pay a round trip each), one cluster barrier follows, and the owner merges what it received and
+// writes the bf16 output; larger trees, whose receive buffers would not fit beside the key ring,
+// keep their partial at home and the owners fetch the rows after the barrier. No global
+// workspace, no atomics.
 //
 // Inside a CTA warp w owns query rows 16w..16w+15 (n <= 128 nodes -> at most 8 warps busy);
 // QK^T and PV are mma.sync m16n8k16 bf16 with fp32 accumulation, scores never leave registers.
@@ -27,7 +31,10 @@ constexpr int kHd = 128;
 constexpr int kKeyTile = 64;
 constexpr int kAtThreads = 256;
 constexpr int kRowBytes = kHd * 2;            // 256-byte rows = 16 chunks of 16 bytes
-constexpr int kWsRow = kHd + 2;               // partial row: 128 outputs, max, sum
+// partial row: 128 outputs, max, sum, padding. 136 floats: rows start on 16 bytes, and the eight rows a
+// warp stores at once (fragment layout: lane / 4 = row) start in banks 8 apart, so that its 8-byte stores
+// do not collide (with 130 floats they did, four ways, and the stores took longer than the merge itself).
+constexpr int kWsRow = kHd + 8;
 constexpr int kMaxSplits = 8;                 // portable cluster size
 constexpr int kMaxStages = 4;
 
@@ -96,10 +103,13 @@ template <int GROUPS, bool COMP>
 __global__ void __launch_bounds__(kAtThreads)
 attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
                     const __nv_bfloat16 *__restrict__ v, int n_heads, int kv_stride, int P, int n, int n_pad,
-                    const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_per_split,
+                    const uint32_t *__restrict__ anc, __nv_bfloat16 *o, int splits, int tiles_base, int tiles_rem,
                     const int32_t *status, unsigned long long *trace, const __nv_bfloat16 *__restrict__ kv_lo,
-                    int n_tree, int q_first, DepWait dep, uint32_t *done_ctr)
+                    int n_tree, int q_first, DepWait dep, uint32_t *done_ctr, int recv_off)
 {
+    // PUSH: partial rows travel to their owners (see the head of the file); recv_off = where the receive
+    // buffer starts in this CTA's shared memory, [splits][rows per CTA][kWsRow] floats behind everything else
+    constexpr bool PUSH = GROUPS == 4;
     // n query rows = the tree nodes q_first .. q_first + n - 1 (all of them in a verification pass,
     // the new ones when a tree is extended); the keys are the prefix and all n_tree tree nodes
     // ring depth: with 128 nodes and the lo planes three stages are what fits in shared memory
@@ -109,6 +119,9 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     const int cta = blockIdx.y * gridDim.x + blockIdx.x;
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 0] = global_timer_ns();
     pdl_launch_dependents();
+    // first cluster barrier, arrival: its completion tells that every CTA of the cluster is running, which a
+    // store into a peer's shared memory requires; waited for just before the first such store
+    if (PUSH) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
     extern __shared__ __align__(128) uint8_t sm[];
     uint8_t *s_q = sm;                                      // [n_pad][256 B], with COMP followed by the lo plane
     uint8_t *s_k = s_q + (size_t)(COMP ? 2 : 1) * n_pad * kRowBytes;   // [kStages][64][256 B]
@@ -122,8 +135,10 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_keys = P + n_tree;
     const int n_tiles = (n_keys + kKeyTile - 1) / kKeyTile;
-    const int t_begin = split * tiles_per_split;
-    const int t_end = min(n_tiles, t_begin + tiles_per_split);
+    // the first tiles_rem splits walk one tile more than the others: the tiles with the tree nodes, which cost
+    // more (remainders, mask) and cannot be requested before the grid dependency, fall to a short split
+    const int t_begin = split * tiles_base + min(split, tiles_rem);
+    const int t_end = min(n_tiles, t_begin + tiles_base + (split < tiles_rem ? 1 : 0));
     const __nv_bfloat16 *kh = k + (size_t)head * kv_stride * kHd;
     const __nv_bfloat16 *vh = v + (size_t)head * kv_stride * kHd;
 
@@ -347,10 +362,9 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
 
     // ---- every warp leaves its unnormalised partial (outputs, max, sum) in shared memory (the
-    // K/V ring is done): wpart[kg][row][130]; the merged partial of the CTA goes to part[row][130]
+    // K/V ring is done): wpart[kg][row][kWsRow]
     __syncthreads();
     float *wpart = reinterpret_cast<float *>(sm);
-    float *part = (GROUPS > 1) ? wpart + (size_t)GROUPS * n_pad * kWsRow : wpart;
     if (active) {
         float *wp = wpart + (size_t)kg * n_pad * kWsRow;
 #pragma unroll
@@ -364,49 +378,40 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
             *reinterpret_cast<float2 *>(wp + (size_t)row1 * kWsRow + kHd) = make_float2(m1, l1);
         }
     }
-    if (GROUPS > 1) {
-        __syncthreads();
-        // merge the key groups of this CTA: out = sum_g O_g 2^(m_g - M), l = sum_g l_g 2^(m_g - M).
-        // First the per-(row, group) weights, once; then every thread combines float4 columns.
-        float *wgt = part + (size_t)n_pad * kWsRow;           // [n_pad][GROUPS]
-        for (int row = tid; row < n_pad; row += kAtThreads) {
-            float mg[GROUPS], M = -INFINITY, L = 0.f;
+    __syncthreads();
+    // The CTA's partial of four outputs of a row, merged over its key groups in group order:
+    // out = sum_g O_g 2^(m_g - M), l = sum_g l_g 2^(m_g - M), M = max_g m_g.
+    auto merged4 = [&](int row, int dim, float2 &ML) {
+        float mg[GROUPS], M = -INFINITY, L = 0.f;
 #pragma unroll
-            for (int g = 0; g < GROUPS; ++g) { mg[g] = wpart[((size_t)g * n_pad + row) * kWsRow + kHd]; M = fmaxf(M, mg[g]); }
+        for (int g = 0; g < GROUPS; ++g) { mg[g] = wpart[((size_t)g * n_pad + row) * kWsRow + kHd]; M = fmaxf(M, mg[g]); }
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int g = 0; g < GROUPS; ++g) {
-                const float w = (mg[g] == -INFINITY) ? 0.f : exp2f(mg[g] - M);
-                wgt[row * GROUPS + g] = w;
-                L += wpart[((size_t)g * n_pad + row) * kWsRow + kHd + 1] * w;
-            }
-            *reinterpret_cast<float2 *>(part + (size_t)row * kWsRow + kHd) = make_float2(M, L);
+        for (int g = 0; g < GROUPS; ++g) {
+            const float w = (mg[g] == -INFINITY) ? 0.f : exp2f(mg[g] - M);
+            const float4 vv = *reinterpret_cast<const float4 *>(wpart + ((size_t)g * n_pad + row) * kWsRow + dim);
+            L += wpart[((size_t)g * n_pad + row) * kWsRow + kHd + 1] * w;
+            acc.x += vv.x * w; acc.y += vv.y * w; acc.z += vv.z * w; acc.w += vv.w * w;
         }
-        __syncthreads();
-        for (int idx = tid; idx < n_pad * (kHd / 2); idx += kAtThreads) {
-            const int row = idx / (kHd / 2), c = (idx % (kHd / 2)) * 2;    // rows are 520 bytes: 8-byte accesses
-            float2 a = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int g = 0; g < GROUPS; ++g) {
-                const float2 vv = *reinterpret_cast<const float2 *>(wpart + ((size_t)g * n_pad + row) * kWsRow + c);
-                const float w = wgt[row * GROUPS + g];
-                a.x += vv.x * w; a.y += vv.y * w;
-            }
-            *reinterpret_cast<float2 *>(part + (size_t)row * kWsRow + c) = a;
-        }
-    }
+        ML = make_float2(M, L);
+        return acc;
+    };
+    // four outputs of one row, normalised, as bf16 hi (and lo) to global memory
+    auto store4 = [&](int row, int dim, float4 acc, float inv) {
+        uint32_t h0, l0w, h1, l1w;
+        pack_split(acc.x * inv, acc.y * inv, h0, l0w);
+        pack_split(acc.z * inv, acc.w * inv, h1, l1w);
+        __nv_bfloat16 *dst = o + ((size_t)row * n_heads + head) * kHd + dim;
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(h0, h1);
+        if (COMP) *reinterpret_cast<uint2 *>(dst + lo_off) = make_uint2(l0w, l1w);
+    };
 
     if (splits == 1) {
-        __syncthreads();
-        for (int idx = tid; idx < n * (kHd / 2); idx += kAtThreads) {
-            const int row = idx / (kHd / 2), dim = (idx % (kHd / 2)) * 2;
-            const float L = part[(size_t)row * kWsRow + kHd + 1];
-            const float inv = L > 0.f ? 1.f / L : 0.f;
-            const float2 ov = *reinterpret_cast<const float2 *>(part + (size_t)row * kWsRow + dim);
-            uint32_t hi, lo;
-            pack_split(ov.x * inv, ov.y * inv, hi, lo);
-            __nv_bfloat16 *dst = o + ((size_t)row * n_heads + head) * kHd + dim;
-            *reinterpret_cast<uint32_t *>(dst) = hi;
-            if (COMP) *reinterpret_cast<uint32_t *>(dst + lo_off) = lo;
+        for (int idx = tid; idx < n * (kHd / 4); idx += kAtThreads) {
+            const int row = idx / (kHd / 4), dim = (idx % (kHd / 4)) * 4;
+            float2 ML;
+            const float4 acc = merged4(row, dim, ML);
+            store4(row, dim, acc, ML.y > 0.f ? 1.f / ML.y : 0.f);
         }
         if (done_ctr != nullptr) {
             __syncthreads();
@@ -416,8 +421,71 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
         return;
     }
 
-    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 4] = global_timer_ns();
     cg::cluster_group cluster = cg::this_cluster();
+    if (PUSH) {
+        // ---- rows to their owners: row r -> CTA r % splits, slot [this split][r / splits] of its receive buffer
+        float *recv = reinterpret_cast<float *>(sm + recv_off);
+        const int rows_cap = (n_pad + splits - 1) / splits;
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");     // every CTA of the cluster is running
+        for (int idx = tid; idx < n * (kHd / 4); idx += kAtThreads) {
+            const int row = idx / (kHd / 4), dim = (idx % (kHd / 4)) * 4;
+            float2 ML;
+            const float4 acc = merged4(row, dim, ML);
+            float *dst = cluster.map_shared_rank(recv, row % splits) + ((size_t)split * rows_cap + row / splits) * kWsRow;
+            *reinterpret_cast<float4 *>(dst + dim) = acc;
+            if (dim == 0) *reinterpret_cast<float2 *>(dst + kHd) = ML;
+        }
+        if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 4] = global_timer_ns();
+        // second cluster barrier: the stores above are released by the arrival and acquired by the wait
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 5] = global_timer_ns();
+        // ---- merge over the splits, in split order: out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M)
+        const int my_rows = (n - split + splits - 1) / splits;   // rows split, split + splits, ... below n
+        for (int idx = tid; idx < my_rows * (kHd / 4); idx += kAtThreads) {
+            const int lr = idx / (kHd / 4), dim = (idx % (kHd / 4)) * 4;
+            float ms[kMaxSplits], M = -INFINITY, L = 0.f;
+#pragma unroll
+            for (int sp = 0; sp < kMaxSplits; ++sp) {
+                ms[sp] = sp < splits ? recv[((size_t)sp * rows_cap + lr) * kWsRow + kHd] : -INFINITY;
+                M = fmaxf(M, ms[sp]);
+            }
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int sp = 0; sp < kMaxSplits; ++sp) {
+                if (sp < splits) {
+                    const float *src = recv + ((size_t)sp * rows_cap + lr) * kWsRow;
+                    const float w = (ms[sp] == -INFINITY) ? 0.f : exp2f(ms[sp] - M);
+                    const float4 vv = *reinterpret_cast<const float4 *>(src + dim);
+                    L += src[kHd + 1] * w;
+                    acc.x += vv.x * w; acc.y += vv.y * w; acc.z += vv.z * w; acc.w += vv.w * w;
+                }
+            }
+            store4(split + lr * splits, dim, acc, L > 0.f ? 1.f / L : 0.f);
+        }
+        if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 6] = global_timer_ns();
+        if (done_ctr != nullptr) {
+            __syncthreads();                                     // this CTA's rows of the output are written
+            if (threadIdx.x == 0) dep_arrive(done_ctr);
+        }
+        // (nobody reads this CTA's shared memory from outside, and what peers stored into it arrived before the
+        // barrier let go: the CTA may leave)
+        if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 12] = global_timer_ns();
+        return;
+    }
+
+    // ---- larger trees: the merged partial of the CTA stays at home, part[row][kWsRow]
+    float *part = (GROUPS > 1) ? wpart + (size_t)GROUPS * n_pad * kWsRow : wpart;
+    if (GROUPS > 1) {
+        for (int idx = tid; idx < n_pad * (kHd / 4); idx += kAtThreads) {
+            const int row = idx / (kHd / 4), dim = (idx % (kHd / 4)) * 4;
+            float2 ML;
+            const float4 acc = merged4(row, dim, ML);
+            *reinterpret_cast<float4 *>(part + (size_t)row * kWsRow + dim) = acc;
+            if (dim == 0) *reinterpret_cast<float2 *>(part + (size_t)row * kWsRow + kHd) = ML;
+        }
+    }
+    if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 4] = global_timer_ns();
     cluster.sync();                                          // all partials of this head are written
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 5] = global_timer_ns();
     // ---- merge rows split, split + splits, ...: out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M)
@@ -425,34 +493,32 @@ attention_tc_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__
 #pragma unroll
     for (int sp = 0; sp < kMaxSplits; ++sp) peer[sp] = sp < splits ? cluster.map_shared_rank(part, sp) : part;
     const int my_rows = (n - split + splits - 1) / splits;   // rows split, split+splits, ... below n
-    for (int idx = tid; idx < my_rows * (kHd / 2); idx += kAtThreads) {
-        const int row = split + (idx / (kHd / 2)) * splits, dim = (idx % (kHd / 2)) * 2;
-        float2 ml[kMaxSplits], ov[kMaxSplits];
+    for (int idx = tid; idx < my_rows * (kHd / 4); idx += kAtThreads) {
+        const int row = split + (idx / (kHd / 4)) * splits, dim = (idx % (kHd / 4)) * 4;
+        float2 ml[kMaxSplits];
+        float4 ov[kMaxSplits];
 #pragma unroll
         for (int sp = 0; sp < kMaxSplits; ++sp) {
             if (sp < splits) {
                 ml[sp] = *reinterpret_cast<const float2 *>(peer[sp] + (size_t)row * kWsRow + kHd);
-                ov[sp] = *reinterpret_cast<const float2 *>(peer[sp] + (size_t)row * kWsRow + dim);
+                ov[sp] = *reinterpret_cast<const float4 *>(peer[sp] + (size_t)row * kWsRow + dim);
             } else {
                 ml[sp] = make_float2(-INFINITY, 0.f);
-                ov[sp] = make_float2(0.f, 0.f);
+                ov[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
         float M = -INFINITY;
 #pragma unroll
         for (int sp = 0; sp < kMaxSplits; ++sp) M = fmaxf(M, ml[sp].x);
-        float L = 0.f, a0 = 0.f, a1 = 0.f;
+        float L = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int sp = 0; sp < kMaxSplits; ++sp) {
-            const float wgt = (ml[sp].x == -INFINITY) ? 0.f : exp2f(ml[sp].x - M);
-            L += ml[sp].y * wgt; a0 += ov[sp].x * wgt; a1 += ov[sp].y * wgt;
+            const float w = (ml[sp].x == -INFINITY) ? 0.f : exp2f(ml[sp].x - M);
+            L += ml[sp].y * w;
+            acc.x += ov[sp].x * w; acc.y += ov[sp].y * w; acc.z += ov[sp].z * w; acc.w += ov[sp].w * w;
         }
-        const float inv = L > 0.f ? 1.f / L : 0.f;
-        uint32_t hi, lo;
-        pack_split(a0 * inv, a1 * inv, hi, lo);
-        __nv_bfloat16 *dst = o + ((size_t)row * n_heads + head) * kHd + dim;
-        *reinterpret_cast<uint32_t *>(dst) = hi;
-        if (COMP) *reinterpret_cast<uint32_t *>(dst + lo_off) = lo;
+        store4(row, dim, acc, L > 0.f ? 1.f / L : 0.f);
     }
     if (trace && threadIdx.x == 0 && cta < 256) trace[(size_t)cta * 16 + 6] = global_timer_ns();
     if (done_ctr != nullptr) {
@@ -484,24 +550,27 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     if (splits > kMaxSplits) splits = kMaxSplits;
     if (splits > n_tiles) splits = n_tiles;
     if (splits < 1) splits = 1;
-    const int tiles_per_split = (n_tiles + splits - 1) / splits;
-    splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
+    const int tiles_base = n_tiles / splits, tiles_rem = n_tiles % splits;   // the first tiles_rem splits take one tile more
     const int q_tiles = n_pad / 16;
     const int groups = q_tiles <= 2 ? 4 : (q_tiles <= 4 ? 2 : 1);
     if (comp && kv_lo == nullptr) return cudaErrorInvalidValue;
     const int stages = (comp && groups == 1) ? 3 : kMaxStages;
     const size_t ring = (size_t)(comp ? 2 : 1) * n_pad * kRowBytes + (size_t)2 * stages * kKeyTile * kRowBytes +
                         (comp ? (size_t)2 * (n_pad + 1) * kRowBytes : 0);
-    const size_t part = (size_t)(groups > 1 ? groups + 1 : 1) * n_pad * kWsRow * sizeof(float) + (size_t)n_pad * groups * sizeof(float);
-    const size_t smem = ring > part ? ring : part;
+    const size_t part = (size_t)(groups > 1 ? groups + 1 : 1) * n_pad * kWsRow * sizeof(float);
+    const size_t recv_off = ((ring > part ? ring : part) + 127) / 128 * 128;
+    // with four key groups (<= 32 nodes) the rows are pushed to their owners: [splits][rows per CTA][kWsRow] behind the rest
+    const size_t recv = groups == 4 ? (size_t)splits * ((n_pad + splits - 1) / splits) * kWsRow * sizeof(float) : 0;
+    const size_t smem = recv_off + recv;
     typedef void (*Kern)(const __nv_bfloat16 *, const __nv_bfloat16 *, const __nv_bfloat16 *, int, int, int, int, int,
-                         const uint32_t *, __nv_bfloat16 *, int, int, const int32_t *, unsigned long long *,
-                         const __nv_bfloat16 *, int, int, DepWait, uint32_t *);
+                         const uint32_t *, __nv_bfloat16 *, int, int, int, const int32_t *, unsigned long long *,
+                         const __nv_bfloat16 *, int, int, DepWait, uint32_t *, int);
     static const Kern kerns[2][3] = {{attention_tc_kernel<1, false>, attention_tc_kernel<2, false>, attention_tc_kernel<4, false>},
                                      {attention_tc_kernel<1, true>, attention_tc_kernel<2, true>, attention_tc_kernel<4, true>}};
     static PerDeviceOnce attr_set;
     if (attr_set.needed()) {
-        const int max_smem = 2 * 128 * kRowBytes + 2 * 3 * kKeyTile * kRowBytes + 2 * 129 * kRowBytes;   // 128 nodes, hi + lo
+        // 128 nodes, hi + lo; with <= 32 nodes: a deeper ring, and the receive buffer behind it
+        const int max_smem = 2 * 128 * kRowBytes + 2 * 3 * kKeyTile * kRowBytes + 2 * 129 * kRowBytes + 128;
         for (int c = 0; c < 2; ++c)
             for (int g = 0; g < 3; ++g) {
                 cudaError_t e = cudaFuncSetAttribute(kerns[c][g], cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
@@ -523,7 +592,8 @@ cudaError_t launch_attention_tc(const void *q, const void *k, const void *v, int
     }
     return cudaLaunchKernelEx(&lc.cfg, kern, (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                               (const __nv_bfloat16 *)v, n_heads, kv_stride, P, n, n_pad, anc, (__nv_bfloat16 *)o, splits,
-                              tiles_per_split, (const int32_t *)status, trace, (const __nv_bfloat16 *)kv_lo, n_tree, q_first, dep, done);
+                              tiles_base, tiles_rem, (const int32_t *)status, trace, (const __nv_bfloat16 *)kv_lo, n_tree, q_first, dep, done,
+                              (int)recv_off);
 }
 
 }  // namespace llmcad
