@@ -396,10 +396,8 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
                 dep = with_sync ? sync.done_ctr : nullptr;
                 dep_target = sync.arrivals;
             }
-            // The first ring-fulls per CTA of the next GEMM's weights go to L2 during this GEMM's tail. Measured on
-            // B200 (7B shape, 32 nodes): 12 items gain 2.5 % of the pass, 24 items gain more for the QKV GEMM
-            // that follows the down projection and lose elsewhere (the burst competes with this GEMM's own
-            // tail); with more than 32 nodes the L2-to-SM path is the busy one and the prefetch only costs.
+            // Optionally (tuning aid, off by default: it measured slower, see launch_gemm_tc) the first items per CTA
+            // of the next GEMM's weights go to L2 during this GEMM's tail.
             if (i + 1 < specs.size() && n_pad <= 32) {
                 const int mode_next = specs[i + 1].ep.mode;
                 gemms[i].p.next = next_weights(gemms[i + 1].p, (mode_next == EPI_QKV || mode_next == EPI_PLAIN) ? 24 : 12);

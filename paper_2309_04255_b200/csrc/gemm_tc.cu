@@ -1080,7 +1080,7 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled, bool
 namespace {
 // tuning aids from the environment, read once per process
 struct Tuning {
-    int pair_k = 0, stages_cap = 0, l2_ahead = 8, next_items = -1;
+    int pair_k = 0, stages_cap = 0, l2_ahead = 0, next_items = 0;
     Tuning()
     {
         if (const char *e = getenv("LLMCAD_GEMM_PAIR_K")) { const int v = atoi(e); if (v == 1 || v == 2) pair_k = v; }
@@ -1127,7 +1127,10 @@ NextWeights next_weights(const GemmParams &planned, int items)
     nx.w_tiled = d.w_tiled;
     nx.n_tiles = d.n_tiles; nx.kb_per_tile = d.kb_per_tile; nx.pair_k = d.pair_k; nx.halves = d.halves;
     nx.items_per_cta = d.items_per_cta; nx.up_tile_offset = d.up_tile_offset; nx.grid = d.grid;
-    nx.items = tuning().next_items >= 0 ? tuning().next_items : items;
+    // Off unless asked for (LLMCAD_GEMM_NEXT_ITEMS): see launch_gemm_tc on what the L2 prefetches measured.
+    (void)items;
+    nx.items = tuning().next_items;
+    if (nx.items <= 0) nx.w_tiled = nullptr;
     return nx;
 }
 
@@ -1189,7 +1192,12 @@ cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_
         if (e != cudaSuccess) return e;
         attr_set.mark();
     }
-    // weight tiles pulled into L2 beyond the ring while the ring is blocked
+    // Weight tiles pulled into L2 beyond the ring while the ring is blocked (LLMCAD_GEMM_L2_AHEAD items), and the
+    // first items of the next GEMM pulled into L2 at the end of this one (LLMCAD_GEMM_NEXT_ITEMS): both off by
+    // default. Measured on B200 (7B shape, 32 nodes, whole passes): 3.12 ms with neither, 3.20-3.34 ms with any
+    // combination of 2-8 items ahead and 4-24 items of the next GEMM (the pair 8 + 12/24 that earlier builds ran
+    // with: 3.21-3.24 ms); at 64 nodes a layer takes 163 us without and 170 us with them. The prefetches bring
+    // nothing in that HBM would not deliver in time anyway, and compete with the stream's own requests.
     p.l2_ahead = tune.l2_ahead;
     if (p.wait_limit_ns == 0) p.wait_limit_ns = kDefaultWaitLimitNs;
     {
