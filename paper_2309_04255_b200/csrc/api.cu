@@ -372,12 +372,9 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
             if (!last) specs.push_back({l + 1, 0, 0, d, qkv_ep(l + 1, tiles4), false});
             else if (logits != nullptr) specs.push_back({-1, 0, 0, d, head_ep(tiles4), false});
         }
-        // every GEMM is planned first, so that each can tell its predecessor where its weights start
         std::vector<TcGemm> gemms(specs.size());
-        for (size_t i = 0; i < specs.size(); ++i) {
+        for (size_t i = 0; i < specs.size(); ++i)
             gemms[i].set(ctx, specs[i].l, specs[i].which, specs[i].act, specs[i].n_in, specs[i].ep, n_pad);
-            CUDA_TRY(plan_gemm_tc(gemms[i].p, ctx->n_sms));
-        }
         // Hand-over between the kernels: completion counters (one per kernel, zeroed here) where both sides are
         // tensor-core kernels of this library, the grid dependency otherwise. `dep` is what the next kernel
         // waits for: null after the embedding kernel and after a plain-ALU attention kernel.
@@ -395,12 +392,6 @@ int run_forward(llmcad_ctx *ctx, const void *packed, void *kv_cache, int P, cons
                                         n_tree, n_old, with_sync ? &sync : nullptr)) != LLMCAD_OK) return rc;
                 dep = with_sync ? sync.done_ctr : nullptr;
                 dep_target = sync.arrivals;
-            }
-            // Optionally (tuning aid, off by default: it measured slower, see launch_gemm_tc) the first items per CTA
-            // of the next GEMM's weights go to L2 during this GEMM's tail.
-            if (i + 1 < specs.size() && n_pad <= 32) {
-                const int mode_next = specs[i + 1].ep.mode;
-                gemms[i].p.next = next_weights(gemms[i + 1].p, (mode_next == EPI_QKV || mode_next == EPI_PLAIN) ? 24 : 12);
             }
             GemmParams &gp = gemms[i].p;
             gp.dep_ctr = dep; gp.dep_target = dep_target;

@@ -597,9 +597,11 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
         // ================================================= weight producer
         // Streams this CTA's weight tiles, in order, as fast as ring slots free up.
         if (lane == 0) {
-            Cursor<PK> cpf;                      // next item to prefetch into L2 (pc: next item to copy into the ring)
-            cpf.init(d);
-            uint32_t prefetched = 0;
+            // (Asking L2 for weights ahead of the ring while it is blocked, or for the first items of the next GEMM
+            // once this CTA's are all requested, or from the finishing kernel while HBM idles, was measured on B200
+            // and costs more than it brings in every combination: 3.12 ms per pass of the 7B shape without against
+            // 3.14-3.34 ms with 2-8 items ahead and 3-24 items of the next GEMM. The stream runs from HBM straight
+            // into the ring.)
             uint64_t t_idle = 0;
             while (!pc.done()) {
                 if (mbar_try(smem_u32(W4 ? &ctl.pempty[ps] : &ctl.empty[ps]), ppar)) {
@@ -607,49 +609,11 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
                     t_idle = 0;
                     continue;
                 }
-                if (W4) {      // the packed ring is deep enough by itself
-                    __nanosleep(32);
-                    if (t_idle == 0) t_idle = global_timer_ns();
-                    else if (*abort_flag || global_timer_ns() - t_idle > wait_limit) { timed_out = true; break; }
-                    continue;
-                }
-                // The ring is full: the consumers wait for their input. Weights do not depend on that,
-                // so pull the next ones from HBM into L2 now; when the ring moves again it refills at
-                // L2 speed.
-                if (prefetched < pissued) {       // the ring overtook the prefetch cursor: catch up
-                    while (prefetched < pissued && !cpf.done()) { cpf.advance(); ++prefetched; }
-                }
-                if (!cpf.done() && prefetched < pissued + (uint32_t)p.stages + (uint32_t)p.l2_ahead) {
-                    if (prefetched >= pissued + (uint32_t)p.stages && d.w_tiled != nullptr) {
-                        const size_t t = (size_t)(cpf.tile + (cpf.half ? d.up_tile_offset : 0)) * d.kb_per_tile + cpf.kb0();
-                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(d.w_tiled + t * kATileBytes),
-                                     "r"((uint32_t)cpf.nk() * kATileBytes) : "memory");
-                    }
-                    cpf.advance();
-                    ++prefetched;
-                    continue;
-                }
                 __nanosleep(32);
                 if (t_idle == 0) t_idle = global_timer_ns();
                 else if (*abort_flag || global_timer_ns() - t_idle > wait_limit) { timed_out = true; break; }
             }
             LLMCAD_TRACE(6);
-            // This CTA's weights are all requested. HBM would now idle through the tail of this GEMM and
-            // the start of the next: ask L2 for the first items of the next GEMM's CTA of the same number.
-            const NextWeights &nx = p.next;
-            if (nx.w_tiled != nullptr && !timed_out && (int)blockIdx.x < nx.grid) {
-                const int ppt = (nx.kb_per_tile + nx.pair_k - 1) / nx.pair_k, ipt = ppt * nx.halves;
-                const int begin = (int)blockIdx.x * nx.items_per_cta;
-                const int end = min(nx.n_tiles * ipt, begin + min(nx.items_per_cta, nx.items));
-                for (int i = begin; i < end; ++i) {
-                    const int tile = i / ipt, q = i - tile * ipt;
-                    const int kp = q / nx.halves, half = q - kp * nx.halves;
-                    const int kb0 = kp * nx.pair_k, nk = min(nx.pair_k, nx.kb_per_tile - kb0);
-                    const size_t t = (size_t)(tile + (half ? nx.up_tile_offset : 0)) * nx.kb_per_tile + kb0;
-                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(nx.w_tiled + t * kATileBytes),
-                                 "r"((uint32_t)nk * kATileBytes) : "memory");
-                }
-            }
         }
     } else if (warp == 6) {
         // ================================================= activation loader
@@ -1080,13 +1044,11 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled, bool
 namespace {
 // tuning aids from the environment, read once per process
 struct Tuning {
-    int pair_k = 0, stages_cap = 0, l2_ahead = 0, next_items = 0;
+    int pair_k = 0, stages_cap = 0;
     Tuning()
     {
         if (const char *e = getenv("LLMCAD_GEMM_PAIR_K")) { const int v = atoi(e); if (v == 1 || v == 2) pair_k = v; }
         if (const char *e = getenv("LLMCAD_GEMM_STAGES")) { const int v = atoi(e); if (v >= 2) stages_cap = v; }
-        if (const char *e = getenv("LLMCAD_GEMM_L2_AHEAD")) l2_ahead = atoi(e);
-        if (const char *e = getenv("LLMCAD_GEMM_NEXT_ITEMS")) next_items = atoi(e);
     }
 };
 const Tuning &tuning()
@@ -1118,20 +1080,6 @@ cudaError_t plan_gemm_tc(GemmParams &p, int n_sms)
     grid = (int)((total + ipc - 1) / ipc);
     d.grid = grid;
     return cudaSuccess;
-}
-
-NextWeights next_weights(const GemmParams &planned, int items)
-{
-    const GemmDesc &d = planned.g;
-    NextWeights nx{};
-    nx.w_tiled = d.w_tiled;
-    nx.n_tiles = d.n_tiles; nx.kb_per_tile = d.kb_per_tile; nx.pair_k = d.pair_k; nx.halves = d.halves;
-    nx.items_per_cta = d.items_per_cta; nx.up_tile_offset = d.up_tile_offset; nx.grid = d.grid;
-    // Off unless asked for (LLMCAD_GEMM_NEXT_ITEMS): see launch_gemm_tc on what the L2 prefetches measured.
-    (void)items;
-    nx.items = tuning().next_items;
-    if (nx.items <= 0) nx.w_tiled = nullptr;
-    return nx;
 }
 
 cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_t partial_floats, cudaStream_t st, int *launched)
@@ -1174,7 +1122,6 @@ cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_
         if (pst < 2) return cudaErrorInvalidConfiguration;
         p.pstages = pst;
         smem = (size_t)stages * stage_bytes + (size_t)pst * pstage + 1024;
-        p.next = NextWeights{};
     }
     p.stages = stages;
     static PerDeviceOnce attr_set;
@@ -1192,13 +1139,6 @@ cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_
         if (e != cudaSuccess) return e;
         attr_set.mark();
     }
-    // Weight tiles pulled into L2 beyond the ring while the ring is blocked (LLMCAD_GEMM_L2_AHEAD items), and the
-    // first items of the next GEMM pulled into L2 at the end of this one (LLMCAD_GEMM_NEXT_ITEMS): both off by
-    // default. Measured on B200 (7B shape, 32 nodes, whole passes): 3.12 ms with neither, 3.20-3.34 ms with any
-    // combination of 2-8 items ahead and 4-24 items of the next GEMM (the pair 8 + 12/24 that earlier builds ran
-    // with: 3.21-3.24 ms); at 64 nodes a layer takes 163 us without and 170 us with them. The prefetches bring
-    // nothing in that HBM would not deliver in time anyway, and compete with the stream's own requests.
-    p.l2_ahead = tune.l2_ahead;
     if (p.wait_limit_ns == 0) p.wait_limit_ns = kDefaultWaitLimitNs;
     {
         LaunchCfg lc(grid, kThreads, smem, st);

@@ -31,15 +31,6 @@ struct GemmMaps {
     CUtensorMap x;  // the activation matrix, box 64 x n_pad rows x planes (hi, lo)
 };
 
-// Where the GEMM that follows in the stream will start reading its weights: when a streaming CTA has
-// issued its last weight copy, it asks L2 for the first items of the same-numbered CTA of the next
-// GEMM, so that HBM keeps working through this GEMM's tail and the next ring fills from L2.
-struct NextWeights {
-    const uint8_t *w_tiled;     // nullptr: nothing to prefetch
-    int n_tiles, kb_per_tile, pair_k, halves, items_per_cta, up_tile_offset, grid;
-    int items;                  // ring items to prefetch per CTA
-};
-
 struct GemmParams {
     int n_pad;          // tree nodes padded to a multiple of 16
     int comp;           // 1: activations come as hi + lo planes; the MMA N is 2 * n_pad and the two columns of a node are added
@@ -51,10 +42,8 @@ struct GemmParams {
                         // tile t held by CTA c sits in slot t + c
     int32_t *status;
     unsigned long long *trace;  // optional [256][16] timeline in ns of this GEMM (nullptr: off)
-    int l2_ahead;       // ring items the producer may prefetch into L2 beyond the ring
     int withhold_act;   // self-test of the wait limit: the activation copies are never issued
     uint64_t wait_limit_ns;   // bound of every device-side wait of the launch
-    NextWeights next;
     // hand-over counters (common.cuh): the streaming kernel waits for `dep` (its input is final, the workspace is
     // free), its four dump warps arrive at s_done; the finishing kernel waits for s_done (4 x grid arrivals) and
     // every CTA of it arrives at f_done (f_grid arrivals, set by the launcher). Null: grid dependencies instead.
@@ -85,10 +74,8 @@ size_t gemm_tc_partial_floats(int n_sms, int max_tiles, int max_n_pad);
 // Describes one GEMM (fills everything but items_per_cta and grid, which the launcher sets).
 GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled = nullptr, bool w4 = false);
 
-// Fixes how the GEMM is cut up (k-blocks per ring item, items per CTA, grid); launch_gemm_tc calls it
-// itself, callers that want to describe a GEMM to its predecessor (next_weights) call it first.
+// Fixes how the GEMM is cut up (k-blocks per ring item, items per CTA, grid); launch_gemm_tc calls it itself.
 cudaError_t plan_gemm_tc(GemmParams &p, int n_sms);
-NextWeights next_weights(const GemmParams &planned, int items);
 
 // Enqueues one GEMM: the streaming kernel, then the finishing kernel (both with programmatic
 // stream serialization). partial_floats is the size of p.partials; cudaErrorInvalidValue if the

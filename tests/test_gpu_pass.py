@@ -283,14 +283,13 @@ print("ok")
 
 
 @pytest.mark.parametrize("env", [{"LLMCAD_PDL": "0"}, {"LLMCAD_SYNC_COUNTERS": "1"}, {"LLMCAD_COMP": "0"},
-                                 {"LLMCAD_GEMM_PAIR_K": "1"}, {"LLMCAD_GEMM_STAGES": "2", "LLMCAD_GEMM_L2_AHEAD": "0"},
-                                 {"LLMCAD_GEMM_L2_AHEAD": "8", "LLMCAD_GEMM_NEXT_ITEMS": "12"},
+                                 {"LLMCAD_GEMM_PAIR_K": "1"}, {"LLMCAD_GEMM_STAGES": "2"},
                                  {"LLMCAD_ATTN_T5_MIN_N": "1"}, {"LLMCAD_ATTN_T5_MIN_N": "0"}])
 def test_tuning_paths_stay_correct(env):
     """The environment knobs select other code paths of the same kernels (no programmatic dependent
     launch, hand-over between kernels through completion counters, plain bf16 activations, ring items
-    of one k-block, a two-stage ring, the L2 prefetches of weight tiles, the tcgen05 attention kernel for
-    every tree size, the mma.sync attention kernel for every tree size): each must still match the oracle. The knobs are read once per
+    of one k-block, a two-stage ring, the tcgen05 attention kernel for every tree size, the mma.sync
+    attention kernel for every tree size): each must still match the oracle. The knobs are read once per
     process, hence the child process."""
     import os, subprocess, sys
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
