@@ -160,7 +160,9 @@ def test_skinny_gemm(shape, mode):
 
 # ----------------------------------------------------------------------------- tree attention
 
-ATTN_CASES = [(0, 1), (0, 15), (5, 8), (64, 33), (300, 32), (1024, 64), (257, 128), (2048, 17), (1000, 97), (4095, 128)]
+ATTN_CASES = [(0, 1), (0, 15), (5, 8), (64, 33), (300, 32), (1024, 64), (257, 128), (2048, 17), (1000, 97), (4095, 128),
+              # fewer query rows than key splits (some CTAs of a cluster own no row), uneven tiles per split
+              (2048, 1), (500, 3), (129, 16), (577, 32)]
 
 
 @pytest.mark.parametrize("case", ATTN_CASES)
