@@ -63,6 +63,7 @@ constexpr size_t kFinSmem = 24 * 1024;   // dynamic shared memory the finishing 
 constexpr int kATileBytes = kTileM * kBlockK * 2;  // 16 KB
 constexpr int kMaxStages = 16;
 constexpr int kMaxPStages = 24;   // INT4 weights: ring of packed tiles
+constexpr int kMaxAStages = 8;    // INT4 weights: ring of activation k-block sets, apart from the expanded weight tiles
 constexpr int kMaxPairK = 2;     // k-blocks per ring item (GemmDesc::pair_k): 2 = one 32 KB weight copy feeds 8 MMAs;
                                  // 1 for wide activation tiles, which would leave too few ring stages otherwise
 
@@ -244,6 +245,8 @@ struct SharedCtl {
     volatile uint32_t a_issued;     // ring items whose weight copy (and expect_tx) has been issued
     uint64_t pfull[kMaxPStages];    // INT4 weights: packed tile landed / packed stage free again
     uint64_t pempty[kMaxPStages];
+    uint64_t afull[kMaxAStages];    // INT4 weights: activation tiles of an item landed / their slot free again
+    uint64_t aempty[kMaxAStages];
 };
 
 // A ring item is (tile, k-block pair, half): up to two consecutive 64-wide k-blocks of one
@@ -504,9 +507,16 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
     const uint32_t stage_bytes = PK * (kATileBytes + b_tile_bytes);
     const uint32_t b_off = PK * kATileBytes;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    // INT4 weights: behind the ring of MMA stages lies a ring of packed items (PK tiles of 4224 bytes each)
+    // INT4 weights: three rings of their own. [p.stages expanded weight items of PK bf16 tiles, written by the dump
+    // warps and read by the MMA][p.astages activation items, PK k-blocks each, filled by the activation loader as far
+    // ahead as slots are free][p.pstages packed items of PK tiles of 4224 bytes each, filled by the weight producer].
+    // Every item needs its activation tiles from L2 (~1.5 us under load) and they are larger than its packed weights:
+    // kept in the stage of the expanded weights, as in the bf16 path, too few of them would be in flight.
     constexpr uint32_t pstage_bytes = PK * kW4TileBytes;
-    const uint32_t packed_base = smem_base + (uint32_t)p.stages * stage_bytes;
+    constexpr uint32_t wstage_bytes = PK * kATileBytes;
+    const uint32_t astage_bytes = PK * b_tile_bytes;
+    const uint32_t act_base = smem_base + (uint32_t)p.stages * wstage_bytes;
+    const uint32_t packed_base = W4 ? act_base + (uint32_t)p.astages * astage_bytes : smem_base + (uint32_t)p.stages * stage_bytes;
     const uint32_t acc_cols = 2u * nb;                    // TMEM columns of one accumulator buffer (gate | up)
     const bool two_bufs = p.acc_bufs == 2;
     const uint64_t wait_limit = p.wait_limit_ns;          // every wait below gives up after this many ns
@@ -556,15 +566,18 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
     };
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            // INT4: a stage is full when its activation bytes have landed (armed by one arrival) and the four
-            // dump warps have written their quarters of the weight tile
-            mbar_init(smem_u32(&ctl.full[s]), W4 ? 5 : 1);
+            // INT4: an expanded weight item is full when the four dump warps have written their quarters of it
+            mbar_init(smem_u32(&ctl.full[s]), W4 ? 4 : 1);
             mbar_init(smem_u32(&ctl.empty[s]), 1);
         }
         if (W4) {
             for (int s = 0; s < p.pstages; ++s) {
                 mbar_init(smem_u32(&ctl.pfull[s]), 1);
                 mbar_init(smem_u32(&ctl.pempty[s]), 4);
+            }
+            for (int s = 0; s < p.astages; ++s) {
+                mbar_init(smem_u32(&ctl.afull[s]), 1);
+                mbar_init(smem_u32(&ctl.aempty[s]), 1);
             }
         }
         for (int b = 0; b < 2; ++b) {
@@ -629,7 +642,22 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
             if (!dep_wait_thread(dep)) timed_out = true;
             fence_proxy_async();          // the activations were written by ordinary stores; the copies below read them
             pdl_launch_dependents();
-            while (!c.done() && !timed_out && !p.withhold_act) {
+            if (W4) {
+                // a ring of its own: item i goes to slot i % astages as soon as the MMAs of item i - astages have read it
+                uint32_t apar = 1;         // a fresh barrier passes a wait on parity 1
+                while (!c.done() && !timed_out && !p.withhold_act) {
+                    if (!mbar_wait(smem_u32(&ctl.aempty[s]), apar, abort_flag, wait_limit)) { timed_out = true; break; }
+                    const uint32_t full = smem_u32(&ctl.afull[s]);
+                    const uint32_t dst = act_base + s * astage_bytes;
+                    const int nk = c.nk();
+                    mbar_expect_tx(full, (uint32_t)nk * b_tile_bytes);
+                    for (int k = 0; k < nk; ++k)
+                        tma_load_3d(dst + k * b_tile_bytes, &maps.x, (c.kb0() + k) * kBlockK, full, pol_keep);
+                    c.advance();
+                    if (++s == p.astages) { s = 0; apar ^= 1u; }
+                }
+            }
+            while (!W4 && !c.done() && !timed_out && !p.withhold_act) {
                 uint64_t t0 = 0;
                 // the stage is ours: the producer has passed its "empty" wait and armed the barrier
                 for (uint32_t spin = 0; (int32_t)(ctl.a_issued - (i + 1)) < 0; ++spin) {
@@ -658,6 +686,8 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
             c.init(d);
             uint32_t seg = 0, ph = 0;   // ph: parity the MMA warp waits for on its stage's "full" barrier
             int s = 0;
+            int as = 0;                 // INT4: slot of the activation ring, and the parity waited for on its "full" barrier
+            uint32_t aph = 0;
             while (!c.done() && !timed_out) {
                 // one segment: the items of one tile that belong to this CTA
                 const int tile = c.tile, halves = c.halves;
@@ -668,15 +698,17 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
                 const uint32_t d0 = tmem_base + buf * acc_cols;
                 for (int q = 0; !c.done() && c.tile == tile; ++q) {
                     if (!mbar_wait(smem_u32(&ctl.full[s]), ph, abort_flag, wait_limit)) { timed_out = true; break; }
+                    if (W4 && !mbar_wait(smem_u32(&ctl.afull[as]), aph, abort_flag, wait_limit)) { timed_out = true; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_base + s * stage_bytes;
+                    const uint32_t a_addr = W4 ? smem_base + s * wstage_bytes : smem_base + s * stage_bytes;
+                    const uint32_t b_addr = W4 ? act_base + as * astage_bytes : a_addr + b_off;
                     // segments of a two-half GEMM start on a gate item, so the first `halves` items
                     // of a segment are the ones that must overwrite their accumulator
                     const uint32_t dcol = d0 + c.half * nb;
                     const int nk = c.nk();
                     for (int k = 0; k < nk; ++k) {
                         const uint64_t a_desc = make_smem_desc(a_addr + k * kATileBytes);
-                        const uint64_t b_desc = make_smem_desc(a_addr + b_off + k * b_tile_bytes);
+                        const uint64_t b_desc = make_smem_desc(b_addr + k * b_tile_bytes);
 #pragma unroll
                         for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
                             // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the >>4 address field
@@ -684,6 +716,10 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
                         }
                     }
                     tc_commit(smem_u32(&ctl.empty[s]));  // frees the stage when these MMAs have read it
+                    if (W4) {
+                        tc_commit(smem_u32(&ctl.aempty[as]));
+                        if (++as == p.astages) { as = 0; aph ^= 1u; }
+                    }
                     c.advance();
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
@@ -708,25 +744,20 @@ gemm_stream_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant_
         const int ipt = pairs_per_tile_c<PK>(d) * d.halves;
         const size_t slot_stride = slot_floats(d.halves, p.n_pad);
         // ---- INT4 weights: these warps also turn every packed item into the bf16 tiles the MMA reads, a quarter
-        // of the rows each, in the MMA stage that they claim for it. Element j of a word sits where
+        // of the rows each, in the next free slot of the ring of expanded items. Element j of a word sits where
         // (word >> 4k) & 0x000f000f picks elements 2k, 2k+1; OR-ing 0x4300 into each half makes the bf16 values
         // 128 + u (u = q + 8), and one fused multiply-add per pair, (128 + u) * 2^e - 136 * 2^e, gives q * 2^e exactly.
         Cursor<PK> dc;
         dc.init(d);
         int ds = 0, dps = 0;
-        uint32_t dpar = 1, dppar = 0, dcount = 0;      // a fresh "empty" barrier passes a wait on parity 1
+        uint32_t dpar = 1, dppar = 0;                  // a fresh "empty" barrier passes a wait on parity 1
         uint8_t *const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
         auto dequant_item = [&]() -> bool {
             const int nk = dc.nk();
             if (!mbar_wait_warp(smem_u32(&ctl.empty[ds]), dpar, abort_flag, lane, wait_limit)) return false;
-            if (warp == 2 && lane == 0) {
-                mbar_expect_tx(smem_u32(&ctl.full[ds]), (uint32_t)nk * b_tile_bytes);
-                __threadfence_block();
-                ctl.a_issued = ++dcount;       // the activation loader may now add its bytes to this stage
-            }
             if (!mbar_wait_warp(smem_u32(&ctl.pfull[dps]), dppar, abort_flag, lane, wait_limit)) return false;
-            const uint8_t *pk = smem_gen + (size_t)p.stages * stage_bytes + (size_t)dps * pstage_bytes;
-            uint8_t *wt = smem_gen + (size_t)ds * stage_bytes;
+            const uint8_t *pk = smem_gen + (packed_base - smem_base) + (size_t)dps * pstage_bytes;
+            uint8_t *wt = smem_gen + (size_t)ds * wstage_bytes;
             // lane = (row within a group of four, chunk): iteration `it` handles row 32 * lane_grp + 4 * it + lane / 8,
             // words and stores of a warp instruction are contiguous (no bank conflicts). All loads of a k-block go
             // out before the first conversion: a warp is alone on its scheduler here, so latency is what counts.
@@ -1044,11 +1075,13 @@ GemmDesc make_gemm_desc(int n_in, const EpiParams &ep, const void *w_tiled, bool
 namespace {
 // tuning aids from the environment, read once per process
 struct Tuning {
-    int pair_k = 0, stages_cap = 0;
+    int pair_k = 0, stages_cap = 0, w4_wstages = 3, w4_pstages = 4;
     Tuning()
     {
         if (const char *e = getenv("LLMCAD_GEMM_PAIR_K")) { const int v = atoi(e); if (v == 1 || v == 2) pair_k = v; }
         if (const char *e = getenv("LLMCAD_GEMM_STAGES")) { const int v = atoi(e); if (v >= 2) stages_cap = v; }
+        if (const char *e = getenv("LLMCAD_W4_WSTAGES")) { const int v = atoi(e); if (v >= 2 && v <= kMaxStages) w4_wstages = v; }
+        if (const char *e = getenv("LLMCAD_W4_PSTAGES")) { const int v = atoi(e); if (v >= 2 && v <= kMaxPStages) w4_pstages = v; }
     }
 };
 const Tuning &tuning()
@@ -1110,18 +1143,25 @@ cudaError_t launch_gemm_tc(const GemmMaps &maps, GemmParams &p, int n_sms, size_
     if (stages < 2) return cudaErrorInvalidConfiguration;
     size_t smem = (size_t)stages * stage_bytes + 1024;
     p.pstages = 0;
+    p.astages = 0;
     if (d.w4) {
-        // INT4 weights: the MMA ring keeps what covers the latency of the activation copies (three stages where
-        // they fit), the rest of the shared memory holds packed items, four times as many weights per byte
+        // INT4 weights: three rings (see the kernel). Three expanded items (8-layer pass of the 7B shape at 32 nodes:
+        // 1.08 ms with two, 0.97 ms with three or four), a few packed items (they are small, 8.4 KB per 32 KB of
+        // bf16; 3 to 12 of them measure the same), and the rest of the shared memory for activation items.
         if (d.w_tiled == nullptr) return cudaErrorInvalidValue;
-        const size_t pstage = (size_t)pair_k * kW4TileBytes;
-        if (stages > 3) stages = 3;
-        while (stages > 2 && full_limit - (size_t)stages * stage_bytes < 8 * pstage) --stages;   // room for eight packed items
-        int pst = (int)((full_limit - (size_t)stages * stage_bytes) / pstage);
+        const size_t pstage = (size_t)pair_k * kW4TileBytes, wstage = (size_t)pair_k * kATileBytes;
+        const size_t astage = (size_t)pair_k * nb * kBlockK * 2;
+        stages = tune.w4_wstages;
+        int pst = tune.w4_pstages;
+        if ((size_t)stages * wstage + (size_t)pst * pstage + 2 * astage > full_limit) return cudaErrorInvalidConfiguration;
+        int ast = (int)((full_limit - (size_t)stages * wstage - (size_t)pst * pstage) / astage);
+        if (ast > kMaxAStages) ast = kMaxAStages;
+        // what the activation ring does not use goes to the packed ring
+        pst = (int)((full_limit - (size_t)stages * wstage - (size_t)ast * astage) / pstage);
         if (pst > kMaxPStages) pst = kMaxPStages;
-        if (pst < 2) return cudaErrorInvalidConfiguration;
         p.pstages = pst;
-        smem = (size_t)stages * stage_bytes + (size_t)pst * pstage + 1024;
+        p.astages = ast;
+        smem = (size_t)stages * wstage + (size_t)ast * astage + (size_t)pst * pstage + 1024;
     }
     p.stages = stages;
     static PerDeviceOnce attr_set;

@@ -35,8 +35,9 @@ struct GemmParams {
     int n_pad;          // tree nodes padded to a multiple of 16
     int comp;           // 1: activations come as hi + lo planes; the MMA N is 2 * n_pad and the two columns of a node are added
     int acc_bufs;       // accumulator buffers in TMEM: 2, or 1 when 2 x (gate | up) x MMA N exceeds the 512 columns
-    int stages;         // depth of the shared-memory ring
+    int stages;         // depth of the shared-memory ring (INT4 weights: of the ring of expanded weight items)
     int pstages;        // INT4 weights: depth of the ring of packed tiles that feeds it
+    int astages;        // INT4 weights: depth of the ring of activation items (with bf16 weights they share the weights' stages)
     int tmem_cols;      // allocated TMEM columns (power of two)
     float *partials;    // segment slots [n_tiles + grid][4 row groups][halves][n_pad][32 rows] fp32: the segment of
                         // tile t held by CTA c sits in slot t + c
