@@ -51,6 +51,22 @@ int llmcad_set_wait_limit_ns(llmcad_ctx *ctx, uint64_t ns);
  * works, or a negative host-detected error. The context is usable afterwards. */
 int llmcad_selftest_wait_timeout(llmcad_ctx *ctx, void *stream);
 
+/* Micro-benchmarks of the machine, context-free, on the current device (no tensor of the library is involved).
+ *
+ * llmcad_probe_bulk_copy: one CTA per SM, one issuing thread each, reads `bytes` (DEVICE buffer `src`, 16-byte
+ * aligned; every byte once, so a buffer much larger than L2 comes from HBM) into shared memory with cp.async.bulk
+ * copies of `copy_bytes` (a multiple of 16), `in_flight` (1..16) of them outstanding per CTA, copy_bytes * in_flight
+ * <= 200 KB: the weight stream of the skinny GEMMs without a consumer. Returns the rate of the slowest CTA's
+ * schedule, GB/s over all SMs, and the mean time from issuing a copy to its completion.
+ * llmcad_probe_mma_sync: `warps` (1..32) warps per SM issue mma.sync.m16n8k16 bf16 into `accumulators` (1, 2, 4, 8)
+ * independent accumulators each: multiply-adds per clock and SM, and SM cycles per MMA of one warp (with one
+ * accumulator and one warp: the latency of a dependent MMA).
+ * Both synchronise `stream`; LLMCAD_ERR_TIMEOUT if a copy does not arrive within the default wait limit. */
+int llmcad_probe_bulk_copy(const void *src /*DEVICE*/, size_t bytes, int32_t copy_bytes, int32_t in_flight, void *stream,
+                           double *gbs /*HOST*/, double *latency_us /*HOST*/);
+int llmcad_probe_mma_sync(int32_t warps, int32_t accumulators, void *stream, double *fma_per_clk_sm /*HOST*/,
+                          double *cycles_per_mma /*HOST*/);
+
 #ifdef __cplusplus
 }
 #endif

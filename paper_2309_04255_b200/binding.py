@@ -34,6 +34,7 @@ EXPORTS = [
     "llmcad_tree_confidence", "llmcad_update_threshold", "llmcad_extend_tree", "llmcad_tree_branches", "llmcad_branch_pacer",
     "llmcad_set_wait_limit_ns", "llmcad_selftest_wait_timeout",
     "llmcad_quantize_int4", "llmcad_tiled_weight_int4_bytes", "llmcad_tile_weight_int4", "llmcad_skinny_gemm_tiled_int4",
+    "llmcad_probe_bulk_copy", "llmcad_probe_mma_sync",
 ]
 
 
@@ -117,6 +118,8 @@ def lib():
         L.llmcad_skinny_gemm_tiled_int4.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
         L.llmcad_set_wait_limit_ns.argtypes = [vp, C.c_uint64]
         L.llmcad_selftest_wait_timeout.argtypes = [vp, vp]
+        L.llmcad_probe_bulk_copy.argtypes = [vp, sz, i32, i32, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.llmcad_probe_mma_sync.argtypes = [i32, i32, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         _lib = L
     return _lib
 
@@ -326,6 +329,21 @@ class Verifier:
         if code < 0:
             raise LlmcadError(code, "llmcad_selftest_wait_timeout")
         return code
+
+
+def probe_bulk_copy(src: torch.Tensor, copy_bytes: int, in_flight: int):
+    """(GB/s, mean latency in us) of cp.async.bulk copies streaming `src` from device memory once (llmcad_profile.h)."""
+    gbs, lat = C.c_double(0.0), C.c_double(0.0)
+    _check(lib().llmcad_probe_bulk_copy(_ptr(src), src.numel() * src.element_size(), int(copy_bytes), int(in_flight),
+                                        _stream(), C.byref(gbs), C.byref(lat)), "llmcad_probe_bulk_copy")
+    return gbs.value, lat.value
+
+
+def probe_mma_sync(warps: int, accumulators: int):
+    """(multiply-adds per clock and SM, SM cycles per MMA of one warp) of mma.sync.m16n8k16 bf16 (llmcad_profile.h)."""
+    rate, cyc = C.c_double(0.0), C.c_double(0.0)
+    _check(lib().llmcad_probe_mma_sync(int(warps), int(accumulators), _stream(), C.byref(rate), C.byref(cyc)), "llmcad_probe_mma_sync")
+    return rate.value, cyc.value
 
 
 def tree_attention_noalloc(q, k, v, prefix_len: int, parent, o, status=None):

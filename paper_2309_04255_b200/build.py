@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libllmcad.so")
 LIB_CHECKS = os.path.join(HERE, "libllmcad_checks.so")     # the same sources with -DLLMCAD_CHECKS (device-side bounds checks)
-SOURCES = ["api.cu", "tree.cu", "gemm_simt.cu", "attention_simt.cu", "gemm_tc.cu", "attention_tc.cu", "attention_t5.cu", "pack.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "tree.cu", "gemm_simt.cu", "attention_simt.cu", "gemm_tc.cu", "attention_tc.cu", "attention_t5.cu", "pack.cu", "noalloc.cu", "probes.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

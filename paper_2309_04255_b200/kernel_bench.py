@@ -6,6 +6,7 @@ reads its operands from HBM, not from L2).
     python -m paper_2309_04255_b200.kernel_bench avnav [--model 7b] [--prefix 512] [--nodes 2,4,...]
     python -m paper_2309_04255_b200.kernel_bench extend [--model 7b] [--prefix 512] [--nodes 32] [--steps 1,2,4,8]
     python -m paper_2309_04255_b200.kernel_bench timeline [--workload C2] [--layers 4] [--int4]   # per-kernel time stamps of one pass
+    python -m paper_2309_04255_b200.kernel_bench probes                                            # bulk-copy and mma.sync rates of the machine
 
 Each line of output is one JSON object. `--reps` launches are timed per case after `--warmup`.
 """
@@ -294,6 +295,28 @@ def bench_timeline(args):
         print(json.dumps(row), flush=True)
 
 
+def bench_probes(args):
+    """What the machine gives to the two access patterns of the pass (llmcad_probe_* of the measurement interface):
+    cp.async.bulk copies streaming a buffer of 8 GB from HBM once, by copy size and copies in flight per SM; and the
+    legacy mma.sync.m16n8k16 bf16 path by warps per SM and independent accumulators per warp."""
+    dev = torch.device("cuda:0")
+    src = torch.empty(args.gb << 30, dtype=torch.uint8, device=dev)
+    src.fill_(1)
+    torch.cuda.synchronize()
+    for size in (4224, 8448, 16384, 32768):
+        for depth in (1, 2, 4, 8, 12):
+            if size * depth > 200 * 1024:
+                continue
+            B.probe_bulk_copy(src, size, depth)          # warm-up
+            gbs, lat = B.probe_bulk_copy(src, size, depth)
+            print(json.dumps({"probe": "bulk_copy", "copy_bytes": size, "in_flight": depth, "gbs": round(gbs, 1),
+                              "latency_us": round(lat, 2)}), flush=True)
+    for warps, acc in ((1, 1), (8, 1), (8, 2), (8, 4), (8, 8), (16, 8), (4, 8)):
+        rate, cyc = B.probe_mma_sync(warps, acc)
+        print(json.dumps({"probe": "mma_sync_m16n8k16_bf16", "warps_per_sm": warps, "accumulators_per_warp": acc,
+                          "fma_per_clk_sm": round(rate, 1), "cycles_per_mma_per_warp": round(cyc, 1)}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -324,11 +347,13 @@ def main():
     t.add_argument("--workload", default="C2")
     t.add_argument("--layers", type=int, default=4)
     t.add_argument("--int4", action="store_true")
+    pr = sub.add_parser("probes")
+    pr.add_argument("--gb", type=int, default=8)
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("kernel_bench needs a CUDA device")
     {"attention": bench_attention, "gemm": bench_gemm, "avnav": bench_avnav, "extend": bench_extend,
-     "timeline": bench_timeline}[args.cmd](args)
+     "timeline": bench_timeline, "probes": bench_probes}[args.cmd](args)
 
 
 if __name__ == "__main__":

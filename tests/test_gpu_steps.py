@@ -262,3 +262,19 @@ def test_attention_head_dim_64_f32():
     ref = orc.tree_attention(q.reshape(n, H * hd), k[:, :P], vv[:, :P], k[:, P:].permute(1, 0, 2).reshape(n, -1),
                              vv[:, P:].permute(1, 0, 2).reshape(n, -1), anc, H, hd)
     assert np.abs(o.double().cpu().numpy().reshape(n, -1) - ref).max() <= 1e-5 * np.abs(ref).max()
+
+
+# ----------------------------------------------------------------------------- machine probes (measurement interface)
+
+def test_machine_probes_run_and_are_plausible():
+    """The micro-benchmarks of llmcad_profile.h return sane figures: a streaming read well above 1 TB/s with a
+    latency of microseconds at most, and an mma.sync rate between 100 and 4096 multiply-adds per clock and SM."""
+    src = torch.ones(1 << 30, dtype=torch.uint8, device=DEV)
+    gbs, lat = B.probe_bulk_copy(src, 32768, 4)
+    assert 1000.0 < gbs < 20000.0 and 0.1 < lat < 50.0, (gbs, lat)
+    gbs1, _ = B.probe_bulk_copy(src, 8448, 1)
+    assert gbs1 < gbs
+    rate, cyc = B.probe_mma_sync(8, 8)
+    assert 100.0 < rate <= 4096.0 and cyc > 1.0, (rate, cyc)
+    with pytest.raises(B.LlmcadError):
+        B.probe_bulk_copy(src, 1000, 4)          # not a multiple of 16
