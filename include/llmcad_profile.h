@@ -29,7 +29,9 @@ int llmcad_get_kernel_timing(llmcad_ctx *ctx, int32_t kind, double *total_ms /*H
  * first weight copy issued (2), grid dependency resolved (3), first accumulator ready (4), last
  * weight copy issued (6), last MMA issued (7), accumulators in the workspace (8), streaming CTA
  * exit (13); finishing CTA entry (9), its grid dependency resolved (10), exit (12). Attention:
- * entry (0), exit (12). Launch order of a pass: QKV GEMM, then per layer attention, O, gate/up,
+ * entry (0), grid dependency resolved (1), first key tile in shared memory (2), key loop done (3),
+ * partial rows merged and handed to their owners (4), cluster barrier passed (5), output stored (6),
+ * exit (12). Launch order of a pass: QKV GEMM, then per layer attention, O, gate/up,
  * down, next QKV (lm_head after the last layer). The stamps cost a predicated store each and do not
  * change how consecutive kernels overlap. */
 int llmcad_set_gemm_trace(llmcad_ctx *ctx, uint64_t *trace, int32_t capacity);
