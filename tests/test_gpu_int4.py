@@ -114,3 +114,42 @@ def test_int4_contexts_are_refused_where_they_cannot_work():
     cfg = gen.ModelConfig("odd", 1, 512, 4, 128, 1000, 512, "bf16")               # FFN width not a multiple of 64
     c = B.make_config(cfg, 64, flags=B.FLAG_INT4_WEIGHTS)
     assert B.lib().llmcad_create(ctypes.byref(c), ctypes.byref(h)) == B.ERR_UNSUPPORTED
+
+
+def test_int4_passes_of_changing_prefix_and_size_are_reproducible():
+    """Passes over different prefix lengths and tree sizes, queued back to back on one INT4 context, each give bit
+    for bit what the same pass gave the first time (the cache is put back before every pass, since a pass writes
+    its tree nodes' slots): the three rings of the INT4 GEMMs and the split merge of the attention kernels leave
+    nothing behind that depends on timing or on the previous launch's shape."""
+    cfg = gen.shrink(gen.MODELS["7b"], 2)
+    S = 640 + 136
+    v = B.Verifier(cfg, S, device=DEV, flags=B.FLAG_INT4_WEIGHTS)
+    v.pack_globals({k: gen.gen_tensor_device(cfg, k, -1, DEV) for k in ("tok_embed", "final_norm", "lm_head")})
+    for l in range(cfg.n_layers):
+        v.pack_layer(l, {k: gen.gen_tensor_device(cfg, k, l, DEV) for k in gen.LAYER_TENSORS})
+    kvv = v.kv_view()
+    kvv[:, :, :, :640] = torch.randn((cfg.n_layers, 2, cfg.n_heads, 640, cfg.head_dim), device=DEV).to(kvv.dtype)
+    saved = kvv.clone()
+    cases = []
+    for P in (1, 64, 577, 640):
+        for n in (1, 17, 32, 33, 128):
+            tokens = torch.as_tensor(gen.gen_tokens(cfg, n, seed=n + P), device=DEV)
+            parent = torch.as_tensor(gen.tree_random(n, 12, "uniform4", n + P) if n > 1 else np.array([-1], np.int32), device=DEV)
+            kvv.copy_(saved)
+            out = v.verify_tree(P, tokens, parent)
+            torch.cuda.synchronize()
+            assert out["scalars"][B.S_STATUS].item() == 0
+            cases.append((P, n, tokens, parent, out["logits"].clone(), out["scalars"].clone()))
+    rng = np.random.default_rng(3)
+    outs = []
+    for _ in range(200):
+        ci = int(rng.integers(len(cases)))
+        P, n, tokens, parent, _, _ = cases[ci]
+        kvv.copy_(saved)
+        o = v.new_outputs(n)
+        v.verify_tree(P, tokens, parent, out=o)
+        outs.append((ci, o))
+    torch.cuda.synchronize()
+    for ci, o in outs:
+        assert torch.equal(o["logits"], cases[ci][4]) and torch.equal(o["scalars"], cases[ci][5]), cases[ci][:2]
+    v.close()
